@@ -1,0 +1,82 @@
+"""Drives the oracle (and, in the GPU tests, the CUDA library beside it) over a workload.
+
+The per-step inputs come from `workloads` (random numbers only). Queries and the current
+token's key/value rows are the harness's stand-in for the backbone model: they are made
+here from the same hidden row with the oracle's projection, so that a token admitted with
+k_new and later rebuilt from x must get the same cache row back.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+
+import workloads as wl
+from oracle import adore_oracle as ao
+
+
+def oracle_config(cfg: wl.WorkloadConfig, batch: Optional[int] = None) -> ao.OracleConfig:
+    return ao.OracleConfig(batch=cfg.batch if batch is None else batch, n_layers=cfg.n_layers,
+                           n_heads=cfg.n_heads, head_dim=cfg.head_dim, hidden=cfg.hidden,
+                           capacity=cfg.capacity, rebuild_max=cfg.rebuild_max, topk=cfg.topk,
+                           max_tokens=cfg.max_tokens, ctrl_hidden=cfg.ctrl_hidden, dtype=cfg.dtype,
+                           rebuild_mode=cfg.rebuild_mode, rope_theta=cfg.rope_theta,
+                           pos_scale=cfg.pos_scale)
+
+
+class Workload:
+    """Seeded inputs of one config, restricted to the first `batch` sequences."""
+
+    def __init__(self, cfg: wl.WorkloadConfig, batch: Optional[int] = None):
+        self.cfg = cfg
+        self.batch = cfg.batch if batch is None else batch
+        self.ctrl = wl.controller_weights(cfg)
+        self.w_kv = [wl.projection_weights(cfg, l) for l in range(cfg.n_layers)]
+        self.w_q = [wl.query_weights(cfg, l) for l in range(cfg.n_layers)]
+        self.r_in = self._r_in()
+
+    def _r_in(self) -> int:
+        if self.cfg.rebuild_mode != "explicit":
+            return 0
+        n = max(self.cfg.max_tokens, 1)
+        mean = n * self.cfg.rebuild_p
+        return int(min(n, np.ceil(mean + 6 * np.sqrt(mean) + 8)))
+
+    def prompt(self, layer: int = 0) -> np.ndarray:
+        return wl.hidden_rows(self.cfg, 0, self.cfg.prompt, layer, self.batch)
+
+    def x_new(self, n: int, layer: int = 0) -> np.ndarray:
+        return wl.hidden_rows(self.cfg, n, 1, layer, self.batch)[:, 0, :]
+
+    def qkv(self, n: int, layer: int, x_row: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+        c = self.cfg
+        B = x_row.shape[0]
+        q = np.empty((B, c.n_heads, c.head_dim), np.float32)
+        k = np.empty_like(q)
+        v = np.empty_like(q)
+        for b in range(B):
+            if c.identity_projection:      # q, k, v i.i.d. N(0,1): q is its own draw
+                qb = wl.gaussian(c.seed, "q", (c.n_heads, c.head_dim), 1.0, c.dtype, idx=(layer, n, b))
+            else:
+                qb = ao.project_q(self.w_q[layer], x_row[b], n, c.n_heads, c.head_dim, c.rope_theta, c.dtype)
+            kb, vb = ao.project_kv(self.w_kv[layer], x_row[b], n, c.n_heads, c.head_dim, c.rope_theta, c.dtype)
+            q[b], k[b], v[b] = qb, kb, vb
+        return q, k, v
+
+    def explicit(self, step: int, n: int) -> Tuple[Optional[np.ndarray], Optional[np.ndarray]]:
+        if self.cfg.rebuild_mode != "explicit":
+            return None, None
+        return wl.rebuild_flags(self.cfg, step, n, self.r_in, self.batch)
+
+
+def make_oracle(w: Workload) -> ao.AdoreOracle:
+    orc = ao.AdoreOracle(oracle_config(w.cfg, w.batch), w.ctrl)
+    for l in range(w.cfg.n_layers):
+        orc.set_projection(l, w.w_kv[l])
+    return orc
+
+
+def explicit_as_lists(lists: Optional[np.ndarray], counts: Optional[np.ndarray]) -> Optional[List[np.ndarray]]:
+    if lists is None:
+        return None
+    return [lists[b, : counts[b]] for b in range(lists.shape[0])]
