@@ -1,0 +1,190 @@
+/*
+ * adore.h - C ABI of the ADORE decode path for NVIDIA B200 (sm_100a).
+ *
+ * ADORE (adaptive token release) keeps a fixed-capacity KV cache during decoding: a small
+ * controller scores every token, the lowest-scoring cached token is released when a new one
+ * arrives, and the most valuable released tokens are recomputed ("rebuilt") so that the next
+ * attention can still see them. One decode step for one layer is
+ *
+ *   1. attention of the current query over the occupied cache slots plus the current token's
+ *      own key/value, restricted to the K largest logits, with the per-slot weights emitted;
+ *   2. (once per step, at layer 0) controller scoring of the new token, release of the least
+ *      valuable retained token, in-place admission of the new token, choice of the rebuild list;
+ *   3. rebuild: K/V projection of the listed tokens' layer-input rows, rotary embedding at the
+ *      token's original position, scatter into the freed slots.
+ *
+ * Conventions
+ *   - Every function returns an adore_status_t. Nothing throws, aborts or traps the device.
+ *   - All device work is queued on the CUDA stream given at create time and is asynchronous;
+ *     only adore_cache_sync_status, adore_decode_step_host (at its end) and
+ *     adore_cache_destroy wait for the device.
+ *   - "device" pointers are CUDA device addresses of the cache's GPU; "host" pointers are
+ *     ordinary (ideally pinned) host memory. The library borrows per-call buffers until the
+ *     stream has passed the call, and borrows projection weights until the cache is destroyed.
+ *   - Element type T is float (ADORE_F32) or bfloat16 (ADORE_BF16), chosen at create time, for
+ *     q, k, v, x, out, the cache and the projection weights. Row-major everywhere.
+ *   - Argument errors are found on the host before anything is launched. Inconsistencies only
+ *     the device can see (an explicit rebuild entry that is out of range, a bounded wait that
+ *     ran out) set a bit in a device error word, turn the offending item into a no-op and are
+ *     reported by adore_cache_sync_status.
+ *   - A cache is not thread-safe; use one thread per cache.
+ *
+ * Sequences of one cache move in lockstep: all B sequences hold the same number of tokens n.
+ */
+#ifndef ADORE_H_
+#define ADORE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct adore_cache adore_cache_t; /* opaque; owned by the library */
+
+typedef enum {
+  ADORE_OK = 0,
+  ADORE_ERR_INVALID_ARG = 1,      /* NULL where not allowed, size or enum out of range          */
+  ADORE_ERR_OOM = 2,              /* device or host allocation failed                           */
+  ADORE_ERR_TOKEN_TABLE_FULL = 3, /* n would exceed max_tokens                                  */
+  ADORE_ERR_STATE = 4,            /* call order (e.g. layer l>0 before layer 0 of the step)     */
+  ADORE_ERR_CUDA = 5,             /* a CUDA runtime/driver call failed                          */
+  ADORE_ERR_DEVICE_FLAG = 6,      /* device error word set: bad explicit entry / bounds check   */
+  ADORE_ERR_TIMEOUT = 7,          /* a bounded device-side wait gave up                         */
+  ADORE_ERR_UNSUPPORTED = 8       /* shape outside what the kernels are built for               */
+} adore_status_t;
+
+typedef enum { ADORE_F32 = 0, ADORE_BF16 = 1 } adore_dtype_t;
+
+/* How the rebuild list is chosen each step (Section 2.3, first sentence).
+ * POLICY:   the min(R_max, #released) released tokens with the highest controller score.
+ * EXPLICIT: the caller names candidate token positions per step; entries that are resident
+ *           are dropped, duplicates removed, and if more than R_max remain the R_max with the
+ *           highest score are kept. */
+typedef enum { ADORE_REBUILD_POLICY = 0, ADORE_REBUILD_EXPLICIT = 1 } adore_rebuild_mode_t;
+
+/* Slot roles in the slot map. */
+enum { ADORE_SLOT_EMPTY = 0, ADORE_SLOT_RETAINED = 1, ADORE_SLOT_REBUILT = 2 };
+
+typedef struct {
+  uint32_t struct_size;  /* sizeof(adore_config_t), for versioning                               */
+  int32_t batch;         /* B  sequences                                                        */
+  int32_t n_layers;      /* L                                                                   */
+  int32_t n_heads;       /* H                                                                   */
+  int32_t head_dim;      /* dh: 64 or 128                                                       */
+  int32_t hidden;        /* d: controller input width and projection inner dimension            */
+  int32_t capacity;      /* C  slots per sequence, 1 <= C <= 4096                               */
+  int32_t rebuild_max;   /* R_max, 0 <= R_max < C; retained budget m = C - R_max (Section 2.3)   */
+  int32_t topk;          /* K >= 1 of the attention mask (Section 2.2); K >= C+1 disables it     */
+  int32_t max_tokens;    /* token-table rows per sequence, <= 8192                              */
+  int32_t ctrl_hidden;   /* d' (Appendix B: 128), <= 256                                        */
+  adore_dtype_t dtype;
+  adore_rebuild_mode_t rebuild_mode;
+  float rope_theta;      /* rotary base; 0 disables the rotation                                 */
+  float pos_scale;       /* position feature of the controller is n / pos_scale                  */
+  uint32_t flags;        /* reserved, must be 0                                                  */
+} adore_config_t;
+
+/* Controller parameters (Section 2.2 Eq. 2 and Appendix B), float32, HOST pointers, copied at
+ * create. Stacked GRU gate order: reset, update, candidate. */
+typedef struct {
+  const float *gru_w_ih; /* [3d', d]  */
+  const float *gru_w_hh; /* [3d', d'] */
+  const float *gru_b_ih; /* [3d']     */
+  const float *gru_b_hh; /* [3d']     */
+  const float *pos_w;    /* [d']   position layer FC(1 -> d') */
+  const float *pos_b;    /* [d']   */
+  const float *mlp_w1;   /* [d', d'] interaction layer (Tanh)  */
+  const float *mlp_b1;   /* [d']   */
+  const float *mlp_w2;   /* [d']   output layer FC(d' -> 1), sigmoid applied to its output */
+  const float *mlp_b2;   /* [1]    */
+} adore_controller_weights_t;
+
+/* Creates an empty cache on the current CUDA device (Section 2.1: a cache of m selected rows per
+ * layer; here C = m + R_max slots). cuda_stream is a cudaStream_t (NULL = default stream). The
+ * library allocates the K/V slots [L][B][H][C][dh], the token table (hidden rows, scores, slot
+ * index per token), controller state and scratch. Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA. */
+adore_status_t adore_cache_create(const adore_config_t *cfg, const adore_controller_weights_t *ctrl,
+                                  void *cuda_stream, adore_cache_t **out);
+
+/* Waits for the stream, frees everything the cache owns. NULL is accepted. */
+adore_status_t adore_cache_destroy(adore_cache_t *cache);
+
+/* Registers the K/V projection of a layer (Section 2.3: rebuilt states are recomputed from token
+ * embeddings). w_kv: device, T[2*H*dh, d] row-major, key rows first then value rows; borrowed
+ * until destroy; must be 16-byte aligned. */
+adore_status_t adore_cache_set_projection(adore_cache_t *cache, int32_t layer, const void *w_kv);
+
+/* Bulk load of T prompt tokens into an EMPTY cache (Section 2.1: user input tokens t_1..t_s).
+ * x: device T[B, T, d]. Runs the controller over the T tokens, retains the newest token plus the
+ * min(m-1, T-1) highest-scoring earlier ones in ascending position from slot 0 (the set that
+ * releasing one token at a time would reach), chooses the rebuild list as in a decode step
+ * (POLICY mode only), and fills every layer whose projection is set from these rows.
+ * Errors: STATE (cache not empty), TOKEN_TABLE_FULL, INVALID_ARG. */
+adore_status_t adore_cache_append_tokens(adore_cache_t *cache, const void *x, int32_t T);
+
+/* Recomputes the K/V rows of every resident token of `layer` from x_table[b, tok, :]
+ * (device T[B, max_tokens, d]); NULL uses the cache's own stored rows. For stacks whose layers
+ * have their own input rows (Section 2.3 recomputes states layer by layer). */
+adore_status_t adore_cache_fill_layer(adore_cache_t *cache, int32_t layer, const void *x_table);
+
+/* One decode step for one layer (Sections 2.1-2.3). Call layer 0 first in every step; it also
+ * runs the controller for the new token, releases / admits / chooses the rebuild list, and
+ * advances n. All pointers are DEVICE pointers.
+ *   q, k_new, v_new : T[B, H, dh]; k_new already carries the rotary embedding of position n.
+ *   x_new           : T[B, d], read at layer 0 only (stored in the token table), else ignored.
+ *   explicit_list   : int32[B, r_in] candidate token positions, explicit_count int32[B] how many
+ *                     are valid per sequence; both NULL in POLICY mode. Read at layer 0 only.
+ *   out             : T[B, H, dh].
+ *   weights         : float[B, H, C+1] or NULL. Entry s < C is slot s, entry C the current
+ *                     token; masked or empty entries are 0.
+ * The attention reads the cache as the previous step left it (retained + last step's rebuilt
+ * rows), i.e. the m+R+1 rows of Section 2.3; the new token's row is then written in place.
+ * Errors: INVALID_ARG, STATE, TOKEN_TABLE_FULL, CUDA. */
+adore_status_t adore_decode_step(adore_cache_t *cache, int32_t layer, const void *q, const void *k_new,
+                                 const void *v_new, const void *x_new, const int32_t *explicit_list,
+                                 const int32_t *explicit_count, int32_t r_in, void *out, float *weights);
+
+/* Same step (Sections 2.1-2.3) with HOST buffers: copies the inputs to the device, runs
+ * adore_decode_step, copies `out` (and `weights` if not NULL) back and waits for the stream.
+ * Pinned host memory makes the copies asynchronous up to the final wait. */
+adore_status_t adore_decode_step_host(adore_cache_t *cache, int32_t layer, const void *q, const void *k_new,
+                                      const void *v_new, const void *x_new, const int32_t *explicit_list,
+                                      const int32_t *explicit_count, int32_t r_in, void *out, float *weights);
+
+/* Rebuild for one layer (Section 2.3): Y = X_L [W_k ; W_v]^T for the rows of this step's rebuild
+ * list, rotary embedding on the key half at each token's original position, rounding to T and
+ * scatter into the list's slots. x_table: device T[B, max_tokens, d] rows indexed by token
+ * position, or NULL for the cache's stored rows. Call after adore_decode_step of the same layer.
+ * Errors: STATE (no projection / no step), INVALID_ARG, CUDA. */
+adore_status_t adore_rebuild(adore_cache_t *cache, int32_t layer, const void *x_table);
+
+/* Read-only DEVICE views of the state of Sections 2.2-2.3 for checking; valid until the next
+ * call that changes the cache. */
+adore_status_t adore_cache_slot_map(adore_cache_t *cache, const int32_t **slot_tok /*[B,C]*/,
+                                    const uint8_t **slot_role /*[B,C]*/);
+adore_status_t adore_cache_rebuild_list(adore_cache_t *cache, const int32_t **tok /*[B,R_max]*/,
+                                        const int32_t **slot /*[B,R_max]*/, const int32_t **count /*[B]*/);
+adore_status_t adore_cache_step_info(adore_cache_t *cache, const int32_t **admit_slot /*[B]*/,
+                                     const int32_t **evicted_tok /*[B]*/);
+adore_status_t adore_cache_scores(adore_cache_t *cache, const float **score /*[B,max_tokens]*/,
+                                  const float **sigma /*[B,max_tokens]*/);
+adore_status_t adore_cache_kv(adore_cache_t *cache, int32_t layer, const void **k, const void **v);
+
+/* Number of tokens n per sequence (host value). */
+int32_t adore_cache_num_tokens(const adore_cache_t *cache);
+
+/* Kernel launches issued by this cache so far (host counter). */
+int64_t adore_cache_launch_count(const adore_cache_t *cache);
+
+/* Waits for the stream and turns the device error word into a status (OK, DEVICE_FLAG, TIMEOUT,
+ * or CUDA if the stream itself failed). The word is cleared. */
+adore_status_t adore_cache_sync_status(adore_cache_t *cache);
+
+const char *adore_status_string(adore_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADORE_H_ */

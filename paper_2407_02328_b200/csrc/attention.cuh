@@ -1,0 +1,277 @@
+// Decode attention over the slot cache with top-K masking and weight emission.
+//
+// Computes, per (sequence b, head h), the target attention of Section 2.1 (unnumbered equation
+// after Eq. 1) / Section 2.3: logits of the query against every occupied slot and against the
+// current token's own key, only the K largest logits keep a weight (Section 2.2, first bullet),
+// softmax over the kept ones, weighted sum of the kept value rows. The kept weights are written
+// out per slot. Finally the current token's key/value row is written into its slot (append of
+// the most recent state, Section 2.2 third bullet).
+//
+// One CTA per (b, h). The K block of a (b, h) is one contiguous C*dh array, so phase 1 streams it
+// with 16-byte loads, phase 2 finds the K-th largest logit with a 4-pass radix select in shared
+// memory, phase 3 is the softmax, phase 4 reads ONLY the kept value rows.
+#pragma once
+
+#include "common.cuh"
+
+namespace adore {
+
+template <typename T>
+struct AttnParams {
+  const T* q;            // [B,H,DH]
+  const T* k_new;        // [B,H,DH]
+  const T* v_new;        // [B,H,DH]
+  T* out;                // [B,H,DH]
+  float* weights;        // [B,H,C+1] or nullptr
+  T* Kc;                 // layer base [B,H,C,DH]
+  T* Vc;
+  const int* slot_tok;   // [B,C] map the cache rows currently follow (<0: empty)
+  const int* admit_slot; // [B] slot that receives the new row, or nullptr
+  int B, H, C, topk;
+  float scale;           // 1/sqrt(DH)
+  unsigned* err;
+};
+
+constexpr int kAttnThreads = 256;
+constexpr int kAttnUnroll = 4;
+
+__host__ __device__ inline size_t attn_smem_bytes(int C, int DH) {
+  const int cp = (C + 1 + 3) & ~3;
+  return sizeof(float) * cp + sizeof(int) * cp + sizeof(unsigned) * 256 +
+         sizeof(float) * (kAttnThreads / 32) * DH + sizeof(float) * 64;
+}
+
+template <int NT>
+__device__ __forceinline__ float block_sum_f(float v, float* tmp) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = warp_sum(v);
+  __syncthreads();                       // tmp may still be read from a previous reduction
+  if (lane == 0) tmp[warp] = v;
+  __syncthreads();
+  float r = 0.f;
+#pragma unroll
+  for (int w = 0; w < NT / 32; ++w) r += tmp[w];
+  return r;
+}
+template <int NT>
+__device__ __forceinline__ float block_max_f(float v, float* tmp) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = warp_max(v);
+  __syncthreads();
+  if (lane == 0) tmp[warp] = v;
+  __syncthreads();
+  float r = tmp[0];
+#pragma unroll
+  for (int w = 1; w < NT / 32; ++w) r = fmaxf(r, tmp[w]);
+  return r;
+}
+
+template <typename T, int DH>
+__global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParams<T> p) {
+  constexpr int NT = kAttnThreads;
+  constexpr int NW = NT / 32;
+  constexpr int EPL = Elem<T>::kPer16B;   // elements per lane (one 16-byte load)
+  constexpr int LPR = DH / EPL;           // lanes that share one row
+  constexpr int RPW = 32 / LPR;           // rows per warp-wide load
+  static_assert(LPR >= 1 && LPR <= 32 && (LPR & (LPR - 1)) == 0, "row must split over a warp");
+  constexpr int U = kAttnUnroll;
+
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int C = p.C, rows = C + 1, cp = (rows + 3) & ~3;
+  float* s_logit = reinterpret_cast<float*>(smem_raw);
+  int* s_list = reinterpret_cast<int*>(s_logit + cp);
+  unsigned* s_hist = reinterpret_cast<unsigned*>(s_list + cp);
+  float* s_red = reinterpret_cast<float*>(s_hist + 256);
+  float* s_tmp = s_red + NW * DH;          // 64 words: reduction scratch [0,32), broadcast [32,64)
+  int* s_sel = reinterpret_cast<int*>(s_tmp + 32);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int sub = lane / LPR, li = lane % LPR;
+  const int bh = blockIdx.x, b = bh / p.H;
+  const size_t row_bytes = size_t(DH) * sizeof(T);
+  const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * row_bytes;
+  const unsigned char* Vb = reinterpret_cast<const unsigned char*>(p.Vc) + size_t(bh) * C * row_bytes;
+  const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * row_bytes;
+  const unsigned char* vnew = reinterpret_cast<const unsigned char*>(p.v_new) + size_t(bh) * row_bytes;
+  const int* map = p.slot_tok + size_t(b) * C;
+
+  // ---- phase 1: logits -------------------------------------------------------------------
+  float qf[EPL];
+  {
+    const uint4 qr = *reinterpret_cast<const uint4*>(
+        reinterpret_cast<const unsigned char*>(p.q) + size_t(bh) * row_bytes + li * 16);
+    Elem<T>::unpack(qr, qf);
+  }
+  for (int r0 = warp * RPW; r0 < rows; r0 += NW * RPW * U) {
+    uint4 kv[U];
+    bool ok[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int row = r0 + u * NW * RPW + sub;
+      ok[u] = row < rows && (row == C || map[row] >= 0);
+      kv[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (ok[u]) kv[u] = ldg_stream((row == C ? knew : Kb + size_t(row) * row_bytes) + li * 16);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int row = r0 + u * NW * RPW + sub;
+      float kf[EPL];
+      Elem<T>::unpack(kv[u], kf);
+      float dot = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kf[e], dot);
+#pragma unroll
+      for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      if (li == 0 && row < rows) s_logit[row] = ok[u] ? dot * p.scale : -INFINITY;
+    }
+  }
+  __syncthreads();
+
+  // ---- phase 2: which logits are kept (K largest, lower index wins ties) -------------------
+  int cnt = 0;
+  for (int i = tid; i < rows; i += NT) cnt += (s_logit[i] > -INFINITY) ? 1 : 0;
+  const int n_cand = __float2int_rn(block_sum_f<NT>(float(cnt), s_tmp));
+  uint32_t thr_key = 0u;                  // keep every candidate unless there are more than K
+  if (n_cand > p.topk) {
+    uint32_t prefix = 0u, mask = 0u;
+    int need = p.topk;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int i = tid; i < 256; i += NT) s_hist[i] = 0u;
+      __syncthreads();
+      for (int i = tid; i < rows; i += NT) {
+        const uint32_t key = float_key(s_logit[i]);
+        if ((key & mask) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (warp == 0) {
+        int c[8], tot = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = int(s_hist[lane * 8 + j]); tot += c[j]; }
+        int incl = tot;                   // suffix sum: this lane's bins and all higher ones
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += t;
+        }
+        const int above = incl - tot;
+        if (above < need && need <= above + tot) {
+          int acc = above;
+#pragma unroll
+          for (int j = 7; j >= 0; --j) {
+            if (acc < need && need <= acc + c[j]) { s_sel[0] = lane * 8 + j; s_sel[1] = need - acc; s_sel[2] = c[j]; }
+            acc += c[j];
+          }
+        }
+      }
+      __syncthreads();
+      prefix |= uint32_t(s_sel[0]) << shift;
+      mask |= 255u << shift;
+      need = s_sel[1];
+    }
+    thr_key = prefix;
+    const int n_eq = s_sel[2];
+    __syncthreads();
+    if (n_eq != need && tid == 0) {       // exact ties at the threshold: keep the lowest indices
+      int left = need;
+      for (int i = 0; i < rows; ++i)
+        if (float_key(s_logit[i]) == thr_key) { if (left > 0) --left; else s_logit[i] = -INFINITY; }
+    }
+    __syncthreads();
+  }
+
+  // ---- phase 3: softmax over the kept logits ----------------------------------------------
+  float mx = -INFINITY;
+  for (int i = tid; i < rows; i += NT) {
+    const float l = s_logit[i];
+    if (l > -INFINITY && float_key(l) >= thr_key) mx = fmaxf(mx, l);
+  }
+  mx = block_max_f<NT>(mx, s_tmp);
+  float part = 0.f;
+  for (int i = tid; i < rows; i += NT) {
+    const float l = s_logit[i];
+    const bool keep = l > -INFINITY && float_key(l) >= thr_key;
+    const float e = keep ? expf(l - mx) : -1.f;   // -1 marks "not kept"
+    s_logit[i] = e;
+    part += keep ? e : 0.f;
+  }
+  const float inv = 1.f / block_sum_f<NT>(part, s_tmp);
+  // ordered compaction of the kept indices; weights replace the logits in place
+  int n_kept = 0;
+  for (int i0 = 0; i0 < rows; i0 += NT) {
+    const int i = i0 + tid;
+    const float e = i < rows ? s_logit[i] : -1.f;
+    const bool keep = e >= 0.f;
+    const unsigned bal = __ballot_sync(0xffffffffu, keep);
+    __syncthreads();
+    if (lane == 0) s_sel[8 + warp] = __popc(bal);
+    __syncthreads();
+    int base = n_kept, total = 0;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) { const int c = s_sel[8 + w]; if (w < warp) base += c; total += c; }
+    const float wgt = keep ? e * inv : 0.f;
+    if (i < rows) {
+      s_logit[i] = wgt;
+      if (p.weights) p.weights[size_t(bh) * rows + i] = wgt;
+    }
+    if (keep) s_list[base + __popc(bal & ((1u << lane) - 1u))] = i;
+    n_kept += total;
+  }
+  __syncthreads();
+
+  // ---- phase 4: weighted sum of the kept value rows ----------------------------------------
+  float acc[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  for (int j0 = warp * RPW; j0 < n_kept; j0 += NW * RPW * U) {
+    uint4 vv[U];
+    float wv[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int j = j0 + u * NW * RPW + sub;
+      vv[u] = make_uint4(0u, 0u, 0u, 0u);
+      wv[u] = 0.f;
+      if (j < n_kept) {
+        const int idx = s_list[j];
+        wv[u] = s_logit[idx];
+        vv[u] = ldg_stream((idx == C ? vnew : Vb + size_t(idx) * row_bytes) + li * 16);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      float vf[EPL];
+      Elem<T>::unpack(vv[u], vf);
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc[e] = fmaf(wv[u], vf[e], acc[e]);
+    }
+  }
+#pragma unroll
+  for (int o = LPR; o < 32; o <<= 1)
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+  if (sub == 0)
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) s_red[warp * DH + li * EPL + e] = acc[e];
+  __syncthreads();
+  for (int e = tid; e < DH; e += NT) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) s += s_red[w * DH + e];
+    p.out[size_t(bh) * DH + e] = Elem<T>::from_float(s);
+  }
+
+  // ---- admit: the current token's row goes into its slot (all reads of this block are done) --
+  if (p.admit_slot != nullptr) {
+    const int s = p.admit_slot[b];
+    if (s >= 0 && s < C) {
+      constexpr int V16 = int(sizeof(T)) * DH / 16;
+      unsigned char* kd = const_cast<unsigned char*>(Kb) + size_t(s) * row_bytes;
+      unsigned char* vd = const_cast<unsigned char*>(Vb) + size_t(s) * row_bytes;
+      if (tid < V16) reinterpret_cast<uint4*>(kd)[tid] = reinterpret_cast<const uint4*>(knew)[tid];
+      else if (tid < 2 * V16) reinterpret_cast<uint4*>(vd)[tid - V16] = reinterpret_cast<const uint4*>(vnew)[tid - V16];
+    } else if (tid == 0) {
+      set_error(p.err, ERRW_BOUNDS);
+    }
+  }
+}
+
+}  // namespace adore
