@@ -1,0 +1,608 @@
+// Host side of the ADORE C ABI: the cache object, argument checks, launch sequences.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/adore.h"
+#include "attention.cuh"
+#include "attention_tma.cuh"
+#include "controller.cuh"
+#include "rebuild_simt.cuh"
+#include "rebuild_tc.cuh"
+#include "select.cuh"
+
+using namespace adore;
+
+namespace {
+
+constexpr int kSelectThreadsSmall = 512;
+constexpr int kMaxPrefillRows = 8192;       // controller rows per chunk during a bulk load
+
+// ---- kernels that glue the device functions together -----------------------------------------
+template <typename T>
+__global__ void ctrl_select_kernel(const RecurParams rp, const SelectParams sp, const T* x_new, T* x_store, int d) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int b = blockIdx.x;
+  // keep the new token's layer-input row: it is what a later rebuild recomputes from
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(x_new + size_t(b) * d);
+    uint4* dst = reinterpret_cast<uint4*>(x_store + (size_t(b) * sp.max_tokens + sp.n) * d);
+    for (int i = threadIdx.x; i < int(d * sizeof(T) / 16); i += blockDim.x) dst[i] = src[i];
+  }
+  controller_tokens(rp, b, reinterpret_cast<double*>(smem));
+  __syncthreads();
+  select_step(sp, smem);
+}
+
+__global__ void ctrl_recur_kernel(const RecurParams rp) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  controller_tokens(rp, blockIdx.x, reinterpret_cast<double*>(smem));
+}
+
+__global__ void bulk_select_kernel(const SelectParams sp) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  select_bulk(sp, smem);
+}
+
+__global__ void fill_i32_kernel(int* p, int v, size_t n) {
+  for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < n; i += size_t(gridDim.x) * blockDim.x) p[i] = v;
+}
+
+int pow2_at_least(int v) {
+  int p = 2;
+  while (p < v) p <<= 1;
+  return p;
+}
+
+}  // namespace
+
+struct adore_cache {
+  adore_config_t cfg{};
+  cudaStream_t stream = nullptr;
+  size_t esz = 2;
+  int n = 0;                    // tokens per sequence
+  int step_layer0_done = 0;     // a step is open (layer 0 ran)
+  int64_t launches = 0;
+  int cur = 0, attn = 0;        // slot-map buffers: target state / state the cache rows follow
+
+  void* Kc = nullptr;
+  void* Vc = nullptr;
+  void* x_store = nullptr;
+  double* z = nullptr;
+  float* score = nullptr;
+  float* sigma = nullptr;
+  int* tok_slot = nullptr;
+  int* slot_tok[2] = {nullptr, nullptr};
+  uint8_t* slot_role[2] = {nullptr, nullptr};
+  int* admit_slot = nullptr;
+  int* evicted_tok = nullptr;
+  int* rebuild_tok = nullptr;
+  int* rebuild_slot = nullptr;
+  int* rebuild_count = nullptr;
+  int* row_off = nullptr;
+  int* row_b = nullptr;
+  int* row_tok = nullptr;
+  int* row_slot = nullptr;
+  int* row_total = nullptr;
+  int* frow_b = nullptr;        // row table of a layer fill (all residents)
+  int* frow_tok = nullptr;
+  int* frow_slot = nullptr;
+  int* frow_total = nullptr;
+  unsigned* done_counter = nullptr;
+  unsigned* err = nullptr;
+  double* part = nullptr;
+  size_t part_doubles = 0;
+  int ksplit = 1;
+  float* rope_cos = nullptr;
+  float* rope_sin = nullptr;
+  // controller parameters on the device
+  float *w_ih = nullptr, *w_hh_t = nullptr, *b_ih = nullptr, *b_hh = nullptr, *pos_w = nullptr, *pos_b = nullptr,
+        *w1_t = nullptr, *b1 = nullptr, *w2 = nullptr, *b2 = nullptr;
+  std::vector<const void*> w_kv;
+  TcState tc;                   // tensor-core rebuild path (tensor maps, gather buffer)
+  // staging for the host-buffer entry point
+  void *h_q = nullptr, *h_k = nullptr, *h_v = nullptr, *h_x = nullptr, *h_out = nullptr;
+  int* h_list = nullptr;
+  int* h_count = nullptr;
+  float* h_weights = nullptr;
+  std::vector<void*> owned;
+};
+
+namespace {
+
+#define CUDA_OK(expr)                                   \
+  do {                                                  \
+    cudaError_t e_ = (expr);                            \
+    if (e_ != cudaSuccess) return cuda_fail(e_);        \
+  } while (0)
+
+adore_status_t cuda_fail(cudaError_t e) {
+  if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return ADORE_ERR_OOM; }
+  return ADORE_ERR_CUDA;
+}
+
+template <typename P>
+adore_status_t dev_alloc(adore_cache* c, P** out, size_t bytes, bool zero) {
+  void* p = nullptr;
+  CUDA_OK(cudaMalloc(&p, bytes ? bytes : 16));
+  c->owned.push_back(p);
+  if (zero) CUDA_OK(cudaMemsetAsync(p, 0, bytes ? bytes : 16, c->stream));
+  *out = static_cast<P*>(p);
+  return ADORE_OK;
+}
+
+adore_status_t upload(adore_cache* c, float** out, const float* host, size_t count) {
+  adore_status_t s = dev_alloc(c, out, count * sizeof(float), false);
+  if (s != ADORE_OK) return s;
+  CUDA_OK(cudaMemcpyAsync(*out, host, count * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));   // the host buffer may be a temporary
+  return ADORE_OK;
+}
+
+adore_status_t fill_i32(adore_cache* c, int* p, int v, size_t n) {
+  const int blocks = int(std::min<size_t>((n + 255) / 256, 1184));
+  fill_i32_kernel<<<blocks ? blocks : 1, 256, 0, c->stream>>>(p, v, n);
+  ++c->launches;
+  CUDA_OK(cudaGetLastError());
+  return ADORE_OK;
+}
+
+int select_threads(const adore_cache* c) { return 3 * c->cfg.ctrl_hidden <= kSelectThreadsSmall ? kSelectThreadsSmall : 1024; }
+
+RecurParams recur_params(adore_cache* c, int rows, int tc, int ksplit, int n0) {
+  RecurParams r{};
+  r.part = c->part; r.ksplit = ksplit; r.rows = rows; r.tc = tc; r.h = c->cfg.ctrl_hidden;
+  r.b_ih = c->b_ih; r.w_hh_t = c->w_hh_t; r.b_hh = c->b_hh; r.pos_w = c->pos_w; r.pos_b = c->pos_b;
+  r.w1_t = c->w1_t; r.b1 = c->b1; r.w2 = c->w2; r.b2 = c->b2;
+  r.z = c->z; r.score = c->score; r.sigma = c->sigma; r.max_tokens = c->cfg.max_tokens; r.n0 = n0;
+  r.pos_scale = double(c->cfg.pos_scale);
+  return r;
+}
+
+SelectParams select_params(adore_cache* c, int n, int P, int old_map, int new_map) {
+  SelectParams s{};
+  s.B = c->cfg.batch; s.C = c->cfg.capacity; s.m = c->cfg.capacity - c->cfg.rebuild_max; s.r_max = c->cfg.rebuild_max;
+  s.n = n; s.max_tokens = c->cfg.max_tokens; s.explicit_mode = c->cfg.rebuild_mode == ADORE_REBUILD_EXPLICIT; s.P = P;
+  s.slot_tok_old = c->slot_tok[old_map]; s.slot_role_old = c->slot_role[old_map];
+  s.slot_tok_new = c->slot_tok[new_map]; s.slot_role_new = c->slot_role[new_map];
+  s.tok_slot = c->tok_slot; s.score = c->score;
+  s.admit_slot = c->admit_slot; s.evicted_tok = c->evicted_tok; s.rebuild_tok = c->rebuild_tok;
+  s.rebuild_slot = c->rebuild_slot; s.rebuild_count = c->rebuild_count;
+  s.row_off = c->row_off; s.row_b = c->row_b; s.row_tok = c->row_tok; s.row_slot = c->row_slot; s.row_total = c->row_total;
+  s.done_counter = c->done_counter; s.err = c->err;
+  return s;
+}
+
+template <typename T>
+adore_status_t launch_gates(adore_cache* c, const T* x, long long seq_stride, int tc, int ksplit) {
+  GateParams<T> g{};
+  g.x = x; g.seq_stride = seq_stride; g.tc = tc; g.rows = c->cfg.batch * tc; g.d = c->cfg.hidden; g.G = 3 * c->cfg.ctrl_hidden;
+  g.w_ih = c->w_ih; g.part = c->part; g.ksplit = ksplit;
+  const int per = (c->cfg.hidden + ksplit - 1) / ksplit;
+  g.kslice = ((per + kGateKChunk - 1) / kGateKChunk) * kGateKChunk;
+  dim3 grid((g.G + kGateTile - 1) / kGateTile, (g.rows + kGateTile - 1) / kGateTile, ksplit);
+  ctrl_gates_kernel<T><<<grid, kGateThreads, 0, c->stream>>>(g);
+  ++c->launches;
+  CUDA_OK(cudaGetLastError());
+  return ADORE_OK;
+}
+
+template <typename T>
+adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const void* k_new, const void* v_new,
+                                void* out, float* weights) {
+  const adore_config_t& f = c->cfg;
+  AttnParams<T> p{};
+  const size_t layer_elems = size_t(f.batch) * f.n_heads * f.capacity * f.head_dim;
+  p.q = static_cast<const T*>(q); p.k_new = static_cast<const T*>(k_new); p.v_new = static_cast<const T*>(v_new);
+  p.out = static_cast<T*>(out); p.weights = weights;
+  p.Kc = static_cast<T*>(c->Kc) + layer * layer_elems; p.Vc = static_cast<T*>(c->Vc) + layer * layer_elems;
+  p.slot_tok = c->slot_tok[c->attn]; p.admit_slot = c->admit_slot;
+  p.B = f.batch; p.H = f.n_heads; p.C = f.capacity; p.topk = f.topk;
+  p.scale = float(1.0 / std::sqrt(double(f.head_dim)));
+  p.err = c->err;
+  const int grid = f.batch * f.n_heads;
+  cudaError_t e;
+  if (attn_tma_usable<T>(f.capacity, f.head_dim)) e = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
+  else if (f.head_dim == 64) {
+    const size_t smem = attn_smem_bytes(f.capacity, 64);
+    attention_kernel<T, 64><<<grid, kAttnThreads, smem, c->stream>>>(p);
+    e = cudaGetLastError();
+  } else {
+    const size_t smem = attn_smem_bytes(f.capacity, 128);
+    attention_kernel<T, 128><<<grid, kAttnThreads, smem, c->stream>>>(p);
+    e = cudaGetLastError();
+  }
+  ++c->launches;
+  CUDA_OK(e);
+  return ADORE_OK;
+}
+
+template <typename T>
+adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, const int* row_b, const int* row_tok,
+                              const int* row_slot, const int* row_total, int m_max) {
+  const adore_config_t& f = c->cfg;
+  if (m_max <= 0) return ADORE_OK;
+  RebuildParams<T> p{};
+  const size_t layer_elems = size_t(f.batch) * f.n_heads * f.capacity * f.head_dim;
+  p.x_table = static_cast<const T*>(x_table ? x_table : c->x_store); p.seq_stride = f.max_tokens; p.d = f.hidden;
+  p.w_kv = static_cast<const T*>(c->w_kv[layer]);
+  p.Kc = static_cast<T*>(c->Kc) + layer * layer_elems; p.Vc = static_cast<T*>(c->Vc) + layer * layer_elems;
+  p.row_b = row_b; p.row_tok = row_tok; p.row_slot = row_slot; p.row_total = row_total;
+  p.rope_cos = f.rope_theta != 0.f ? c->rope_cos : nullptr; p.rope_sin = f.rope_theta != 0.f ? c->rope_sin : nullptr;
+  p.H = f.n_heads; p.DH = f.head_dim; p.C = f.capacity; p.N = 2 * f.n_heads * f.head_dim; p.err = c->err;
+  if (tc_usable<T>(c->tc)) {
+    int launched = 0;
+    cudaError_t e = launch_rebuild_tc(c->tc, p, layer, m_max, c->stream, &launched);
+    c->launches += launched;
+    CUDA_OK(e);
+    return ADORE_OK;
+  }
+  dim3 grid(p.N / kSimtTile, (m_max + kSimtTile - 1) / kSimtTile);
+  rebuild_simt_kernel<T><<<grid, 256, 0, c->stream>>>(p);
+  ++c->launches;
+  CUDA_OK(cudaGetLastError());
+  return ADORE_OK;
+}
+
+adore_status_t fill_layer_impl(adore_cache* c, int layer, const void* x_table) {
+  const adore_config_t& f = c->cfg;
+  resident_rows_kernel<<<1, 1024, 0, c->stream>>>(c->slot_tok[c->cur], f.batch, f.capacity, c->frow_b, c->frow_tok,
+                                                  c->frow_slot, c->frow_total);
+  ++c->launches;
+  CUDA_OK(cudaGetLastError());
+  if (f.dtype == ADORE_F32)
+    return launch_rebuild<float>(c, layer, x_table, c->frow_b, c->frow_tok, c->frow_slot, c->frow_total, f.batch * f.capacity);
+  return launch_rebuild<__nv_bfloat16>(c, layer, x_table, c->frow_b, c->frow_tok, c->frow_slot, c->frow_total,
+                                       f.batch * f.capacity);
+}
+
+adore_status_t check_config(const adore_config_t* f) {
+  if (f->struct_size != sizeof(adore_config_t)) return ADORE_ERR_INVALID_ARG;
+  if (f->batch < 1 || f->n_layers < 1 || f->n_heads < 1 || f->hidden < 1 || f->capacity < 1 || f->topk < 1 ||
+      f->max_tokens < 1 || f->ctrl_hidden < 1 || f->rebuild_max < 0 || f->rebuild_max >= f->capacity || f->flags != 0 ||
+      !(f->pos_scale > 0.f) || f->rope_theta < 0.f)
+    return ADORE_ERR_INVALID_ARG;
+  if (f->dtype != ADORE_F32 && f->dtype != ADORE_BF16) return ADORE_ERR_INVALID_ARG;
+  if (f->rebuild_mode != ADORE_REBUILD_POLICY && f->rebuild_mode != ADORE_REBUILD_EXPLICIT) return ADORE_ERR_INVALID_ARG;
+  if (f->head_dim != 64 && f->head_dim != 128) return ADORE_ERR_UNSUPPORTED;
+  if (f->capacity > 4096 || f->max_tokens > 8192 || f->ctrl_hidden > 256 || f->hidden % 64 != 0)
+    return ADORE_ERR_UNSUPPORTED;
+  return ADORE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* adore_status_string(adore_status_t s) {
+  switch (s) {
+    case ADORE_OK: return "ok";
+    case ADORE_ERR_INVALID_ARG: return "invalid argument";
+    case ADORE_ERR_OOM: return "out of memory";
+    case ADORE_ERR_TOKEN_TABLE_FULL: return "token table full";
+    case ADORE_ERR_STATE: return "call out of order";
+    case ADORE_ERR_CUDA: return "CUDA call failed";
+    case ADORE_ERR_DEVICE_FLAG: return "device error word set";
+    case ADORE_ERR_TIMEOUT: return "bounded device wait gave up";
+    case ADORE_ERR_UNSUPPORTED: return "unsupported shape";
+  }
+  return "unknown status";
+}
+
+adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_controller_weights_t* w, void* cuda_stream,
+                                  adore_cache_t** out) {
+  if (!cfg || !w || !out) return ADORE_ERR_INVALID_ARG;
+  *out = nullptr;
+  adore_status_t st = check_config(cfg);
+  if (st != ADORE_OK) return st;
+  if (!w->gru_w_ih || !w->gru_w_hh || !w->gru_b_ih || !w->gru_b_hh || !w->pos_w || !w->pos_b || !w->mlp_w1 ||
+      !w->mlp_b1 || !w->mlp_w2 || !w->mlp_b2)
+    return ADORE_ERR_INVALID_ARG;
+  adore_cache* c = new (std::nothrow) adore_cache();
+  if (!c) return ADORE_ERR_OOM;
+  c->cfg = *cfg;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->esz = cfg->dtype == ADORE_F32 ? 4 : 2;
+  c->w_kv.assign(cfg->n_layers, nullptr);
+  const adore_config_t& f = c->cfg;
+  const size_t B = f.batch, C = f.capacity, MT = f.max_tokens, h = f.ctrl_hidden, d = f.hidden, G = 3 * h;
+  const size_t kv_bytes = size_t(f.n_layers) * B * f.n_heads * C * f.head_dim * c->esz;
+  const size_t rmax1 = f.rebuild_max > 0 ? f.rebuild_max : 1;
+#define TRY(x) do { st = (x); if (st != ADORE_OK) { adore_cache_destroy(c); return st; } } while (0)
+  TRY(dev_alloc(c, &c->Kc, kv_bytes, true));
+  TRY(dev_alloc(c, &c->Vc, kv_bytes, true));
+  TRY(dev_alloc(c, &c->x_store, B * MT * d * c->esz, false));
+  TRY(dev_alloc(c, &c->z, B * h * sizeof(double), true));
+  TRY(dev_alloc(c, &c->score, B * MT * sizeof(float), true));
+  TRY(dev_alloc(c, &c->sigma, B * MT * sizeof(float), true));
+  TRY(dev_alloc(c, &c->tok_slot, B * MT * sizeof(int), false));
+  for (int i = 0; i < 2; ++i) {
+    TRY(dev_alloc(c, &c->slot_tok[i], B * C * sizeof(int), false));
+    TRY(dev_alloc(c, &c->slot_role[i], B * C, true));
+    TRY(fill_i32(c, c->slot_tok[i], -1, B * C));
+  }
+  TRY(fill_i32(c, c->tok_slot, -1, B * MT));
+  TRY(dev_alloc(c, &c->admit_slot, B * sizeof(int), true));
+  TRY(dev_alloc(c, &c->evicted_tok, B * sizeof(int), true));
+  TRY(dev_alloc(c, &c->rebuild_tok, B * rmax1 * sizeof(int), true));
+  TRY(dev_alloc(c, &c->rebuild_slot, B * rmax1 * sizeof(int), true));
+  TRY(dev_alloc(c, &c->rebuild_count, B * sizeof(int), true));
+  TRY(dev_alloc(c, &c->row_off, (B + 1) * sizeof(int), true));
+  TRY(dev_alloc(c, &c->row_b, B * rmax1 * sizeof(int), true));
+  TRY(dev_alloc(c, &c->row_tok, B * rmax1 * sizeof(int), true));
+  TRY(dev_alloc(c, &c->row_slot, B * rmax1 * sizeof(int), true));
+  TRY(dev_alloc(c, &c->row_total, sizeof(int), true));
+  TRY(dev_alloc(c, &c->frow_b, B * C * sizeof(int), true));
+  TRY(dev_alloc(c, &c->frow_tok, B * C * sizeof(int), true));
+  TRY(dev_alloc(c, &c->frow_slot, B * C * sizeof(int), true));
+  TRY(dev_alloc(c, &c->frow_total, sizeof(int), true));
+  TRY(dev_alloc(c, &c->done_counter, sizeof(unsigned), true));
+  TRY(dev_alloc(c, &c->err, sizeof(unsigned), true));
+  // decode splits the d-long dot products so that roughly one wave of CTAs is busy
+  {
+    const int tiles = int((G + kGateTile - 1) / kGateTile) * int((B + kGateTile - 1) / kGateTile);
+    int ks = 1;
+    while (ks < 16 && tiles * ks * 2 <= 296 && int(d) / (ks * 2) >= kGateKChunk) ks *= 2;
+    c->ksplit = ks;
+    const size_t rows_prefill = std::min<size_t>(B * MT, std::max<size_t>(kMaxPrefillRows, B));
+    c->part_doubles = std::max<size_t>(size_t(ks) * B, rows_prefill) * G;
+    TRY(dev_alloc(c, &c->part, c->part_doubles * sizeof(double), false));
+  }
+  // controller parameters (two matrices transposed so that threads read them coalesced)
+  {
+    std::vector<float> t(G * h);
+    for (size_t g = 0; g < G; ++g) for (size_t j = 0; j < h; ++j) t[j * G + g] = w->gru_w_hh[g * h + j];
+    TRY(upload(c, &c->w_hh_t, t.data(), G * h));
+    std::vector<float> t1(h * h);
+    for (size_t i = 0; i < h; ++i) for (size_t j = 0; j < h; ++j) t1[j * h + i] = w->mlp_w1[i * h + j];
+    TRY(upload(c, &c->w1_t, t1.data(), h * h));
+  }
+  TRY(upload(c, &c->w_ih, w->gru_w_ih, G * d));
+  TRY(upload(c, &c->b_ih, w->gru_b_ih, G));
+  TRY(upload(c, &c->b_hh, w->gru_b_hh, G));
+  TRY(upload(c, &c->pos_w, w->pos_w, h));
+  TRY(upload(c, &c->pos_b, w->pos_b, h));
+  TRY(upload(c, &c->b1, w->mlp_b1, h));
+  TRY(upload(c, &c->w2, w->mlp_w2, h));
+  TRY(upload(c, &c->b2, w->mlp_b2, 1));
+  if (f.rope_theta != 0.f) {   // rotation angle of pair j at position p: p * theta^(-2j/dh)
+    const size_t half = f.head_dim / 2;
+    std::vector<float> cs(MT * half), sn(MT * half);
+    for (size_t j = 0; j < half; ++j) {
+      const double inv = std::pow(double(f.rope_theta), -2.0 * double(j) / double(f.head_dim));
+      for (size_t pos = 0; pos < MT; ++pos) {
+        cs[pos * half + j] = float(std::cos(double(pos) * inv));
+        sn[pos * half + j] = float(std::sin(double(pos) * inv));
+      }
+    }
+    TRY(upload(c, &c->rope_cos, cs.data(), MT * half));
+    TRY(upload(c, &c->rope_sin, sn.data(), MT * half));
+  }
+  // opt in to large dynamic shared memory where a kernel may need it
+  {
+    const int big = 200 * 1024;
+    cudaFuncSetAttribute(ctrl_select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    cudaFuncSetAttribute(ctrl_select_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    cudaFuncSetAttribute(bulk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    if (cudaGetLastError() != cudaSuccess) { adore_cache_destroy(c); return ADORE_ERR_CUDA; }
+  }
+  if (f.dtype == ADORE_BF16) {
+    st = tc_init(c->tc, f, c->owned, c->stream);
+    if (st != ADORE_OK) { adore_cache_destroy(c); return st; }
+  }
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) { adore_cache_destroy(c); return ADORE_ERR_CUDA; }
+#undef TRY
+  *out = c;
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_destroy(adore_cache_t* c) {
+  if (!c) return ADORE_OK;
+  cudaStreamSynchronize(c->stream);
+  for (void* p : c->owned) cudaFree(p);
+  void* hosts[] = {c->h_q, c->h_k, c->h_v, c->h_x, c->h_out, c->h_list, c->h_count, c->h_weights};
+  for (void* p : hosts) if (p) cudaFree(p);
+  cudaGetLastError();
+  delete c;
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_set_projection(adore_cache_t* c, int32_t layer, const void* w_kv) {
+  if (!c || !w_kv || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(w_kv) % 16 != 0) return ADORE_ERR_INVALID_ARG;
+  c->w_kv[layer] = w_kv;
+  if (c->cfg.dtype == ADORE_BF16) return tc_set_weights(c->tc, layer, w_kv);
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_append_tokens(adore_cache_t* c, const void* x, int32_t T) {
+  if (!c || !x || T < 1) return ADORE_ERR_INVALID_ARG;
+  if (c->n != 0) return ADORE_ERR_STATE;
+  const adore_config_t& f = c->cfg;
+  if (T > f.max_tokens) return ADORE_ERR_TOKEN_TABLE_FULL;
+  const size_t row = size_t(f.hidden) * c->esz;
+  CUDA_OK(cudaMemcpy2DAsync(c->x_store, size_t(f.max_tokens) * row, x, size_t(T) * row, size_t(T) * row, f.batch,
+                            cudaMemcpyDeviceToDevice, c->stream));
+  int chunk = int(c->part_doubles / (size_t(3) * f.ctrl_hidden) / f.batch);
+  if (chunk < 1) chunk = 1;
+  for (int t0 = 0; t0 < T; t0 += chunk) {
+    const int tc = std::min(chunk, T - t0);
+    adore_status_t st;
+    if (f.dtype == ADORE_F32)
+      st = launch_gates<float>(c, static_cast<const float*>(c->x_store) + size_t(t0) * f.hidden, f.max_tokens, tc, 1);
+    else
+      st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(c->x_store) + size_t(t0) * f.hidden,
+                                       f.max_tokens, tc, 1);
+    if (st != ADORE_OK) return st;
+    RecurParams rp = recur_params(c, f.batch * tc, tc, 1, t0);
+    ctrl_recur_kernel<<<f.batch, select_threads(c), recur_smem_bytes(f.ctrl_hidden), c->stream>>>(rp);
+    ++c->launches;
+    CUDA_OK(cudaGetLastError());
+  }
+  const int P = pow2_at_least(T);
+  SelectParams sp = select_params(c, T, P, c->cur, c->cur);
+  bulk_select_kernel<<<f.batch, select_threads(c), select_smem_bytes(f.capacity, P), c->stream>>>(sp);
+  ++c->launches;
+  CUDA_OK(cudaGetLastError());
+  c->n = T;
+  c->attn = c->cur;
+  for (int l = 0; l < f.n_layers; ++l)
+    if (c->w_kv[l]) {
+      adore_status_t st = fill_layer_impl(c, l, nullptr);
+      if (st != ADORE_OK) return st;
+    }
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_fill_layer(adore_cache_t* c, int32_t layer, const void* x_table) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (!c->w_kv[layer]) return ADORE_ERR_STATE;
+  return fill_layer_impl(c, layer, x_table);
+}
+
+adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q, const void* k_new, const void* v_new,
+                                 const void* x_new, const int32_t* explicit_list, const int32_t* explicit_count,
+                                 int32_t r_in, void* out, float* weights) {
+  if (!c || !q || !k_new || !v_new || !out || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  const adore_config_t& f = c->cfg;
+  if (layer == 0) {
+    if (!x_new) return ADORE_ERR_INVALID_ARG;
+    if (c->n >= f.max_tokens) return ADORE_ERR_TOKEN_TABLE_FULL;
+    const bool ex = f.rebuild_mode == ADORE_REBUILD_EXPLICIT;
+    if (r_in < 0 || (ex && r_in > 0 && (!explicit_list || !explicit_count))) return ADORE_ERR_INVALID_ARG;
+    if (ex && r_in > 8192) return ADORE_ERR_UNSUPPORTED;
+    // controller + selection for the step; the attention below still reads the previous map
+    adore_status_t st;
+    if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit);
+    else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit);
+    if (st != ADORE_OK) return st;
+    const int P = ex ? pow2_at_least(r_in) : pow2_at_least(c->n);
+    RecurParams rp = recur_params(c, f.batch, 1, c->ksplit, c->n);
+    SelectParams sp = select_params(c, c->n, P, c->cur, 1 - c->cur);
+    sp.explicit_list = ex && r_in > 0 ? explicit_list : nullptr;
+    sp.explicit_count = ex && r_in > 0 ? explicit_count : nullptr;
+    sp.r_in = r_in;
+    const size_t smem = std::max(select_smem_bytes(f.capacity, P), recur_smem_bytes(f.ctrl_hidden));
+    if (f.dtype == ADORE_F32)
+      ctrl_select_kernel<float><<<f.batch, select_threads(c), smem, c->stream>>>(
+          rp, sp, static_cast<const float*>(x_new), static_cast<float*>(c->x_store), f.hidden);
+    else
+      ctrl_select_kernel<__nv_bfloat16><<<f.batch, select_threads(c), smem, c->stream>>>(
+          rp, sp, static_cast<const __nv_bfloat16*>(x_new), static_cast<__nv_bfloat16*>(c->x_store), f.hidden);
+    ++c->launches;
+    CUDA_OK(cudaGetLastError());
+    c->attn = c->cur;
+    c->cur = 1 - c->cur;
+    c->n += 1;
+    c->step_layer0_done = 1;
+  } else if (!c->step_layer0_done) {
+    return ADORE_ERR_STATE;
+  }
+  if (f.dtype == ADORE_F32) return launch_attention<float>(c, layer, q, k_new, v_new, out, weights);
+  return launch_attention<__nv_bfloat16>(c, layer, q, k_new, v_new, out, weights);
+}
+
+adore_status_t adore_decode_step_host(adore_cache_t* c, int32_t layer, const void* q, const void* k_new,
+                                      const void* v_new, const void* x_new, const int32_t* explicit_list,
+                                      const int32_t* explicit_count, int32_t r_in, void* out, float* weights) {
+  if (!c || !q || !k_new || !v_new || !out) return ADORE_ERR_INVALID_ARG;
+  const adore_config_t& f = c->cfg;
+  const size_t qb = size_t(f.batch) * f.n_heads * f.head_dim * c->esz, xb = size_t(f.batch) * f.hidden * c->esz;
+  const size_t wb = size_t(f.batch) * f.n_heads * (f.capacity + 1) * sizeof(float);
+  if (!c->h_q) {
+    CUDA_OK(cudaMalloc(&c->h_q, qb)); CUDA_OK(cudaMalloc(&c->h_k, qb)); CUDA_OK(cudaMalloc(&c->h_v, qb));
+    CUDA_OK(cudaMalloc(&c->h_out, qb)); CUDA_OK(cudaMalloc(&c->h_x, xb));
+    CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->h_list), size_t(f.batch) * f.max_tokens * sizeof(int)));
+    CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->h_count), size_t(f.batch) * sizeof(int)));
+  }
+  if (weights && !c->h_weights) CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->h_weights), wb));
+  if (r_in < 0 || r_in > f.max_tokens) return ADORE_ERR_INVALID_ARG;
+  CUDA_OK(cudaMemcpyAsync(c->h_q, q, qb, cudaMemcpyHostToDevice, c->stream));
+  CUDA_OK(cudaMemcpyAsync(c->h_k, k_new, qb, cudaMemcpyHostToDevice, c->stream));
+  CUDA_OK(cudaMemcpyAsync(c->h_v, v_new, qb, cudaMemcpyHostToDevice, c->stream));
+  const bool lists = layer == 0 && explicit_list && explicit_count && r_in > 0;
+  if (layer == 0) {
+    if (!x_new) return ADORE_ERR_INVALID_ARG;
+    CUDA_OK(cudaMemcpyAsync(c->h_x, x_new, xb, cudaMemcpyHostToDevice, c->stream));
+    if (lists) {
+      CUDA_OK(cudaMemcpyAsync(c->h_list, explicit_list, size_t(f.batch) * r_in * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+      CUDA_OK(cudaMemcpyAsync(c->h_count, explicit_count, size_t(f.batch) * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+    }
+  }
+  adore_status_t st = adore_decode_step(c, layer, c->h_q, c->h_k, c->h_v, c->h_x, lists ? c->h_list : nullptr,
+                                        lists ? c->h_count : nullptr, lists ? r_in : 0, c->h_out,
+                                        weights ? c->h_weights : nullptr);
+  if (st != ADORE_OK) return st;
+  CUDA_OK(cudaMemcpyAsync(out, c->h_out, qb, cudaMemcpyDeviceToHost, c->stream));
+  if (weights) CUDA_OK(cudaMemcpyAsync(weights, c->h_weights, wb, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  return ADORE_OK;
+}
+
+adore_status_t adore_rebuild(adore_cache_t* c, int32_t layer, const void* x_table) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (!c->w_kv[layer] || !c->step_layer0_done) return ADORE_ERR_STATE;
+  const adore_config_t& f = c->cfg;
+  if (f.dtype == ADORE_F32)
+    return launch_rebuild<float>(c, layer, x_table, c->row_b, c->row_tok, c->row_slot, c->row_total, f.batch * f.rebuild_max);
+  return launch_rebuild<__nv_bfloat16>(c, layer, x_table, c->row_b, c->row_tok, c->row_slot, c->row_total,
+                                       f.batch * f.rebuild_max);
+}
+
+adore_status_t adore_cache_slot_map(adore_cache_t* c, const int32_t** slot_tok, const uint8_t** slot_role) {
+  if (!c) return ADORE_ERR_INVALID_ARG;
+  if (slot_tok) *slot_tok = c->slot_tok[c->cur];
+  if (slot_role) *slot_role = c->slot_role[c->cur];
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_rebuild_list(adore_cache_t* c, const int32_t** tok, const int32_t** slot, const int32_t** count) {
+  if (!c) return ADORE_ERR_INVALID_ARG;
+  if (tok) *tok = c->rebuild_tok;
+  if (slot) *slot = c->rebuild_slot;
+  if (count) *count = c->rebuild_count;
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_step_info(adore_cache_t* c, const int32_t** admit_slot, const int32_t** evicted_tok) {
+  if (!c) return ADORE_ERR_INVALID_ARG;
+  if (admit_slot) *admit_slot = c->admit_slot;
+  if (evicted_tok) *evicted_tok = c->evicted_tok;
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_scores(adore_cache_t* c, const float** score, const float** sigma) {
+  if (!c) return ADORE_ERR_INVALID_ARG;
+  if (score) *score = c->score;
+  if (sigma) *sigma = c->sigma;
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_kv(adore_cache_t* c, int32_t layer, const void** k, const void** v) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  const size_t off = size_t(layer) * c->cfg.batch * c->cfg.n_heads * c->cfg.capacity * c->cfg.head_dim * c->esz;
+  if (k) *k = static_cast<const unsigned char*>(c->Kc) + off;
+  if (v) *v = static_cast<const unsigned char*>(c->Vc) + off;
+  return ADORE_OK;
+}
+
+int32_t adore_cache_num_tokens(const adore_cache_t* c) { return c ? c->n : -1; }
+
+int64_t adore_cache_launch_count(const adore_cache_t* c) { return c ? c->launches : -1; }
+
+adore_status_t adore_cache_sync_status(adore_cache_t* c) {
+  if (!c) return ADORE_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
+  unsigned word = 0;
+  if (cudaMemcpy(&word, c->err, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return ADORE_ERR_CUDA;
+  if (word != 0) {
+    if (cudaMemset(c->err, 0, sizeof(word)) != cudaSuccess) return ADORE_ERR_CUDA;
+    return (word & ERRW_TIMEOUT) ? ADORE_ERR_TIMEOUT : ADORE_ERR_DEVICE_FLAG;
+  }
+  return ADORE_OK;
+}
+
+}  // extern "C"

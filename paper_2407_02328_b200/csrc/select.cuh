@@ -1,0 +1,324 @@
+// Release / admit / rebuild-list selection and the slot map (one CTA per sequence).
+//
+// Section 2.2: when the cache is full the retained token with the lowest controller score is
+// released and the newest token is appended; one decision per token serves all layers and heads.
+// Section 2.3: among released tokens, the R with the highest score are rebuilt for the next step.
+// Tokens are compared by (score, position): higher score first, the newer token on equal scores.
+// The order is materialised as one 64-bit key per token and sorted in shared memory.
+#pragma once
+
+#include <limits.h>
+
+#include "common.cuh"
+
+namespace adore {
+
+// ---- block-wide helpers (any blockDim.x that is a multiple of 32, scratch of 64 words) --------
+__device__ __forceinline__ int block_sum_i(int v, int* tmp) {
+  v = warp_sum(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) tmp[threadIdx.x >> 5] = v;
+  __syncthreads();
+  int r = 0;
+  for (int w = 0; w < int(blockDim.x >> 5); ++w) r += tmp[w];
+  return r;
+}
+__device__ __forceinline__ int block_min_i(int v, int* tmp) {
+  v = warp_min(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) tmp[threadIdx.x >> 5] = v;
+  __syncthreads();
+  int r = INT_MAX;
+  for (int w = 0; w < int(blockDim.x >> 5); ++w) r = min(r, tmp[w]);
+  return r;
+}
+__device__ __forceinline__ unsigned long long block_min_u64(unsigned long long v, unsigned long long* tmp) {
+  v = warp_min(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) tmp[threadIdx.x >> 5] = v;
+  __syncthreads();
+  unsigned long long r = ~0ull;
+  for (int w = 0; w < int(blockDim.x >> 5); ++w) r = tmp[w] < r ? tmp[w] : r;
+  return r;
+}
+// Exclusive position of this thread's flag among the block's flags (thread order); total out.
+__device__ __forceinline__ int block_rank(bool flag, int* tmp, int* total) {
+  const unsigned bal = __ballot_sync(0xffffffffu, flag);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __syncthreads();
+  if (lane == 0) tmp[warp] = __popc(bal);
+  __syncthreads();
+  int base = 0, tot = 0;
+  for (int w = 0; w < int(blockDim.x >> 5); ++w) { const int c = tmp[w]; if (w < warp) base += c; tot += c; }
+  *total = tot;
+  return base + __popc(bal & ((1u << lane) - 1u));
+}
+
+// Sorts keys[0..P) in DESCENDING order; P is a power of two. All threads of the block call it.
+__device__ inline void bitonic_sort_desc(unsigned long long* keys, int P) {
+  for (int k = 2; k <= P; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      __syncthreads();
+      for (int t = threadIdx.x; t < (P >> 1); t += blockDim.x) {
+        const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // lower index of the pair
+        const int l = i | j;
+        const unsigned long long a = keys[i], c = keys[l];
+        const bool desc = (i & k) == 0;
+        if (desc ? (a < c) : (a > c)) { keys[i] = c; keys[l] = a; }
+      }
+    }
+  }
+  __syncthreads();
+}
+
+struct SelectParams {
+  int B, C, m, r_max, n;      // n: position of the token being admitted
+  int max_tokens;
+  int explicit_mode;
+  int P;                      // sort width: power of two >= number of candidate entries
+  const int* slot_tok_old;    // [B,C]
+  const uint8_t* slot_role_old;
+  int* slot_tok_new;
+  uint8_t* slot_role_new;
+  int* tok_slot;              // [B,max_tokens]
+  const float* score;         // [B,max_tokens]
+  const int* explicit_list;   // [B,r_in]
+  const int* explicit_count;  // [B]
+  int r_in;
+  int* admit_slot;            // [B]
+  int* evicted_tok;           // [B]
+  int* rebuild_tok;           // [B,r_max]
+  int* rebuild_slot;          // [B,r_max]
+  int* rebuild_count;         // [B]
+  // compact row table over the batch, built by the last CTA to finish
+  int* row_off;               // [B+1]
+  int* row_b;                 // [B*r_max]
+  int* row_tok;
+  int* row_slot;
+  int* row_total;             // [1]
+  unsigned* done_counter;     // [1], returns to 0
+  unsigned* err;
+};
+
+__host__ __device__ inline size_t select_smem_bytes(int C, int P) {
+  // keys[P] u64 | tok[C] | lst[C] | slots[C] int | role[C] u8 (padded) | 64 words scratch | 32 u64
+  return sizeof(unsigned long long) * size_t(P) + sizeof(int) * 3 * size_t(C) + ((size_t(C) + 15) & ~size_t(15)) +
+         sizeof(int) * 64 + sizeof(unsigned long long) * 32;
+}
+
+struct SelectSmem {
+  unsigned long long* keys;
+  int* tok;
+  int* lst;
+  int* slots;
+  uint8_t* role;
+  int* tmp;
+  unsigned long long* tmp64;
+  __device__ SelectSmem(unsigned char* base, int C, int P) {
+    tmp64 = reinterpret_cast<unsigned long long*>(base);
+    keys = tmp64 + 32;
+    tok = reinterpret_cast<int*>(keys + P);
+    lst = tok + C;
+    slots = lst + C;
+    tmp = slots + C;
+    role = reinterpret_cast<uint8_t*>(tmp + 64);
+  }
+};
+
+// Candidate keys -> sorted -> first r_max distinct tokens -> ascending empty slots.
+// Expects sm.tok / sm.role to hold the map with the new token already placed. Returns the count.
+__device__ inline int assign_rebuild_list(const SelectParams& p, const SelectSmem& sm, int b, int* tok_slot,
+                                          int n_seen) {
+  const int tid = threadIdx.x, NT = blockDim.x;
+  const float* score = p.score + size_t(b) * p.max_tokens;
+  if (p.explicit_mode) {
+    const int cnt = p.explicit_list ? min(p.explicit_count[b], p.r_in) : 0;
+    for (int i = tid; i < p.P; i += NT) {
+      unsigned long long key = 0ull;
+      if (i < cnt) {
+        const int e = p.explicit_list[size_t(b) * p.r_in + i];
+        if (e < 0 || e >= n_seen) set_error(p.err, ERRW_BAD_LIST);
+        else if (tok_slot[e] < 0) key = value_key(score[e], e);
+      }
+      sm.keys[i] = key;
+    }
+  } else {
+    for (int i = tid; i < p.P; i += NT)
+      sm.keys[i] = (i < n_seen && tok_slot[i] < 0) ? value_key(score[i], i) : 0ull;
+  }
+  bitonic_sort_desc(sm.keys, p.P);
+  int found = 0;
+  for (int i0 = 0; i0 < p.P && found < p.r_max; i0 += NT) {
+    if (sm.keys[i0] == 0ull) break;                       // sorted: nothing but padding follows
+    const int i = i0 + tid;
+    const bool f = i < p.P && sm.keys[i] != 0ull && (i == 0 || sm.keys[i] != sm.keys[i - 1]);
+    int tot;
+    const int pos = found + block_rank(f, sm.tmp, &tot);
+    if (f && pos < p.r_max) sm.lst[pos] = int(sm.keys[i] & 0xffffffffull);
+    found += tot;
+  }
+  const int cnt = min(found, p.r_max);
+  int seen = 0;
+  for (int s0 = 0; s0 < p.C && seen < cnt; s0 += NT) {
+    const int s = s0 + tid;
+    const bool f = s < p.C && sm.role[s] == ROLE_EMPTY;
+    int tot;
+    const int pos = seen + block_rank(f, sm.tmp, &tot);
+    if (f && pos < cnt) sm.slots[pos] = s;
+    seen += tot;
+  }
+  __syncthreads();
+  for (int j = tid; j < p.r_max; j += NT) {
+    int tok = -1, s = -1;
+    if (j < cnt) {
+      tok = sm.lst[j];
+      s = sm.slots[j];
+      sm.tok[s] = tok;
+      sm.role[s] = ROLE_REBUILT;
+      tok_slot[tok] = s;
+    }
+    p.rebuild_tok[size_t(b) * p.r_max + j] = tok;
+    p.rebuild_slot[size_t(b) * p.r_max + j] = s;
+  }
+  if (tid == 0) p.rebuild_count[b] = cnt;
+  __syncthreads();
+  return cnt;
+}
+
+// The last CTA to arrive turns the per-sequence lists into one compact row table.
+__device__ inline void finish_row_table(const SelectParams& p, int* tmp) {
+  const int tid = threadIdx.x, NT = blockDim.x;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) tmp[0] = (atomicAdd(p.done_counter, 1u) == unsigned(p.B - 1)) ? 1 : 0;
+  __syncthreads();
+  if (!tmp[0]) return;
+  __threadfence();
+  if (tid == 0) {
+    int off = 0;
+    for (int b = 0; b < p.B; ++b) { p.row_off[b] = off; off += __ldcg(p.rebuild_count + b); }
+    p.row_off[p.B] = off;
+    *p.row_total = off;
+    *p.done_counter = 0u;
+  }
+  __syncthreads();
+  for (int i = tid; i < p.B * p.r_max; i += NT) {
+    const int b = i / p.r_max, j = i % p.r_max;
+    if (j < __ldcg(p.rebuild_count + b)) {
+      const int r = p.row_off[b] + j;
+      p.row_b[r] = b;
+      p.row_tok[r] = __ldcg(p.rebuild_tok + i);
+      p.row_slot[r] = __ldcg(p.rebuild_slot + i);
+    }
+  }
+}
+
+// One decode step's selection for sequence blockIdx.x.
+__device__ inline void select_step(const SelectParams& p, unsigned char* smem) {
+  const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x, C = p.C;
+  SelectSmem sm(smem, C, p.P);
+  int* tok_slot = p.tok_slot + size_t(b) * p.max_tokens;
+  const float* score = p.score + size_t(b) * p.max_tokens;
+  // 1. rebuilt states live for one step: free them
+  for (int s = tid; s < C; s += NT) {
+    int t = p.slot_tok_old[size_t(b) * C + s];
+    uint8_t r = p.slot_role_old[size_t(b) * C + s];
+    if (r == ROLE_REBUILT) { tok_slot[t] = -1; t = -1; r = ROLE_EMPTY; }
+    sm.tok[s] = t;
+    sm.role[s] = r;
+  }
+  __syncthreads();
+  // 2. full => release the least valuable retained token
+  int cnt = 0;
+  unsigned long long kmin = ~0ull;
+  for (int s = tid; s < C; s += NT)
+    if (sm.role[s] == ROLE_RETAINED) {
+      ++cnt;
+      const unsigned long long k = value_key(score[sm.tok[s]], sm.tok[s]);
+      kmin = k < kmin ? k : kmin;
+    }
+  const int n_ret = block_sum_i(cnt, sm.tmp);
+  kmin = block_min_u64(kmin, sm.tmp64);
+  const int evicted = (n_ret >= p.m) ? int(kmin & 0xffffffffull) : -1;
+  if (evicted >= 0)
+    for (int s = tid; s < C; s += NT)
+      if (sm.tok[s] == evicted) { sm.tok[s] = -1; sm.role[s] = ROLE_EMPTY; tok_slot[evicted] = -1; }
+  __syncthreads();
+  // 3. the new token takes the lowest-index empty slot
+  int amin = INT_MAX;
+  for (int s = tid; s < C; s += NT) if (sm.role[s] == ROLE_EMPTY) amin = min(amin, s);
+  amin = block_min_i(amin, sm.tmp);
+  if (tid == 0) {
+    if (amin < C) { sm.tok[amin] = p.n; sm.role[amin] = ROLE_RETAINED; tok_slot[p.n] = amin; }
+    else set_error(p.err, ERRW_BOUNDS);
+    p.admit_slot[b] = amin < C ? amin : -1;
+    p.evicted_tok[b] = evicted;
+  }
+  __syncthreads();
+  // 4./5. rebuild list among the released tokens, into the empty slots
+  assign_rebuild_list(p, sm, b, tok_slot, p.n);
+  for (int s = tid; s < C; s += NT) {
+    p.slot_tok_new[size_t(b) * C + s] = sm.tok[s];
+    p.slot_role_new[size_t(b) * C + s] = sm.role[s];
+  }
+  finish_row_table(p, sm.tmp);
+}
+
+// Bulk load of T tokens into an empty cache: the newest token plus the min(m-1, T-1) most
+// valuable earlier ones are retained, in ascending position from slot 0; then the rebuild list.
+// p.n = T (tokens seen), p.P >= T.
+__device__ inline void select_bulk(const SelectParams& p, unsigned char* smem) {
+  const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x, C = p.C, T = p.n;
+  SelectSmem sm(smem, C, p.P);
+  int* tok_slot = p.tok_slot + size_t(b) * p.max_tokens;
+  const float* score = p.score + size_t(b) * p.max_tokens;
+  for (int s = tid; s < C; s += NT) { sm.tok[s] = -1; sm.role[s] = ROLE_EMPTY; }
+  for (int i = tid; i < p.P; i += NT) sm.keys[i] = (i < T - 1) ? value_key(score[i], i) : 0ull;
+  for (int i = tid; i < T; i += NT) tok_slot[i] = -1;
+  bitonic_sort_desc(sm.keys, p.P);
+  const int n_keep = min(p.m - 1, T - 1);
+  for (int i = tid; i < n_keep; i += NT) tok_slot[int(sm.keys[i] & 0xffffffffull)] = -2;   // mark
+  if (tid == 0) tok_slot[T - 1] = -2;
+  __syncthreads();
+  int placed = 0;
+  for (int t0 = 0; t0 < T; t0 += NT) {
+    const int t = t0 + tid;
+    const bool f = t < T && tok_slot[t] == -2;
+    int tot;
+    const int pos = placed + block_rank(f, sm.tmp, &tot);
+    if (f) { sm.tok[pos] = t; sm.role[pos] = ROLE_RETAINED; tok_slot[t] = pos; }
+    placed += tot;
+  }
+  if (tid == 0) { p.admit_slot[b] = -1; p.evicted_tok[b] = -1; }
+  __syncthreads();
+  if (p.explicit_mode) {     // no candidates are named for a prompt
+    for (int j = tid; j < p.r_max; j += NT) { p.rebuild_tok[size_t(b) * p.r_max + j] = -1; p.rebuild_slot[size_t(b) * p.r_max + j] = -1; }
+    if (tid == 0) p.rebuild_count[b] = 0;
+    __syncthreads();
+  } else {
+    assign_rebuild_list(p, sm, b, tok_slot, T);
+  }
+  for (int s = tid; s < C; s += NT) {
+    p.slot_tok_new[size_t(b) * C + s] = sm.tok[s];
+    p.slot_role_new[size_t(b) * C + s] = sm.role[s];
+  }
+  finish_row_table(p, sm.tmp);
+}
+
+// Row table of every occupied slot (for filling a layer): one CTA.
+__global__ void resident_rows_kernel(const int* slot_tok, int B, int C, int* row_b, int* row_tok, int* row_slot,
+                                     int* row_total) {
+  __shared__ int tmp[64];
+  int base = 0;
+  for (int i0 = 0; i0 < B * C; i0 += blockDim.x) {
+    const int i = i0 + threadIdx.x;
+    const bool f = i < B * C && slot_tok[i] >= 0;
+    int tot;
+    const int pos = base + block_rank(f, tmp, &tot);
+    if (f) { row_b[pos] = i / C; row_tok[pos] = slot_tok[i]; row_slot[pos] = i % C; }
+    base += tot;
+  }
+  if (threadIdx.x == 0) *row_total = base;
+}
+
+}  // namespace adore

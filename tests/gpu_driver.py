@@ -1,0 +1,251 @@
+"""Runs the CUDA library and the oracle side by side on one workload and compares them.
+
+Bit-exact: slot maps, roles, admitted slot, evicted token, rebuild lists. Floating point:
+attention output and weights within the dtype's tolerance, cache rows within one unit in the
+last place of the cache type. Attention top-K sets must be equal except where the oracle's own
+logits of the swapped entries differ by less than 1e-6 of the row's largest |logit| (the GPU
+ranks float32 logits, the oracle float64 ones); such near-ties are counted and reported.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+import workloads as wl
+from oracle import adore_oracle as ao
+from paper_2407_02328_b200 import adore as lib
+from tests.harness import Workload, make_oracle, explicit_as_lists
+
+TOL = {"bf16": dict(out_abs=2e-2, out_rel=1e-2, w_abs=1e-3), "f32": dict(out_abs=1e-4, out_rel=1e-4, w_abs=1e-5)}
+NEAR_TIE_REL = 1e-6
+
+
+def torch_dtype(cfg: wl.WorkloadConfig):
+    return torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+
+
+def to_dev(a: np.ndarray, cfg: wl.WorkloadConfig) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a)).to("cuda").to(torch_dtype(cfg)).contiguous()
+
+
+@dataclass
+class Report:
+    steps: int = 0
+    near_ties: int = 0
+    topk_rows: int = 0
+    max_out_err: float = 0.0
+    max_w_err: float = 0.0
+    max_kv_ulp: float = 0.0
+    score_mismatch: int = 0
+    notes: List[str] = field(default_factory=list)
+
+
+class GpuCache:
+    """The library's cache for a workload, with torch-owned device buffers for the per-step I/O."""
+
+    def __init__(self, w: Workload):
+        c = self.cfg = w.cfg
+        self.w = w
+        self.B = w.batch
+        self.handle = lib.adore_cache_create(
+            lib.make_config(batch=self.B, n_layers=c.n_layers, n_heads=c.n_heads, head_dim=c.head_dim,
+                            hidden=c.hidden, capacity=c.capacity, rebuild_max=c.rebuild_max, topk=c.topk,
+                            max_tokens=c.max_tokens, ctrl_hidden=c.ctrl_hidden, dtype=c.dtype,
+                            rebuild_mode=c.rebuild_mode, rope_theta=c.rope_theta, pos_scale=c.pos_scale),
+            w.ctrl, torch.cuda.current_stream().cuda_stream)
+        self.w_kv_dev = [to_dev(m, c) for m in w.w_kv]
+        for l, m in enumerate(self.w_kv_dev):
+            lib.adore_cache_set_projection(self.handle, l, m)
+        self.out = torch.empty((self.B, c.n_heads, c.head_dim), dtype=torch_dtype(c), device="cuda")
+        self.weights = torch.empty((self.B, c.n_heads, c.capacity + 1), dtype=torch.float32, device="cuda")
+
+    def close(self):
+        if self.handle:
+            lib.adore_cache_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
+
+    # ---- views ----
+    def slot_map(self):
+        st, sr = lib.adore_cache_slot_map(self.handle)
+        c = self.cfg
+        return (lib.device_view(st, (self.B, c.capacity), torch.int32).cpu().numpy(),
+                lib.device_view(sr, (self.B, c.capacity), torch.uint8).cpu().numpy())
+
+    def step_info(self):
+        a, e = lib.adore_cache_step_info(self.handle)
+        return (lib.device_view(a, (self.B,), torch.int32).cpu().numpy(),
+                lib.device_view(e, (self.B,), torch.int32).cpu().numpy())
+
+    def rebuild_list(self):
+        c = self.cfg
+        if c.rebuild_max == 0:
+            z = np.zeros((self.B, 0), np.int32)
+            return z, z, np.zeros(self.B, np.int32)
+        t, s, n = lib.adore_cache_rebuild_list(self.handle)
+        return (lib.device_view(t, (self.B, c.rebuild_max), torch.int32).cpu().numpy(),
+                lib.device_view(s, (self.B, c.rebuild_max), torch.int32).cpu().numpy(),
+                lib.device_view(n, (self.B,), torch.int32).cpu().numpy())
+
+    def scores(self, n):
+        s, g = lib.adore_cache_scores(self.handle)
+        c = self.cfg
+        return (lib.device_view(s, (self.B, c.max_tokens), torch.float32)[:, :n].cpu().numpy(),
+                lib.device_view(g, (self.B, c.max_tokens), torch.float32)[:, :n].cpu().numpy())
+
+    def kv(self, layer):
+        k, v = lib.adore_cache_kv(self.handle, layer)
+        c = self.cfg
+        shape = (self.B, c.n_heads, c.capacity, c.head_dim)
+        return (lib.device_view(k, shape, torch_dtype(c)).float().cpu().numpy(),
+                lib.device_view(v, shape, torch_dtype(c)).float().cpu().numpy())
+
+
+def _ulp(ref: np.ndarray, dtype: str) -> np.ndarray:
+    """Size of one unit in the last place of the cache type at |ref| (floor at the smallest normal scale used)."""
+    mant = 8 if dtype == "bf16" else 24
+    e = np.floor(np.log2(np.maximum(np.abs(ref), 1e-30)))
+    return np.exp2(e - (mant - 1))
+
+
+def compare_attention(rep: Report, cfg, q, orc: ao.AdoreOracle, layer, k_new, attn_map, out_g, w_g, out_o, w_o,
+                      Kc_before):
+    tol = TOL[cfg.dtype]
+    err = np.abs(out_g - out_o)
+    bound = tol["out_abs"] + tol["out_rel"] * np.abs(out_o)
+    assert (err <= bound).all(), f"attention output off by {err.max():.3e} (step {rep.steps}, layer {layer})"
+    rep.max_out_err = max(rep.max_out_err, float(err.max()))
+    keep_g, keep_o = w_g > 0, w_o > 0
+    rep.topk_rows += keep_o.shape[0] * keep_o.shape[1]
+    bad = np.argwhere((keep_g != keep_o).any(-1))
+    w_ok = np.ones_like(keep_o)
+    for b, h in bad:
+        Kall = np.concatenate([Kc_before[b, h].astype(np.float64), k_new[b, h][None].astype(np.float64)])
+        logit = Kall @ q[b, h].astype(np.float64) / np.sqrt(cfg.head_dim)
+        valid = np.concatenate([attn_map[b] >= 0, [True]])
+        scale = max(1.0, float(np.abs(logit[valid]).max()))
+        diff = np.nonzero(keep_g[b, h] != keep_o[b, h])[0]
+        assert keep_g[b, h].sum() == keep_o[b, h].sum(), "kept count differs"
+        assert valid[diff].all(), "an empty slot was kept"
+        thr = logit[keep_o[b, h]].min()
+        gap = np.abs(logit[diff] - thr).max()
+        assert gap <= NEAR_TIE_REL * scale, f"top-K sets differ beyond a near-tie: gap {gap:.3e} scale {scale:.3e}"
+        rep.near_ties += 1
+        w_ok[b, h, diff] = False
+    werr = np.abs(w_g - w_o)[w_ok]
+    assert (werr <= tol["w_abs"]).all(), f"attention weights off by {werr.max():.3e}"
+    rep.max_w_err = max(rep.max_w_err, float(werr.max()))
+    s = w_g.sum(-1)
+    assert np.allclose(s, 1.0, atol=1e-4), "weights do not sum to one"
+
+
+def compare_state(rep: Report, g: GpuCache, orc: ao.AdoreOracle, layers, check_scores=True):
+    cfg = g.cfg
+    st, sr = g.slot_map()
+    assert np.array_equal(st, orc.slot_tok), f"slot map differs at step {rep.steps}"
+    assert np.array_equal(sr, orc.slot_role), f"slot roles differ at step {rep.steps}"
+    adm, ev = g.step_info()
+    assert np.array_equal(adm, orc.info.admit_slot) and np.array_equal(ev, orc.info.evicted_tok)
+    lt, ls, ln = g.rebuild_list()
+    for b in range(g.B):
+        k = len(orc.info.rebuild_tok[b])
+        assert ln[b] == k, f"rebuild count differs (b={b}): {ln[b]} vs {k}"
+        assert np.array_equal(lt[b, :k], orc.info.rebuild_tok[b]) and np.array_equal(ls[b, :k], orc.info.rebuild_slot[b])
+    if check_scores:
+        sc, sg = g.scores(orc.n)
+        mism = int((sc != orc.score[:, : orc.n]).sum())
+        rep.score_mismatch += mism
+        assert np.allclose(sc, orc.score[:, : orc.n], rtol=1e-6, atol=1e-9)
+        assert np.allclose(sg, orc.sigma[:, : orc.n], rtol=1e-6, atol=1e-9)
+    occ = orc.slot_tok >= 0
+    for l in layers:
+        Kg, Vg = g.kv(l)
+        for name, G, O in (("K", Kg, orc.Kc[l]), ("V", Vg, orc.Vc[l])):
+            m = np.broadcast_to(occ[:, None, :, None], G.shape)
+            d = np.abs(G - O)[m]
+            u = _ulp(O, cfg.dtype)[m]
+            lim = 1.0 if cfg.dtype == "bf16" else 64.0      # f32: float32 accumulation over d terms
+            # float32 accumulation of the d-long dot products leaves an absolute error that one unit
+            # in the last place cannot cover for outputs that nearly cancel to zero
+            floor = 1e-4 if cfg.dtype == "bf16" else 1e-5
+            worst = float((d / u).max()) if d.size else 0.0
+            assert (d <= lim * u + floor).all(), f"{name} cache rows off by {worst:.2f} ulp at step {rep.steps}"
+            rep.max_kv_ulp = max(rep.max_kv_ulp, worst)
+
+
+def run_parity(cfg: wl.WorkloadConfig, batch: Optional[int] = None, steps: Optional[int] = None,
+               state_every: int = 1, host_entry: bool = False) -> Report:
+    """Free-running parity: both sides consume the same inputs and must agree at every step."""
+    w = Workload(cfg, batch)
+    orc = make_oracle(w)
+    g = GpuCache(w)
+    rep = Report()
+    L = cfg.n_layers
+    tables = None
+    try:
+        if cfg.prompt:
+            xp = w.prompt()
+            orc.append_tokens(xp)
+            lib.adore_cache_append_tokens(g.handle, to_dev(xp, cfg), cfg.prompt)
+            if cfg.per_layer_inputs:
+                tables = [torch.zeros((g.B, cfg.max_tokens, cfg.hidden), dtype=torch_dtype(cfg), device="cuda")
+                          for _ in range(L)]
+                otab = [np.zeros((g.B, cfg.max_tokens, cfg.hidden), np.float32) for _ in range(L)]
+                for l in range(L):
+                    xl = xp if l == 0 else w.prompt(l)
+                    otab[l][:, : cfg.prompt] = xl
+                    tables[l][:, : cfg.prompt] = to_dev(xl, cfg)
+                    if l > 0:
+                        orc.fill_layer(l, otab[l])
+                        lib.adore_cache_fill_layer(g.handle, l, tables[l])
+            lib.adore_cache_sync_status(g.handle)
+            compare_state(rep, g, orc, range(L))
+        elif cfg.per_layer_inputs:
+            tables = [torch.zeros((g.B, cfg.max_tokens, cfg.hidden), dtype=torch_dtype(cfg), device="cuda") for _ in range(L)]
+            otab = [np.zeros((g.B, cfg.max_tokens, cfg.hidden), np.float32) for _ in range(L)]
+        n_steps = cfg.steps if steps is None else steps
+        for s in range(n_steps):
+            n = orc.n
+            lists, counts = w.explicit(s, n)
+            ex = explicit_as_lists(lists, counts)
+            dl = torch.from_numpy(lists).cuda() if lists is not None else None
+            dc = torch.from_numpy(counts).cuda() if counts is not None else None
+            for l in range(L):
+                x = w.x_new(n, l if cfg.per_layer_inputs else 0)
+                q, k, v = w.qkv(n, l, x)
+                if cfg.per_layer_inputs:
+                    otab[l][:, n] = x
+                    tables[l][:, n] = to_dev(x, cfg)
+                attn_map = orc.slot_tok.copy() if l == 0 else orc.attn_slot_tok.copy()
+                K_before = orc.Kc[l].copy()
+                out_o, w_o = orc.decode_step(l, q, k, v, x if l == 0 else None, ex if l == 0 else None)
+                if host_entry:
+                    ho = np.zeros((g.B, cfg.n_heads, cfg.head_dim), np.float32)
+                    hq, hk, hv, hx = (to_dev(a, cfg).cpu() for a in (q, k, v, x))
+                    hout = torch.zeros((g.B, cfg.n_heads, cfg.head_dim), dtype=torch_dtype(cfg))
+                    hw = torch.zeros((g.B, cfg.n_heads, cfg.capacity + 1), dtype=torch.float32)
+                    lib.adore_decode_step_host(g.handle, l, hq, hk, hv, hx, lists if l == 0 else None,
+                                               counts if l == 0 else None, w.r_in if l == 0 else 0, hout, hw)
+                    out_g, w_g = hout.float().numpy(), hw.numpy()
+                else:
+                    lib.adore_decode_step(g.handle, l, to_dev(q, cfg), to_dev(k, cfg), to_dev(v, cfg), to_dev(x, cfg),
+                                          dl if l == 0 else None, dc if l == 0 else None, w.r_in if l == 0 else 0,
+                                          g.out, g.weights)
+                    out_g, w_g = g.out.float().cpu().numpy(), g.weights.cpu().numpy()
+                compare_attention(rep, cfg, q, orc, l, k, attn_map, out_g, w_g, out_o, w_o, K_before)
+                orc.rebuild(l, otab[l] if (cfg.per_layer_inputs and l > 0) else None)
+                lib.adore_rebuild(g.handle, l, tables[l] if (cfg.per_layer_inputs and l > 0) else None)
+            rep.steps += 1
+            if (s + 1) % state_every == 0 or s == n_steps - 1:
+                lib.adore_cache_sync_status(g.handle)
+                orc.check_invariants()
+                compare_state(rep, g, orc, range(L))
+        lib.adore_cache_sync_status(g.handle)
+    finally:
+        g.close()
+    return rep

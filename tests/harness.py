@@ -33,6 +33,8 @@ class Workload:
         self.ctrl = wl.controller_weights(cfg)
         self.w_kv = [wl.projection_weights(cfg, l) for l in range(cfg.n_layers)]
         self.w_q = [wl.query_weights(cfg, l) for l in range(cfg.n_layers)]
+        self.w_kv64 = [w.astype(np.float64) for w in self.w_kv]
+        self.w_q64 = [w.astype(np.float64) for w in self.w_q]
         self.r_in = self._r_in()
 
     def _r_in(self) -> int:
@@ -49,18 +51,19 @@ class Workload:
         return wl.hidden_rows(self.cfg, n, 1, layer, self.batch)[:, 0, :]
 
     def qkv(self, n: int, layer: int, x_row: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+        """q, k_new, v_new [B, H, dh] of the token at position n (all sequences in one product)."""
         c = self.cfg
-        B = x_row.shape[0]
-        q = np.empty((B, c.n_heads, c.head_dim), np.float32)
-        k = np.empty_like(q)
-        v = np.empty_like(q)
-        for b in range(B):
-            if c.identity_projection:      # q, k, v i.i.d. N(0,1): q is its own draw
-                qb = wl.gaussian(c.seed, "q", (c.n_heads, c.head_dim), 1.0, c.dtype, idx=(layer, n, b))
-            else:
-                qb = ao.project_q(self.w_q[layer], x_row[b], n, c.n_heads, c.head_dim, c.rope_theta, c.dtype)
-            kb, vb = ao.project_kv(self.w_kv[layer], x_row[b], n, c.n_heads, c.head_dim, c.rope_theta, c.dtype)
-            q[b], k[b], v[b] = qb, kb, vb
+        B, hd = x_row.shape[0], c.n_heads * c.head_dim
+        x64 = x_row.astype(np.float64)
+        ykv = x64 @ self.w_kv64[layer].T
+        k = ao.round_store(ao.rope_rotate(ykv[:, :hd].reshape(B, c.n_heads, c.head_dim), n, c.rope_theta), c.dtype)
+        v = ao.round_store(ykv[:, hd:].reshape(B, c.n_heads, c.head_dim), c.dtype)
+        if c.identity_projection:          # q, k, v i.i.d. N(0,1): q is its own draw
+            q = np.stack([wl.gaussian(c.seed, "q", (c.n_heads, c.head_dim), 1.0, c.dtype, idx=(layer, n, b))
+                          for b in range(B)])
+        else:
+            yq = x64 @ self.w_q64[layer].T
+            q = ao.round_store(ao.rope_rotate(yq.reshape(B, c.n_heads, c.head_dim), n, c.rope_theta), c.dtype)
         return q, k, v
 
     def explicit(self, step: int, n: int) -> Tuple[Optional[np.ndarray], Optional[np.ndarray]]:
@@ -72,7 +75,7 @@ class Workload:
 def make_oracle(w: Workload) -> ao.AdoreOracle:
     orc = ao.AdoreOracle(oracle_config(w.cfg, w.batch), w.ctrl)
     for l in range(w.cfg.n_layers):
-        orc.set_projection(l, w.w_kv[l])
+        orc.set_projection(l, w.w_kv64[l])
     return orc
 
 

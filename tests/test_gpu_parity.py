@@ -1,0 +1,70 @@
+"""GPU parity: the CUDA library against the oracle, through the C ABI, on seeded workloads."""
+import numpy as np
+import pytest
+
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+SMALL = wl.WorkloadConfig(name="small_bf16", dtype="bf16", n_layers=1, batch=3, n_heads=4, head_dim=128,
+                          hidden=256, capacity=40, topk=16, rebuild_max=4, prompt=50, steps=40,
+                          rope_theta=1.0e4, rebuild_mode="policy", rebuild_p=0.0, seed=101, ctrl_hidden=128)
+
+
+def _run(cfg, **kw):
+    from tests.gpu_driver import run_parity
+    rep = run_parity(cfg, **kw)
+    print(f"\n[{cfg.name}] steps={rep.steps} near_ties={rep.near_ties}/{rep.topk_rows} rows "
+          f"max_out_err={rep.max_out_err:.3e} max_w_err={rep.max_w_err:.3e} max_kv_ulp={rep.max_kv_ulp:.2f} "
+          f"score_mismatch={rep.score_mismatch}")
+    assert rep.near_ties <= max(2, rep.topk_rows // 1000)
+    return rep
+
+
+def test_config1_fp32_full_run():
+    _run(wl.get_config(1))
+
+
+def test_small_bf16_policy_with_prompt():
+    _run(SMALL)
+
+
+def test_small_bf16_no_prompt_grows_from_empty():
+    _run(SMALL.scaled(name="small_bf16_empty", prompt=0, steps=70, seed=102))
+
+
+def test_small_bf16_explicit_large_rebuild_budget():
+    _run(SMALL.scaled(name="small_bf16_explicit", rebuild_mode="explicit", rebuild_p=0.3, rebuild_max=20,
+                      capacity=48, topk=24, prompt=0, steps=90, seed=103))
+
+
+def test_head_dim_64_bf16_and_fp32_with_rope():
+    _run(SMALL.scaled(name="dh64_bf16", head_dim=64, n_heads=3, hidden=192, seed=104))
+    _run(SMALL.scaled(name="dh128_f32", dtype="f32", n_heads=2, hidden=128, capacity=33, topk=7, seed=105))
+
+
+def test_topk_disabled_and_topk_one():
+    _run(SMALL.scaled(name="topk_off", topk=1000, seed=106))
+    _run(SMALL.scaled(name="topk_one", topk=1, seed=107))
+
+
+def test_no_rebuild_budget_is_plain_release():
+    _run(SMALL.scaled(name="r0", rebuild_max=0, seed=108))
+
+
+def test_three_layers_with_their_own_inputs():
+    _run(SMALL.scaled(name="L3", n_layers=3, batch=2, per_layer_inputs=True, seed=109, steps=20))
+
+
+def test_host_buffer_entry_point():
+    _run(SMALL.scaled(name="host_entry", steps=12, seed=110), host_entry=True)
+    _run(wl.get_config(1).scaled(steps=40), host_entry=True)
+
+
+def test_capacity_spanning_several_tiles_with_ragged_tail():
+    _run(SMALL.scaled(name="c517", capacity=517, topk=200, rebuild_max=37, prompt=700, steps=12, batch=2,
+                      n_heads=2, seed=111))
+
+
+def test_config2_sub_batch():
+    _run(wl.get_config(2), batch=2, steps=24, state_every=4)
