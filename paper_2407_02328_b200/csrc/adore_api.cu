@@ -2,6 +2,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -24,7 +25,7 @@ constexpr int kMaxPrefillRows = 8192;       // controller rows per chunk during 
 // ---- kernels that glue the device functions together -----------------------------------------
 template <typename T>
 __global__ void ctrl_select_kernel(const RecurParams rp, const SelectParams sp, const T* x_new, T* x_store, int d) {
-  extern __shared__ __align__(16) unsigned char smem[];
+  extern __shared__ __align__(128) unsigned char smem[];
   const int b = blockIdx.x;
   // keep the new token's layer-input row: it is what a later rebuild recomputes from
   {
@@ -38,12 +39,12 @@ __global__ void ctrl_select_kernel(const RecurParams rp, const SelectParams sp, 
 }
 
 __global__ void ctrl_recur_kernel(const RecurParams rp) {
-  extern __shared__ __align__(16) unsigned char smem[];
+  extern __shared__ __align__(128) unsigned char smem[];
   controller_tokens(rp, blockIdx.x, reinterpret_cast<double*>(smem));
 }
 
 __global__ void bulk_select_kernel(const SelectParams sp) {
-  extern __shared__ __align__(16) unsigned char smem[];
+  extern __shared__ __align__(128) unsigned char smem[];
   select_bulk(sp, smem);
 }
 
@@ -205,7 +206,9 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
   p.err = c->err;
   const int grid = f.batch * f.n_heads;
   cudaError_t e;
-  if (attn_tma_usable<T>(f.capacity, f.head_dim)) e = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
+  // ADORE_ATTN_DIRECT=1 selects the variant without shared-memory staging (for A/B timing)
+  static const bool direct = std::getenv("ADORE_ATTN_DIRECT") != nullptr;
+  if (!direct && attn_tma_usable<T>(f.capacity, f.head_dim)) e = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
   else if (f.head_dim == 64) {
     const size_t smem = attn_smem_bytes(f.capacity, 64);
     attention_kernel<T, 64><<<grid, kAttnThreads, smem, c->stream>>>(p);

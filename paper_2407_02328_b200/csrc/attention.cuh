@@ -66,66 +66,51 @@ __device__ __forceinline__ float block_max_f(float v, float* tmp) {
   return r;
 }
 
+// Shared-memory carve-up common to the attention kernels.
+template <int DH>
+struct AttnSmem {
+  float* logit;
+  int* list;
+  unsigned* hist;
+  float* red;
+  float* tmp;     // 64 words: reduction scratch [0,32), broadcast [32,64)
+  int* sel;
+  __device__ AttnSmem(unsigned char* base, int rows) {
+    const int cp = (rows + 3) & ~3;
+    logit = reinterpret_cast<float*>(base);
+    list = reinterpret_cast<int*>(logit + cp);
+    hist = reinterpret_cast<unsigned*>(list + cp);
+    red = reinterpret_cast<float*>(hist + 256);
+    tmp = red + (kAttnThreads / 32) * DH;
+    sel = reinterpret_cast<int*>(tmp + 32);
+  }
+};
+
+// Phases 2-4 and the admit write, given the logits of all C+1 rows in shared memory
+// (-inf for empty slots). Every thread of the block calls it after a __syncthreads().
 template <typename T, int DH>
-__global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParams<T> p) {
+__device__ __forceinline__ void attention_tail(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh) {
   constexpr int NT = kAttnThreads;
   constexpr int NW = NT / 32;
-  constexpr int EPL = Elem<T>::kPer16B;   // elements per lane (one 16-byte load)
-  constexpr int LPR = DH / EPL;           // lanes that share one row
-  constexpr int RPW = 32 / LPR;           // rows per warp-wide load
-  static_assert(LPR >= 1 && LPR <= 32 && (LPR & (LPR - 1)) == 0, "row must split over a warp");
+  constexpr int EPL = Elem<T>::kPer16B;
+  constexpr int LPR = DH / EPL;
+  constexpr int RPW = 32 / LPR;
   constexpr int U = kAttnUnroll;
-
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int C = p.C, rows = C + 1, cp = (rows + 3) & ~3;
-  float* s_logit = reinterpret_cast<float*>(smem_raw);
-  int* s_list = reinterpret_cast<int*>(s_logit + cp);
-  unsigned* s_hist = reinterpret_cast<unsigned*>(s_list + cp);
-  float* s_red = reinterpret_cast<float*>(s_hist + 256);
-  float* s_tmp = s_red + NW * DH;          // 64 words: reduction scratch [0,32), broadcast [32,64)
-  int* s_sel = reinterpret_cast<int*>(s_tmp + 32);
-
+  float* s_logit = sm.logit;
+  int* s_list = sm.list;
+  unsigned* s_hist = sm.hist;
+  float* s_red = sm.red;
+  float* s_tmp = sm.tmp;
+  int* s_sel = sm.sel;
+  const int C = p.C, rows = C + 1;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane / LPR, li = lane % LPR;
-  const int bh = blockIdx.x, b = bh / p.H;
+  const int b = bh / p.H;
   const size_t row_bytes = size_t(DH) * sizeof(T);
   const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * row_bytes;
   const unsigned char* Vb = reinterpret_cast<const unsigned char*>(p.Vc) + size_t(bh) * C * row_bytes;
   const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * row_bytes;
   const unsigned char* vnew = reinterpret_cast<const unsigned char*>(p.v_new) + size_t(bh) * row_bytes;
-  const int* map = p.slot_tok + size_t(b) * C;
-
-  // ---- phase 1: logits -------------------------------------------------------------------
-  float qf[EPL];
-  {
-    const uint4 qr = *reinterpret_cast<const uint4*>(
-        reinterpret_cast<const unsigned char*>(p.q) + size_t(bh) * row_bytes + li * 16);
-    Elem<T>::unpack(qr, qf);
-  }
-  for (int r0 = warp * RPW; r0 < rows; r0 += NW * RPW * U) {
-    uint4 kv[U];
-    bool ok[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int row = r0 + u * NW * RPW + sub;
-      ok[u] = row < rows && (row == C || map[row] >= 0);
-      kv[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (ok[u]) kv[u] = ldg_stream((row == C ? knew : Kb + size_t(row) * row_bytes) + li * 16);
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int row = r0 + u * NW * RPW + sub;
-      float kf[EPL];
-      Elem<T>::unpack(kv[u], kf);
-      float dot = 0.f;
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kf[e], dot);
-#pragma unroll
-      for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-      if (li == 0 && row < rows) s_logit[row] = ok[u] ? dot * p.scale : -INFINITY;
-    }
-  }
-  __syncthreads();
 
   // ---- phase 2: which logits are kept (K largest, lower index wins ties) -------------------
   int cnt = 0;
@@ -272,6 +257,64 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParam
       set_error(p.err, ERRW_BOUNDS);
     }
   }
+}
+
+template <typename T, int DH>
+__global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParams<T> p) {
+  constexpr int NT = kAttnThreads;
+  constexpr int NW = NT / 32;
+  constexpr int EPL = Elem<T>::kPer16B;   // elements per lane (one 16-byte load)
+  constexpr int LPR = DH / EPL;           // lanes that share one row
+  constexpr int RPW = 32 / LPR;           // rows per warp-wide load
+  static_assert(LPR >= 1 && LPR <= 32 && (LPR & (LPR - 1)) == 0, "row must split over a warp");
+  constexpr int U = kAttnUnroll;
+
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int C = p.C, rows = C + 1;
+  const AttnSmem<DH> sm(smem_raw, rows);
+  float* s_logit = sm.logit;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int sub = lane / LPR, li = lane % LPR;
+  const int bh = blockIdx.x, b = bh / p.H;
+  const size_t row_bytes = size_t(DH) * sizeof(T);
+  const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * row_bytes;
+  const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * row_bytes;
+  const int* map = p.slot_tok + size_t(b) * C;
+
+  // ---- phase 1: logits -------------------------------------------------------------------
+  float qf[EPL];
+  {
+    const uint4 qr = *reinterpret_cast<const uint4*>(
+        reinterpret_cast<const unsigned char*>(p.q) + size_t(bh) * row_bytes + li * 16);
+    Elem<T>::unpack(qr, qf);
+  }
+  for (int r0 = warp * RPW; r0 < rows; r0 += NW * RPW * U) {
+    uint4 kv[U];
+    bool ok[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int row = r0 + u * NW * RPW + sub;
+      ok[u] = row < rows && (row == C || map[row] >= 0);
+      kv[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (ok[u]) kv[u] = ldg_stream((row == C ? knew : Kb + size_t(row) * row_bytes) + li * 16);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int row = r0 + u * NW * RPW + sub;
+      float kf[EPL];
+      Elem<T>::unpack(kv[u], kf);
+      float dot = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kf[e], dot);
+#pragma unroll
+      for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      if (li == 0 && row < rows) s_logit[row] = ok[u] ? dot * p.scale : -INFINITY;
+    }
+  }
+  __syncthreads();
+
+  attention_tail<T, DH>(p, sm, bh);
 }
 
 }  // namespace adore

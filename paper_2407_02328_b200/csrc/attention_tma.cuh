@@ -1,14 +1,177 @@
-// Bulk-copy (TMA) staged variant of the decode attention; selected when the shape allows it.
+// Decode attention, phase 1 staged through shared memory by the bulk-copy engine (TMA).
+//
+// Same computation as attention_kernel (Section 2.1 target attention with the top-K mask of
+// Section 2.2); only the way the key rows reach the SM differs. The K block of one (sequence,
+// head) is a contiguous C*dh array, so one elected thread streams it in 8 KB chunks with
+// cp.async.bulk into a 4-deep ring; an mbarrier per stage counts the bytes. The warps read the
+// rows from shared memory (conflict-free 16-byte accesses). This keeps 24-32 KB in flight per
+// CTA without spending registers or issue slots on the loads, which is what the HBM roofline
+// needs with several CTAs per SM. The kept value rows are still gathered with direct loads.
+//
+// Every wait is bounded: if a stage never fills, the CTA sets the timeout bit of the error word,
+// drains what it issued with short waits and finishes with whatever it has (the step is then
+// reported as failed by adore_cache_sync_status).
 #pragma once
 
 #include "attention.cuh"
 
 namespace adore {
 
-template <typename T>
-inline bool attn_tma_usable(int /*C*/, int /*DH*/) { return false; }
+constexpr int kRingStages = 4;
+constexpr int kRingChunkBytes = 8192;
+constexpr uint32_t kWaitPolls = 1u << 22;      // upper bound on mbarrier polls
+constexpr uint32_t kDrainPolls = 1u << 10;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t max_polls) {
+  for (uint32_t i = 0; i < max_polls; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// global -> shared bulk copy; both addresses 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+__host__ __device__ inline size_t attn_tma_smem_bytes(int C, int DH) {
+  // ring first (needs 128-byte alignment at most), then barriers, then the common carve-up
+  return size_t(kRingStages) * kRingChunkBytes + 64 + attn_smem_bytes(C, DH);
+}
+
+template <typename T, int DH>
+__global__ void __launch_bounds__(kAttnThreads) attention_tma_kernel(const AttnParams<T> p) {
+  constexpr int NT = kAttnThreads;
+  constexpr int NW = NT / 32;
+  constexpr int EPL = Elem<T>::kPer16B;
+  constexpr int LPR = DH / EPL;
+  constexpr int RPW = 32 / LPR;
+  constexpr int ROW_BYTES = DH * int(sizeof(T));
+  constexpr int CHUNK_ROWS = kRingChunkBytes / ROW_BYTES;
+  static_assert(CHUNK_ROWS % (NW * RPW) == 0, "a chunk must be a whole number of block-wide passes");
+  constexpr int PASSES = CHUNK_ROWS / (NW * RPW);
+
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  unsigned char* ring = smem_raw;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + size_t(kRingStages) * kRingChunkBytes);
+  const int C = p.C, rows = C + 1;
+  const AttnSmem<DH> sm(smem_raw + size_t(kRingStages) * kRingChunkBytes + 64, rows);
+  float* s_logit = sm.logit;
+  int* s_fail = sm.sel + 24;               // one word of the broadcast area
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int sub = lane / LPR, li = lane % LPR;
+  const int bh = blockIdx.x, b = bh / p.H;
+  const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * ROW_BYTES;
+  const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * ROW_BYTES;
+  const int* map = p.slot_tok + size_t(b) * C;
+  const int n_chunks = (C + CHUNK_ROWS - 1) / CHUNK_ROWS;
+
+  if (tid == 0) {
+#pragma unroll
+    for (int s = 0; s < kRingStages; ++s) mbar_init(&full[s], 1u);
+    *s_fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  auto issue = [&](int chunk) {
+    const int stage = chunk % kRingStages;
+    const int r0 = chunk * CHUNK_ROWS;
+    const uint32_t bytes = uint32_t(min(CHUNK_ROWS, C - r0)) * ROW_BYTES;
+    mbar_expect_tx(&full[stage], bytes);
+    bulk_g2s(ring + size_t(stage) * kRingChunkBytes, Kb + size_t(r0) * ROW_BYTES, bytes, &full[stage]);
+  };
+  if (tid == 0)
+    for (int c = 0; c < min(kRingStages, n_chunks); ++c) issue(c);
+
+  float qf[EPL];
+  {
+    const uint4 qr = *reinterpret_cast<const uint4*>(
+        reinterpret_cast<const unsigned char*>(p.q) + size_t(bh) * ROW_BYTES + li * 16);
+    Elem<T>::unpack(qr, qf);
+  }
+  // the current token's own key (row index C) does not go through the ring
+  if (warp == NW - 1 && sub == 0) {
+    float kf[EPL];
+    Elem<T>::unpack(*reinterpret_cast<const uint4*>(knew + li * 16), kf);
+    float dot = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kf[e], dot);
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu >> (32 - LPR), dot, o);
+    if (li == 0) s_logit[C] = dot * p.scale;
+  }
+
+  bool failed = false;
+  for (int c = 0; c < n_chunks; ++c) {
+    const int stage = c % kRingStages;
+    const uint32_t parity = uint32_t(c / kRingStages) & 1u;
+    if (!mbar_wait_bounded(&full[stage], parity, failed ? kDrainPolls : kWaitPolls)) {
+      if (!failed) { set_error(p.err, ERRW_TIMEOUT); *s_fail = 1; }
+      failed = true;
+    }
+    const unsigned char* src = ring + size_t(stage) * kRingChunkBytes;
+    const int r0 = c * CHUNK_ROWS;
+#pragma unroll
+    for (int ps = 0; ps < PASSES; ++ps) {
+      const int lr = ps * NW * RPW + warp * RPW + sub;      // row inside the chunk
+      const int row = r0 + lr;
+      const bool ok = row < C && map[row] >= 0;
+      float kf[EPL];
+      // rows past C in a ragged last chunk hold stale bytes of an earlier chunk: read, not used
+      Elem<T>::unpack(*reinterpret_cast<const uint4*>(src + size_t(lr) * ROW_BYTES + li * 16), kf);
+      float dot = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kf[e], dot);
+#pragma unroll
+      for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      if (li == 0 && row < C) s_logit[row] = ok ? dot * p.scale : -INFINITY;
+    }
+    __syncthreads();                                         // everyone is done with this stage
+    failed = failed || (*s_fail != 0);
+    if (tid == 0 && !failed && c + kRingStages < n_chunks) issue(c + kRingStages);
+  }
+  // (the loop's last __syncthreads also publishes the logits)
+  attention_tail<T, DH>(p, sm, bh);
+}
 
 template <typename T>
-inline cudaError_t launch_attention_tma(const AttnParams<T>&, int, int, cudaStream_t) { return cudaErrorNotSupported; }
+inline bool attn_tma_usable(int /*C*/, int DH) { return DH == 64 || DH == 128; }
+
+template <typename T, int DH>
+inline cudaError_t launch_attention_tma_dh(const AttnParams<T>& p, int grid, cudaStream_t stream) {
+  const size_t smem = attn_tma_smem_bytes(p.C, DH);
+  static bool opted_in = false;            // per instantiation; the attribute is per function
+  if (!opted_in) {
+    cudaError_t e = cudaFuncSetAttribute(attention_tma_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (e != cudaSuccess) return e;
+    opted_in = true;
+  }
+  attention_tma_kernel<T, DH><<<grid, kAttnThreads, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+template <typename T>
+inline cudaError_t launch_attention_tma(const AttnParams<T>& p, int DH, int grid, cudaStream_t stream) {
+  if (DH == 64) return launch_attention_tma_dh<T, 64>(p, grid, stream);
+  return launch_attention_tma_dh<T, 128>(p, grid, stream);
+}
 
 }  // namespace adore
