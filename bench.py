@@ -1,0 +1,545 @@
+"""Benchmark of the ADORE decode path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..4] [--impl ours|reference]
+
+A step is one pass of the whole hot path for one new token per sequence: for every layer the
+top-K attention over the slot cache (with weight emission and the in-place admit), once per
+step the controller + selection, and for every layer the rebuild projection + RoPE + scatter.
+Inputs are synthetic (seeded Gaussians of the workload's shapes) and resident in HBM when the
+timed region starts; the `e2e` number repeats the steps through the host-buffer entry point.
+One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "decode tokens/s (= batch x decode steps/s) at batch B, cache C"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries,
+# keyed by (kernel, workload); None until captured for the kernel as it stands.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def default_steps(cfg: wl.WorkloadConfig):
+    return {1: 80, 2: 150, 3: 30, 4: 12}.get(cfg_index(cfg), 30)
+
+
+def cfg_index(cfg):
+    for k, v in wl.CONFIGS.items():
+        if v.name == cfg.name:
+            return k
+    return 0
+
+
+# ------------------------------------------------------------------------------------------------
+# distributed plumbing (replicas: sequences are independent, no data-path collective)
+# ------------------------------------------------------------------------------------------------
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    """Largest `value` over all ranks (the slowest rank defines the job's time)."""
+    if world == 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(batch_per_rank: int, steps: int, world: int, ms_max: float) -> float:
+    return batch_per_rank * world * steps / (ms_max * 1e-3)
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(prefix="adore_clocks_", suffix=".csv")
+        self.proc = None
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, reasons, mx = [], set(), None
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    mx = float(parts[2])
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+# device-side synthetic workload
+# ------------------------------------------------------------------------------------------------
+class DeviceRun:
+    """Cache + pre-generated per-step inputs on the GPU for `total_steps` decode steps."""
+
+    def __init__(self, cfg: wl.WorkloadConfig, total_steps: int, rank: int):
+        import torch
+        from paper_2407_02328_b200 import adore as lib
+        self.torch, self.lib, self.cfg = torch, lib, cfg
+        c = cfg
+        assert total_steps <= c.steps, f"{total_steps} steps asked, the workload has {c.steps}"
+        self.dt = torch.float32 if c.dtype == "f32" else torch.bfloat16
+        dev = torch.device("cuda")
+        g = torch.Generator(device=dev)
+        g.manual_seed(c.seed * 1000 + rank)
+        B, L, H, dh, d = c.batch, c.n_layers, c.n_heads, c.head_dim, c.hidden
+        N = H * dh
+        self.stream = torch.cuda.current_stream().cuda_stream
+        self.handle = lib.adore_cache_create(
+            lib.make_config(batch=B, n_layers=L, n_heads=H, head_dim=dh, hidden=d, capacity=c.capacity,
+                            rebuild_max=c.rebuild_max, topk=c.topk, max_tokens=c.max_tokens,
+                            ctrl_hidden=c.ctrl_hidden, dtype=c.dtype, rebuild_mode=c.rebuild_mode,
+                            rope_theta=c.rope_theta, pos_scale=c.pos_scale),
+            wl.controller_weights(c), self.stream)
+
+        def randn(*shape, std=1.0):
+            return (torch.randn(*shape, generator=g, device=dev, dtype=torch.float32) * std)
+
+        def rows(*shape):
+            x = randn(*shape)
+            if c.per_layer_inputs:
+                x = x * torch.rsqrt(x.pow(2).mean(-1, keepdim=True) + 1e-5)
+            return x.to(self.dt)
+
+        if c.identity_projection:
+            eye = torch.eye(N, device=dev, dtype=self.dt)
+            self.w_kv = [torch.cat([eye, eye], 0).contiguous() for _ in range(L)]
+        else:
+            self.w_kv = [randn(2 * N, d, std=0.02).to(self.dt).contiguous() for _ in range(L)]
+        self.w_q = [randn(N, d, std=0.02).to(self.dt).contiguous() for _ in range(L)]
+        for l in range(L):
+            lib.adore_cache_set_projection(self.handle, l, self.w_kv[l])
+        # prompt
+        self.tables = None
+        if c.per_layer_inputs:
+            self.tables = [torch.zeros((B, c.max_tokens, d), dtype=self.dt, device=dev) for _ in range(L)]
+        if c.prompt:
+            xp = rows(B, c.prompt, d).contiguous()
+            lib.adore_cache_append_tokens(self.handle, xp, c.prompt)
+            if c.per_layer_inputs:
+                self.tables[0][:, : c.prompt] = xp
+                for l in range(1, L):
+                    self.tables[l][:, : c.prompt] = rows(B, c.prompt, d)
+                    lib.adore_cache_fill_layer(self.handle, l, self.tables[l])
+            del xp
+        # per-step inputs
+        S = self.S = total_steps
+        n_x = L if c.per_layer_inputs else 1
+        self.x = rows(S, n_x, B, d).contiguous()
+        self.q = torch.empty((S, L, B, H, dh), dtype=self.dt, device=dev)
+        self.k = torch.empty_like(self.q)
+        self.v = torch.empty_like(self.q)
+        for s in range(S):
+            n = c.prompt + s
+            for l in range(L):
+                xl = self.x[s, l if c.per_layer_inputs else 0].float()
+                kv = xl @ self.w_kv[l].float().t()
+                self.k[s, l] = self._rope(kv[:, :N].reshape(B, H, dh), n).to(self.dt)
+                self.v[s, l] = kv[:, N:].reshape(B, H, dh).to(self.dt)
+                if c.identity_projection:
+                    self.q[s, l] = randn(B, H, dh).to(self.dt)
+                else:
+                    self.q[s, l] = self._rope((xl @ self.w_q[l].float().t()).reshape(B, H, dh), n).to(self.dt)
+                if c.per_layer_inputs:
+                    self.tables[l][:, n] = self.x[s, l]
+        self.r_in = 0
+        self.lists = self.counts = None
+        if c.rebuild_mode == "explicit":
+            mean = c.max_tokens * c.rebuild_p
+            self.r_in = int(min(c.max_tokens, math.ceil(mean + 6 * math.sqrt(mean) + 8)))
+            self.lists = torch.full((S, B, self.r_in), -1, dtype=torch.int32, device=dev)
+            self.counts = torch.zeros((S, B), dtype=torch.int32, device=dev)
+            for s in range(S):
+                n = c.prompt + s
+                if n == 0:
+                    continue
+                flag = torch.rand((B, n), generator=g, device=dev) < c.rebuild_p
+                key = torch.where(flag, torch.arange(n, device=dev).expand(B, n), torch.full((B, n), 1 << 30, device=dev))
+                srt = key.sort(dim=1).values[:, : self.r_in]
+                cnt = flag.sum(1).clamp(max=self.r_in).to(torch.int32)
+                w = srt.shape[1]
+                self.lists[s, :, :w] = torch.where(srt < (1 << 30), srt, torch.full_like(srt, -1)).to(torch.int32)
+                self.counts[s] = cnt
+        self.out = torch.empty((B, H, dh), dtype=self.dt, device=dev)
+        self.weights = torch.empty((B, H, c.capacity + 1), dtype=torch.float32, device=dev)
+        self.next = 0
+        lib.adore_cache_sync_status(self.handle)
+
+    def _rope(self, y, n):
+        c, torch = self.cfg, self.torch
+        if c.rope_theta == 0.0:
+            return y
+        j = torch.arange(c.head_dim // 2, device=y.device, dtype=torch.float64)
+        ang = (n * torch.pow(torch.tensor(c.rope_theta, dtype=torch.float64, device=y.device), -2.0 * j / c.head_dim))
+        cs, sn = torch.cos(ang).float(), torch.sin(ang).float()
+        a, b = y[..., 0::2], y[..., 1::2]
+        out = torch.empty_like(y)
+        out[..., 0::2] = a * cs - b * sn
+        out[..., 1::2] = a * sn + b * cs
+        return out
+
+    def step(self):
+        lib, c, s = self.lib, self.cfg, self.next
+        for l in range(c.n_layers):
+            lib.adore_decode_step(self.handle, l, self.q[s, l], self.k[s, l], self.v[s, l], self.x[s, 0],
+                                  None if self.lists is None else self.lists[s],
+                                  None if self.counts is None else self.counts[s], self.r_in, self.out, self.weights)
+            lib.adore_rebuild(self.handle, l, self.tables[l] if (self.tables is not None and l > 0) else None)
+        self.next += 1
+
+    def make_host_inputs(self, first: int, count: int):
+        """Pinned host copies of the inputs of steps first..first+count-1 (for the end-to-end pass)."""
+        t = self.torch
+        sl = slice(first, first + count)
+        pin = lambda a: a.cpu().pin_memory()
+        self.h = dict(q=pin(self.q[sl]), k=pin(self.k[sl]), v=pin(self.v[sl]), x=pin(self.x[sl]),
+                      lists=None if self.lists is None else pin(self.lists[sl]),
+                      counts=None if self.counts is None else pin(self.counts[sl]),
+                      out=t.empty(self.out.shape, dtype=self.dt).pin_memory(),
+                      weights=t.empty(self.weights.shape, dtype=t.float32).pin_memory())
+        self.h_first = first
+
+    def step_host(self):
+        lib, c, s = self.lib, self.cfg, self.next
+        i, h = s - self.h_first, self.h
+        for l in range(c.n_layers):
+            lib.adore_decode_step_host(self.handle, l, h["q"][i, l], h["k"][i, l], h["v"][i, l], h["x"][i, 0],
+                                       None if h["lists"] is None else h["lists"][i],
+                                       None if h["counts"] is None else h["counts"][i], self.r_in, h["out"], h["weights"])
+            lib.adore_rebuild(self.handle, l, self.tables[l] if (self.tables is not None and l > 0) else None)
+        self.next += 1
+
+    def host_bytes_per_step(self):
+        c, e = self.cfg, self.cfg.elem_bytes
+        qkv = 3 * c.batch * c.n_heads * c.head_dim * e * c.n_layers
+        x = c.batch * c.hidden * e
+        lists = (c.batch * self.r_in * 4 + c.batch * 4) if self.lists is not None else 0
+        out = c.n_layers * (c.batch * c.n_heads * c.head_dim * e + c.batch * c.n_heads * (c.capacity + 1) * 4)
+        return qkv + x + lists, out
+
+    def close(self):
+        if self.handle:
+            self.lib.adore_cache_destroy(self.handle)
+            self.handle = None
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU baseline (the oracle as it stands, on a bounded sample of the workload)
+# ------------------------------------------------------------------------------------------------
+def time_oracle(cfg: wl.WorkloadConfig, steps: int, warmup: int, budget_s: float = 25.0):
+    """Times the numpy oracle on the first sequences (and, for deep stacks, the first layers) of
+    the workload. Returns tokens/s scaled to all layers, the threads used and a description."""
+    from oracle.harness import Workload, make_oracle, explicit_as_lists
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    b = 1 if cfg.batch == 1 else 2
+    layers = min(cfg.n_layers, 2)
+    sample = cfg.scaled(n_layers=layers)
+    w = Workload(sample, b)
+    orc = make_oracle(w)
+    if sample.prompt:
+        orc.append_tokens(w.prompt())
+    done, t_total = 0, 0.0
+    for s in range(warmup + steps):
+        n = orc.n
+        lists, counts = w.explicit(s, n)
+        ex = explicit_as_lists(lists, counts)
+        inputs = []
+        for l in range(layers):
+            x = w.x_new(n, 0)
+            inputs.append((x,) + w.qkv(n, l, x))
+        t0 = time.perf_counter()
+        for l in range(layers):
+            x, q, k, v = inputs[l]
+            orc.decode_step(l, q, k, v, x if l == 0 else None, ex if l == 0 else None)
+            orc.rebuild(l)
+        dt = time.perf_counter() - t0
+        if s >= warmup:
+            done += 1
+            t_total += dt
+            if t_total > budget_s:
+                break
+    per_step = t_total / max(done, 1) * (cfg.n_layers / layers)
+    desc = (f"first {b} of {cfg.batch} sequences, {layers} of {cfg.n_layers} layers (time scaled by layers), "
+            f"{done} decode steps after the prompt; numpy float64 oracle")
+    return b / per_step, threads, desc, per_step * 1e3
+
+
+def run_reference(args, cfg):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    value, threads, desc, ms = time_oracle(cfg, args.steps, args.warmup, budget_s=120.0)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": workload_desc(cfg),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_desc(cfg):
+    return {"workload": cfg.name, "batch": cfg.batch, "layers": cfg.n_layers, "heads": cfg.n_heads,
+            "head_dim": cfg.head_dim, "hidden": cfg.hidden, "capacity": cfg.capacity, "topk": cfg.topk,
+            "rebuild_max": cfg.rebuild_max, "rebuild_mode": cfg.rebuild_mode, "rebuild_p": cfg.rebuild_p,
+            "prompt": cfg.prompt, "parallelism": "replicas",
+            "l2": "inputs larger than L2 (KV cache per step >> 126 MB)" if kv_bytes(cfg) > 2.5e8
+            else "L2 flushed between timed iterations"}
+
+
+def kv_bytes(cfg):
+    return 2 * cfg.n_layers * cfg.batch * cfg.n_heads * cfg.capacity * cfg.head_dim * cfg.elem_bytes
+
+
+# ------------------------------------------------------------------------------------------------
+# roofline arithmetic
+# ------------------------------------------------------------------------------------------------
+def attention_bytes_per_launch(cfg, occ: float) -> float:
+    """Algorithmic bytes of one attention launch: all occupied key rows + the current token's, only
+    the kept value rows, q and out, the emitted weights, and the admitted K/V row."""
+    e, dh = cfg.elem_bytes, cfg.head_dim
+    cand = occ + 1
+    per_bh = (cand + min(cfg.topk, cand) + 2) * dh * e + (cfg.capacity + 1) * 4 + 2 * dh * e
+    return cfg.batch * cfg.n_heads * per_bh
+
+
+def rebuild_flops_bytes_per_launch(cfg, rows: float):
+    n_out = 2 * cfg.n_heads * cfg.head_dim
+    flops = 2.0 * rows * cfg.hidden * n_out
+    bytes_ = (n_out * cfg.hidden + rows * cfg.hidden + rows * n_out) * cfg.elem_bytes
+    return flops, bytes_
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=3, help="workload 1..4 (default 3: the largest single-layer config)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    cfg = wl.get_config(args.config)
+    if args.steps is None:
+        args.steps = default_steps(cfg) if args.impl == "ours" else 3
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2407_02328_b200 import build
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2407_02328_b200 import adore as lib
+
+    K, W = args.steps, args.warmup
+    with_e2e = not args.no_e2e
+    total = W + K + (K if with_e2e else 0) + K          # warm-up, timed, end-to-end, per-stage pass
+    run = DeviceRun(cfg, total, rank)
+    flush = None
+    if kv_bytes(cfg) <= 2.5e8:
+        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(W):
+        run.step()
+    lib.adore_cache_sync_status(run.handle)
+
+    # ---- timed region: K steps, device time, max over ranks ----
+    launches0 = lib.adore_cache_launch_count(run.handle)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    barrier()
+    if flush is None:
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(K):
+            run.step()
+        ev1.record()
+        barrier()
+        ms_local = ev0.elapsed_time(ev1)
+    else:                                               # small workloads: flush L2 between steps
+        pairs = []
+        for _ in range(K):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            run.step()
+            b.record()
+            pairs.append((a, b))
+        barrier()
+        ms_local = sum(a.elapsed_time(b) for a, b in pairs)
+    clocks = sampler.stop() if sampler else None
+    launches = lib.adore_cache_launch_count(run.handle) - launches0
+    lib.adore_cache_sync_status(run.handle)
+    ms_total = max_over_ranks(ms_local, world, dev)
+    value = whole_job_tokens_per_s(cfg.batch, K, world, ms_total)
+
+    # ---- end to end through the host-buffer entry point ----
+    e2e = None
+    if with_e2e:
+        run.make_host_inputs(run.next, K)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(K):
+            run.step_host()
+        torch.cuda.synchronize()
+        e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, world, dev)
+        h2d, d2h = run.host_bytes_per_step()
+        e2e = {"value": whole_job_tokens_per_s(cfg.batch, K, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms / K,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    # ---- per-stage pass (events around every launch) for the roofline figures ----
+    rows0 = lib.adore_cache_rebuild_rows(run.handle)
+    lib.adore_cache_set_stage_timing(run.handle, True)
+    lib.adore_cache_stage_times(run.handle)
+    for _ in range(K):
+        if flush is not None:
+            flush.zero_()
+        run.step()
+    st_ms, st_n = lib.adore_cache_stage_times(run.handle)
+    lib.adore_cache_set_stage_timing(run.handle, False)
+    rows = (lib.adore_cache_rebuild_rows(run.handle) - rows0) / max(K, 1)      # rebuilt rows per step
+    lib.adore_cache_sync_status(run.handle)
+
+    peaks, peak_kind = measured_peaks()
+    occ = min(cfg.capacity, cfg.retained_max + rows / cfg.batch)
+    att_ms = st_ms[0] / max(st_n[0], 1)
+    sel_ms = st_ms[1] / max(K, 1)
+    reb_ms = st_ms[2] / max(st_n[2], 1)
+    att_bytes = attention_bytes_per_launch(cfg, occ)
+    reb_flops, reb_bytes = rebuild_flops_bytes_per_launch(cfg, rows)
+    att_gbs = att_bytes / (att_ms * 1e-3) / 1e9 if att_ms > 0 else 0.0
+    stages = {
+        "attention": {"bound": "hbm", "ms_per_launch": att_ms, "launches_per_step": cfg.n_layers,
+                      "algorithmic_bytes": att_bytes, "achieved": att_gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                      "frac": att_gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": att_gbs / NOMINAL_HBM_GBS},
+        "controller_select": {"ms_per_step": sel_ms},
+    }
+    sel_bytes = 4 * (3 * cfg.ctrl_hidden * (cfg.hidden + cfg.ctrl_hidden)) + cfg.batch * cfg.hidden * cfg.elem_bytes
+    both_ms = att_ms * cfg.n_layers + sel_ms
+    both_gbs = (att_bytes * cfg.n_layers + sel_bytes) / (both_ms * 1e-3) / 1e9 if both_ms > 0 else 0.0
+    stages["attention_plus_selection"] = {"bound": "hbm", "achieved": both_gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                                          "frac": both_gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": both_gbs / NOMINAL_HBM_GBS}
+    tensor_bound = cfg.dtype == "bf16" and rows >= 300
+    if reb_ms > 0 and rows > 0:
+        if tensor_bound:
+            tf = reb_flops / (reb_ms * 1e-3) / 1e12
+            stages["rebuild"] = {"bound": "tensor", "ms_per_launch": reb_ms, "rows_per_launch": rows, "flops": reb_flops,
+                                 "achieved": tf, "unit": "TFLOP/s", "peak": peaks["bf16_tflops_sustained"],
+                                 "frac": tf / peaks["bf16_tflops_sustained"], "frac_of_burst": tf / peaks["bf16_tflops"]}
+        else:
+            gb = reb_bytes / (reb_ms * 1e-3) / 1e9
+            stages["rebuild"] = {"bound": "hbm", "ms_per_launch": reb_ms, "rows_per_launch": rows,
+                                 "algorithmic_bytes": reb_bytes, "achieved": gb, "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                                 "frac": gb / peaks["hbm_gbs"]}
+    dominant = "rebuild" if ("rebuild" in stages and st_ms[2] > st_ms[0]) else "attention"
+    d = stages[dominant]
+    kernel_name = {"attention": "attention_tma_kernel", "rebuild": "rebuild projection"}[dominant]
+    roofline = {"kernel": kernel_name, "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"], "unit": d["unit"],
+                "frac": d["frac"], "peak_source": f"{peak_kind} ({'sustained' if d['bound'] == 'tensor' else 'copy'})",
+                "traffic": NCU_TRAFFIC_BYTES.get((kernel_name, cfg.name)),
+                "share_of_step": {"attention": st_ms[0] / max(sum(st_ms), 1e-9), "controller_select": st_ms[1] / max(sum(st_ms), 1e-9),
+                                  "rebuild": st_ms[2] / max(sum(st_ms), 1e-9)}}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, threads, desc, _ = time_oracle(cfg, 3, 1)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                "ms_per_step": ms_total / K, "steps_per_s": K / (ms_total * 1e-3), "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+                "config": workload_desc(cfg), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+                "roofline": roofline, "stages": stages, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    run.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

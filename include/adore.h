@@ -178,6 +178,20 @@ int32_t adore_cache_num_tokens(const adore_cache_t *cache);
 /* Kernel launches issued by this cache so far (host counter). */
 int64_t adore_cache_launch_count(const adore_cache_t *cache);
 
+/* Per-stage device timing for benchmarks (no counterpart in the paper beyond its Appendix D
+ * runtime split between the controller and the rest). When enabled, every kernel launch of the
+ * cache is bracketed by CUDA events on its stream. adore_cache_stage_times waits for the stream,
+ * adds up the elapsed milliseconds and launch counts per stage since the last call and resets
+ * them. Stage index: 0 attention (+admit), 1 controller + selection, 2 rebuild projection.
+ * ms and launches: HOST arrays of 3. Event recording costs a few microseconds per launch, so
+ * whole-step throughput should be measured with timing disabled. */
+adore_status_t adore_cache_set_stage_timing(adore_cache_t *cache, int32_t enable);
+adore_status_t adore_cache_stage_times(adore_cache_t *cache, double *ms, int64_t *launches);
+
+/* Total number of rows rebuilt by decode steps so far (Section 2.3: sum over steps and sequences
+ * of the rebuild-list lengths); waits for the stream. rows: HOST pointer. */
+adore_status_t adore_cache_rebuild_rows(adore_cache_t *cache, int64_t *rows);
+
 /* Waits for the stream and turns the device error word into a status (OK, DEVICE_FLAG, TIMEOUT,
  * or CUDA if the stream itself failed). The word is cleared. */
 adore_status_t adore_cache_sync_status(adore_cache_t *cache);

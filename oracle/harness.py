@@ -1,4 +1,4 @@
-"""Drives the oracle (and, in the GPU tests, the CUDA library beside it) over a workload.
+"""Drives the oracle over a workload (test infrastructure, like the rest of this package).
 
 The per-step inputs come from `workloads` (random numbers only). Queries and the current
 token's key/value rows are the harness's stand-in for the backbone model: they are made

@@ -46,7 +46,8 @@ EXPORTS = ["adore_cache_create", "adore_cache_destroy", "adore_cache_set_project
            "adore_cache_append_tokens", "adore_cache_fill_layer", "adore_decode_step",
            "adore_decode_step_host", "adore_rebuild", "adore_cache_slot_map", "adore_cache_rebuild_list",
            "adore_cache_step_info", "adore_cache_scores", "adore_cache_kv", "adore_cache_num_tokens",
-           "adore_cache_launch_count", "adore_cache_sync_status", "adore_status_string"]
+           "adore_cache_launch_count", "adore_cache_sync_status", "adore_status_string",
+           "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows"]
 
 
 def _lib():
@@ -77,6 +78,9 @@ def _lib():
         lib.adore_cache_launch_count.argtypes = [vp]
         lib.adore_cache_launch_count.restype = C.c_int64
         lib.adore_cache_sync_status.argtypes = [vp]
+        lib.adore_cache_set_stage_timing.argtypes = [vp, i32]
+        lib.adore_cache_stage_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+        lib.adore_cache_rebuild_rows.argtypes = [vp, C.POINTER(C.c_int64)]
         _LIB = lib
     return _LIB
 
@@ -177,6 +181,24 @@ def adore_cache_launch_count(cache: int) -> int:
 
 def adore_cache_sync_status(cache: int) -> None:
     _check(_lib().adore_cache_sync_status(cache), "adore_cache_sync_status")
+
+
+def adore_cache_set_stage_timing(cache: int, enable: bool) -> None:
+    _check(_lib().adore_cache_set_stage_timing(cache, int(enable)), "adore_cache_set_stage_timing")
+
+
+def adore_cache_stage_times(cache: int):
+    """Returns ([ms attention, ms controller+select, ms rebuild], [launch counts]) since the last call."""
+    ms = (C.c_double * 3)()
+    n = (C.c_int64 * 3)()
+    _check(_lib().adore_cache_stage_times(cache, ms, n), "adore_cache_stage_times")
+    return list(ms), list(n)
+
+
+def adore_cache_rebuild_rows(cache: int) -> int:
+    v = C.c_int64()
+    _check(_lib().adore_cache_rebuild_rows(cache, C.byref(v)), "adore_cache_rebuild_rows")
+    return v.value
 
 
 def adore_status_string(status: int) -> str:

@@ -93,7 +93,15 @@ struct adore_cache {
   int* frow_slot = nullptr;
   int* frow_total = nullptr;
   unsigned* done_counter = nullptr;
+  unsigned long long* rows_accum = nullptr;
   unsigned* err = nullptr;
+  // optional per-stage timing
+  bool timing = false;
+  std::vector<cudaEvent_t> ev_pool;        // start/stop pairs, reused after each read-out
+  size_t ev_used = 0;
+  std::vector<int> ev_stage;
+  double stage_ms[3] = {0, 0, 0};
+  int64_t stage_launches[3] = {0, 0, 0};
   double* part = nullptr;
   size_t part_doubles = 0;
   int ksplit = 1;
@@ -119,6 +127,28 @@ namespace {
     cudaError_t e_ = (expr);                            \
     if (e_ != cudaSuccess) return cuda_fail(e_);        \
   } while (0)
+
+// Brackets the launches made during its lifetime with a pair of events when timing is on.
+struct StageScope {
+  adore_cache* c;
+  size_t idx = 0;
+  bool on = false;
+  StageScope(adore_cache* cache, int stage) : c(cache) {
+    if (!c->timing) return;
+    if (c->ev_used + 2 > c->ev_pool.size()) {
+      cudaEvent_t a, b;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+      c->ev_pool.push_back(a);
+      c->ev_pool.push_back(b);
+    }
+    idx = c->ev_used;
+    c->ev_used += 2;
+    c->ev_stage.push_back(stage);
+    cudaEventRecord(c->ev_pool[idx], c->stream);
+    on = true;
+  }
+  ~StageScope() { if (on) cudaEventRecord(c->ev_pool[idx + 1], c->stream); }
+};
 
 adore_status_t cuda_fail(cudaError_t e) {
   if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return ADORE_ERR_OOM; }
@@ -173,7 +203,7 @@ SelectParams select_params(adore_cache* c, int n, int P, int old_map, int new_ma
   s.admit_slot = c->admit_slot; s.evicted_tok = c->evicted_tok; s.rebuild_tok = c->rebuild_tok;
   s.rebuild_slot = c->rebuild_slot; s.rebuild_count = c->rebuild_count;
   s.row_off = c->row_off; s.row_b = c->row_b; s.row_tok = c->row_tok; s.row_slot = c->row_slot; s.row_total = c->row_total;
-  s.done_counter = c->done_counter; s.err = c->err;
+  s.done_counter = c->done_counter; s.rows_accum = nullptr; s.err = c->err;
   return s;
 }
 
@@ -205,6 +235,7 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
   p.scale = float(1.0 / std::sqrt(double(f.head_dim)));
   p.err = c->err;
   const int grid = f.batch * f.n_heads;
+  StageScope scope(c, 0);
   cudaError_t e;
   // ADORE_ATTN_DIRECT=1 selects the variant without shared-memory staging (for A/B timing)
   static const bool direct = std::getenv("ADORE_ATTN_DIRECT") != nullptr;
@@ -236,6 +267,7 @@ adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, co
   p.row_b = row_b; p.row_tok = row_tok; p.row_slot = row_slot; p.row_total = row_total;
   p.rope_cos = f.rope_theta != 0.f ? c->rope_cos : nullptr; p.rope_sin = f.rope_theta != 0.f ? c->rope_sin : nullptr;
   p.H = f.n_heads; p.DH = f.head_dim; p.C = f.capacity; p.N = 2 * f.n_heads * f.head_dim; p.err = c->err;
+  StageScope scope(c, 2);
   if (tc_usable<T>(c->tc)) {
     int launched = 0;
     cudaError_t e = launch_rebuild_tc(c->tc, p, layer, m_max, c->stream, &launched);
@@ -343,6 +375,7 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   TRY(dev_alloc(c, &c->frow_slot, B * C * sizeof(int), true));
   TRY(dev_alloc(c, &c->frow_total, sizeof(int), true));
   TRY(dev_alloc(c, &c->done_counter, sizeof(unsigned), true));
+  TRY(dev_alloc(c, &c->rows_accum, sizeof(unsigned long long), true));
   TRY(dev_alloc(c, &c->err, sizeof(unsigned), true));
   // decode splits the d-long dot products so that roughly one wave of CTAs is busy
   {
@@ -406,6 +439,7 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (!c) return ADORE_OK;
   cudaStreamSynchronize(c->stream);
   for (void* p : c->owned) cudaFree(p);
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   void* hosts[] = {c->h_q, c->h_k, c->h_v, c->h_x, c->h_out, c->h_list, c->h_count, c->h_weights};
   for (void* p : hosts) if (p) cudaFree(p);
   cudaGetLastError();
@@ -479,8 +513,11 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     if (ex && r_in > 8192) return ADORE_ERR_UNSUPPORTED;
     // controller + selection for the step; the attention below still reads the previous map
     adore_status_t st;
-    if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit);
-    else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit);
+    {
+      StageScope scope(c, 1);
+      if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit);
+      else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit);
+    }
     if (st != ADORE_OK) return st;
     const int P = ex ? pow2_at_least(r_in) : pow2_at_least(c->n);
     RecurParams rp = recur_params(c, f.batch, 1, c->ksplit, c->n);
@@ -488,6 +525,8 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     sp.explicit_list = ex && r_in > 0 ? explicit_list : nullptr;
     sp.explicit_count = ex && r_in > 0 ? explicit_count : nullptr;
     sp.r_in = r_in;
+    sp.rows_accum = c->rows_accum;
+    StageScope scope(c, 1);
     const size_t smem = std::max(select_smem_bytes(f.capacity, P), recur_smem_bytes(f.ctrl_hidden));
     if (f.dtype == ADORE_F32)
       ctrl_select_kernel<float><<<f.batch, select_threads(c), smem, c->stream>>>(
@@ -595,6 +634,41 @@ adore_status_t adore_cache_kv(adore_cache_t* c, int32_t layer, const void** k, c
 int32_t adore_cache_num_tokens(const adore_cache_t* c) { return c ? c->n : -1; }
 
 int64_t adore_cache_launch_count(const adore_cache_t* c) { return c ? c->launches : -1; }
+
+adore_status_t adore_cache_set_stage_timing(adore_cache_t* c, int32_t enable) {
+  if (!c) return ADORE_ERR_INVALID_ARG;
+  c->timing = enable != 0;
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_stage_times(adore_cache_t* c, double* ms, int64_t* launches) {
+  if (!c || !ms || !launches) return ADORE_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
+  for (size_t i = 0; i < c->ev_stage.size(); ++i) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, c->ev_pool[2 * i], c->ev_pool[2 * i + 1]) != cudaSuccess) return ADORE_ERR_CUDA;
+    c->stage_ms[c->ev_stage[i]] += double(t);
+    c->stage_launches[c->ev_stage[i]] += 1;
+  }
+  c->ev_stage.clear();
+  c->ev_used = 0;
+  for (int s = 0; s < 3; ++s) {
+    ms[s] = c->stage_ms[s];
+    launches[s] = c->stage_launches[s];
+    c->stage_ms[s] = 0;
+    c->stage_launches[s] = 0;
+  }
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_rebuild_rows(adore_cache_t* c, int64_t* rows) {
+  if (!c || !rows) return ADORE_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
+  unsigned long long v = 0;
+  if (cudaMemcpy(&v, c->rows_accum, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return ADORE_ERR_CUDA;
+  *rows = int64_t(v);
+  return ADORE_OK;
+}
 
 adore_status_t adore_cache_sync_status(adore_cache_t* c) {
   if (!c) return ADORE_ERR_INVALID_ARG;

@@ -97,6 +97,7 @@ struct SelectParams {
   int* row_slot;
   int* row_total;             // [1]
   unsigned* done_counter;     // [1], returns to 0
+  unsigned long long* rows_accum;  // [1] running total of rebuilt rows, or nullptr
   unsigned* err;
 };
 
@@ -199,6 +200,7 @@ __device__ inline void finish_row_table(const SelectParams& p, int* tmp) {
     for (int b = 0; b < p.B; ++b) { p.row_off[b] = off; off += __ldcg(p.rebuild_count + b); }
     p.row_off[p.B] = off;
     *p.row_total = off;
+    if (p.rows_accum) *p.rows_accum += static_cast<unsigned long long>(off);
     *p.done_counter = 0u;
   }
   __syncthreads();

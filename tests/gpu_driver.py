@@ -17,7 +17,7 @@ import torch
 import workloads as wl
 from oracle import adore_oracle as ao
 from paper_2407_02328_b200 import adore as lib
-from tests.harness import Workload, make_oracle, explicit_as_lists
+from oracle.harness import Workload, make_oracle, explicit_as_lists
 
 TOL = {"bf16": dict(out_abs=2e-2, out_rel=1e-2, w_abs=1e-3), "f32": dict(out_abs=1e-4, out_rel=1e-4, w_abs=1e-5)}
 NEAR_TIE_REL = 1e-6

@@ -12,7 +12,7 @@ import torch
 
 import workloads as wl
 from oracle import adore_oracle as ao
-from tests.harness import Workload, make_oracle, explicit_as_lists
+from oracle.harness import Workload, make_oracle, explicit_as_lists
 
 TINY = wl.WorkloadConfig(name="tiny", dtype="f32", n_layers=1, batch=2, n_heads=2, head_dim=8,
                          hidden=16, capacity=8, topk=4, rebuild_max=2, prompt=0, steps=24,
