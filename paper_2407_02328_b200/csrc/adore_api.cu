@@ -264,7 +264,7 @@ adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, co
   p.x_table = static_cast<const T*>(x_table ? x_table : c->x_store); p.seq_stride = f.max_tokens; p.d = f.hidden;
   p.w_kv = static_cast<const T*>(c->w_kv[layer]);
   p.Kc = static_cast<T*>(c->Kc) + layer * layer_elems; p.Vc = static_cast<T*>(c->Vc) + layer * layer_elems;
-  p.row_b = row_b; p.row_tok = row_tok; p.row_slot = row_slot; p.row_total = row_total;
+  p.row_b = row_b; p.row_tok = row_tok; p.row_slot = row_slot; p.row_total = row_total; p.row_base = 0; p.row_limit = m_max;
   p.rope_cos = f.rope_theta != 0.f ? c->rope_cos : nullptr; p.rope_sin = f.rope_theta != 0.f ? c->rope_sin : nullptr;
   p.H = f.n_heads; p.DH = f.head_dim; p.C = f.capacity; p.N = 2 * f.n_heads * f.head_dim; p.err = c->err;
   StageScope scope(c, 2);

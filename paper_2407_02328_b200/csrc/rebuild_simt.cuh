@@ -21,7 +21,9 @@ struct RebuildParams {
   const int* row_b;
   const int* row_tok;
   const int* row_slot;
-  const int* row_total;   // device scalar M
+  const int* row_total;   // device scalar: rows in the whole table
+  int row_base;           // this launch covers table rows [row_base, row_base + row_limit) (row_* point at row_base)
+  int row_limit;
   const float* rope_cos;  // [max_tokens, DH/2] or nullptr
   const float* rope_sin;
   int H, DH, C, N;
@@ -36,7 +38,7 @@ __global__ void __launch_bounds__(256) rebuild_simt_kernel(const RebuildParams<T
   __shared__ float As[kSimtK][kSimtTile + 4];
   __shared__ float Ws[kSimtK][kSimtTile + 4];
   __shared__ long long s_rowoff[kSimtTile];
-  const int M = *p.row_total;
+  const int M = min(max(*p.row_total - p.row_base, 0), p.row_limit);
   const int m0 = blockIdx.y * kSimtTile, n0 = blockIdx.x * kSimtTile;
   if (m0 >= M) return;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
