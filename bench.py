@@ -47,7 +47,7 @@ def measured_peaks():
 
 
 def default_steps(cfg: wl.WorkloadConfig):
-    return {1: 80, 2: 150, 3: 30, 4: 12}.get(cfg_index(cfg), 30)
+    return {1: 80, 2: 150, 3: 300, 4: 40}.get(cfg_index(cfg), 30)
 
 
 def cfg_index(cfg):
@@ -83,7 +83,7 @@ def whole_job_tokens_per_s(batch_per_rank: int, steps: int, world: int, ms_max: 
 # clocks
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -93,12 +93,15 @@ class ClockSampler:
         try:
             self.f = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+                                          "-lms", "50", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self, t_begin: float, t_end: float):
+        """Median SM clock and throttle reasons of the samples taken between two time.time() stamps."""
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0,
+               "window": "timed region + end-to-end pass + per-stage pass"}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -115,6 +118,9 @@ class ClockSampler:
                 if len(parts) < 9:
                     continue
                 try:
+                    ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    if ts < t_begin - 0.05 or ts > t_end + 0.05:
+                        continue
                     sm.append(float(parts[1]))
                     mx = float(parts[2])
                 except ValueError:
@@ -431,7 +437,10 @@ def main():
     # ---- timed region: K steps, device time, max over ranks ----
     launches0 = lib.adore_cache_launch_count(run.handle)
     sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        time.sleep(0.5)                                 # let the sampler come up
     barrier()
+    t_clock0 = time.time()
     if flush is None:
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record()
@@ -451,7 +460,6 @@ def main():
             pairs.append((a, b))
         barrier()
         ms_local = sum(a.elapsed_time(b) for a, b in pairs)
-    clocks = sampler.stop() if sampler else None
     launches = lib.adore_cache_launch_count(run.handle) - launches0
     lib.adore_cache_sync_status(run.handle)
     ms_total = max_over_ranks(ms_local, world, dev)
@@ -483,6 +491,7 @@ def main():
     lib.adore_cache_set_stage_timing(run.handle, False)
     rows = (lib.adore_cache_rebuild_rows(run.handle) - rows0) / max(K, 1)      # rebuilt rows per step
     lib.adore_cache_sync_status(run.handle)
+    clocks = sampler.stop(t_clock0, time.time()) if sampler else None
 
     peaks, peak_kind = measured_peaks()
     occ = min(cfg.capacity, cfg.retained_max + rows / cfg.batch)

@@ -35,6 +35,7 @@ def to_dev(a: np.ndarray, cfg: wl.WorkloadConfig) -> torch.Tensor:
 class Report:
     steps: int = 0
     near_ties: int = 0
+    rounding_ties: int = 0
     topk_rows: int = 0
     max_out_err: float = 0.0
     max_w_err: float = 0.0
@@ -114,7 +115,7 @@ def _ulp(ref: np.ndarray, dtype: str) -> np.ndarray:
 
 
 def compare_attention(rep: Report, cfg, q, orc: ao.AdoreOracle, layer, k_new, attn_map, out_g, w_g, out_o, w_o,
-                      Kc_before):
+                      Kc_before, gpu_k=None, admit_slot=None):
     tol = TOL[cfg.dtype]
     err = np.abs(out_g - out_o)
     bound = tol["out_abs"] + tol["out_rel"] * np.abs(out_o)
@@ -134,8 +135,24 @@ def compare_attention(rep: Report, cfg, q, orc: ao.AdoreOracle, layer, k_new, at
         assert valid[diff].all(), "an empty slot was kept"
         thr = logit[keep_o[b, h]].min()
         gap = np.abs(logit[diff] - thr).max()
-        assert gap <= NEAR_TIE_REL * scale, f"top-K sets differ beyond a near-tie: gap {gap:.3e} scale {scale:.3e}"
-        rep.near_ties += 1
+        if gap <= NEAR_TIE_REL * scale:
+            rep.near_ties += 1
+        else:
+            # Rebuilt cache rows may differ from the oracle's by one unit in the last place (float32
+            # against float64 accumulation before the rounding; checked by compare_state). Such a row
+            # moves its logit by far more than 1e-6, so the GPU's choice is judged on the rows it
+            # actually holds: with float64 logits of ITS cache bytes the kept set must be the top K.
+            assert gpu_k is not None, f"top-K sets differ beyond a near-tie: gap {gap:.3e} scale {scale:.3e}"
+            Kg = gpu_k()[b, h].astype(np.float64)
+            a = int(admit_slot[b])
+            Kg[a] = Kc_before[b, h, a]            # that slot already holds the new token's row
+            lg = np.concatenate([Kg, k_new[b, h][None].astype(np.float64)]) @ q[b, h].astype(np.float64) / np.sqrt(cfg.head_dim)
+            lowest_kept = lg[keep_g[b, h]].min()
+            highest_dropped = lg[valid & ~keep_g[b, h]].max()
+            assert lowest_kept >= highest_dropped - NEAR_TIE_REL * scale, \
+                f"top-K set is not the top K of the GPU's own cache rows: {lowest_kept:.6e} < {highest_dropped:.6e}"
+            assert np.abs(lg - logit)[valid].max() <= 0.05 * scale
+            rep.rounding_ties += 1
         w_ok[b, h, diff] = False
     werr = np.abs(w_g - w_o)[w_ok]
     assert (werr <= tol["w_abs"]).all(), f"attention weights off by {werr.max():.3e}"
@@ -237,7 +254,8 @@ def run_parity(cfg: wl.WorkloadConfig, batch: Optional[int] = None, steps: Optio
                                           dl if l == 0 else None, dc if l == 0 else None, w.r_in if l == 0 else 0,
                                           g.out, g.weights)
                     out_g, w_g = g.out.float().cpu().numpy(), g.weights.cpu().numpy()
-                compare_attention(rep, cfg, q, orc, l, k, attn_map, out_g, w_g, out_o, w_o, K_before)
+                compare_attention(rep, cfg, q, orc, l, k, attn_map, out_g, w_g, out_o, w_o, K_before,
+                                  gpu_k=lambda l=l: g.kv(l)[0], admit_slot=orc.info.admit_slot)
                 orc.rebuild(l, otab[l] if (cfg.per_layer_inputs and l > 0) else None)
                 lib.adore_rebuild(g.handle, l, tables[l] if (cfg.per_layer_inputs and l > 0) else None)
             rep.steps += 1
