@@ -192,6 +192,44 @@ adore_status_t adore_cache_stage_times(adore_cache_t *cache, double *ms, int64_t
  * of the rebuild-list lengths); waits for the stream. rows: HOST pointer. */
 adore_status_t adore_cache_rebuild_rows(adore_cache_t *cache, int64_t *rows);
 
+/* Controller scoring for callers that cannot allocate device memory. (The paper has no
+ * counterpart: this is a packaging of its controller, Section 2.2 Eq. 2, for a constrained
+ * caller.) Some users of this library run where cudaMalloc is off limits: a scheduler thread
+ * that scores tokens while another thread is capturing or replaying CUDA graphs, a service whose
+ * device memory was carved up once at start-up and is owned by a different allocator, or code
+ * that must not take the driver's allocation lock on its latency path. The cache-based path
+ * gets its scratch (the k-split partial sums of the gate product W_ih x) from cudaMalloc in
+ * adore_cache_create; this entry point keeps the same scratch in a fixed 2 MiB array inside
+ * the library image instead, and needs no cache object at all.
+ *
+ * It scores ONE new token per sequence: z <- GRU(x, z), score = MLP(p + z), sigma = sigmoid.
+ *   w         : HOST struct of DEVICE pointers to the float32 parameters, same shapes and gate
+ *               order as adore_controller_weights_t describes (row-major, not transposed).
+ *   x         : device T[batch, hidden] rows of the new tokens (T by `dtype`).
+ *   z         : device double[batch, ctrl_hidden], the GRU state; read and overwritten (start a
+ *               sequence with zeros).
+ *   position  : position n of the new token; the position feature is n / pos_scale.
+ *   score, sigma : device float[batch] outputs (pre-sigmoid score and sigma).
+ * The arithmetic is the cache-based path's (float64, rounded to float32 at the end); only the
+ * number of k-slices may differ, so results agree to the last float32 digit or one unit of it.
+ *
+ * Limits and rules:
+ *   - batch * 3 * ctrl_hidden doubles must fit the 2 MiB array (batch <= 682 for d' = 128);
+ *     larger requests return ADORE_ERR_UNSUPPORTED and launch nothing.
+ *   - The array is part of the library image: every GPU on which the library runs holds
+ *     these 2 MiB until the process exits.
+ *   - The first call on each device looks up the array's device address (no allocation). Make
+ *     that first call outside any stream capture.
+ *   - All calls on a device share the array. It is fully rewritten by each call, so nothing
+ *     needs clearing, but two calls whose kernels overlap on the GPU (different streams) race;
+ *     keep calls on one stream or order them with events.
+ *   - No cudaMalloc, cudaFree or other allocating routine is called; work is queued on
+ *     cuda_stream (a cudaStream_t, NULL = default stream) and not waited for. */
+adore_status_t adore_controller_score_static(const adore_controller_weights_t *w, adore_dtype_t dtype,
+                                             int32_t batch, int32_t hidden, int32_t ctrl_hidden, const void *x,
+                                             double *z, int32_t position, float pos_scale, float *score,
+                                             float *sigma, void *cuda_stream);
+
 /* Waits for the stream and turns the device error word into a status (OK, DEVICE_FLAG, TIMEOUT,
  * or CUDA if the stream itself failed). The word is cleared. */
 adore_status_t adore_cache_sync_status(adore_cache_t *cache);

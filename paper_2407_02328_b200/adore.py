@@ -47,7 +47,8 @@ EXPORTS = ["adore_cache_create", "adore_cache_destroy", "adore_cache_set_project
            "adore_decode_step_host", "adore_rebuild", "adore_cache_slot_map", "adore_cache_rebuild_list",
            "adore_cache_step_info", "adore_cache_scores", "adore_cache_kv", "adore_cache_num_tokens",
            "adore_cache_launch_count", "adore_cache_sync_status", "adore_status_string",
-           "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows"]
+           "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows",
+           "adore_controller_score_static"]
 
 
 def _lib():
@@ -81,6 +82,8 @@ def _lib():
         lib.adore_cache_set_stage_timing.argtypes = [vp, i32]
         lib.adore_cache_stage_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         lib.adore_cache_rebuild_rows.argtypes = [vp, C.POINTER(C.c_int64)]
+        lib.adore_controller_score_static.argtypes = [C.POINTER(adore_controller_weights_t), C.c_int, i32, i32, i32, vp, vp,
+                                                      i32, C.c_float, vp, vp, vp]
         _LIB = lib
     return _LIB
 
@@ -199,6 +202,16 @@ def adore_cache_rebuild_rows(cache: int) -> int:
     v = C.c_int64()
     _check(_lib().adore_cache_rebuild_rows(cache, C.byref(v)), "adore_cache_rebuild_rows")
     return v.value
+
+
+def adore_controller_score_static(weights_dev: Dict[str, object], dtype: str, batch: int, hidden: int, ctrl_hidden: int,
+                                  x, z, position: int, pos_scale: float, score, sigma, cuda_stream: int = 0) -> None:
+    """Scores one new token per sequence without any allocation; `weights_dev` maps the parameter
+    names of adore_controller_weights_t to float32 CUDA tensors (or raw device addresses)."""
+    w = adore_controller_weights_t(**{k: _ptr(weights_dev[k]) for k, _ in adore_controller_weights_t._fields_})
+    _check(_lib().adore_controller_score_static(C.byref(w), ADORE_F32 if dtype == "f32" else ADORE_BF16, batch, hidden,
+                                                ctrl_hidden, _ptr(x), _ptr(z), position, pos_scale, _ptr(score),
+                                                _ptr(sigma), cuda_stream or None), "adore_controller_score_static")
 
 
 def adore_status_string(status: int) -> str:
