@@ -13,7 +13,8 @@ from typing import Dict, Optional, Tuple
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libadore.so")
+# ADORE_LIB points at another build of the same library (e.g. an instrumented one)
+LIB_PATH = os.environ.get("ADORE_LIB") or os.path.join(_HERE, "libadore.so")
 
 ADORE_F32, ADORE_BF16 = 0, 1
 ADORE_REBUILD_POLICY, ADORE_REBUILD_EXPLICIT = 0, 1

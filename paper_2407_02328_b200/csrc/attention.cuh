@@ -86,31 +86,21 @@ struct AttnSmem {
   }
 };
 
-// Phases 2-4 and the admit write, given the logits of all C+1 rows in shared memory
-// (-inf for empty slots). Every thread of the block calls it after a __syncthreads().
+// Phases 2-3, given the logits of all C+1 rows in shared memory (-inf for empty slots): decides the
+// kept set, turns the logits into weights in place (0 for rows not kept), writes the weights out and
+// builds the ordered list of kept row indices. Returns the number of kept rows. Every thread of the
+// block calls it after a __syncthreads(); the results are published by a final __syncthreads().
 template <typename T, int DH>
-__device__ __forceinline__ void attention_tail(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh) {
+__device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh) {
   constexpr int NT = kAttnThreads;
   constexpr int NW = NT / 32;
-  constexpr int EPL = Elem<T>::kPer16B;
-  constexpr int LPR = DH / EPL;
-  constexpr int RPW = 32 / LPR;
-  constexpr int U = kAttnUnroll;
   float* s_logit = sm.logit;
   int* s_list = sm.list;
   unsigned* s_hist = sm.hist;
-  float* s_red = sm.red;
   float* s_tmp = sm.tmp;
   int* s_sel = sm.sel;
-  const int C = p.C, rows = C + 1;
+  const int rows = p.C + 1;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int sub = lane / LPR, li = lane % LPR;
-  const int b = bh / p.H;
-  const size_t row_bytes = size_t(DH) * sizeof(T);
-  const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * row_bytes;
-  const unsigned char* Vb = reinterpret_cast<const unsigned char*>(p.Vc) + size_t(bh) * C * row_bytes;
-  const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * row_bytes;
-  const unsigned char* vnew = reinterpret_cast<const unsigned char*>(p.v_new) + size_t(bh) * row_bytes;
 
   // ---- phase 2: which logits are kept (K largest, lower index wins ties) -------------------
   int cnt = 0;
@@ -202,11 +192,35 @@ __device__ __forceinline__ void attention_tail(const AttnParams<T>& p, const Att
     n_kept += total;
   }
   __syncthreads();
+  return n_kept;
+}
 
+// Phase 4 with direct loads: adds w_s * V[s] of the kept rows into acc (this lane's 16-byte column
+// slice; lanes of different row groups and warps hold partial sums).
+template <typename T, int DH>
+__device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh, int n_kept,
+                                                        float (&acc)[Elem<T>::kPer16B]) {
+  constexpr int NT = kAttnThreads;
+  constexpr int NW = NT / 32;
+  constexpr int EPL = Elem<T>::kPer16B;
+  constexpr int LPR = DH / EPL;
+  constexpr int RPW = 32 / LPR;
+  constexpr int U = kAttnUnroll;
+  float* s_logit = sm.logit;
+  int* s_list = sm.list;
+  float* s_red = sm.red;
+  const int C = p.C;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int sub = lane / LPR, li = lane % LPR;
+  const int b = bh / p.H;
+  const size_t row_bytes = size_t(DH) * sizeof(T);
+  const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * row_bytes;
+  const unsigned char* Vb = reinterpret_cast<const unsigned char*>(p.Vc) + size_t(bh) * C * row_bytes;
+  const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * row_bytes;
+  const unsigned char* vnew = reinterpret_cast<const unsigned char*>(p.v_new) + size_t(bh) * row_bytes;
+  (void)NW; (void)RPW; (void)U; (void)s_logit; (void)s_list; (void)s_red; (void)warp; (void)sub; (void)li; (void)b;
+  (void)Kb; (void)Vb; (void)knew; (void)vnew;
   // ---- phase 4: weighted sum of the kept value rows ----------------------------------------
-  float acc[EPL];
-#pragma unroll
-  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
   for (int j0 = warp * RPW; j0 < n_kept; j0 += NW * RPW * U) {
     uint4 vv[U];
     float wv[U];
@@ -229,6 +243,33 @@ __device__ __forceinline__ void attention_tail(const AttnParams<T>& p, const Att
       for (int e = 0; e < EPL; ++e) acc[e] = fmaf(wv[u], vf[e], acc[e]);
     }
   }
+}
+
+// Adds the partial sums of all row groups and warps, writes `out`, then writes the current token's
+// row into its slot (append of the most recent state, Section 2.2 third bullet).
+template <typename T, int DH>
+__device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh,
+                                                 float (&acc)[Elem<T>::kPer16B]) {
+  constexpr int NT = kAttnThreads;
+  constexpr int NW = NT / 32;
+  constexpr int EPL = Elem<T>::kPer16B;
+  constexpr int LPR = DH / EPL;
+  constexpr int RPW = 32 / LPR;
+  constexpr int U = kAttnUnroll;
+  float* s_logit = sm.logit;
+  int* s_list = sm.list;
+  float* s_red = sm.red;
+  const int C = p.C;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int sub = lane / LPR, li = lane % LPR;
+  const int b = bh / p.H;
+  const size_t row_bytes = size_t(DH) * sizeof(T);
+  const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * row_bytes;
+  const unsigned char* Vb = reinterpret_cast<const unsigned char*>(p.Vc) + size_t(bh) * C * row_bytes;
+  const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * row_bytes;
+  const unsigned char* vnew = reinterpret_cast<const unsigned char*>(p.v_new) + size_t(bh) * row_bytes;
+  (void)NW; (void)RPW; (void)U; (void)s_logit; (void)s_list; (void)s_red; (void)warp; (void)sub; (void)li; (void)b;
+  (void)Kb; (void)Vb; (void)knew; (void)vnew;
 #pragma unroll
   for (int o = LPR; o < 32; o <<= 1)
 #pragma unroll
@@ -257,6 +298,17 @@ __device__ __forceinline__ void attention_tail(const AttnParams<T>& p, const Att
       set_error(p.err, ERRW_BOUNDS);
     }
   }
+}
+
+// Phases 2-4 and the admit write for kernels that gather the value rows with direct loads.
+template <typename T, int DH>
+__device__ __forceinline__ void attention_tail(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh) {
+  const int n_kept = attention_keep_and_weights<T, DH>(p, sm, bh);
+  float acc[Elem<T>::kPer16B];
+#pragma unroll
+  for (int e = 0; e < Elem<T>::kPer16B; ++e) acc[e] = 0.f;
+  attention_values_direct<T, DH>(p, sm, bh, n_kept, acc);
+  attention_finish<T, DH>(p, sm, bh, acc);
 }
 
 template <typename T, int DH>

@@ -6,7 +6,7 @@
 // cp.async.bulk into a 4-deep ring; an mbarrier per stage counts the bytes. The warps read the
 // rows from shared memory (conflict-free 16-byte accesses). This keeps 24-32 KB in flight per
 // CTA without spending registers or issue slots on the loads, which is what the HBM roofline
-// needs with several CTAs per SM. The kept value rows are still gathered with direct loads.
+// needs with several CTAs per SM. The kept value rows are gathered with direct loads.
 //
 // Every wait is bounded: if a stage never fills, the CTA sets the timeout bit of the error word,
 // drains what it issued with short waits and finishes with whatever it has (the step is then
@@ -149,7 +149,15 @@ __global__ void __launch_bounds__(kAttnThreads) attention_tma_kernel(const AttnP
     if (tid == 0 && !failed && c + kRingStages < n_chunks) issue(c + kRingStages);
   }
   // (the loop's last __syncthreads also publishes the logits)
-  attention_tail<T, DH>(p, sm, bh);
+  const int n_kept = attention_keep_and_weights<T, DH>(p, sm, bh);
+
+  // ---- phase 4: only the kept value rows, gathered with direct 16-byte loads (one bulk copy per
+  // 256-byte row was measured slower than the loads: the copy engine's per-operation cost dominates)
+  float acc[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  attention_values_direct<T, DH>(p, sm, bh, n_kept, acc);
+  attention_finish<T, DH>(p, sm, bh, acc);
 }
 
 template <typename T>

@@ -14,74 +14,117 @@
 
 namespace adore {
 
-constexpr int kGateTile = 32;     // rows x gates per CTA
+constexpr int kGateTileG = 64;     // gates per CTA
+constexpr int kGateTileR = 32;     // rows per CTA
 constexpr int kGateKChunk = 64;
 constexpr int kGateThreads = 256;
 
 template <typename T>
 struct GateParams {
-  const T* x;            // row r = b*tc + t lives at x + ((b*seq_stride + t) * d)
+  const T* x;            // row r = b*tc + t lives at x + ((b*seq_stride + t) * d); 16-byte aligned rows
   long long seq_stride;  // tokens between consecutive sequences in x
   int tc;                // tokens per sequence in this call
   int rows;              // B * tc
-  int d, G;              // input width, 3*d'
+  int d, G;              // input width (multiple of 64), 3*d'
   const float* w_ih;     // [G, d]
   double* part;          // [ksplit, rows, G]
   int ksplit, kslice;    // kslice is a multiple of kGateKChunk
 };
 
+// 64 gates x 32 rows per CTA, 4 x 2 outputs per thread, float64 FMA, k in chunks of 32. The next
+// chunk is fetched into registers while the current one is consumed from shared memory.
+constexpr int kGateKInner = 32;
+
 template <typename T>
 __global__ void __launch_bounds__(kGateThreads) ctrl_gates_kernel(const GateParams<T> p) {
-  __shared__ double Ws[kGateTile][kGateKChunk + 1];
-  __shared__ double Xs[kGateTile][kGateKChunk + 1];
+  constexpr int WS = kGateTileG + 2, XS = kGateTileR + 2;       // padded, rows stay 16-byte aligned
+  __shared__ __align__(16) double Ws[kGateKInner][WS];
+  __shared__ __align__(16) double Xs[kGateKInner][XS];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const int g0 = blockIdx.x * kGateTile, r0 = blockIdx.y * kGateTile, ks = blockIdx.z;
+  const int g0 = blockIdx.x * kGateTileG, r0 = blockIdx.y * kGateTileR, ks = blockIdx.z;
   const int k_begin = ks * p.kslice, k_end = min(p.d, k_begin + p.kslice);
-  double acc[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
-  for (int k0 = k_begin; k0 < k_end; k0 += kGateKChunk) {
-    for (int i = tid; i < kGateTile * kGateKChunk; i += kGateThreads) {
-      const int rr = i / kGateKChunk, kk = i % kGateKChunk;
-      const int k = k0 + kk;
-      const int g = g0 + rr, r = r0 + rr;
-      Ws[rr][kk] = (g < p.G && k < k_end) ? double(p.w_ih[size_t(g) * p.d + k]) : 0.0;
-      double xv = 0.0;
-      if (r < p.rows && k < k_end) {
-        const long long b = r / p.tc, t = r % p.tc;
-        xv = double(Elem<T>::to_float(p.x[(b * p.seq_stride + t) * p.d + k]));
-      }
-      Xs[rr][kk] = xv;
+  // per chunk this thread fetches two float4 of W (gates wg, wg+32; k offset 4*wk) and 4 elements of one x row
+  const int wk = tid & 7, wg = tid >> 3;
+  const int xr = tid >> 3, xk = tid & 7;
+  const float* wsrc[2];
+  bool wok[2];
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int g = g0 + wg + 32 * j;
+    wok[j] = g < p.G;
+    wsrc[j] = p.w_ih + size_t(wok[j] ? g : 0) * p.d + 4 * wk;
+  }
+  const bool xok = r0 + xr < p.rows;
+  const T* xsrc = p.x;
+  if (xok) {
+    const long long r = r0 + xr, b = r / p.tc, t = r % p.tc;
+    xsrc = p.x + (b * p.seq_stride + t) * p.d + 4 * xk;
+  }
+  float4 wreg[2];
+  float xreg[4];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+      wreg[j] = wok[j] ? __ldg(reinterpret_cast<const float4*>(wsrc[j] + k0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    if (!xok) {
+      xreg[0] = xreg[1] = xreg[2] = xreg[3] = 0.f;
+    } else if (sizeof(T) == 2) {
+      const uint2 v = __ldg(reinterpret_cast<const uint2*>(xsrc + k0));
+      xreg[0] = __uint_as_float(v.x << 16); xreg[1] = __uint_as_float(v.x & 0xffff0000u);
+      xreg[2] = __uint_as_float(v.y << 16); xreg[3] = __uint_as_float(v.y & 0xffff0000u);
+    } else {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(xsrc + k0));
+      xreg[0] = v.x; xreg[1] = v.y; xreg[2] = v.z; xreg[3] = v.w;
     }
+  };
+  double acc[4][2];
+#pragma unroll
+  for (int a = 0; a < 4; ++a) { acc[a][0] = 0.0; acc[a][1] = 0.0; }
+  if (k_begin < k_end) fetch(k_begin);
+  for (int k0 = k_begin; k0 < k_end; k0 += kGateKInner) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int g = wg + 32 * j;
+      Ws[4 * wk + 0][g] = double(wreg[j].x);
+      Ws[4 * wk + 1][g] = double(wreg[j].y);
+      Ws[4 * wk + 2][g] = double(wreg[j].z);
+      Ws[4 * wk + 3][g] = double(wreg[j].w);
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) Xs[4 * xk + e][xr] = double(xreg[e]);
     __syncthreads();
+    if (k0 + kGateKInner < k_end) fetch(k0 + kGateKInner);
 #pragma unroll 8
-    for (int kk = 0; kk < kGateKChunk; ++kk) {
-      const double w0 = Ws[tx][kk], w1 = Ws[tx + 16][kk];
-      const double x0 = Xs[ty][kk], x1 = Xs[ty + 16][kk];
-      acc[0][0] = fma(w0, x0, acc[0][0]);
-      acc[0][1] = fma(w0, x1, acc[0][1]);
-      acc[1][0] = fma(w1, x0, acc[1][0]);
-      acc[1][1] = fma(w1, x1, acc[1][1]);
+    for (int kk = 0; kk < kGateKInner; ++kk) {
+      const double2 wa = *reinterpret_cast<const double2*>(&Ws[kk][2 * tx]);        // gates 2tx, 2tx+1
+      const double2 wb = *reinterpret_cast<const double2*>(&Ws[kk][32 + 2 * tx]);   // gates 32+2tx, 33+2tx
+      const double2 xv = *reinterpret_cast<const double2*>(&Xs[kk][2 * ty]);
+      acc[0][0] = fma(wa.x, xv.x, acc[0][0]); acc[0][1] = fma(wa.x, xv.y, acc[0][1]);
+      acc[1][0] = fma(wa.y, xv.x, acc[1][0]); acc[1][1] = fma(wa.y, xv.y, acc[1][1]);
+      acc[2][0] = fma(wb.x, xv.x, acc[2][0]); acc[2][1] = fma(wb.x, xv.y, acc[2][1]);
+      acc[3][0] = fma(wb.y, xv.x, acc[3][0]); acc[3][1] = fma(wb.y, xv.y, acc[3][1]);
     }
     __syncthreads();
   }
 #pragma unroll
-  for (int a = 0; a < 2; ++a)
+  for (int a = 0; a < 4; ++a)
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
-      const int g = g0 + tx + 16 * a, r = r0 + ty + 16 * c;
+      const int g = g0 + 2 * tx + (a & 1) + 32 * (a >> 1), r = r0 + 2 * ty + c;
       if (g < p.G && r < p.rows) p.part[(size_t(ks) * p.rows + r) * p.G + g] = acc[a][c];
     }
 }
 
 struct RecurParams {
-  const double* part;    // [ksplit, rows, G], row = b*tc + t
+  const double* part;    // [ksplit, rows, G], row = b*tc + t; ksplit <= 32
   int ksplit, rows, tc;
   int h;                 // d'
   const float* b_ih;     // [3h]
-  const float* w_hh_t;   // [h, 3h]   transposed recurrent matrix
+  const float* w_hh;     // [3h, h]   recurrent matrix, row-major
   const float* b_hh;     // [3h]
   const float* pos_w;    // [h]
   const float* pos_b;    // [h]
-  const float* w1_t;     // [h, h]    transposed interaction matrix
+  const float* w1;       // [h, h]    interaction matrix, row-major
   const float* b1;       // [h]
   const float* w2;       // [h]
   const float* b2;       // [1]
@@ -93,29 +136,59 @@ struct RecurParams {
   double pos_scale;
 };
 
-// Shared memory needed by controller_tokens: 6*h + 32 doubles.
-__host__ __device__ inline size_t recur_smem_bytes(int h) { return sizeof(double) * (6 * h + 32); }
+constexpr int kCtrlJ = 8;          // ceil(max d' / 32): inner-index elements per lane
+
+// Shared memory needed by controller_tokens: 7*h + 32 doubles.
+__host__ __device__ inline size_t recur_smem_bytes(int h) { return sizeof(double) * (7 * h + 32); }
 
 // Runs p.tc tokens of sequence b through the recurrent half of the GRU and the MLP.
-// All threads of the block must call it; blockDim.x >= 3*h.
+// All threads of the block must call it. Every matrix-vector product is spread over the whole
+// block: a warp owns an output row, its lanes split the inner index (coalesced loads that are all
+// in flight at once) and a shuffle tree adds the lane partials, in a fixed order.
 __device__ inline void controller_tokens(const RecurParams& p, int b, double* sm) {
-  const int h = p.h, G = 3 * h, tid = threadIdx.x;
+  const int h = p.h, G = 3 * h, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
   double* s_z = sm;            // [h]
-  double* s_gi = sm + h;       // [3h]
-  double* s_gh = sm + 4 * h;   // [h] only the candidate's hidden-side term is kept apart
+  double* s_gi = sm + h;       // [3h]  reset/update: input + hidden side; candidate: input side
+  double* s_gh = sm + 4 * h;   // [h]   candidate: hidden side
   double* s_pz = sm + 5 * h;   // [h]
-  double* s_c = sm + 6 * h;    // [32] warp partials
+  double* s_t = sm + 6 * h;    // [h]   w2[i] * tanh(.)
   if (tid < h) s_z[tid] = p.z[size_t(b) * h + tid];
   __syncthreads();
   for (int t = 0; t < p.tc; ++t) {
     const int row = b * p.tc + t;
-    if (tid < G) {
-      double gi = double(p.b_ih[tid]);
-      for (int ks = 0; ks < p.ksplit; ++ks) gi += p.part[(size_t(ks) * p.rows + row) * G + tid];
-      double gh = double(p.b_hh[tid]);
-      for (int j = 0; j < h; ++j) gh = fma(double(p.w_hh_t[size_t(j) * G + tid]), s_z[j], gh);
-      if (tid < 2 * h) s_gi[tid] = gi + gh;          // reset and update gates: sum of both sides
-      else { s_gi[tid] = gi; s_gh[tid - 2 * h] = gh; }
+    // four output rows per warp at a time: all their loads are issued before the first is used
+    for (int g0 = warp * 4; g0 < G; g0 += nw * 4) {
+      float w[4][kCtrlJ];
+      double in_part[4];
+      float bh[4], bi[4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int g = min(g0 + a, G - 1);
+#pragma unroll
+        for (int jj = 0; jj < kCtrlJ; ++jj) {
+          const int j = lane + 32 * jj;
+          w[a][jj] = j < h ? __ldg(p.w_hh + size_t(g) * h + j) : 0.f;
+        }
+        in_part[a] = lane < p.ksplit ? p.part[(size_t(lane) * p.rows + row) * G + g] : 0.0;
+        bh[a] = __ldg(p.b_hh + g);
+        bi[a] = __ldg(p.b_ih + g);
+      }
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int g = g0 + a;
+        double acc = 0.0;
+#pragma unroll
+        for (int jj = 0; jj < kCtrlJ; ++jj) {
+          const int j = lane + 32 * jj;
+          if (j < h) acc = fma(double(w[a][jj]), s_z[j], acc);
+        }
+        const double gh = warp_sum(acc) + double(bh[a]);
+        const double gi = warp_sum(in_part[a]) + double(bi[a]);
+        if (lane == 0 && g < G) {
+          if (g < 2 * h) s_gi[g] = gi + gh;
+          else { s_gi[g] = gi; s_gh[g - 2 * h] = gh; }
+        }
+      }
     }
     __syncthreads();
     const int pos = p.n0 + t;
@@ -129,20 +202,43 @@ __device__ inline void controller_tokens(const RecurParams& p, int b, double* sm
       s_pz[tid] = double(p.pos_w[tid]) * upos + double(p.pos_b[tid]) + zn;
     }
     __syncthreads();
-    double contrib = 0.0;
-    if (tid < h) {
-      double a = double(p.b1[tid]);
-      for (int j = 0; j < h; ++j) a = fma(double(p.w1_t[size_t(j) * h + tid]), s_pz[j], a);
-      contrib = double(p.w2[tid]) * tanh(a);
+    for (int i0 = warp * 4; i0 < h; i0 += nw * 4) {
+      float w[4][kCtrlJ];
+      float bb[4], ww[4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int i = min(i0 + a, h - 1);
+#pragma unroll
+        for (int jj = 0; jj < kCtrlJ; ++jj) {
+          const int j = lane + 32 * jj;
+          w[a][jj] = j < h ? __ldg(p.w1 + size_t(i) * h + j) : 0.f;
+        }
+        bb[a] = __ldg(p.b1 + i);
+        ww[a] = __ldg(p.w2 + i);
+      }
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int i = i0 + a;
+        double acc = 0.0;
+#pragma unroll
+        for (int jj = 0; jj < kCtrlJ; ++jj) {
+          const int j = lane + 32 * jj;
+          if (j < h) acc = fma(double(w[a][jj]), s_pz[j], acc);
+        }
+        acc = warp_sum(acc);
+        if (lane == 0 && i < h) s_t[i] = double(ww[a]) * tanh(acc + double(bb[a]));
+      }
     }
-    contrib = warp_sum(contrib);
-    if ((tid & 31) == 0) s_c[tid >> 5] = contrib;
     __syncthreads();
-    if (tid == 0) {
-      double s = double(p.b2[0]);
-      for (int w = 0; w < (h + 31) / 32; ++w) s += s_c[w];
-      p.score[size_t(b) * p.max_tokens + pos] = float(s);
-      p.sigma[size_t(b) * p.max_tokens + pos] = float(1.0 / (1.0 + exp(-s)));
+    if (warp == 0) {
+      double acc = 0.0;
+      for (int i = lane; i < h; i += 32) acc += s_t[i];
+      acc = warp_sum(acc);
+      if (lane == 0) {
+        const double sc = acc + double(p.b2[0]);
+        p.score[size_t(b) * p.max_tokens + pos] = float(sc);
+        p.sigma[size_t(b) * p.max_tokens + pos] = float(1.0 / (1.0 + exp(-sc)));
+      }
     }
     __syncthreads();
   }

@@ -106,7 +106,7 @@ extern "C" adore_status_t adore_controller_score_static(const adore_controller_w
   while (ksplit < 16 && size_t(2 * ksplit) * batch * G <= kStaticPartDoubles && hidden / (2 * ksplit) >= kGateKChunk) ksplit *= 2;
   const int per = (hidden + ksplit - 1) / ksplit;
   const int kslice = ((per + kGateKChunk - 1) / kGateKChunk) * kGateKChunk;
-  dim3 grid((G + kGateTile - 1) / kGateTile, (batch + kGateTile - 1) / kGateTile, ksplit);
+  dim3 grid((G + kGateTileG - 1) / kGateTileG, (batch + kGateTileR - 1) / kGateTileR, ksplit);
   if (dtype == ADORE_F32) {
     GateParams<float> g{};
     g.x = static_cast<const float*>(x); g.seq_stride = 1; g.tc = 1; g.rows = batch; g.d = hidden; g.G = G;

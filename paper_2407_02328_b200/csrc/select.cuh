@@ -55,16 +55,27 @@ __device__ __forceinline__ int block_rank(bool flag, int* tmp, int* total) {
 }
 
 // Sorts keys[0..P) in DESCENDING order; P is a power of two. All threads of the block call it.
+// Each warp owns a contiguous block of E >= 64 keys; compare-exchange stages whose partners are at
+// most E/2 apart stay inside one warp's block and need only a warp barrier.
 __device__ inline void bitonic_sort_desc(unsigned long long* keys, int P) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const int E = (P >= 64 * nw) ? P / nw : (P >= 64 ? 64 : P);
+  const int active = P / E;                       // warps that own keys
+  bool prev_block_wide = true;                    // the keys were written by arbitrary threads
   for (int k = 2; k <= P; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
-      __syncthreads();
-      for (int t = threadIdx.x; t < (P >> 1); t += blockDim.x) {
-        const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // lower index of the pair
-        const int l = i | j;
-        const unsigned long long a = keys[i], c = keys[l];
-        const bool desc = (i & k) == 0;
-        if (desc ? (a < c) : (a > c)) { keys[i] = c; keys[l] = a; }
+      const bool block_wide = 2 * j > E;
+      if (block_wide || prev_block_wide) __syncthreads(); else __syncwarp();
+      prev_block_wide = block_wide;
+      if (warp < active) {
+        for (int q = lane; q < (E >> 1); q += 32) {
+          const int t = warp * (E >> 1) + q;
+          const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // lower index of the pair
+          const int l = i | j;
+          const unsigned long long a = keys[i], c = keys[l];
+          const bool desc = (i & k) == 0;
+          if (desc ? (a < c) : (a > c)) { keys[i] = c; keys[l] = a; }
+        }
       }
     }
   }
@@ -90,14 +101,6 @@ struct SelectParams {
   int* rebuild_tok;           // [B,r_max]
   int* rebuild_slot;          // [B,r_max]
   int* rebuild_count;         // [B]
-  // compact row table over the batch, built by the last CTA to finish
-  int* row_off;               // [B+1]
-  int* row_b;                 // [B*r_max]
-  int* row_tok;
-  int* row_slot;
-  int* row_total;             // [1]
-  unsigned* done_counter;     // [1], returns to 0
-  unsigned long long* rows_accum;  // [1] running total of rebuilt rows, or nullptr
   unsigned* err;
 };
 
@@ -186,32 +189,30 @@ __device__ inline int assign_rebuild_list(const SelectParams& p, const SelectSme
   return cnt;
 }
 
-// The last CTA to arrive turns the per-sequence lists into one compact row table.
-__device__ inline void finish_row_table(const SelectParams& p, int* tmp) {
-  const int tid = threadIdx.x, NT = blockDim.x;
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) tmp[0] = (atomicAdd(p.done_counter, 1u) == unsigned(p.B - 1)) ? 1 : 0;
-  __syncthreads();
-  if (!tmp[0]) return;
-  __threadfence();
-  if (tid == 0) {
-    int off = 0;
-    for (int b = 0; b < p.B; ++b) { p.row_off[b] = off; off += __ldcg(p.rebuild_count + b); }
-    p.row_off[p.B] = off;
-    *p.row_total = off;
-    if (p.rows_accum) *p.rows_accum += static_cast<unsigned long long>(off);
-    *p.done_counter = 0u;
+// Turns the per-sequence rebuild lists into one compact row table (b-major, list order): CTA b sums
+// the counts of the sequences before it and writes its own rows. One small launch after the selection.
+__global__ void __launch_bounds__(128) row_table_kernel(const int* rebuild_tok, const int* rebuild_slot,
+                                                        const int* rebuild_count, int B, int r_max, int* row_b, int* row_tok,
+                                                        int* row_slot, int* row_total, unsigned long long* rows_accum) {
+  __shared__ int tmp[64];
+  const int b = blockIdx.x, tid = threadIdx.x;
+  int before = 0, all = 0;
+  for (int i = tid; i < B; i += blockDim.x) {
+    const int c = rebuild_count[i];
+    all += c;
+    if (i < b) before += c;
   }
-  __syncthreads();
-  for (int i = tid; i < p.B * p.r_max; i += NT) {
-    const int b = i / p.r_max, j = i % p.r_max;
-    if (j < __ldcg(p.rebuild_count + b)) {
-      const int r = p.row_off[b] + j;
-      p.row_b[r] = b;
-      p.row_tok[r] = __ldcg(p.rebuild_tok + i);
-      p.row_slot[r] = __ldcg(p.rebuild_slot + i);
-    }
+  const int off = block_sum_i(before, tmp);
+  const int total = block_sum_i(all, tmp);
+  const int cnt = rebuild_count[b];
+  for (int j = tid; j < cnt; j += blockDim.x) {
+    row_b[off + j] = b;
+    row_tok[off + j] = rebuild_tok[size_t(b) * r_max + j];
+    row_slot[off + j] = rebuild_slot[size_t(b) * r_max + j];
+  }
+  if (b == 0 && tid == 0) {
+    *row_total = total;
+    if (rows_accum) *rows_accum += static_cast<unsigned long long>(total);
   }
 }
 
@@ -263,7 +264,6 @@ __device__ inline void select_step(const SelectParams& p, unsigned char* smem) {
     p.slot_tok_new[size_t(b) * C + s] = sm.tok[s];
     p.slot_role_new[size_t(b) * C + s] = sm.role[s];
   }
-  finish_row_table(p, sm.tmp);
 }
 
 // Bulk load of T tokens into an empty cache: the newest token plus the min(m-1, T-1) most
@@ -304,7 +304,6 @@ __device__ inline void select_bulk(const SelectParams& p, unsigned char* smem) {
     p.slot_tok_new[size_t(b) * C + s] = sm.tok[s];
     p.slot_role_new[size_t(b) * C + s] = sm.role[s];
   }
-  finish_row_table(p, sm.tmp);
 }
 
 // Row table of every occupied slot (for filling a layer): one CTA.
