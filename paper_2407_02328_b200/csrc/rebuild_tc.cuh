@@ -163,6 +163,20 @@ struct TcSmem {
   static constexpr size_t kTotal = size_t(kStages) * kStageBytes + kBarrierBytes + 1024;   // + alignment slack
 };
 
+// Tile order: the output columns are walked in bands of kTcBandCols weight rows (about 34 MB of W), all
+// row tiles inside a band, columns fastest. A band of W then stays L2-resident while the rows stream
+// past it once, instead of the whole 67 MB weight matrix being re-read from DRAM for every wave.
+constexpr int kTcBandCols = 4096;
+template <int BN>
+__device__ __forceinline__ void tc_tile_origin(int t, int m_tiles, int n_tiles, int& m0, int& n0) {
+  constexpr int kBand = kTcBandCols / BN;                 // column tiles per band
+  const int per_band = m_tiles * kBand;
+  const int band = t / per_band, r = t - band * per_band;
+  const int width = min(kBand, n_tiles - band * kBand);   // the last band may be narrower
+  m0 = (r / width) * kTcBM;
+  n0 = (band * kBand + r % width) * BN;
+}
+
 template <int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const TcGemmParams p) {
@@ -205,7 +219,8 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       uint32_t phase = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const int m0 = (t / n_tiles) * kTcBM, n0 = (t % n_tiles) * BN;
+        int m0, n0;
+        tc_tile_origin<BN>(t, m_tiles, n_tiles, m0, n0);
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!tc_mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
           unsigned char* sa = tiles + size_t(stage) * S::kStageBytes;
@@ -255,7 +270,8 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
       const int acc = it & 1;
       const uint32_t acc_phase = uint32_t(it >> 1) & 1u;
-      const int m0 = (t / n_tiles) * kTcBM, n0 = (t % n_tiles) * BN;
+      int m0, n0;
+      tc_tile_origin<BN>(t, m_tiles, n_tiles, m0, n0);
       const int r = m0 + quarter * 32 + lane;
       const bool valid = r < M;
       int b = 0, tok = 0, slot = 0;
