@@ -265,8 +265,7 @@ class DeviceRun:
         self.h = dict(q=pin(self.q[sl]), k=pin(self.k[sl]), v=pin(self.v[sl]), x=pin(self.x[sl]),
                       lists=None if self.lists is None else pin(self.lists[sl]),
                       counts=None if self.counts is None else pin(self.counts[sl]),
-                      out=t.empty(self.out.shape, dtype=self.dt).pin_memory(),
-                      weights=t.empty(self.weights.shape, dtype=t.float32).pin_memory())
+                      out=t.empty(self.out.shape, dtype=self.dt).pin_memory())
         self.h_first = first
 
     def step_host(self):
@@ -275,7 +274,7 @@ class DeviceRun:
         for l in range(c.n_layers):
             lib.adore_decode_step_host(self.handle, l, h["q"][i, l], h["k"][i, l], h["v"][i, l], h["x"][i, 0],
                                        None if h["lists"] is None else h["lists"][i],
-                                       None if h["counts"] is None else h["counts"][i], self.r_in, h["out"], h["weights"])
+                                       None if h["counts"] is None else h["counts"][i], self.r_in, h["out"], self.weights)
             lib.adore_rebuild(self.handle, l, self.tables[l] if (self.tables is not None and l > 0) else None)
         self.next += 1
 
@@ -284,7 +283,7 @@ class DeviceRun:
         qkv = 3 * c.batch * c.n_heads * c.head_dim * e * c.n_layers
         x = c.batch * c.hidden * e
         lists = (c.batch * self.r_in * 4 + c.batch * 4) if self.lists is not None else 0
-        out = c.n_layers * (c.batch * c.n_heads * c.head_dim * e + c.batch * c.n_heads * (c.capacity + 1) * 4)
+        out = c.n_layers * c.batch * c.n_heads * c.head_dim * e      # the weights stay on the device
         return qkv + x + lists, out
 
     def close(self):

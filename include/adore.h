@@ -146,9 +146,11 @@ adore_status_t adore_decode_step(adore_cache_t *cache, int32_t layer, const void
                                  const void *v_new, const void *x_new, const int32_t *explicit_list,
                                  const int32_t *explicit_count, int32_t r_in, void *out, float *weights);
 
-/* Same step (Sections 2.1-2.3) with HOST buffers: copies the inputs to the device, runs
- * adore_decode_step, copies `out` (and `weights` if not NULL) back and waits for the stream.
- * Pinned host memory makes the copies asynchronous up to the final wait. */
+/* Same step (Sections 2.1-2.3) with HOST buffers: copies q, k_new, v_new, x_new and the explicit
+ * list to the device, runs adore_decode_step, copies `out` back and waits for the stream. Pinned
+ * host memory makes the copies asynchronous up to the final wait. `weights` stays a DEVICE pointer
+ * (float[B, H, C+1]) or NULL: the per-slot weights are eight times the size of `out` and are meant
+ * for consumers on the device, so they are emitted there and not copied. */
 adore_status_t adore_decode_step_host(adore_cache_t *cache, int32_t layer, const void *q, const void *k_new,
                                       const void *v_new, const void *x_new, const int32_t *explicit_list,
                                       const int32_t *explicit_count, int32_t r_in, void *out, float *weights);

@@ -130,7 +130,6 @@ struct adore_cache {
   void *h_q = nullptr, *h_k = nullptr, *h_v = nullptr, *h_x = nullptr, *h_out = nullptr;
   int* h_list = nullptr;
   int* h_count = nullptr;
-  float* h_weights = nullptr;
   std::vector<void*> owned;
 };
 
@@ -465,7 +464,7 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   for (void* p : c->owned) cudaFree(p);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
-  void* hosts[] = {c->h_q, c->h_k, c->h_v, c->h_x, c->h_out, c->h_list, c->h_count, c->h_weights};
+  void* hosts[] = {c->h_q, c->h_k, c->h_v, c->h_x, c->h_out, c->h_list, c->h_count};
   for (void* p : hosts) if (p) cudaFree(p);
   cudaGetLastError();
   delete c;
@@ -606,14 +605,12 @@ adore_status_t adore_decode_step_host(adore_cache_t* c, int32_t layer, const voi
   if (!c || !q || !k_new || !v_new || !out) return ADORE_ERR_INVALID_ARG;
   const adore_config_t& f = c->cfg;
   const size_t qb = size_t(f.batch) * f.n_heads * f.head_dim * c->esz, xb = size_t(f.batch) * f.hidden * c->esz;
-  const size_t wb = size_t(f.batch) * f.n_heads * (f.capacity + 1) * sizeof(float);
   if (!c->h_q) {
     CUDA_OK(cudaMalloc(&c->h_q, qb)); CUDA_OK(cudaMalloc(&c->h_k, qb)); CUDA_OK(cudaMalloc(&c->h_v, qb));
     CUDA_OK(cudaMalloc(&c->h_out, qb)); CUDA_OK(cudaMalloc(&c->h_x, xb));
     CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->h_list), size_t(f.batch) * f.max_tokens * sizeof(int)));
     CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->h_count), size_t(f.batch) * sizeof(int)));
   }
-  if (weights && !c->h_weights) CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->h_weights), wb));
   if (r_in < 0 || r_in > f.max_tokens) return ADORE_ERR_INVALID_ARG;
   CUDA_OK(cudaMemcpyAsync(c->h_q, q, qb, cudaMemcpyHostToDevice, c->stream));
   CUDA_OK(cudaMemcpyAsync(c->h_k, k_new, qb, cudaMemcpyHostToDevice, c->stream));
@@ -628,11 +625,9 @@ adore_status_t adore_decode_step_host(adore_cache_t* c, int32_t layer, const voi
     }
   }
   adore_status_t st = adore_decode_step(c, layer, c->h_q, c->h_k, c->h_v, c->h_x, lists ? c->h_list : nullptr,
-                                        lists ? c->h_count : nullptr, lists ? r_in : 0, c->h_out,
-                                        weights ? c->h_weights : nullptr);
+                                        lists ? c->h_count : nullptr, lists ? r_in : 0, c->h_out, weights);
   if (st != ADORE_OK) return st;
   CUDA_OK(cudaMemcpyAsync(out, c->h_out, qb, cudaMemcpyDeviceToHost, c->stream));
-  if (weights) CUDA_OK(cudaMemcpyAsync(weights, c->h_weights, wb, cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(cudaStreamSynchronize(c->stream));
   return ADORE_OK;
 }

@@ -245,10 +245,9 @@ def run_parity(cfg: wl.WorkloadConfig, batch: Optional[int] = None, steps: Optio
                     ho = np.zeros((g.B, cfg.n_heads, cfg.head_dim), np.float32)
                     hq, hk, hv, hx = (to_dev(a, cfg).cpu() for a in (q, k, v, x))
                     hout = torch.zeros((g.B, cfg.n_heads, cfg.head_dim), dtype=torch_dtype(cfg))
-                    hw = torch.zeros((g.B, cfg.n_heads, cfg.capacity + 1), dtype=torch.float32)
                     lib.adore_decode_step_host(g.handle, l, hq, hk, hv, hx, lists if l == 0 else None,
-                                               counts if l == 0 else None, w.r_in if l == 0 else 0, hout, hw)
-                    out_g, w_g = hout.float().numpy(), hw.numpy()
+                                               counts if l == 0 else None, w.r_in if l == 0 else 0, hout, g.weights)
+                    out_g, w_g = hout.float().numpy(), g.weights.cpu().numpy()
                 else:
                     lib.adore_decode_step(g.handle, l, to_dev(q, cfg), to_dev(k, cfg), to_dev(v, cfg), to_dev(x, cfg),
                                           dl if l == 0 else None, dc if l == 0 else None, w.r_in if l == 0 else 0,

