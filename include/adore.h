@@ -184,8 +184,10 @@ int64_t adore_cache_launch_count(const adore_cache_t *cache);
  * runtime split between the controller and the rest). When enabled, every kernel launch of the
  * cache is bracketed by CUDA events on its stream. adore_cache_stage_times waits for the stream,
  * adds up the elapsed milliseconds and launch counts per stage since the last call and resets
- * them. Stage index: 0 attention (+admit), 1 controller + selection, 2 rebuild projection.
- * ms and launches: HOST arrays of 3. Event recording costs a few microseconds per launch, so
+ * them. Stage index: 0 attention (with the fused admit of layers > 0), 1 controller + selection,
+ * 2 rebuild projection (gather + GEMM), 3 the separate admit launch of layer 0.
+ * ms and launches: HOST arrays of 4. While timing is enabled the controller runs on the main
+ * stream instead of beside the attention, so that the stage times add up. Event recording costs a few microseconds per launch, so
  * whole-step throughput should be measured with timing disabled. */
 adore_status_t adore_cache_set_stage_timing(adore_cache_t *cache, int32_t enable);
 adore_status_t adore_cache_stage_times(adore_cache_t *cache, double *ms, int64_t *launches);

@@ -192,9 +192,9 @@ def adore_cache_set_stage_timing(cache: int, enable: bool) -> None:
 
 
 def adore_cache_stage_times(cache: int):
-    """Returns ([ms attention, ms controller+select, ms rebuild], [launch counts]) since the last call."""
-    ms = (C.c_double * 3)()
-    n = (C.c_int64 * 3)()
+    """Returns ([ms attention, controller+select, rebuild, layer-0 admit], [launch counts]) since the last call."""
+    ms = (C.c_double * 4)()
+    n = (C.c_int64 * 4)()
     _check(_lib().adore_cache_stage_times(cache, ms, n), "adore_cache_stage_times")
     return list(ms), list(n)
 

@@ -700,11 +700,7 @@ adore_status_t adore_cache_stage_times(adore_cache_t* c, double* ms, int64_t* la
   }
   c->ev_stage.clear();
   c->ev_used = 0;
-  // the separate admit launch of layer 0 belongs to the attention stage's time, not to its launch count
-  c->stage_ms[0] += c->stage_ms[3];
-  c->stage_ms[3] = 0;
-  c->stage_launches[3] = 0;
-  for (int s = 0; s < 3; ++s) {
+  for (int s = 0; s < 4; ++s) {
     ms[s] = c->stage_ms[s];
     launches[s] = c->stage_launches[s];
     c->stage_ms[s] = 0;
