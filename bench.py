@@ -62,7 +62,35 @@ def measured_peaks():
 
 
 def default_steps(cfg: wl.WorkloadConfig):
-    return {1: 80, 2: 150, 3: 300, 4: 40}.get(cfg_index(cfg), 30)
+    return {1: 80, 2: 150, 3: 300, 4: 40}.get(cfg_index(cfg), 40)
+
+
+def sweep_point(capacity: int, batch: int) -> wl.WorkloadConfig:
+    for cap, b, cfg in wl.sweep_points():
+        if cap == capacity and b == batch:
+            return cfg
+    raise SystemExit(f"no sweep point C={capacity} B={batch}")
+
+
+def run_sweep(args):
+    """Capacity x batch sweep: every point in its own process (a fresh context per point)."""
+    for cap, b, cfg in wl.sweep_points():
+        cmd = [sys.executable, os.path.abspath(__file__), "--config", "5", "--capacity", str(cap), "--batch", str(b),
+               "--no-cpu-baseline", "--no-e2e", "--warmup", str(args.warmup)]
+        if args.steps is not None:
+            cmd += ["--steps", str(args.steps)]
+        res = subprocess.run(cmd, capture_output=True, text=True)
+        if res.returncode != 0:
+            print(json.dumps({"workload": cfg.name, "error": res.stderr.strip().splitlines()[-1:]}), flush=True)
+            continue
+        d = json.loads(res.stdout.strip().splitlines()[-1])
+        st = d["stages"]
+        print(json.dumps({"workload": cfg.name, "capacity": cap, "batch": b, "steps_per_s": d["steps_per_s"],
+                          "tokens_per_s": d["value"], "ms_per_step": d["ms_per_step"],
+                          "attention_hbm_frac": st["attention"]["frac"],
+                          "attention_plus_selection_hbm_frac": st["attention_plus_selection"]["frac"],
+                          "rebuild": {k: st.get("rebuild", {}).get(k) for k in ("bound", "frac", "rows_per_launch", "ms_per_launch")},
+                          "clocks": d["clocks"]}), flush=True)
 
 
 def cfg_index(cfg):
@@ -186,6 +214,13 @@ class DeviceRun:
                 x = x * torch.rsqrt(x.pow(2).mean(-1, keepdim=True) + 1e-5)
             return x.to(self.dt)
 
+        def prompt_rows():          # [B, prompt, d], drawn 256 tokens at a time to bound the fp32 temporary
+            out = torch.empty((B, c.prompt, d), dtype=self.dt, device=dev)
+            for t0 in range(0, c.prompt, 256):
+                t1 = min(c.prompt, t0 + 256)
+                out[:, t0:t1] = rows(B, t1 - t0, d)
+            return out
+
         if c.identity_projection:
             eye = torch.eye(N, device=dev, dtype=self.dt)
             self.w_kv = [torch.cat([eye, eye], 0).contiguous() for _ in range(L)]
@@ -199,12 +234,12 @@ class DeviceRun:
         if c.per_layer_inputs:
             self.tables = [torch.zeros((B, c.max_tokens, d), dtype=self.dt, device=dev) for _ in range(L)]
         if c.prompt:
-            xp = rows(B, c.prompt, d).contiguous()
+            xp = prompt_rows()
             lib.adore_cache_append_tokens(self.handle, xp, c.prompt)
             if c.per_layer_inputs:
                 self.tables[0][:, : c.prompt] = xp
                 for l in range(1, L):
-                    self.tables[l][:, : c.prompt] = rows(B, c.prompt, d)
+                    self.tables[l][:, : c.prompt] = prompt_rows()
                     lib.adore_cache_fill_layer(self.handle, l, self.tables[l])
             del xp
         # per-step inputs
@@ -402,12 +437,20 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=3, help="workload 1..4 (default 3: the largest single-layer config)")
+    ap.add_argument("--config", type=int, default=3,
+                    help="workload 1..4 (default 3: the largest single-layer config); 5 = one point of the capacity x batch "
+                         "sweep, chosen with --capacity and --batch")
+    ap.add_argument("--capacity", type=int, default=512, help="sweep point: C in {128,256,512,1024,2048}")
+    ap.add_argument("--batch", type=int, default=32, help="sweep point: B in {1,8,32,128,256}")
+    ap.add_argument("--sweep", action="store_true", help="run all 25 sweep points, one short JSON line each")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
-    cfg = wl.get_config(args.config)
+    if args.sweep:
+        run_sweep(args)
+        return
+    cfg = sweep_point(args.capacity, args.batch) if args.config == 5 else wl.get_config(args.config)
     if args.steps is None:
         args.steps = default_steps(cfg) if args.impl == "ours" else 3
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
