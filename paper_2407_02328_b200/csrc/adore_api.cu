@@ -10,6 +10,7 @@
 #include "../../include/adore.h"
 #include "attention.cuh"
 #include "attention_tma.cuh"
+#include "attention_split.cuh"
 #include "controller.cuh"
 #include "rebuild_simt.cuh"
 #include "rebuild_tc.cuh"
@@ -19,12 +20,12 @@ using namespace adore;
 
 namespace {
 
-constexpr int kSelectThreadsSmall = 512;
 constexpr int kMaxPrefillRows = 8192;       // controller rows per chunk during a bulk load
 
 // ---- kernels that glue the device functions together -----------------------------------------
 template <typename T>
-__global__ void ctrl_select_kernel(const RecurParams rp, const SelectParams sp, const T* x_new, T* x_store, int d) {
+__global__ void __launch_bounds__(512) ctrl_select_kernel(const RecurParams rp, const SelectParams sp, const T* x_new, T* x_store, int d,
+                                                          int resident) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int b = blockIdx.x;
   // keep the new token's layer-input row: it is what a later rebuild recomputes from
@@ -33,17 +34,19 @@ __global__ void ctrl_select_kernel(const RecurParams rp, const SelectParams sp, 
     uint4* dst = reinterpret_cast<uint4*>(x_store + (size_t(b) * sp.max_tokens + sp.n) * d);
     for (int i = threadIdx.x; i < int(d * sizeof(T) / 16); i += blockDim.x) dst[i] = src[i];
   }
-  controller_tokens(rp, b, reinterpret_cast<double*>(smem));
+  if (resident) controller_tokens_resident(rp, b, smem, sp.err);
+  else controller_tokens(rp, b, reinterpret_cast<double*>(smem));
   __syncthreads();
   select_step(sp, smem);
 }
 
-__global__ void ctrl_recur_kernel(const RecurParams rp) {
+__global__ void __launch_bounds__(512) ctrl_recur_kernel(const RecurParams rp, int resident, unsigned* err) {
   extern __shared__ __align__(128) unsigned char smem[];
-  controller_tokens(rp, blockIdx.x, reinterpret_cast<double*>(smem));
+  if (resident) controller_tokens_resident(rp, blockIdx.x, smem, err);
+  else controller_tokens(rp, blockIdx.x, reinterpret_cast<double*>(smem));
 }
 
-__global__ void bulk_select_kernel(const SelectParams sp) {
+__global__ void __launch_bounds__(512) bulk_select_kernel(const SelectParams sp) {
   extern __shared__ __align__(128) unsigned char smem[];
   select_bulk(sp, smem);
 }
@@ -104,6 +107,7 @@ struct adore_cache {
   int* frow_slot = nullptr;
   int* frow_total = nullptr;
   unsigned long long* rows_accum = nullptr;
+  int sms = 148;
   unsigned* err = nullptr;
   // optional per-stage timing
   bool timing = false;
@@ -195,7 +199,13 @@ adore_status_t fill_i32(adore_cache* c, int* p, int v, size_t n) {
   return ADORE_OK;
 }
 
-int select_threads(const adore_cache* c) { return 3 * c->cfg.ctrl_hidden <= kSelectThreadsSmall ? kSelectThreadsSmall : 1024; }
+// One CTA per sequence owns an SM for a latency-bound chain (GRU, MLP, sort): the more warps, the better
+// the loads and barriers are hidden.
+int select_threads(const adore_cache*) { return 512; }
+size_t ctrl_smem(const adore_cache* c) {
+  const int h = c->cfg.ctrl_hidden;
+  return ctrl_resident_ok(h) ? ctrl_resident_smem_bytes(h) : recur_smem_bytes(h);
+}
 
 RecurParams recur_params(adore_cache* c, int rows, int tc, int ksplit, int n0) {
   RecurParams r{};
@@ -252,7 +262,10 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
   cudaError_t e;
   // ADORE_ATTN_DIRECT=1 selects the variant without shared-memory staging (for A/B timing)
   static const bool direct = std::getenv("ADORE_ATTN_DIRECT") != nullptr;
-  if (!direct && attn_tma_usable<T>(f.capacity, f.head_dim)) e = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
+  // few (b, h) pairs: a cluster of CTAs shares each of them
+  const int split = direct ? 1 : attn_split_factor(grid, f.capacity, c->sms);
+  if (split > 1) e = launch_attention_split<T>(p, f.head_dim, grid, split, c->stream);
+  else if (!direct && attn_tma_usable<T>(f.capacity, f.head_dim)) e = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
   else if (f.head_dim == 64) {
     const size_t smem = attn_smem_bytes(f.capacity, 64);
     attention_kernel<T, 64><<<grid, kAttnThreads, smem, c->stream>>>(p);
@@ -398,6 +411,10 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   TRY(dev_alloc(c, &c->frow_slot, B * C * sizeof(int), true));
   TRY(dev_alloc(c, &c->frow_total, sizeof(int), true));
   TRY(dev_alloc(c, &c->rows_accum, sizeof(unsigned long long), true));
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, dev);
+  }
   TRY(dev_alloc(c, &c->err, sizeof(unsigned), true));
   // decode splits the d-long dot products so that roughly one wave of CTAs is busy
   {
@@ -434,7 +451,8 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   }
   // opt in to large dynamic shared memory where a kernel may need it
   {
-    const int big = 200 * 1024;
+    const int big = 227 * 1024;
+    cudaFuncSetAttribute(ctrl_recur_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     cudaFuncSetAttribute(ctrl_select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     cudaFuncSetAttribute(ctrl_select_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     cudaFuncSetAttribute(bulk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
@@ -499,7 +517,7 @@ adore_status_t adore_cache_append_tokens(adore_cache_t* c, const void* x, int32_
                                        f.max_tokens, tc, 1, c->stream);
     if (st != ADORE_OK) return st;
     RecurParams rp = recur_params(c, f.batch * tc, tc, 1, t0);
-    ctrl_recur_kernel<<<f.batch, select_threads(c), recur_smem_bytes(f.ctrl_hidden), c->stream>>>(rp);
+    ctrl_recur_kernel<<<f.batch, select_threads(c), ctrl_smem(c), c->stream>>>(rp, ctrl_resident_ok(f.ctrl_hidden) ? 1 : 0, c->err);
     ++c->launches;
     CUDA_OK(cudaGetLastError());
   }
@@ -560,13 +578,14 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
       sp.explicit_list = ex && r_in > 0 ? explicit_list : nullptr;
       sp.explicit_count = ex && r_in > 0 ? explicit_count : nullptr;
       sp.r_in = r_in;
-      const size_t smem = std::max(select_smem_bytes(f.capacity, P), recur_smem_bytes(f.ctrl_hidden));
+      const size_t smem = std::max(select_smem_bytes(f.capacity, P), ctrl_smem(c));
+      const int resident = ctrl_resident_ok(f.ctrl_hidden) ? 1 : 0;
       if (f.dtype == ADORE_F32)
         ctrl_select_kernel<float><<<f.batch, select_threads(c), smem, side>>>(
-            rp, sp, static_cast<const float*>(x_new), static_cast<float*>(c->x_store), f.hidden);
+            rp, sp, static_cast<const float*>(x_new), static_cast<float*>(c->x_store), f.hidden, resident);
       else
         ctrl_select_kernel<__nv_bfloat16><<<f.batch, select_threads(c), smem, side>>>(
-            rp, sp, static_cast<const __nv_bfloat16*>(x_new), static_cast<__nv_bfloat16*>(c->x_store), f.hidden);
+            rp, sp, static_cast<const __nv_bfloat16*>(x_new), static_cast<__nv_bfloat16*>(c->x_store), f.hidden, resident);
       ++c->launches;
       CUDA_OK(cudaGetLastError());
       st = launch_row_table(c, true, side);

@@ -195,11 +195,11 @@ __device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p
   return n_kept;
 }
 
-// Phase 4 with direct loads: adds w_s * V[s] of the kept rows into acc (this lane's 16-byte column
+// Phase 4 with direct loads: adds w_s * V[s] of the kept rows [j_begin, n_kept) of the list into acc (this lane's 16-byte column
 // slice; lanes of different row groups and warps hold partial sums).
 template <typename T, int DH>
 __device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh, int n_kept,
-                                                        float (&acc)[Elem<T>::kPer16B]) {
+                                                        float (&acc)[Elem<T>::kPer16B], int j_begin = 0) {
   constexpr int NT = kAttnThreads;
   constexpr int NW = NT / 32;
   constexpr int EPL = Elem<T>::kPer16B;
@@ -221,7 +221,7 @@ __device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, 
   (void)NW; (void)RPW; (void)U; (void)s_logit; (void)s_list; (void)s_red; (void)warp; (void)sub; (void)li; (void)b;
   (void)Kb; (void)Vb; (void)knew; (void)vnew;
   // ---- phase 4: weighted sum of the kept value rows ----------------------------------------
-  for (int j0 = warp * RPW; j0 < n_kept; j0 += NW * RPW * U) {
+  for (int j0 = j_begin + warp * RPW; j0 < n_kept; j0 += NW * RPW * U) {   // entries [j_begin, n_kept) of the kept list
     uint4 vv[U];
     float wv[U];
 #pragma unroll

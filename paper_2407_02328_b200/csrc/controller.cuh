@@ -11,6 +11,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "mbarrier.cuh"
 
 namespace adore {
 
@@ -136,7 +137,6 @@ struct RecurParams {
   double pos_scale;
 };
 
-constexpr int kCtrlJ = 8;          // ceil(max d' / 32): inner-index elements per lane
 
 // Shared memory needed by controller_tokens: 7*h + 32 doubles.
 __host__ __device__ inline size_t recur_smem_bytes(int h) { return sizeof(double) * (7 * h + 32); }
@@ -145,7 +145,8 @@ __host__ __device__ inline size_t recur_smem_bytes(int h) { return sizeof(double
 // All threads of the block must call it. Every matrix-vector product is spread over the whole
 // block: a warp owns an output row, its lanes split the inner index (coalesced loads that are all
 // in flight at once) and a shuffle tree adds the lane partials, in a fixed order.
-__device__ inline void controller_tokens(const RecurParams& p, int b, double* sm) {
+template <int kCtrlJ>               // inner-index elements per lane: ceil(d' / 32) rounded up to 4 or 8
+__device__ __forceinline__ void controller_tokens_impl(const RecurParams& p, int b, double* sm) {
   const int h = p.h, G = 3 * h, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
   double* s_z = sm;            // [h]
   double* s_gi = sm + h;       // [3h]  reset/update: input + hidden side; candidate: input side
@@ -243,6 +244,175 @@ __device__ inline void controller_tokens(const RecurParams& p, int b, double* sm
     __syncthreads();
   }
   if (tid < h) p.z[size_t(b) * h + tid] = s_z[tid];
+}
+
+// ---- variant with the recurrent matrix resident in shared memory ---------------------------------
+// For d' <= 128 (and a multiple of 4) the whole recurrent matrix (3 d' x d' floats, 192 KB at d' = 128)
+// fits in shared memory: one elected thread fetches it with bulk copies while the other parameters
+// are loaded, the interaction matrix lives in registers (each warp owns d'/16 of its rows), and
+// every token then costs only shared-memory reads. This is what makes a long prompt scan cheap and
+// takes the weight-load latency off the decode step.
+constexpr int kCtrlWarps = 16;                 // the resident variant runs with 512 threads
+
+__host__ __device__ inline bool ctrl_resident_ok(int h) { return h <= 128 && h % 4 == 0; }
+// shared memory: matrix | 13h doubles (state, gate sums, input sums) | 8h floats (small vectors) | barrier
+__host__ __device__ inline size_t ctrl_resident_smem_bytes(int h) {
+  return size_t(3) * h * h * sizeof(float) + sizeof(double) * (13 * h + 32) + sizeof(float) * 8 * h + 16;
+}
+
+__device__ __forceinline__ void controller_tokens_resident(const RecurParams& p, int b, unsigned char* smem, unsigned* err) {
+  const int h = p.h, G = 3 * h, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float* s_w = reinterpret_cast<float*>(smem);                    // [3h][h]
+  double* sd = reinterpret_cast<double*>(smem + size_t(G) * h * sizeof(float));
+  double* s_z = sd;             // [h]
+  double* s_gi = sd + h;        // [3h]
+  double* s_gh = sd + 4 * h;    // [h]
+  double* s_pz = sd + 5 * h;    // [h]
+  double* s_t = sd + 6 * h;     // [h]
+  double* s_gin = sd + 7 * h;   // [3h] input-side sums (+ bias) of the current token
+  float* sf = reinterpret_cast<float*>(sd + 13 * h + 32);
+  float* s_bhh = sf;            // [3h]
+  float* s_posw = sf + 3 * h;   // [h]
+  float* s_posb = sf + 4 * h;   // [h]
+  float* s_b1 = sf + 5 * h;     // [h]
+  float* s_w2 = sf + 6 * h;     // [h]
+  uint64_t* bar = reinterpret_cast<uint64_t*>(sf + 8 * h);
+
+  if (tid == 0) {
+    mbar_init(bar, 1u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    const uint32_t total = uint32_t(G) * h * sizeof(float);
+    mbar_expect_tx(bar, total);
+    for (uint32_t off = 0; off < total; off += 65536u)
+      bulk_g2s(smem + off, reinterpret_cast<const unsigned char*>(p.w_hh) + off, min(65536u, total - off), bar);
+  }
+  // the interaction matrix in registers: warp w owns rows w*RW .. w*RW+RW-1, lane l columns l, l+32, ...
+  constexpr int RW = 8, JN = 4;
+  const int rw = (h + kCtrlWarps - 1) / kCtrlWarps;               // rows per warp actually used (<= RW)
+  float w1r[RW][JN];
+#pragma unroll
+  for (int a = 0; a < RW; ++a) {
+    const int i = warp * rw + a;
+#pragma unroll
+    for (int jj = 0; jj < JN; ++jj) {
+      const int j = lane + 32 * jj;
+      w1r[a][jj] = (a < rw && i < h && j < h) ? __ldg(p.w1 + size_t(i) * h + j) : 0.f;
+    }
+  }
+  for (int i = tid; i < G; i += blockDim.x) s_bhh[i] = p.b_hh[i];
+  for (int i = tid; i < h; i += blockDim.x) {
+    s_posw[i] = p.pos_w[i]; s_posb[i] = p.pos_b[i]; s_b1[i] = p.b1[i]; s_w2[i] = p.w2[i];
+    s_z[i] = p.z[size_t(b) * h + i];
+  }
+  const float b2 = __ldg(p.b2);
+  __syncthreads();
+  bool have_w = false;
+  for (int t = 0; t < p.tc; ++t) {
+    const int row = b * p.tc + t;
+    // input-side sums: the k-slices are added in a fixed order
+    for (int g = tid; g < G; g += blockDim.x) {
+      double gi = double(__ldg(p.b_ih + g));
+#pragma unroll 4
+      for (int ks = 0; ks < p.ksplit; ++ks) gi += p.part[(size_t(ks) * p.rows + row) * G + g];
+      s_gin[g] = gi;
+    }
+    if (!have_w) {                                  // first token: the matrix must have landed
+      if (!mbar_wait_bounded(bar, 0u, kWaitPolls) && tid == 0) set_error(err, ERRW_TIMEOUT);
+      have_w = true;
+    }
+    __syncthreads();
+    // recurrent half: a warp per gate row, a lane per four columns
+    {
+      double z4[4] = {0.0, 0.0, 0.0, 0.0};
+      const int j0 = lane * 4;
+      if (j0 < h) { z4[0] = s_z[j0]; z4[1] = s_z[j0 + 1]; z4[2] = s_z[j0 + 2]; z4[3] = s_z[j0 + 3]; }
+      // eight rows at a time, so that their shuffle reductions overlap instead of queueing up
+      for (int gb = warp; gb < G; gb += kCtrlWarps * 8) {
+        double acc[8];
+#pragma unroll
+        for (int a = 0; a < 8; ++a) {
+          const int g = gb + a * kCtrlWarps;
+          acc[a] = 0.0;
+          if (g < G && j0 < h) {
+            const float4 w4 = *reinterpret_cast<const float4*>(s_w + size_t(g) * h + j0);
+            acc[a] = fma(double(w4.x), z4[0], acc[a]);
+            acc[a] = fma(double(w4.y), z4[1], acc[a]);
+            acc[a] = fma(double(w4.z), z4[2], acc[a]);
+            acc[a] = fma(double(w4.w), z4[3], acc[a]);
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+          for (int a = 0; a < 8; ++a) acc[a] += __shfl_xor_sync(0xffffffffu, acc[a], o);
+        if (lane == 0) {
+#pragma unroll
+          for (int a = 0; a < 8; ++a) {
+            const int g = gb + a * kCtrlWarps;
+            if (g < G) {
+              const double gh = acc[a] + double(s_bhh[g]);
+              if (g < 2 * h) s_gi[g] = s_gin[g] + gh;
+              else { s_gi[g] = s_gin[g]; s_gh[g - 2 * h] = gh; }
+            }
+          }
+        }
+      }
+    }
+    __syncthreads();
+    const int pos = p.n0 + t;
+    if (tid < h) {
+      const double r = 1.0 / (1.0 + exp(-s_gi[tid]));
+      const double u = 1.0 / (1.0 + exp(-s_gi[h + tid]));
+      const double c = tanh(s_gi[2 * h + tid] + r * s_gh[tid]);
+      const double zn = (1.0 - u) * c + u * s_z[tid];
+      s_z[tid] = zn;
+      s_pz[tid] = double(s_posw[tid]) * (double(pos) / p.pos_scale) + double(s_posb[tid]) + zn;
+    }
+    __syncthreads();
+    {
+      double pz[JN];
+#pragma unroll
+      for (int jj = 0; jj < JN; ++jj) pz[jj] = (lane + 32 * jj < h) ? s_pz[lane + 32 * jj] : 0.0;
+      double acc[RW];
+#pragma unroll
+      for (int a = 0; a < RW; ++a) {
+        acc[a] = 0.0;
+#pragma unroll
+        for (int jj = 0; jj < JN; ++jj) acc[a] = fma(double(w1r[a][jj]), pz[jj], acc[a]);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int a = 0; a < RW; ++a) acc[a] += __shfl_xor_sync(0xffffffffu, acc[a], o);
+      // the tanh of the eight rows is spread over eight lanes
+      if (lane < RW) {
+        double mine = acc[0];
+#pragma unroll
+        for (int a = 1; a < RW; ++a) if (lane == a) mine = acc[a];
+        const int i = warp * rw + lane;
+        if (lane < rw && i < h) s_t[i] = double(s_w2[i]) * tanh(mine + double(s_b1[i]));
+      }
+    }
+    __syncthreads();
+    if (warp == 0) {
+      double acc = 0.0;
+      for (int i = lane; i < h; i += 32) acc += s_t[i];
+      acc = warp_sum(acc);
+      if (lane == 0) {
+        const double sc = acc + double(b2);
+        p.score[size_t(b) * p.max_tokens + pos] = float(sc);
+        p.sigma[size_t(b) * p.max_tokens + pos] = float(1.0 / (1.0 + exp(-sc)));
+      }
+    }
+    __syncthreads();
+  }
+  if (tid < h) p.z[size_t(b) * h + tid] = s_z[tid];
+}
+
+__device__ inline void controller_tokens(const RecurParams& p, int b, double* sm) {
+  if (p.h <= 128) controller_tokens_impl<4>(p, b, sm);
+  else controller_tokens_impl<8>(p, b, sm);
 }
 
 }  // namespace adore

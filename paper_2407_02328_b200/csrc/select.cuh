@@ -54,32 +54,104 @@ __device__ __forceinline__ int block_rank(bool flag, int* tmp, int* total) {
   return base + __popc(bal & ((1u << lane) - 1u));
 }
 
-// Sorts keys[0..P) in DESCENDING order; P is a power of two. All threads of the block call it.
-// Each warp owns a contiguous block of E >= 64 keys; compare-exchange stages whose partners are at
-// most E/2 apart stay inside one warp's block and need only a warp barrier.
-__device__ inline void bitonic_sort_desc(unsigned long long* keys, int P) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
-  const int E = (P >= 64 * nw) ? P / nw : (P >= 64 ? 64 : P);
-  const int active = P / E;                       // warps that own keys
-  bool prev_block_wide = true;                    // the keys were written by arbitrary threads
+// ---- bitonic sort, DESCENDING, P a power of two -------------------------------------------------
+// Each warp owns a contiguous block of E = 32*R keys and keeps them in registers (R per lane, key
+// x = base + 32*r + lane). Compare-exchange stages whose partners are less than E apart never leave
+// the warp: a distance below 32 is a shuffle, a distance of 32 or more is another register of the same
+// lane. Only the stages that cross warps go through shared memory, one block barrier each.
+template <int R>
+__device__ __forceinline__ void bitonic_warp_run(unsigned long long (&v)[R], int base, int lane, int k, int j_start) {
+#pragma unroll
+  for (int sft = 9; sft >= 0; --sft) {               // j = 512 .. 1, compile-time after unrolling
+    const int j = 1 << sft;
+    if (j >= 32 * R || j > j_start) continue;
+    if (j >= 32) {
+      const int dr = j >> 5;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if ((r & dr) == 0) {
+          const bool desc = ((base + r * 32 + lane) & k) == 0;
+          const unsigned long long a = v[r], c = v[r | dr];
+          if (desc ? (a < c) : (a > c)) { v[r] = c; v[r | dr] = a; }
+        }
+      }
+    } else {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, v[r], j);
+        const bool desc = ((base + r * 32 + lane) & k) == 0;
+        const bool take_max = ((lane & j) == 0) == desc;
+        const unsigned long long hi = v[r] > other ? v[r] : other, lo = v[r] > other ? other : v[r];
+        v[r] = take_max ? hi : lo;
+      }
+    }
+  }
+}
+
+template <int R>
+__device__ __forceinline__ void bitonic_sort_desc_regs(unsigned long long* keys, int P) {
+  constexpr int E = 32 * R;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const bool active = warp < P / E;
+  const int base = warp * E;
+  unsigned long long v[R];
+  __syncthreads();                                    // the keys were written by arbitrary threads
+#pragma unroll
+  for (int r = 0; r < R; ++r) v[r] = active ? keys[base + r * 32 + lane] : 0ull;
+  for (int k = 2; k <= E; k <<= 1) bitonic_warp_run<R>(v, base, lane, k, k >> 1);
+  for (int k = 2 * E; k <= P; k <<= 1) {
+    if (active) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) keys[base + r * 32 + lane] = v[r];
+    }
+    __syncthreads();
+    for (int j = k >> 1; j >= E; j >>= 1) {           // partners in other warps' blocks
+      for (int t = threadIdx.x; t < (P >> 1); t += blockDim.x) {
+        const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+        const int l = i | j;
+        const unsigned long long a = keys[i], c = keys[l];
+        const bool desc = (i & k) == 0;
+        if (desc ? (a < c) : (a > c)) { keys[i] = c; keys[l] = a; }
+      }
+      __syncthreads();
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) v[r] = active ? keys[base + r * 32 + lane] : 0ull;
+    bitonic_warp_run<R>(v, base, lane, k, E >> 1);
+  }
+  if (active) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) keys[base + r * 32 + lane] = v[r];
+  }
+  __syncthreads();
+}
+
+// Small inputs (P < 64): everything in shared memory.
+__device__ inline void bitonic_sort_desc_small(unsigned long long* keys, int P) {
   for (int k = 2; k <= P; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
-      const bool block_wide = 2 * j > E;
-      if (block_wide || prev_block_wide) __syncthreads(); else __syncwarp();
-      prev_block_wide = block_wide;
-      if (warp < active) {
-        for (int q = lane; q < (E >> 1); q += 32) {
-          const int t = warp * (E >> 1) + q;
-          const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // lower index of the pair
-          const int l = i | j;
-          const unsigned long long a = keys[i], c = keys[l];
-          const bool desc = (i & k) == 0;
-          if (desc ? (a < c) : (a > c)) { keys[i] = c; keys[l] = a; }
-        }
+      __syncthreads();
+      for (int t = threadIdx.x; t < (P >> 1); t += blockDim.x) {
+        const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+        const int l = i | j;
+        const unsigned long long a = keys[i], c = keys[l];
+        const bool desc = (i & k) == 0;
+        if (desc ? (a < c) : (a > c)) { keys[i] = c; keys[l] = a; }
       }
     }
   }
   __syncthreads();
+}
+
+// All threads of the block call it; blockDim.x a multiple of 32; P <= 512 * (blockDim.x / 32).
+__device__ inline void bitonic_sort_desc(unsigned long long* keys, int P) {
+  const int nw = blockDim.x >> 5;
+  if (P < 64) { bitonic_sort_desc_small(keys, P); return; }
+  const int E = max(64, P / nw);                      // keys per warp
+  if (E == 64) bitonic_sort_desc_regs<2>(keys, P);
+  else if (E == 128) bitonic_sort_desc_regs<4>(keys, P);
+  else if (E == 256) bitonic_sort_desc_regs<8>(keys, P);
+  else bitonic_sort_desc_regs<16>(keys, P);
 }
 
 struct SelectParams {
