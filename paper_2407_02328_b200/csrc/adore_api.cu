@@ -262,8 +262,10 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
   cudaError_t e;
   // ADORE_ATTN_DIRECT=1 selects the variant without shared-memory staging (for A/B timing)
   static const bool direct = std::getenv("ADORE_ATTN_DIRECT") != nullptr;
-  // few (b, h) pairs: a cluster of CTAs shares each of them
-  const int split = direct ? 1 : attn_split_factor(grid, f.capacity, c->sms);
+  // Few (b, h) pairs: a cluster of CTAs shares each of them. Not at layer 0: there the controller's
+  // one-CTA-per-sequence kernel (200 KB of shared memory each) runs beside the attention and needs
+  // SMs that the extra CTAs would occupy; measured at batch 1 the step got slower, not faster.
+  const int split = (direct || layer == 0) ? 1 : attn_split_factor(grid, f.capacity, c->sms);
   if (split > 1) e = launch_attention_split<T>(p, f.head_dim, grid, split, c->stream);
   else if (!direct && attn_tma_usable<T>(f.capacity, f.head_dim)) e = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
   else if (f.head_dim == 64) {

@@ -70,12 +70,14 @@ def test_capacity_spanning_several_tiles_with_ragged_tail():
 
 
 def test_split_slot_clusters_for_few_heads():
-    """Few (b, h) pairs: 2, 4 or 8 CTAs of a cluster share one pair's slots (ragged slices, bf16 and fp32)."""
-    _run(SMALL.scaled(name="split8", batch=1, n_heads=4, capacity=300, topk=100, rebuild_max=20, prompt=400, steps=10, seed=112))
+    """Few (b, h) pairs: in the layers after the first, 2, 4 or 8 CTAs of a cluster share one pair's slots
+    (ragged slices, bf16 and fp32)."""
+    two = dict(n_layers=2, per_layer_inputs=True)
+    _run(SMALL.scaled(name="split8", batch=1, n_heads=4, capacity=300, topk=100, rebuild_max=20, prompt=400, steps=10, seed=112, **two))
     _run(SMALL.scaled(name="split4_f32", dtype="f32", batch=1, n_heads=2, hidden=128, capacity=131, topk=50, rebuild_max=9,
-                      prompt=0, steps=150, seed=113))
+                      prompt=0, steps=150, seed=113, **two))
     _run(SMALL.scaled(name="split2_dh64", head_dim=64, batch=2, n_heads=3, hidden=192, capacity=70, topk=70, rebuild_max=5,
-                      prompt=90, steps=10, seed=114))
+                      prompt=90, steps=10, seed=114, **two))
 
 
 def test_config2_sub_batch():
