@@ -127,6 +127,9 @@ struct adore_cache {
   // side stream: the controller and the selection run beside the attention of layer 0
   cudaStream_t aux = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  // uploads of the host-buffer entry point run on their own stream, beside the previous rebuild
+  cudaStream_t copy = nullptr;
+  cudaEvent_t ev_copy = nullptr;
   bool joined = true;
   std::vector<const void*> w_kv;
   TcState tc;                   // tensor-core rebuild path (tensor maps, gather buffer)
@@ -462,7 +465,9 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   }
   if (cudaStreamCreateWithFlags(&c->aux, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+      cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_copy, cudaEventDisableTiming) != cudaSuccess) {
     adore_cache_destroy(c);
     return ADORE_ERR_CUDA;
   }
@@ -480,6 +485,8 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (!c) return ADORE_OK;
   cudaStreamSynchronize(c->stream);
   if (c->aux) { cudaStreamSynchronize(c->aux); cudaStreamDestroy(c->aux); }
+  if (c->copy) { cudaStreamSynchronize(c->copy); cudaStreamDestroy(c->copy); }
+  if (c->ev_copy) cudaEventDestroy(c->ev_copy);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   for (void* p : c->owned) cudaFree(p);
@@ -633,18 +640,22 @@ adore_status_t adore_decode_step_host(adore_cache_t* c, int32_t layer, const voi
     CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->h_count), size_t(f.batch) * sizeof(int)));
   }
   if (r_in < 0 || r_in > f.max_tokens) return ADORE_ERR_INVALID_ARG;
-  CUDA_OK(cudaMemcpyAsync(c->h_q, q, qb, cudaMemcpyHostToDevice, c->stream));
-  CUDA_OK(cudaMemcpyAsync(c->h_k, k_new, qb, cudaMemcpyHostToDevice, c->stream));
-  CUDA_OK(cudaMemcpyAsync(c->h_v, v_new, qb, cudaMemcpyHostToDevice, c->stream));
+  // The staging buffers are free (the previous call waited for every kernel that read them), so the
+  // uploads need not queue behind the rebuild that may still be running on the main stream.
+  CUDA_OK(cudaMemcpyAsync(c->h_q, q, qb, cudaMemcpyHostToDevice, c->copy));
+  CUDA_OK(cudaMemcpyAsync(c->h_k, k_new, qb, cudaMemcpyHostToDevice, c->copy));
+  CUDA_OK(cudaMemcpyAsync(c->h_v, v_new, qb, cudaMemcpyHostToDevice, c->copy));
   const bool lists = layer == 0 && explicit_list && explicit_count && r_in > 0;
   if (layer == 0) {
     if (!x_new) return ADORE_ERR_INVALID_ARG;
-    CUDA_OK(cudaMemcpyAsync(c->h_x, x_new, xb, cudaMemcpyHostToDevice, c->stream));
+    CUDA_OK(cudaMemcpyAsync(c->h_x, x_new, xb, cudaMemcpyHostToDevice, c->copy));
     if (lists) {
-      CUDA_OK(cudaMemcpyAsync(c->h_list, explicit_list, size_t(f.batch) * r_in * sizeof(int), cudaMemcpyHostToDevice, c->stream));
-      CUDA_OK(cudaMemcpyAsync(c->h_count, explicit_count, size_t(f.batch) * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+      CUDA_OK(cudaMemcpyAsync(c->h_list, explicit_list, size_t(f.batch) * r_in * sizeof(int), cudaMemcpyHostToDevice, c->copy));
+      CUDA_OK(cudaMemcpyAsync(c->h_count, explicit_count, size_t(f.batch) * sizeof(int), cudaMemcpyHostToDevice, c->copy));
     }
   }
+  CUDA_OK(cudaEventRecord(c->ev_copy, c->copy));
+  CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_copy, 0));
   adore_status_t st = adore_decode_step(c, layer, c->h_q, c->h_k, c->h_v, c->h_x, lists ? c->h_list : nullptr,
                                         lists ? c->h_count : nullptr, lists ? r_in : 0, c->h_out, weights);
   if (st != ADORE_OK) return st;

@@ -95,3 +95,10 @@ def test_config4_shapes_two_layers_full_batch():
     """Config 4's batch, capacity, top-K and prompt with two of its 32 layers (the oracle's float64
     projection of all 32 would take an hour); layers only share the slot map, so two cover the path."""
     _run(wl.get_config(4).scaled(name="cfg4_two_layers", n_layers=2), steps=2)
+
+
+def test_controller_widths_off_the_default():
+    """d' = 160 takes the controller path that streams its matrices from global memory, d' = 96 the
+    shared-memory-resident one with partly filled warps."""
+    _run(SMALL.scaled(name="ctrl160", ctrl_hidden=160, steps=25, seed=115))
+    _run(SMALL.scaled(name="ctrl96", ctrl_hidden=96, steps=25, seed=116))
