@@ -432,6 +432,33 @@ def rebuild_flops_bytes_per_launch(cfg, rows: float):
     return flops, bytes_
 
 
+def probe_pattern_ceiling(run, flush):
+    """Times a plain read kernel on the layer-0 cache with the attention's two access patterns: all key
+    blocks streamed, then `topk` of the C value rows of every (b, h) gathered. Returns GB/s of each."""
+    import torch
+    lib, c = run.lib, run.cfg
+    kptr, vptr = lib.adore_cache_kv(run.handle, 0)
+    n_blocks, row_bytes = c.batch * c.n_heads, c.head_dim * c.elem_bytes
+    sink = torch.zeros(4, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    out = {}
+    for name, ptr, kept, gather in (("stream", kptr, c.capacity, False), ("gather", vptr, min(c.topk, c.capacity), True)):
+        best = None
+        for _ in range(5):
+            if flush is not None:
+                flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            lib.adore_probe_read_bandwidth(ptr, n_blocks, c.capacity, row_bytes, kept, gather, 148 * 8, sink, stream)
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b)
+            best = ms if best is None else min(best, ms)
+        out[name + "_gbs"] = n_blocks * kept * row_bytes / (best * 1e-3) / 1e9
+        out[name + "_us"] = best * 1e3
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -550,6 +577,8 @@ def main():
     lib.adore_cache_sync_status(run.handle)
     clocks = sampler.stop(t_clock0, time.time()) if sampler else None
 
+    ceiling = probe_pattern_ceiling(run, flush)
+
     peaks, peak_kind = measured_peaks()
     occ = min(cfg.capacity, cfg.retained_max + rows / cfg.batch)
     att_ms = st_ms[0] / max(st_n[0], 1)
@@ -603,6 +632,10 @@ def main():
                 "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
                 "config": workload_desc(cfg), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
                 "roofline": roofline, "stages": stages, "cpu_baseline": cpu}
+        # the plain read kernel's time for the same bytes: what the access pattern allows on this GPU
+        ideal_us = ceiling["stream_us"] + ceiling["gather_us"]
+        line["attention_pattern_ceiling"] = dict(ceiling, ideal_us=ideal_us, kernel_us=att_ms * 1e3,
+                                                 kernel_over_ideal=att_ms * 1e3 / ideal_us if ideal_us > 0 else None)
         print(json.dumps(line))
     run.close()
     if world > 1:

@@ -196,6 +196,17 @@ adore_status_t adore_cache_stage_times(adore_cache_t *cache, double *ms, int64_t
  * of the rebuild-list lengths); waits for the stream. rows: HOST pointer. */
 adore_status_t adore_cache_rebuild_rows(adore_cache_t *cache, int64_t *rows);
 
+/* Measurement aid (no counterpart in the paper): reads `buffer`, laid out as n_blocks blocks of
+ * block_rows rows of row_bytes (128, 256 or 512) bytes, with plain 16-byte loads and `ctas` CTAs of
+ * 256 threads. gather == 0 streams every block whole (the key pass of the attention);
+ * gather != 0 reads kept_rows rows per block, spread over the block with a pseudo-random jitter
+ * (the kept value rows of a top-K mask). Nothing is written except possibly 4 bytes at scratch4
+ * (device). The caller times the launch on cuda_stream; bytes read = n_blocks * rows * row_bytes.
+ * buffer: DEVICE pointer, 16-byte aligned. Errors: INVALID_ARG, CUDA. */
+adore_status_t adore_probe_read_bandwidth(const void *buffer, int32_t n_blocks, int32_t block_rows,
+                                          int32_t row_bytes, int32_t kept_rows, int32_t gather,
+                                          int32_t ctas, void *scratch4, void *cuda_stream);
+
 /* Controller scoring for callers that cannot allocate device memory. (The paper has no
  * counterpart: this is a packaging of its controller, Section 2.2 Eq. 2, for a constrained
  * caller.) Some users of this library run where cudaMalloc is off limits: a scheduler thread

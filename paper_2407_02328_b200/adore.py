@@ -49,7 +49,7 @@ EXPORTS = ["adore_cache_create", "adore_cache_destroy", "adore_cache_set_project
            "adore_cache_step_info", "adore_cache_scores", "adore_cache_kv", "adore_cache_num_tokens",
            "adore_cache_launch_count", "adore_cache_sync_status", "adore_status_string",
            "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows",
-           "adore_controller_score_static"]
+           "adore_controller_score_static", "adore_probe_read_bandwidth"]
 
 
 def _lib():
@@ -83,6 +83,7 @@ def _lib():
         lib.adore_cache_set_stage_timing.argtypes = [vp, i32]
         lib.adore_cache_stage_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         lib.adore_cache_rebuild_rows.argtypes = [vp, C.POINTER(C.c_int64)]
+        lib.adore_probe_read_bandwidth.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp]
         lib.adore_controller_score_static.argtypes = [C.POINTER(adore_controller_weights_t), C.c_int, i32, i32, i32, vp, vp,
                                                       i32, C.c_float, vp, vp, vp]
         _LIB = lib
@@ -213,6 +214,12 @@ def adore_controller_score_static(weights_dev: Dict[str, object], dtype: str, ba
     _check(_lib().adore_controller_score_static(C.byref(w), ADORE_F32 if dtype == "f32" else ADORE_BF16, batch, hidden,
                                                 ctrl_hidden, _ptr(x), _ptr(z), position, pos_scale, _ptr(score),
                                                 _ptr(sigma), cuda_stream or None), "adore_controller_score_static")
+
+
+def adore_probe_read_bandwidth(buffer, n_blocks: int, block_rows: int, row_bytes: int, kept_rows: int, gather: bool,
+                               ctas: int, scratch4, cuda_stream: int = 0) -> None:
+    _check(_lib().adore_probe_read_bandwidth(_ptr(buffer), n_blocks, block_rows, row_bytes, kept_rows, int(gather), ctas,
+                                             _ptr(scratch4), cuda_stream or None), "adore_probe_read_bandwidth")
 
 
 def adore_status_string(status: int) -> str:

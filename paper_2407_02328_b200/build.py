@@ -8,7 +8,8 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB = os.path.join(HERE, "libadore.so")
-SOURCES = [os.path.join(HERE, "csrc", "adore_api.cu"), os.path.join(HERE, "csrc", "controller_static.cu")]
+SOURCES = [os.path.join(HERE, "csrc", "adore_api.cu"), os.path.join(HERE, "csrc", "controller_static.cu"),
+           os.path.join(HERE, "csrc", "probe.cu")]
 
 
 def _newest_source_mtime() -> float:
