@@ -35,10 +35,10 @@ struct AttnParams {
 constexpr int kAttnThreads = 256;
 constexpr int kAttnUnroll = 4;
 
-__host__ __device__ inline size_t attn_smem_bytes(int C, int DH) {
+__host__ __device__ inline size_t attn_smem_bytes(int C, int DH, int threads = kAttnThreads) {
   const int cp = (C + 1 + 3) & ~3;
   return sizeof(float) * cp + sizeof(int) * cp + sizeof(unsigned) * 256 +
-         sizeof(float) * (kAttnThreads / 32) * DH + sizeof(float) * 64;
+         sizeof(float) * (threads / 32) * DH + sizeof(float) * 64;
 }
 
 template <int NT>
@@ -67,7 +67,7 @@ __device__ __forceinline__ float block_max_f(float v, float* tmp) {
 }
 
 // Shared-memory carve-up common to the attention kernels.
-template <int DH>
+template <int DH, int NT = kAttnThreads>
 struct AttnSmem {
   float* logit;
   int* list;
@@ -81,7 +81,7 @@ struct AttnSmem {
     list = reinterpret_cast<int*>(logit + cp);
     hist = reinterpret_cast<unsigned*>(list + cp);
     red = reinterpret_cast<float*>(hist + 256);
-    tmp = red + (kAttnThreads / 32) * DH;
+    tmp = red + (NT / 32) * DH;
     sel = reinterpret_cast<int*>(tmp + 32);
   }
 };
@@ -90,9 +90,8 @@ struct AttnSmem {
 // kept set, turns the logits into weights in place (0 for rows not kept), writes the weights out and
 // builds the ordered list of kept row indices. Returns the number of kept rows. Every thread of the
 // block calls it after a __syncthreads(); the results are published by a final __syncthreads().
-template <typename T, int DH>
-__device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh) {
-  constexpr int NT = kAttnThreads;
+template <typename T, int DH, int NT = kAttnThreads>
+__device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh) {
   constexpr int NW = NT / 32;
   float* s_logit = sm.logit;
   int* s_list = sm.list;
@@ -197,10 +196,9 @@ __device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p
 
 // Phase 4 with direct loads: adds w_s * V[s] of the kept rows [j_begin, n_kept) of the list into acc (this lane's 16-byte column
 // slice; lanes of different row groups and warps hold partial sums).
-template <typename T, int DH>
-__device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh, int n_kept,
+template <typename T, int DH, int NT = kAttnThreads>
+__device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh, int n_kept,
                                                         float (&acc)[Elem<T>::kPer16B], int j_begin = 0) {
-  constexpr int NT = kAttnThreads;
   constexpr int NW = NT / 32;
   constexpr int EPL = Elem<T>::kPer16B;
   constexpr int LPR = DH / EPL;
@@ -247,10 +245,9 @@ __device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, 
 
 // Adds the partial sums of all row groups and warps, writes `out`, then writes the current token's
 // row into its slot (append of the most recent state, Section 2.2 third bullet).
-template <typename T, int DH>
-__device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh,
+template <typename T, int DH, int NT = kAttnThreads>
+__device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh,
                                                  float (&acc)[Elem<T>::kPer16B]) {
-  constexpr int NT = kAttnThreads;
   constexpr int NW = NT / 32;
   constexpr int EPL = Elem<T>::kPer16B;
   constexpr int LPR = DH / EPL;
@@ -301,14 +298,14 @@ __device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const A
 }
 
 // Phases 2-4 and the admit write for kernels that gather the value rows with direct loads.
-template <typename T, int DH>
-__device__ __forceinline__ void attention_tail(const AttnParams<T>& p, const AttnSmem<DH>& sm, int bh) {
-  const int n_kept = attention_keep_and_weights<T, DH>(p, sm, bh);
+template <typename T, int DH, int NT = kAttnThreads>
+__device__ __forceinline__ void attention_tail(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh) {
+  const int n_kept = attention_keep_and_weights<T, DH, NT>(p, sm, bh);
   float acc[Elem<T>::kPer16B];
 #pragma unroll
   for (int e = 0; e < Elem<T>::kPer16B; ++e) acc[e] = 0.f;
-  attention_values_direct<T, DH>(p, sm, bh, n_kept, acc);
-  attention_finish<T, DH>(p, sm, bh, acc);
+  attention_values_direct<T, DH, NT>(p, sm, bh, n_kept, acc);
+  attention_finish<T, DH, NT>(p, sm, bh, acc);
 }
 
 template <typename T, int DH>

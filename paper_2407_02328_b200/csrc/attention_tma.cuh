@@ -18,16 +18,17 @@
 
 namespace adore {
 
-constexpr int kRingStages = 4;
 constexpr int kRingChunkBytes = 8192;
-__host__ __device__ inline size_t attn_tma_smem_bytes(int C, int DH) {
+__host__ __device__ inline size_t attn_tma_smem_bytes(int C, int DH, int threads, int kRingStages) {
   // ring first (needs 128-byte alignment at most), then barriers, then the common carve-up
-  return size_t(kRingStages) * kRingChunkBytes + 64 + attn_smem_bytes(C, DH);
+  return size_t(kRingStages) * kRingChunkBytes + 64 + attn_smem_bytes(C, DH, threads);
 }
 
-template <typename T, int DH>
-__global__ void __launch_bounds__(kAttnThreads) attention_tma_kernel(const AttnParams<T> p) {
-  constexpr int NT = kAttnThreads;
+// NT threads per CTA and kRingStages ring stages are chosen per launch: 128 threads / 2 stages put
+// 8-10 CTAs on an SM (fewer, shorter waves when there are many (b, h) pairs), 256 threads / 4 stages
+// give each pair more threads (better when there are few pairs or very long key blocks).
+template <typename T, int DH, int NT, int kRingStages>
+__global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p) {
   constexpr int NW = NT / 32;
   constexpr int EPL = Elem<T>::kPer16B;
   constexpr int LPR = DH / EPL;
@@ -41,7 +42,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_tma_kernel(const AttnP
   unsigned char* ring = smem_raw;
   uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + size_t(kRingStages) * kRingChunkBytes);
   const int C = p.C, rows = C + 1;
-  const AttnSmem<DH> sm(smem_raw + size_t(kRingStages) * kRingChunkBytes + 64, rows);
+  const AttnSmem<DH, NT> sm(smem_raw + size_t(kRingStages) * kRingChunkBytes + 64, rows);
   float* s_logit = sm.logit;
   int* s_fail = sm.sel + 24;               // one word of the broadcast area
 
@@ -119,37 +120,44 @@ __global__ void __launch_bounds__(kAttnThreads) attention_tma_kernel(const AttnP
     if (tid == 0 && !failed && c + kRingStages < n_chunks) issue(c + kRingStages);
   }
   // (the loop's last __syncthreads also publishes the logits)
-  const int n_kept = attention_keep_and_weights<T, DH>(p, sm, bh);
+  const int n_kept = attention_keep_and_weights<T, DH, NT>(p, sm, bh);
 
   // ---- phase 4: only the kept value rows, gathered with direct 16-byte loads (one bulk copy per
   // 256-byte row was measured slower than the loads: the copy engine's per-operation cost dominates)
   float acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-  attention_values_direct<T, DH>(p, sm, bh, n_kept, acc);
-  attention_finish<T, DH>(p, sm, bh, acc);
+  attention_values_direct<T, DH, NT>(p, sm, bh, n_kept, acc);
+  attention_finish<T, DH, NT>(p, sm, bh, acc);
 }
 
 template <typename T>
 inline bool attn_tma_usable(int /*C*/, int DH) { return DH == 64 || DH == 128; }
 
-template <typename T, int DH>
-inline cudaError_t launch_attention_tma_dh(const AttnParams<T>& p, int grid, cudaStream_t stream) {
-  const size_t smem = attn_tma_smem_bytes(p.C, DH);
+template <typename T, int DH, int NT, int STAGES>
+inline cudaError_t launch_attention_tma_cfg(const AttnParams<T>& p, int grid, cudaStream_t stream) {
+  const size_t smem = attn_tma_smem_bytes(p.C, DH, NT, STAGES);
   static bool opted_in = false;            // per instantiation; the attribute is per function
   if (!opted_in) {
-    cudaError_t e = cudaFuncSetAttribute(attention_tma_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(attention_tma_kernel<T, DH, NT, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
     if (e != cudaSuccess) return e;
     opted_in = true;
   }
-  attention_tma_kernel<T, DH><<<grid, kAttnThreads, smem, stream>>>(p);
+  attention_tma_kernel<T, DH, NT, STAGES><<<grid, NT, smem, stream>>>(p);
   return cudaGetLastError();
 }
 
+// Many (b, h) pairs with key blocks of moderate length: small CTAs; otherwise large ones (measured on the
+// capacity x batch sweep: 128 threads win from ~1000 pairs on up to C = 1024, 256 threads elsewhere).
 template <typename T>
 inline cudaError_t launch_attention_tma(const AttnParams<T>& p, int DH, int grid, cudaStream_t stream) {
-  if (DH == 64) return launch_attention_tma_dh<T, 64>(p, grid, stream);
-  return launch_attention_tma_dh<T, 128>(p, grid, stream);
+  const bool small_ctas = grid >= 1024 && p.C <= 1024;
+  if (DH == 64) {
+    if (small_ctas) return launch_attention_tma_cfg<T, 64, 128, 2>(p, grid, stream);
+    return launch_attention_tma_cfg<T, 64, 256, 4>(p, grid, stream);
+  }
+  if (small_ctas) return launch_attention_tma_cfg<T, 128, 128, 2>(p, grid, stream);
+  return launch_attention_tma_cfg<T, 128, 256, 4>(p, grid, stream);
 }
 
 }  // namespace adore
