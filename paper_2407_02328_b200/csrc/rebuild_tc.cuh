@@ -167,14 +167,64 @@ struct TcSmem {
 // row tiles inside a band, columns fastest. A band of W then stays L2-resident while the rows stream
 // past it once, instead of the whole 67 MB weight matrix being re-read from DRAM for every wave.
 constexpr int kTcBandCols = 4096;
-template <int BN>
+template <int BN, int BM = kTcBM>
 __device__ __forceinline__ void tc_tile_origin(int t, int m_tiles, int n_tiles, int& m0, int& n0) {
   constexpr int kBand = kTcBandCols / BN;                 // column tiles per band
   const int per_band = m_tiles * kBand;
   const int band = t / per_band, r = t - band * per_band;
   const int width = min(kBand, n_tiles - band * kBand);   // the last band may be narrower
-  m0 = (r / width) * kTcBM;
+  m0 = (r / width) * BM;
   n0 = (band * kBand + r % width) * BN;
+}
+
+// Epilogue of one accumulator for one output row per lane: reads the row's BN fp32 values from TMEM (32 columns
+// at a time; `taddr` addresses this warp's lane quarter and the accumulator's first column), applies the rotary
+// embedding to the key half, rounds to bf16 and stores each head's segment at the token's slot. Rows with
+// in_range == false take part in the warp-collective TMEM loads and store nothing.
+template <int BN>
+__device__ __forceinline__ void tc_epilogue_row(const TcGemmParams& p, uint32_t taddr, int n0, bool in_range, int b, int tok,
+                                                int slot) {
+  const int HD = p.H * p.DH;
+#pragma unroll 1
+  for (int c = 0; c < BN / 32; ++c) {
+    uint32_t v[32];
+    __syncwarp();                               // the TMEM load is warp-collective
+    tc_ld_32x32(taddr + uint32_t(c * 32), v);
+    const int col0 = n0 + c * 32;
+    const int part = col0 / HD, h = (col0 % HD) / p.DH, e0 = col0 % p.DH;
+    if (in_range) {
+      float y[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(v[i]);
+      if (part == 0 && p.rope_cos != nullptr) {
+        const float4* cs = reinterpret_cast<const float4*>(p.rope_cos + size_t(tok) * (p.DH / 2) + e0 / 2);
+        const float4* sn = reinterpret_cast<const float4*>(p.rope_sin + size_t(tok) * (p.DH / 2) + e0 / 2);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const float4 c4 = __ldg(cs + g), s4 = __ldg(sn + g);
+          const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float a0 = y[8 * g + 2 * j], a1 = y[8 * g + 2 * j + 1];
+            y[8 * g + 2 * j] = a0 * cc[j] - a1 * ss[j];
+            y[8 * g + 2 * j + 1] = a0 * ss[j] + a1 * cc[j];
+          }
+        }
+      }
+      __nv_bfloat16* dst = (part == 0 ? p.Kc : p.Vc) + ((size_t(b) * p.H + h) * p.C + slot) * p.DH + e0;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        uint4 o;
+        __nv_bfloat162 t0 = __floats2bfloat162_rn(y[8 * g + 0], y[8 * g + 1]);
+        __nv_bfloat162 t1 = __floats2bfloat162_rn(y[8 * g + 2], y[8 * g + 3]);
+        __nv_bfloat162 t2 = __floats2bfloat162_rn(y[8 * g + 4], y[8 * g + 5]);
+        __nv_bfloat162 t3 = __floats2bfloat162_rn(y[8 * g + 6], y[8 * g + 7]);
+        o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
+        o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
+        reinterpret_cast<uint4*>(dst)[g] = o;
+      }
+    }
+  }
 }
 
 template <int BN>
@@ -264,7 +314,6 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   } else {
     // ---------------- epilogue (warps 2..5; TMEM lane quarter = warp % 4) ----------------
     const int quarter = warp & 3;
-    const int HD = p.H * p.DH;
     bool ok = true;
     int it = 0;
     for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
@@ -281,46 +330,7 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (!tc_mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * BN);
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t v[32];
-        __syncwarp();                               // the TMEM load is warp-collective
-        tc_ld_32x32(taddr + uint32_t(c * 32), v);
-        const int col0 = n0 + c * 32;
-        const int part = col0 / HD, h = (col0 % HD) / p.DH, e0 = col0 % p.DH;
-        if (in_range) {
-          float y[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(v[i]);
-          if (part == 0 && p.rope_cos != nullptr) {
-            const float4* cs = reinterpret_cast<const float4*>(p.rope_cos + size_t(tok) * (p.DH / 2) + e0 / 2);
-            const float4* sn = reinterpret_cast<const float4*>(p.rope_sin + size_t(tok) * (p.DH / 2) + e0 / 2);
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              const float4 c4 = __ldg(cs + g), s4 = __ldg(sn + g);
-              const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const float a0 = y[8 * g + 2 * j], a1 = y[8 * g + 2 * j + 1];
-                y[8 * g + 2 * j] = a0 * cc[j] - a1 * ss[j];
-                y[8 * g + 2 * j + 1] = a0 * ss[j] + a1 * cc[j];
-              }
-            }
-          }
-          __nv_bfloat16* dst = (part == 0 ? p.Kc : p.Vc) + ((size_t(b) * p.H + h) * p.C + slot) * p.DH + e0;
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint4 o;
-            __nv_bfloat162 t0 = __floats2bfloat162_rn(y[8 * g + 0], y[8 * g + 1]);
-            __nv_bfloat162 t1 = __floats2bfloat162_rn(y[8 * g + 2], y[8 * g + 3]);
-            __nv_bfloat162 t2 = __floats2bfloat162_rn(y[8 * g + 4], y[8 * g + 5]);
-            __nv_bfloat162 t3 = __floats2bfloat162_rn(y[8 * g + 6], y[8 * g + 7]);
-            o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
-            o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
-            reinterpret_cast<uint4*>(dst)[g] = o;
-          }
-        }
-      }
+      tc_epilogue_row<BN>(p, taddr, n0, in_range, b, tok, slot);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) tc_mbar_arrive(&acc_empty[acc]);   // this warp has drained its quarter
@@ -335,6 +345,12 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   if (warp == 0) { __syncwarp(); tc_dealloc(tmem_base, kTmemCols); }
 }
 
+}  // namespace adore
+
+#include "rebuild_tc_pair.cuh"   // the two-SM variant of the kernel above (uses its wrappers and epilogue)
+
+namespace adore {
+
 // ---- host side -------------------------------------------------------------------------------------
 typedef CUresult (*TcEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -345,7 +361,8 @@ struct TcState {
   TcEncodeFn encode = nullptr;
   int sms = 148;
   int N = 0, K = 0;
-  size_t a_rows = 0;                  // rows of the gather buffer (multiple of 128)
+  int pairs = 0;                      // CTA pairs the two-SM kernel runs with (0: not available)
+  size_t a_rows = 0;                  // rows of the gather buffer (multiple of 256)
   __nv_bfloat16* a_buf = nullptr;
   CUtensorMap map_a{};
   std::vector<CUtensorMap> map_w256;  // per layer, W tile of 256 rows (only if N % 256 == 0)
@@ -382,8 +399,8 @@ inline adore_status_t tc_init(TcState& s, const adore_config_t& f, std::vector<v
   cudaDeviceGetAttribute(&s.sms, cudaDevAttrMultiProcessorCount, dev);
   const size_t want = size_t(f.batch) * size_t(std::max(f.rebuild_max, std::min(f.capacity, 32768 / std::max(1, f.batch) + 1)));
   const size_t full = size_t(f.batch) * f.capacity;
-  s.a_rows = ((std::min(std::max(want, size_t(f.batch) * f.rebuild_max), full) + kTcBM - 1) / kTcBM) * kTcBM;
-  if (s.a_rows < size_t(kTcBM)) s.a_rows = kTcBM;
+  s.a_rows = ((std::min(std::max(want, size_t(f.batch) * f.rebuild_max), full) + 2 * kTcBM - 1) / (2 * kTcBM)) * (2 * kTcBM);
+  if (s.a_rows < size_t(2 * kTcBM)) s.a_rows = 2 * kTcBM;
   void* ptr = nullptr;
   if (cudaMalloc(&ptr, s.a_rows * s.K * 2) != cudaSuccess) { cudaGetLastError(); return ADORE_ERR_OOM; }
   owned.push_back(ptr);
@@ -396,6 +413,19 @@ inline adore_status_t tc_init(TcState& s, const adore_config_t& f, std::vector<v
   if (cudaFuncSetAttribute(rebuild_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(TcSmem<256>::kTotal)) != cudaSuccess ||
       cudaFuncSetAttribute(rebuild_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(TcSmem<128>::kTotal)) != cudaSuccess)
     return ADORE_ERR_CUDA;
+  // the two-SM kernel needs pairs of SMs that can host a cluster of two 1-CTA-per-SM blocks
+  if (s.N % kPairBN == 0 && std::getenv("ADORE_REBUILD_ONE_SM") == nullptr &&
+      cudaFuncSetAttribute(rebuild_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kPairSmemBytes)) == cudaSuccess) {
+    cudaLaunchConfig_t lc{};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    lc.gridDim = dim3(unsigned(s.sms / 2 * 2)); lc.blockDim = dim3(kTcThreads); lc.dynamicSmemBytes = kPairSmemBytes;
+    lc.attrs = at; lc.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, rebuild_tc_pair_kernel, &lc) == cudaSuccess) s.pairs = std::min(clusters, s.sms / 2);
+  }
+  cudaGetLastError();
   s.ready = true;
   return ADORE_OK;
 }
@@ -430,6 +460,20 @@ inline cudaError_t launch_rebuild_tc<__nv_bfloat16>(TcState& s, const RebuildPar
     g.Kc = rp.Kc; g.Vc = rp.Vc; g.row_b = rp.row_b + base; g.row_tok = rp.row_tok + base; g.row_slot = rp.row_slot + base;
     g.row_total = rp.row_total; g.row_base = base; g.row_limit = limit;
     g.rope_cos = rp.rope_cos; g.rope_sin = rp.rope_sin; g.H = rp.H; g.DH = rp.DH; g.C = rp.C; g.N = rp.N; g.K = rp.d; g.err = rp.err;
+    // enough 256 x 256 tiles for every pair of SMs: the two-SM kernel
+    const int pair_tiles = ((limit + 2 * kTcBM - 1) / (2 * kTcBM)) * (s.N / kPairBN);
+    if (s.pairs > 0 && s.N % kPairBN == 0 && pair_tiles >= s.pairs) {
+      cudaLaunchConfig_t lc{};
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      lc.gridDim = dim3(unsigned(2 * s.pairs)); lc.blockDim = dim3(kTcThreads); lc.dynamicSmemBytes = kPairSmemBytes;
+      lc.stream = stream; lc.attrs = at; lc.numAttrs = 1;
+      e = cudaLaunchKernelEx(&lc, rebuild_tc_pair_kernel, s.map_a, s.map_w128[layer], g);
+      ++*launched;
+      if (e != cudaSuccess) return e;
+      continue;
+    }
     // the 256-wide tile pays once there are enough tiles to fill the machine; otherwise more, smaller tiles
     const int m_tiles = (limit + kTcBM - 1) / kTcBM;
     const bool wide = s.N % 256 == 0 && m_tiles * (s.N / 256) >= s.sms;

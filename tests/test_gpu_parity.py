@@ -80,6 +80,13 @@ def test_split_slot_clusters_for_few_heads():
                       prompt=90, steps=10, seed=114, **two))
 
 
+def test_rebuild_on_sm_pairs_with_ragged_row_count():
+    # 20 x 120 = 2400 listed rows at most and N = 2048: ten 256-row tile rows x eight 256-column tiles, enough for
+    # the two-SM kernel; the rows actually flagged per step vary, so the last tile row is ragged
+    _run(SMALL.scaled(name="pair_gemm", batch=20, n_heads=8, capacity=160, topk=64, rebuild_max=120, prompt=300, steps=6,
+                      rebuild_mode="explicit", rebuild_p=0.6, seed=117))
+
+
 def test_config2_sub_batch():
     _run(wl.get_config(2), batch=2, steps=24, state_every=4)
 
