@@ -16,8 +16,8 @@
  * Conventions
  *   - Every function returns an adore_status_t. Nothing throws, aborts or traps the device.
  *   - All device work is queued on the CUDA stream given at create time and is asynchronous;
- *     only adore_cache_sync_status, adore_decode_step_host (at its end) and
- *     adore_cache_destroy wait for the device.
+ *     only adore_cache_sync_status, adore_decode_step_host (at its end), the state snapshot
+ *     calls and adore_cache_destroy wait for the device.
  *   - "device" pointers are CUDA device addresses of the cache's GPU; "host" pointers are
  *     ordinary (ideally pinned) host memory. The library borrows per-call buffers until the
  *     stream has passed the call, and borrows projection weights until the cache is destroyed.
@@ -244,6 +244,22 @@ adore_status_t adore_controller_score_static(const adore_controller_weights_t *w
                                              int32_t batch, int32_t hidden, int32_t ctrl_hidden, const void *x,
                                              double *z, int32_t position, float pos_scale, float *score,
                                              float *sigma, void *cuda_stream);
+
+/* Snapshot of the small per-sequence state that scoring and selection carry from step to step
+ * (Section 2.2: which tokens hold which slots, every token's controller score and the GRU state z;
+ * Section 2.3: the step's rebuild list): both slot-map buffers, the token-to-slot table, score and sigma
+ * of all tokens, z, the step's admit/evict/rebuild lists and row table, and n. NOT included: the K/V
+ * cache rows and the stored layer-input rows (they are large; a caller that wants to rewind a cache keeps
+ * or recomputes them itself).
+ *   export: host_buf == NULL stores the size needed in *bytes. Otherwise *bytes is the capacity of
+ *           host_buf (HOST memory, written by the call) and receives the size written; too small a
+ *           buffer returns ADORE_ERR_INVALID_ARG with the size needed in *bytes.
+ *   import: host_buf is a snapshot taken from a cache created with the same batch, capacity,
+ *           rebuild_max, max_tokens and ctrl_hidden; anything else returns ADORE_ERR_INVALID_ARG and
+ *           changes nothing.
+ * Both wait for the cache's streams before copying (synchronous calls). */
+adore_status_t adore_cache_export_state(adore_cache_t *cache, void *host_buf, size_t *bytes);
+adore_status_t adore_cache_import_state(adore_cache_t *cache, const void *host_buf, size_t bytes);
 
 /* Waits for the stream and turns the device error word into a status (OK, DEVICE_FLAG, TIMEOUT,
  * or CUDA if the stream itself failed). The word is cleared. */

@@ -49,7 +49,8 @@ EXPORTS = ["adore_cache_create", "adore_cache_destroy", "adore_cache_set_project
            "adore_cache_step_info", "adore_cache_scores", "adore_cache_kv", "adore_cache_num_tokens",
            "adore_cache_launch_count", "adore_cache_sync_status", "adore_status_string",
            "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows",
-           "adore_controller_score_static", "adore_probe_read_bandwidth"]
+           "adore_controller_score_static", "adore_probe_read_bandwidth",
+           "adore_cache_export_state", "adore_cache_import_state"]
 
 
 def _lib():
@@ -83,6 +84,8 @@ def _lib():
         lib.adore_cache_set_stage_timing.argtypes = [vp, i32]
         lib.adore_cache_stage_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         lib.adore_cache_rebuild_rows.argtypes = [vp, C.POINTER(C.c_int64)]
+        lib.adore_cache_export_state.argtypes = [vp, vp, C.POINTER(C.c_size_t)]
+        lib.adore_cache_import_state.argtypes = [vp, vp, C.c_size_t]
         lib.adore_probe_read_bandwidth.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp]
         lib.adore_controller_score_static.argtypes = [C.POINTER(adore_controller_weights_t), C.c_int, i32, i32, i32, vp, vp,
                                                       i32, C.c_float, vp, vp, vp]
@@ -186,6 +189,17 @@ def adore_cache_launch_count(cache: int) -> int:
 
 def adore_cache_sync_status(cache: int) -> None:
     _check(_lib().adore_cache_sync_status(cache), "adore_cache_sync_status")
+
+
+def adore_cache_export_state(cache: int, host_buf: Optional[np.ndarray] = None) -> int:
+    """Bytes needed (host_buf None) or written into the uint8 array host_buf."""
+    n = C.c_size_t(0 if host_buf is None else host_buf.nbytes)
+    _check(_lib().adore_cache_export_state(cache, _ptr(host_buf), C.byref(n)), "adore_cache_export_state")
+    return int(n.value)
+
+
+def adore_cache_import_state(cache: int, host_buf: np.ndarray) -> None:
+    _check(_lib().adore_cache_import_state(cache, _ptr(host_buf), host_buf.nbytes), "adore_cache_import_state")
 
 
 def adore_cache_set_stage_timing(cache: int, enable: bool) -> None:

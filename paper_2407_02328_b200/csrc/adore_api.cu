@@ -750,6 +750,92 @@ adore_status_t adore_cache_rebuild_rows(adore_cache_t* c, int64_t* rows) {
   return ADORE_OK;
 }
 
+// ---- small-state snapshot ------------------------------------------------------------------------
+namespace {
+
+struct StateHeader {
+  uint32_t magic, version;
+  int32_t batch, capacity, rebuild_max, max_tokens, ctrl_hidden, n, cur, attn, step_open;
+  uint32_t reserved[5];
+};
+static_assert(sizeof(StateHeader) == 64, "snapshot header is 64 bytes");
+constexpr uint32_t kStateMagic = 0x54534441u;   // "ADST"
+
+struct StateSection { void* ptr; size_t bytes; };
+
+// Everything selection and scoring carry from step to step, in snapshot order (each section padded to 8 bytes).
+std::vector<StateSection> state_sections(adore_cache* c) {
+  const adore_config_t& f = c->cfg;
+  const size_t B = f.batch, C = f.capacity, MT = f.max_tokens, h = f.ctrl_hidden;
+  const size_t rmax1 = f.rebuild_max > 0 ? f.rebuild_max : 1;
+  return {
+      {c->slot_tok[0], B * C * sizeof(int)}, {c->slot_tok[1], B * C * sizeof(int)},
+      {c->slot_role[0], B * C},              {c->slot_role[1], B * C},
+      {c->tok_slot, B * MT * sizeof(int)},   {c->score, B * MT * sizeof(float)},  {c->sigma, B * MT * sizeof(float)},
+      {c->z, B * h * sizeof(double)},
+      {c->admit_slot, B * sizeof(int)},      {c->evicted_tok, B * sizeof(int)},
+      {c->rebuild_tok, B * rmax1 * sizeof(int)}, {c->rebuild_slot, B * rmax1 * sizeof(int)}, {c->rebuild_count, B * sizeof(int)},
+      {c->row_b, B * rmax1 * sizeof(int)},   {c->row_tok, B * rmax1 * sizeof(int)}, {c->row_slot, B * rmax1 * sizeof(int)},
+      {c->row_total, sizeof(int)},
+  };
+}
+inline size_t pad8(size_t v) { return (v + 7) & ~size_t(7); }
+
+}  // namespace
+
+adore_status_t adore_cache_export_state(adore_cache_t* c, void* host_buf, size_t* bytes) {
+  if (!c || !bytes) return ADORE_ERR_INVALID_ARG;
+  const std::vector<StateSection> sec = state_sections(c);
+  size_t need = sizeof(StateHeader);
+  for (const StateSection& s : sec) need += pad8(s.bytes);
+  if (!host_buf) { *bytes = need; return ADORE_OK; }
+  if (*bytes < need) { *bytes = need; return ADORE_ERR_INVALID_ARG; }
+  *bytes = need;
+  // the side stream's work is joined into the main stream by the calls that use it; wait for both anyway
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
+  if (c->aux && cudaStreamSynchronize(c->aux) != cudaSuccess) return ADORE_ERR_CUDA;
+  StateHeader hd{};
+  hd.magic = kStateMagic; hd.version = 1;
+  hd.batch = c->cfg.batch; hd.capacity = c->cfg.capacity; hd.rebuild_max = c->cfg.rebuild_max;
+  hd.max_tokens = c->cfg.max_tokens; hd.ctrl_hidden = c->cfg.ctrl_hidden;
+  hd.n = c->n; hd.cur = c->cur; hd.attn = c->attn; hd.step_open = c->step_layer0_done;
+  unsigned char* dst = static_cast<unsigned char*>(host_buf);
+  std::memset(dst, 0, need);
+  std::memcpy(dst, &hd, sizeof(hd));
+  size_t off = sizeof(hd);
+  for (const StateSection& s : sec) {
+    CUDA_OK(cudaMemcpy(dst + off, s.ptr, s.bytes, cudaMemcpyDeviceToHost));
+    off += pad8(s.bytes);
+  }
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_import_state(adore_cache_t* c, const void* host_buf, size_t bytes) {
+  if (!c || !host_buf || bytes < sizeof(StateHeader)) return ADORE_ERR_INVALID_ARG;
+  StateHeader hd;
+  std::memcpy(&hd, host_buf, sizeof(hd));
+  const adore_config_t& f = c->cfg;
+  if (hd.magic != kStateMagic || hd.version != 1 || hd.batch != f.batch || hd.capacity != f.capacity ||
+      hd.rebuild_max != f.rebuild_max || hd.max_tokens != f.max_tokens || hd.ctrl_hidden != f.ctrl_hidden ||
+      hd.n < 0 || hd.n > f.max_tokens || (hd.cur != 0 && hd.cur != 1) || (hd.attn != 0 && hd.attn != 1))
+    return ADORE_ERR_INVALID_ARG;
+  const std::vector<StateSection> sec = state_sections(c);
+  size_t need = sizeof(StateHeader);
+  for (const StateSection& s : sec) need += pad8(s.bytes);
+  if (bytes < need) return ADORE_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
+  if (c->aux && cudaStreamSynchronize(c->aux) != cudaSuccess) return ADORE_ERR_CUDA;
+  const unsigned char* src = static_cast<const unsigned char*>(host_buf);
+  size_t off = sizeof(hd);
+  for (const StateSection& s : sec) {
+    CUDA_OK(cudaMemcpy(s.ptr, src + off, s.bytes, cudaMemcpyHostToDevice));
+    off += pad8(s.bytes);
+  }
+  c->n = hd.n; c->cur = hd.cur; c->attn = hd.attn; c->step_layer0_done = hd.step_open;
+  c->joined = true;
+  return ADORE_OK;
+}
+
 adore_status_t adore_cache_sync_status(adore_cache_t* c) {
   if (!c) return ADORE_ERR_INVALID_ARG;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
