@@ -23,9 +23,11 @@ namespace {
 constexpr int kMaxPrefillRows = 8192;       // controller rows per chunk during a bulk load
 
 // ---- kernels that glue the device functions together -----------------------------------------
+// One step's selection for sequence blockIdx.x. It ranks tokens 0..n-1 by the scores they already have, so it
+// does not wait for the controller's score of the new token n (that score is first read at step n+1) and runs
+// beside the controller kernels.
 template <typename T>
-__global__ void __launch_bounds__(512) ctrl_select_kernel(const RecurParams rp, const SelectParams sp, const T* x_new, T* x_store, int d,
-                                                          int resident) {
+__global__ void __launch_bounds__(512) select_kernel(const SelectParams sp, const T* x_new, T* x_store, int d) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int b = blockIdx.x;
   // keep the new token's layer-input row: it is what a later rebuild recomputes from
@@ -34,9 +36,6 @@ __global__ void __launch_bounds__(512) ctrl_select_kernel(const RecurParams rp, 
     uint4* dst = reinterpret_cast<uint4*>(x_store + (size_t(b) * sp.max_tokens + sp.n) * d);
     for (int i = threadIdx.x; i < int(d * sizeof(T) / 16); i += blockDim.x) dst[i] = src[i];
   }
-  if (resident) controller_tokens_resident(rp, b, smem, sp.err);
-  else controller_tokens(rp, b, reinterpret_cast<double*>(smem));
-  __syncthreads();
   select_step(sp, smem);
 }
 
@@ -127,6 +126,11 @@ struct adore_cache {
   // side stream: the controller and the selection run beside the attention of layer 0
   cudaStream_t aux = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  // second side stream: the controller (gates, then GRU + MLP) of the new token. Its score is first needed by
+  // the NEXT step's selection, so it may run on past the end of the step that launched it.
+  cudaStream_t ctl = nullptr;
+  cudaEvent_t ev_gates = nullptr, ev_ctrl = nullptr;
+  bool ctrl_pending = false;    // ev_ctrl was recorded and the main stream has not waited for it yet
   // uploads of the host-buffer entry point run on their own stream, beside the previous rebuild
   cudaStream_t copy = nullptr;
   cudaEvent_t ev_copy = nullptr;
@@ -174,6 +178,15 @@ struct StageScope {
 adore_status_t cuda_fail(cudaError_t e) {
   if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return ADORE_ERR_OOM; }
   return ADORE_ERR_CUDA;
+}
+
+// Makes the main stream wait for a controller launch that is still running on its side stream.
+adore_status_t join_controller(adore_cache* c) {
+  if (c->ctrl_pending) {
+    CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_ctrl, 0));
+    c->ctrl_pending = false;
+  }
+  return ADORE_OK;
 }
 
 template <typename P>
@@ -458,14 +471,17 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   {
     const int big = 227 * 1024;
     cudaFuncSetAttribute(ctrl_recur_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-    cudaFuncSetAttribute(ctrl_select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-    cudaFuncSetAttribute(ctrl_select_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    cudaFuncSetAttribute(select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    cudaFuncSetAttribute(select_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     cudaFuncSetAttribute(bulk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     if (cudaGetLastError() != cudaSuccess) { adore_cache_destroy(c); return ADORE_ERR_CUDA; }
   }
   if (cudaStreamCreateWithFlags(&c->aux, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&c->ctl, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_gates, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_ctrl, cudaEventDisableTiming) != cudaSuccess ||
       cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_copy, cudaEventDisableTiming) != cudaSuccess) {
     adore_cache_destroy(c);
@@ -485,6 +501,9 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (!c) return ADORE_OK;
   cudaStreamSynchronize(c->stream);
   if (c->aux) { cudaStreamSynchronize(c->aux); cudaStreamDestroy(c->aux); }
+  if (c->ctl) { cudaStreamSynchronize(c->ctl); cudaStreamDestroy(c->ctl); }
+  if (c->ev_gates) cudaEventDestroy(c->ev_gates);
+  if (c->ev_ctrl) cudaEventDestroy(c->ev_ctrl);
   if (c->copy) { cudaStreamSynchronize(c->copy); cudaStreamDestroy(c->copy); }
   if (c->ev_copy) cudaEventDestroy(c->ev_copy);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
@@ -511,6 +530,7 @@ adore_status_t adore_cache_append_tokens(adore_cache_t* c, const void* x, int32_
   if (c->n != 0) return ADORE_ERR_STATE;
   const adore_config_t& f = c->cfg;
   if (T > f.max_tokens) return ADORE_ERR_TOKEN_TABLE_FULL;
+  if (join_controller(c) != ADORE_OK) return ADORE_ERR_CUDA;
   const size_t row = size_t(f.hidden) * c->esz;
   CUDA_OK(cudaMemcpy2DAsync(c->x_store, size_t(f.max_tokens) * row, x, size_t(T) * row, size_t(T) * row, f.batch,
                             cudaMemcpyDeviceToDevice, c->stream));
@@ -566,42 +586,51 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     const bool ex = f.rebuild_mode == ADORE_REBUILD_EXPLICIT;
     if (r_in < 0 || (ex && r_in > 0 && (!explicit_list || !explicit_count))) return ADORE_ERR_INVALID_ARG;
     if (ex && r_in > 8192) return ADORE_ERR_UNSUPPORTED;
-    // Controller + selection for the step run on the side stream while the attention of this layer,
-    // which still reads the previous map, runs on the main one; the new token's row is written once
-    // both are done.
-    // (With per-stage timing on, everything stays on the main stream so that the stage times add up.)
-    cudaStream_t side = c->timing ? c->stream : c->aux;
-    if (side != c->stream) {
-      CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
-      CUDA_OK(cudaStreamWaitEvent(side, c->ev_fork, 0));
-    }
+    // Three things start here and run side by side: the attention of this layer on the main stream, reading the
+    // cache through the previous slot map; the selection on one side stream (it needs the scores of tokens < n
+    // only); the controller of token n on another (gate products, then GRU + MLP + score). The new token's row is
+    // written once attention and selection are done. The controller may run on past this step: the next step's
+    // selection waits for it, and so does every call that reads or replaces the controller state.
+    // (With per-stage timing on, the selection stays on the main stream and the controller is joined before the
+    // stage's closing event, so that the stage times add up.)
+    cudaStream_t sel = c->timing ? c->stream : c->aux;
     adore_status_t st;
     {
-      StageScope scope(c, 1, side);
-      if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit, side);
-      else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit, side);
+      StageScope scope(c, 1);
+      CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
+      if (sel != c->stream) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_fork, 0));
+      CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
+      if (c->ctrl_pending) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_ctrl, 0));   // scores of token n-1
+      if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit, c->ctl);
+      else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit, c->ctl);
       if (st != ADORE_OK) return st;
+      CUDA_OK(cudaEventRecord(c->ev_gates, c->ctl));
       const int P = ex ? pow2_at_least(r_in) : pow2_at_least(c->n);
-      RecurParams rp = recur_params(c, f.batch, 1, c->ksplit, c->n);
       SelectParams sp = select_params(c, c->n, P, c->cur, 1 - c->cur);
       sp.explicit_list = ex && r_in > 0 ? explicit_list : nullptr;
       sp.explicit_count = ex && r_in > 0 ? explicit_count : nullptr;
       sp.r_in = r_in;
-      const size_t smem = std::max(select_smem_bytes(f.capacity, P), ctrl_smem(c));
-      const int resident = ctrl_resident_ok(f.ctrl_hidden) ? 1 : 0;
+      const size_t smem = select_smem_bytes(f.capacity, P);
       if (f.dtype == ADORE_F32)
-        ctrl_select_kernel<float><<<f.batch, select_threads(c), smem, side>>>(
-            rp, sp, static_cast<const float*>(x_new), static_cast<float*>(c->x_store), f.hidden, resident);
+        select_kernel<float><<<f.batch, select_threads(c), smem, sel>>>(
+            sp, static_cast<const float*>(x_new), static_cast<float*>(c->x_store), f.hidden);
       else
-        ctrl_select_kernel<__nv_bfloat16><<<f.batch, select_threads(c), smem, side>>>(
-            rp, sp, static_cast<const __nv_bfloat16*>(x_new), static_cast<__nv_bfloat16*>(c->x_store), f.hidden, resident);
+        select_kernel<__nv_bfloat16><<<f.batch, select_threads(c), smem, sel>>>(
+            sp, static_cast<const __nv_bfloat16*>(x_new), static_cast<__nv_bfloat16*>(c->x_store), f.hidden);
       ++c->launches;
       CUDA_OK(cudaGetLastError());
-      st = launch_row_table(c, true, side);
+      st = launch_row_table(c, true, sel);
       if (st != ADORE_OK) return st;
+      RecurParams rp = recur_params(c, f.batch, 1, c->ksplit, c->n);
+      ctrl_recur_kernel<<<f.batch, select_threads(c), ctrl_smem(c), c->ctl>>>(rp, ctrl_resident_ok(f.ctrl_hidden) ? 1 : 0, c->err);
+      ++c->launches;
+      CUDA_OK(cudaGetLastError());
+      CUDA_OK(cudaEventRecord(c->ev_ctrl, c->ctl));
+      c->ctrl_pending = true;
+      if (c->timing) { CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_ctrl, 0)); c->ctrl_pending = false; }
     }
-    c->joined = side == c->stream;
-    if (!c->joined) CUDA_OK(cudaEventRecord(c->ev_join, side));
+    c->joined = sel == c->stream;
+    if (!c->joined) CUDA_OK(cudaEventRecord(c->ev_join, sel));
     c->attn = c->cur;
     c->cur = 1 - c->cur;
     c->n += 1;
@@ -615,6 +644,7 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
   if (st != ADORE_OK || fused) return st;
   if (!c->joined) CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
   c->joined = true;
+  CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_gates, 0));   // x_new is borrowed only until the main stream passes the call
   {
     StageScope scope(c, 3);
     const size_t row_bytes = size_t(f.head_dim) * c->esz;
@@ -792,8 +822,10 @@ adore_status_t adore_cache_export_state(adore_cache_t* c, void* host_buf, size_t
   if (*bytes < need) { *bytes = need; return ADORE_ERR_INVALID_ARG; }
   *bytes = need;
   // the side stream's work is joined into the main stream by the calls that use it; wait for both anyway
+  if (join_controller(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
   if (c->aux && cudaStreamSynchronize(c->aux) != cudaSuccess) return ADORE_ERR_CUDA;
+  if (c->ctl && cudaStreamSynchronize(c->ctl) != cudaSuccess) return ADORE_ERR_CUDA;
   StateHeader hd{};
   hd.magic = kStateMagic; hd.version = 1;
   hd.batch = c->cfg.batch; hd.capacity = c->cfg.capacity; hd.rebuild_max = c->cfg.rebuild_max;
@@ -823,8 +855,10 @@ adore_status_t adore_cache_import_state(adore_cache_t* c, const void* host_buf, 
   size_t need = sizeof(StateHeader);
   for (const StateSection& s : sec) need += pad8(s.bytes);
   if (bytes < need) return ADORE_ERR_INVALID_ARG;
+  if (join_controller(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
   if (c->aux && cudaStreamSynchronize(c->aux) != cudaSuccess) return ADORE_ERR_CUDA;
+  if (c->ctl && cudaStreamSynchronize(c->ctl) != cudaSuccess) return ADORE_ERR_CUDA;
   const unsigned char* src = static_cast<const unsigned char*>(host_buf);
   size_t off = sizeof(hd);
   for (const StateSection& s : sec) {
@@ -838,6 +872,7 @@ adore_status_t adore_cache_import_state(adore_cache_t* c, const void* host_buf, 
 
 adore_status_t adore_cache_sync_status(adore_cache_t* c) {
   if (!c) return ADORE_ERR_INVALID_ARG;
+  if (join_controller(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
   unsigned word = 0;
   if (cudaMemcpy(&word, c->err, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return ADORE_ERR_CUDA;
