@@ -151,6 +151,12 @@ struct TcGemmParams {
   const float* rope_sin;
   int H, DH, C, N, K;
   unsigned* err;
+  // split of the K dimension over `ksplit` work units per tile (1 = off). Every unit stores its fp32
+  // accumulator in `partial`; the unit that arrives last at the tile's counter adds the parts in ascending
+  // order (so the sum does not depend on who was last) and runs the epilogue. Nobody waits for anybody.
+  int ksplit;
+  float* partial;             // [units][BN * 128] floats per CTA-sized accumulator
+  unsigned* unit_cnt;         // [tiles (x 2 CTAs of a pair)][4 lane quarters], zero between launches
 };
 
 template <int BN>
@@ -181,9 +187,27 @@ __device__ __forceinline__ void tc_tile_origin(int t, int m_tiles, int n_tiles, 
 // at a time; `taddr` addresses this warp's lane quarter and the accumulator's first column), applies the rotary
 // embedding to the key half, rounds to bf16 and stores each head's segment at the token's slot. Rows with
 // in_range == false take part in the warp-collective TMEM loads and store nothing.
+// Layout of one stored accumulator (BN columns x 128 rows): [BN/32 chunks][4 lane quarters][32 columns][32 lanes],
+// so that the 32 lanes of a warp write and read consecutive floats.
+template <int BN>
+__device__ __forceinline__ void tc_store_partial(uint32_t taddr, float* dst, int quarter, int lane) {
+#pragma unroll 1
+  for (int c = 0; c < BN / 32; ++c) {
+    uint32_t v[32];
+    __syncwarp();
+    tc_ld_32x32(taddr + uint32_t(c * 32), v);
+    float* d = dst + (size_t(c * 4 + quarter) * 32) * 32 + lane;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) d[i * 32] = __uint_as_float(v[i]);
+  }
+}
+
+// `parts` > 1: the row's values are the sum over the stored accumulators parts_base + q * part_stride, q ascending,
+// with this unit's own part (`my_part`) taken from TMEM.
 template <int BN>
 __device__ __forceinline__ void tc_epilogue_row(const TcGemmParams& p, uint32_t taddr, int n0, bool in_range, int b, int tok,
-                                                int slot) {
+                                                int slot, int quarter = 0, int lane = 0, int parts = 1, int my_part = 0,
+                                                const float* parts_base = nullptr, size_t part_stride = 0) {
   const int HD = p.H * p.DH;
 #pragma unroll 1
   for (int c = 0; c < BN / 32; ++c) {
@@ -194,8 +218,23 @@ __device__ __forceinline__ void tc_epilogue_row(const TcGemmParams& p, uint32_t 
     const int part = col0 / HD, h = (col0 % HD) / p.DH, e0 = col0 % p.DH;
     if (in_range) {
       float y[32];
+      if (parts > 1) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(v[i]);
+        for (int i = 0; i < 32; ++i) y[i] = 0.f;
+        for (int q = 0; q < parts; ++q) {
+          if (q == my_part) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) y[i] += __uint_as_float(v[i]);
+          } else {
+            const float* src = parts_base + size_t(q) * part_stride + (size_t(c * 4 + quarter) * 32) * 32 + lane;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) y[i] += __ldcg(src + i * 32);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(v[i]);
+      }
       if (part == 0 && p.rope_cos != nullptr) {
         const float4* cs = reinterpret_cast<const float4*>(p.rope_cos + size_t(tok) * (p.DH / 2) + e0 / 2);
         const float4* sn = reinterpret_cast<const float4*>(p.rope_sin + size_t(tok) * (p.DH / 2) + e0 / 2);
@@ -227,6 +266,25 @@ __device__ __forceinline__ void tc_epilogue_row(const TcGemmParams& p, uint32_t 
   }
 }
 
+// Split-K hand-over for one warp (one lane quarter of one CTA-sized accumulator): stores the accumulator, then
+// counts itself in. Returns true for the warp that arrived last; it also puts the counter back to zero.
+template <int BN>
+__device__ __forceinline__ bool tc_split_arrive(const TcGemmParams& p, uint32_t taddr, float* my_slot, unsigned* cnt,
+                                                int quarter, int lane) {
+  tc_store_partial<BN>(taddr, my_slot, quarter, lane);
+  __threadfence();
+  __syncwarp();
+  unsigned old = 0;
+  if (lane == 0) old = atomicAdd(cnt, 1u);
+  old = __shfl_sync(0xffffffffu, old, 0);
+  const bool last = old == unsigned(p.ksplit - 1);
+  if (last) {
+    if (lane == 0) *cnt = 0u;
+    __threadfence();
+  }
+  return last;
+}
+
 template <int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const TcGemmParams p) {
@@ -246,7 +304,7 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int M = min(max(*p.row_total - p.row_base, 0), p.row_limit);
   const int m_tiles = (M + kTcBM - 1) / kTcBM, n_tiles = p.N / BN;
-  const int total_tiles = m_tiles * n_tiles;
+  const int total_tiles = m_tiles * n_tiles * p.ksplit;      // work units: (tile, part of K), parts of a tile adjacent
   const int k_blocks = p.K / kTcBK;
 
   if (threadIdx.x == 0) {
@@ -268,10 +326,12 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      for (int u = blockIdx.x; u < total_tiles && ok; u += gridDim.x) {
+        const int t = u / p.ksplit, part = u - t * p.ksplit;
         int m0, n0;
         tc_tile_origin<BN>(t, m_tiles, n_tiles, m0, n0);
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        const int kb_end = (part + 1) * k_blocks / p.ksplit;
+        for (int kb = part * k_blocks / p.ksplit; kb < kb_end; ++kb) {
           if (!tc_mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
           unsigned char* sa = tiles + size_t(stage) * S::kStageBytes;
           tc_mbar_expect_tx(&full[stage], uint32_t(S::kStageBytes));
@@ -290,20 +350,22 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       uint32_t phase = 0;
       bool ok = true;
       int it = 0;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+      for (int u = blockIdx.x; u < total_tiles && ok; u += gridDim.x, ++it) {
+        const int part = u % p.ksplit;
         const int acc = it & 1;
         const uint32_t acc_phase = uint32_t(it >> 1) & 1u;
         if (!tc_mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + uint32_t(acc * BN);
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        const int kb_begin = part * k_blocks / p.ksplit, kb_end = (part + 1) * k_blocks / p.ksplit;
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!tc_mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const unsigned char* sa = tiles + size_t(stage) * S::kStageBytes;
           const uint64_t adesc = tc_smem_desc(sa), bdesc = tc_smem_desc(sa + S::kABytes);
 #pragma unroll
           for (int k = 0; k < kTcBK / 16; ++k)      // 16 bf16 = 32 bytes further along K: +2 in 16-byte units
-            tc_mma_bf16(d_tmem, adesc + uint64_t(2 * k), bdesc + uint64_t(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+            tc_mma_bf16(d_tmem, adesc + uint64_t(2 * k), bdesc + uint64_t(2 * k), idesc, (kb > kb_begin || k != 0) ? 1u : 0u);
           tc_commit(&empty[stage]);                 // stage reusable once these MMAs have read it
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -316,7 +378,8 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const int quarter = warp & 3;
     bool ok = true;
     int it = 0;
-    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+    for (int u = blockIdx.x; u < total_tiles && ok; u += gridDim.x, ++it) {
+      const int t = u / p.ksplit, part = u - t * p.ksplit;
       const int acc = it & 1;
       const uint32_t acc_phase = uint32_t(it >> 1) & 1u;
       int m0, n0;
@@ -330,7 +393,14 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (!tc_mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * BN);
-      tc_epilogue_row<BN>(p, taddr, n0, in_range, b, tok, slot);
+      if (p.ksplit == 1) {
+        tc_epilogue_row<BN>(p, taddr, n0, in_range, b, tok, slot);
+      } else {
+        constexpr size_t kPart = size_t(BN) * 128;
+        float* tile_parts = p.partial + size_t(t) * p.ksplit * kPart;
+        if (tc_split_arrive<BN>(p, taddr, tile_parts + size_t(part) * kPart, p.unit_cnt + t * 4 + quarter, quarter, lane))
+          tc_epilogue_row<BN>(p, taddr, n0, in_range, b, tok, slot, quarter, lane, p.ksplit, part, tile_parts, kPart);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) tc_mbar_arrive(&acc_empty[acc]);   // this warp has drained its quarter
@@ -364,11 +434,32 @@ struct TcState {
   int pairs = 0;                      // CTA pairs the two-SM kernel runs with (0: not available)
   size_t a_rows = 0;                  // rows of the gather buffer (multiple of 256)
   __nv_bfloat16* a_buf = nullptr;
+  float* partial = nullptr;           // split-K accumulators: one 128 x 256 fp32 block per SM
+  unsigned* unit_cnt = nullptr;       // split-K arrival counters (kTcCounters words, zero between launches)
   CUtensorMap map_a{};
   std::vector<CUtensorMap> map_w256;  // per layer, W tile of 256 rows (only if N % 256 == 0)
   std::vector<CUtensorMap> map_w128;  // per layer, W tile of 128 rows
   std::vector<char> has_w;
 };
+
+constexpr int kTcCounters = 4096;
+constexpr size_t kTcPartialFloatsPerSm = size_t(256) * 128;
+
+// Which kernel and which split of K serve a launch of at most `rows` rows. Enough 256 x 256 tiles for every SM pair:
+// the two-SM kernel (tensor-bound). Enough 128 x 256 tiles for every SM: those. Otherwise the launch is bound by the
+// latency of streaming each weight tile once (measured: ~1.5 us per 32 KB stage with six stages in flight, i.e.
+// ~0.3 us per k-block whatever the tile), so 128 x 128 tiles, and K split in two when that still leaves SMs idle.
+struct TcPlan { int kind; int ksplit; int grid; };   // kind 0: 128-wide tiles, 1: 256-wide tiles, 2: SM pairs
+inline TcPlan tc_plan(int rows, int N, int K, int sms, int pairs, int max_split) {
+  const int kb = K / kTcBK;
+  const int mt128 = (rows + kTcBM - 1) / kTcBM, mt256 = (rows + 2 * kTcBM - 1) / (2 * kTcBM);
+  if (pairs > 0 && N % 256 == 0 && mt256 * (N / 256) >= pairs) return TcPlan{2, 1, 2 * pairs};
+  if (N % 256 == 0 && mt128 * (N / 256) >= sms) return TcPlan{1, 1, sms};
+  const int tiles = mt128 * (N / 128);
+  const bool split = max_split >= 2 && kb % 2 == 0 && kb / 2 >= 4 && 2 * tiles <= sms && 4 * tiles <= kTcCounters;
+  const int units = split ? 2 * tiles : tiles;
+  return TcPlan{0, split ? 2 : 1, std::max(1, std::min(sms, units))};
+}
 
 inline bool tc_encode_2d(TcState& s, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
   const cuuint64_t dims[2] = {cols, rows};
@@ -407,6 +498,13 @@ inline adore_status_t tc_init(TcState& s, const adore_config_t& f, std::vector<v
   s.a_buf = static_cast<__nv_bfloat16*>(ptr);
   if (cudaMemset(ptr, 0, s.a_rows * s.K * 2) != cudaSuccess) return ADORE_ERR_CUDA;
   if (!tc_encode_2d(s, &s.map_a, s.a_buf, s.a_rows, s.K, kTcBM)) return ADORE_ERR_CUDA;
+  if (cudaMalloc(&ptr, size_t(s.sms) * kTcPartialFloatsPerSm * sizeof(float)) != cudaSuccess) { cudaGetLastError(); return ADORE_ERR_OOM; }
+  owned.push_back(ptr);
+  s.partial = static_cast<float*>(ptr);
+  if (cudaMalloc(&ptr, kTcCounters * sizeof(unsigned)) != cudaSuccess) { cudaGetLastError(); return ADORE_ERR_OOM; }
+  owned.push_back(ptr);
+  s.unit_cnt = static_cast<unsigned*>(ptr);
+  if (cudaMemset(ptr, 0, kTcCounters * sizeof(unsigned)) != cudaSuccess) return ADORE_ERR_CUDA;
   s.map_w256.resize(f.n_layers);
   s.map_w128.resize(f.n_layers);
   s.has_w.assign(f.n_layers, 0);
@@ -460,27 +558,23 @@ inline cudaError_t launch_rebuild_tc<__nv_bfloat16>(TcState& s, const RebuildPar
     g.Kc = rp.Kc; g.Vc = rp.Vc; g.row_b = rp.row_b + base; g.row_tok = rp.row_tok + base; g.row_slot = rp.row_slot + base;
     g.row_total = rp.row_total; g.row_base = base; g.row_limit = limit;
     g.rope_cos = rp.rope_cos; g.rope_sin = rp.rope_sin; g.H = rp.H; g.DH = rp.DH; g.C = rp.C; g.N = rp.N; g.K = rp.d; g.err = rp.err;
-    // enough 256 x 256 tiles for every pair of SMs: the two-SM kernel
-    const int pair_tiles = ((limit + 2 * kTcBM - 1) / (2 * kTcBM)) * (s.N / kPairBN);
-    if (s.pairs > 0 && s.N % kPairBN == 0 && pair_tiles >= s.pairs) {
+    static const int max_split = std::getenv("ADORE_TC_KSPLIT_MAX") ? std::atoi(std::getenv("ADORE_TC_KSPLIT_MAX")) : 4;
+    const TcPlan plan = tc_plan(limit, s.N, s.K, s.sms, s.pairs, max_split);
+    g.ksplit = plan.ksplit; g.partial = s.partial; g.unit_cnt = s.unit_cnt;
+    if (plan.kind == 2) {
       cudaLaunchConfig_t lc{};
       cudaLaunchAttribute at[1];
       at[0].id = cudaLaunchAttributeClusterDimension;
       at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-      lc.gridDim = dim3(unsigned(2 * s.pairs)); lc.blockDim = dim3(kTcThreads); lc.dynamicSmemBytes = kPairSmemBytes;
+      lc.gridDim = dim3(unsigned(plan.grid)); lc.blockDim = dim3(kTcThreads); lc.dynamicSmemBytes = kPairSmemBytes;
       lc.stream = stream; lc.attrs = at; lc.numAttrs = 1;
       e = cudaLaunchKernelEx(&lc, rebuild_tc_pair_kernel, s.map_a, s.map_w128[layer], g);
       ++*launched;
       if (e != cudaSuccess) return e;
       continue;
     }
-    // the 256-wide tile pays once there are enough tiles to fill the machine; otherwise more, smaller tiles
-    const int m_tiles = (limit + kTcBM - 1) / kTcBM;
-    const bool wide = s.N % 256 == 0 && m_tiles * (s.N / 256) >= s.sms;
-    const int max_tiles = m_tiles * (s.N / (wide ? 256 : 128));
-    const int grid = std::max(1, std::min(s.sms, max_tiles));
-    if (wide) rebuild_tc_kernel<256><<<grid, kTcThreads, TcSmem<256>::kTotal, stream>>>(s.map_a, s.map_w256[layer], g);
-    else rebuild_tc_kernel<128><<<grid, kTcThreads, TcSmem<128>::kTotal, stream>>>(s.map_a, s.map_w128[layer], g);
+    if (plan.kind == 1) rebuild_tc_kernel<256><<<plan.grid, kTcThreads, TcSmem<256>::kTotal, stream>>>(s.map_a, s.map_w256[layer], g);
+    else rebuild_tc_kernel<128><<<plan.grid, kTcThreads, TcSmem<128>::kTotal, stream>>>(s.map_a, s.map_w128[layer], g);
     ++*launched;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;

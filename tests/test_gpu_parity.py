@@ -87,6 +87,15 @@ def test_rebuild_on_sm_pairs_with_ragged_row_count():
                       rebuild_mode="explicit", rebuild_p=0.6, seed=117))
 
 
+def test_rebuild_with_the_reduction_dimension_split_over_work_units():
+    # few output tiles: the launch plan splits K in two so that more SMs stream the weights; whichever unit of a tile
+    # finishes last adds the two parts in a fixed order
+    _run(SMALL.scaled(name="ksplit2", hidden=1024, rebuild_max=12, capacity=48, topk=20, rebuild_mode="explicit", rebuild_p=0.5,
+                      prompt=60, steps=8, seed=118))
+    _run(SMALL.scaled(name="ksplit2_two_row_tiles", hidden=1024, batch=5, rebuild_max=40, capacity=100, topk=40,
+                      rebuild_mode="explicit", rebuild_p=0.7, prompt=160, steps=6, seed=120))   # 200 rows: 2 x 8 tiles x 2 parts
+
+
 def test_config2_sub_batch():
     _run(wl.get_config(2), batch=2, steps=24, state_every=4)
 
