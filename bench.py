@@ -283,6 +283,14 @@ class DeviceRun:
         self.out = torch.empty((B, H, dh), dtype=self.dt, device=dev)
         self.weights = torch.empty((B, H, c.capacity + 1), dtype=torch.float32, device=dev)
         self.next = 0
+        # device addresses of every step's inputs, taken once: the timed loop then only passes integers
+        ptrs = lambda a: [[a[s, l].data_ptr() for l in range(a.shape[1])] for s in range(a.shape[0])]
+        self.pq, self.pk, self.pv = ptrs(self.q), ptrs(self.k), ptrs(self.v)
+        self.px = [self.x[s, 0].data_ptr() for s in range(self.x.shape[0])]
+        self.pl = None if self.lists is None else [self.lists[s].data_ptr() for s in range(self.lists.shape[0])]
+        self.pc = None if self.counts is None else [self.counts[s].data_ptr() for s in range(self.counts.shape[0])]
+        self.pt = None if self.tables is None else [t.data_ptr() for t in self.tables]
+        self.pout, self.pw = self.out.data_ptr(), self.weights.data_ptr()
         lib.adore_cache_sync_status(self.handle)
 
     def _rope(self, y, n):
@@ -300,11 +308,12 @@ class DeviceRun:
 
     def step(self):
         lib, c, s = self.lib, self.cfg, self.next
+        pl = None if self.pl is None else self.pl[s]
+        pc = None if self.pc is None else self.pc[s]
         for l in range(c.n_layers):
-            lib.adore_decode_step(self.handle, l, self.q[s, l], self.k[s, l], self.v[s, l], self.x[s, 0],
-                                  None if self.lists is None else self.lists[s],
-                                  None if self.counts is None else self.counts[s], self.r_in, self.out, self.weights)
-            lib.adore_rebuild(self.handle, l, self.tables[l] if (self.tables is not None and l > 0) else None)
+            lib.adore_decode_step(self.handle, l, self.pq[s][l], self.pk[s][l], self.pv[s][l], self.px[s], pl, pc, self.r_in,
+                                  self.pout, self.pw)
+            lib.adore_rebuild(self.handle, l, self.pt[l] if (self.pt is not None and l > 0) else None)
         self.next += 1
 
     def make_host_inputs(self, first: int, count: int):

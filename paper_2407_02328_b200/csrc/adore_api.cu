@@ -30,6 +30,7 @@ template <typename T>
 __global__ void __launch_bounds__(512) select_kernel(const SelectParams sp, const T* x_new, T* x_store, int d) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int b = blockIdx.x;
+  let_next_grid_start();
   // keep the new token's layer-input row: it is what a later rebuild recomputes from
   {
     const uint4* src = reinterpret_cast<const uint4*>(x_new + size_t(b) * d);
@@ -53,6 +54,7 @@ __global__ void __launch_bounds__(512) bulk_select_kernel(const SelectParams sp)
 // Writes the new token's key/value rows of layer 0 into the admitted slot: one warp per (b, h).
 __global__ void admit_rows_kernel(unsigned char* Kc, unsigned char* Vc, const unsigned char* k_new, const unsigned char* v_new,
                                   const int* admit_slot, int H, int C, int row_bytes, unsigned* err) {
+  let_next_grid_start();
   const int bh = blockIdx.x, b = bh / H, s = admit_slot[b];
   if (s < 0 || s >= C) { if (threadIdx.x == 0) set_error(err, ERRW_BOUNDS); return; }
   const size_t dst = (size_t(bh) * C + s) * row_bytes, src = size_t(bh) * row_bytes;
@@ -137,6 +139,7 @@ struct adore_cache {
   bool joined = true;
   std::vector<const void*> w_kv;
   TcState tc;                   // tensor-core rebuild path (tensor maps, gather buffer)
+  bool rows_gathered = false;   // the gather buffer holds this step's listed rows, taken from the token store
   // staging for the host-buffer entry point
   void *h_q = nullptr, *h_k = nullptr, *h_v = nullptr, *h_x = nullptr, *h_out = nullptr;
   int* h_list = nullptr;
@@ -300,7 +303,7 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
 
 template <typename T>
 adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, const int* row_b, const int* row_tok,
-                              const int* row_slot, const int* row_total, int m_max) {
+                              const int* row_slot, const int* row_total, int m_max, bool step_table) {
   const adore_config_t& f = c->cfg;
   if (m_max <= 0) return ADORE_OK;
   RebuildParams<T> p{};
@@ -313,9 +316,12 @@ adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, co
   p.H = f.n_heads; p.DH = f.head_dim; p.C = f.capacity; p.N = 2 * f.n_heads * f.head_dim; p.err = c->err;
   StageScope scope(c, 2);
   if (tc_usable<T>(c->tc)) {
+    // Rows gathered from the token store for this step's table serve every layer that rebuilds from the store.
+    const bool from_store = step_table && x_table == nullptr && size_t(m_max) <= c->tc.a_rows;
     int launched = 0;
-    cudaError_t e = launch_rebuild_tc(c->tc, p, layer, m_max, c->stream, &launched);
+    cudaError_t e = launch_rebuild_tc(c->tc, p, layer, m_max, c->stream, &launched, from_store && c->rows_gathered);
     c->launches += launched;
+    c->rows_gathered = from_store;
     CUDA_OK(e);
     return ADORE_OK;
   }
@@ -329,11 +335,10 @@ adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, co
 adore_status_t launch_row_table(adore_cache* c, bool count_rows, cudaStream_t stream) {
   const adore_config_t& f = c->cfg;
   if (f.rebuild_max == 0) return ADORE_OK;          // row_total stays 0
-  row_table_kernel<<<f.batch, 128, 0, stream>>>(c->rebuild_tok, c->rebuild_slot, c->rebuild_count, f.batch, f.rebuild_max,
-                                                   c->row_b, c->row_tok, c->row_slot, c->row_total,
-                                                   count_rows ? c->rows_accum : nullptr);
+  CUDA_OK(launch_dependent(row_table_kernel, dim3(f.batch), dim3(128), 0, stream, c->rebuild_tok, c->rebuild_slot,
+                           c->rebuild_count, f.batch, f.rebuild_max, c->row_b, c->row_tok, c->row_slot, c->row_total,
+                           count_rows ? c->rows_accum : nullptr));
   ++c->launches;
-  CUDA_OK(cudaGetLastError());
   return ADORE_OK;
 }
 
@@ -344,9 +349,9 @@ adore_status_t fill_layer_impl(adore_cache* c, int layer, const void* x_table) {
   ++c->launches;
   CUDA_OK(cudaGetLastError());
   if (f.dtype == ADORE_F32)
-    return launch_rebuild<float>(c, layer, x_table, c->frow_b, c->frow_tok, c->frow_slot, c->frow_total, f.batch * f.capacity);
+    return launch_rebuild<float>(c, layer, x_table, c->frow_b, c->frow_tok, c->frow_slot, c->frow_total, f.batch * f.capacity, false);
   return launch_rebuild<__nv_bfloat16>(c, layer, x_table, c->frow_b, c->frow_tok, c->frow_slot, c->frow_total,
-                                       f.batch * f.capacity);
+                                       f.batch * f.capacity, false);
 }
 
 adore_status_t check_config(const adore_config_t* f) {
@@ -476,10 +481,14 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
     cudaFuncSetAttribute(bulk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     if (cudaGetLastError() != cudaSuccess) { adore_cache_destroy(c); return ADORE_ERR_CUDA; }
   }
-  if (cudaStreamCreateWithFlags(&c->aux, cudaStreamNonBlocking) != cudaSuccess ||
+  // the side streams carry short kernels that the step's critical path waits for: their CTAs go ahead of the
+  // attention kernel's pending ones
+  int prio_low = 0, prio_high = 0;
+  cudaDeviceGetStreamPriorityRange(&prio_low, &prio_high);
+  if (cudaStreamCreateWithPriority(&c->aux, cudaStreamNonBlocking, prio_high) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
-      cudaStreamCreateWithFlags(&c->ctl, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaStreamCreateWithPriority(&c->ctl, cudaStreamNonBlocking, prio_high) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_gates, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_ctrl, cudaEventDisableTiming) != cudaSuccess ||
       cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess ||
@@ -595,11 +604,18 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     // stage's closing event, so that the stage times add up.)
     cudaStream_t sel = c->timing ? c->stream : c->aux;
     adore_status_t st;
+    // the attention is the longest of the three and is launched first; the side streams start from the same point
+    // (with per-stage timing on: from the end of the attention, so that no stage overlaps another)
+    if (!c->timing) CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
+    c->attn = c->cur;
+    st = f.dtype == ADORE_F32 ? launch_attention<float>(c, 0, q, k_new, v_new, out, weights, false)
+                              : launch_attention<__nv_bfloat16>(c, 0, q, k_new, v_new, out, weights, false);
+    if (st != ADORE_OK) return st;
+    if (c->timing) CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
+    if (sel != c->stream) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_fork, 0));
+    CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
     {
       StageScope scope(c, 1);
-      CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
-      if (sel != c->stream) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_fork, 0));
-      CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
       if (c->ctrl_pending) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_ctrl, 0));   // scores of token n-1
       if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit, c->ctl);
       else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit, c->ctl);
@@ -629,19 +645,32 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
       c->ctrl_pending = true;
       if (c->timing) { CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_ctrl, 0)); c->ctrl_pending = false; }
     }
+    // The listed rows are copied out of the token store into the GEMM's compact input right away, beside the
+    // attention, so that the rebuild that follows starts with its GEMM. (Not with per-stage timing on: there the
+    // copy stays with the rebuild stage.)
+    c->rows_gathered = false;
+    {
+      const int m_max = f.batch * f.rebuild_max;
+      if (!c->timing && f.dtype == ADORE_BF16 && tc_usable<__nv_bfloat16>(c->tc) && m_max > 0 && size_t(m_max) <= c->tc.a_rows) {
+        RebuildParams<__nv_bfloat16> gp{};
+        gp.x_table = static_cast<const __nv_bfloat16*>(c->x_store); gp.seq_stride = f.max_tokens; gp.d = f.hidden;
+        gp.row_b = c->row_b; gp.row_tok = c->row_tok; gp.row_total = c->row_total;
+        CUDA_OK(launch_gather_tc<__nv_bfloat16>(c->tc, gp, m_max, sel));
+        ++c->launches;
+        c->rows_gathered = true;
+      }
+    }
     c->joined = sel == c->stream;
     if (!c->joined) CUDA_OK(cudaEventRecord(c->ev_join, sel));
-    c->attn = c->cur;
     c->cur = 1 - c->cur;
     c->n += 1;
     c->step_layer0_done = 1;
   } else if (!c->step_layer0_done) {
     return ADORE_ERR_STATE;
   }
-  const bool fused = layer != 0;
-  adore_status_t st = f.dtype == ADORE_F32 ? launch_attention<float>(c, layer, q, k_new, v_new, out, weights, fused)
-                                           : launch_attention<__nv_bfloat16>(c, layer, q, k_new, v_new, out, weights, fused);
-  if (st != ADORE_OK || fused) return st;
+  if (layer != 0)
+    return f.dtype == ADORE_F32 ? launch_attention<float>(c, layer, q, k_new, v_new, out, weights, true)
+                                : launch_attention<__nv_bfloat16>(c, layer, q, k_new, v_new, out, weights, true);
   if (!c->joined) CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
   c->joined = true;
   CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_gates, 0));   // x_new is borrowed only until the main stream passes the call
@@ -699,9 +728,9 @@ adore_status_t adore_rebuild(adore_cache_t* c, int32_t layer, const void* x_tabl
   if (!c->w_kv[layer] || !c->step_layer0_done) return ADORE_ERR_STATE;
   const adore_config_t& f = c->cfg;
   if (f.dtype == ADORE_F32)
-    return launch_rebuild<float>(c, layer, x_table, c->row_b, c->row_tok, c->row_slot, c->row_total, f.batch * f.rebuild_max);
+    return launch_rebuild<float>(c, layer, x_table, c->row_b, c->row_tok, c->row_slot, c->row_total, f.batch * f.rebuild_max, true);
   return launch_rebuild<__nv_bfloat16>(c, layer, x_table, c->row_b, c->row_tok, c->row_slot, c->row_total,
-                                       f.batch * f.rebuild_max);
+                                       f.batch * f.rebuild_max, true);
 }
 
 adore_status_t adore_cache_slot_map(adore_cache_t* c, const int32_t** slot_tok, const uint8_t** slot_role) {
@@ -867,6 +896,7 @@ adore_status_t adore_cache_import_state(adore_cache_t* c, const void* host_buf, 
   }
   c->n = hd.n; c->cur = hd.cur; c->attn = hd.attn; c->step_layer0_done = hd.step_open;
   c->joined = true;
+  c->rows_gathered = false;
   return ADORE_OK;
 }
 

@@ -62,6 +62,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+  wait_for_prior_grid();     // the cache rows, the slot map and q, k, v come from earlier kernels
   auto issue = [&](int chunk) {
     const int stage = chunk % kRingStages;
     const int r0 = chunk * CHUNK_ROWS;
@@ -143,8 +144,7 @@ inline cudaError_t launch_attention_tma_cfg(const AttnParams<T>& p, int grid, cu
     if (e != cudaSuccess) return e;
     opted_in = true;
   }
-  attention_tma_kernel<T, DH, NT, STAGES><<<grid, NT, smem, stream>>>(p);
-  return cudaGetLastError();
+  return launch_dependent(attention_tma_kernel<T, DH, NT, STAGES>, dim3(grid), dim3(NT), smem, stream, p);
 }
 
 // Many (b, h) pairs with key blocks of moderate length: small CTAs; otherwise large ones (measured on the

@@ -2,6 +2,8 @@
 // warp/block reductions, order-preserving keys.
 #pragma once
 
+#include <cstdlib>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -94,6 +96,29 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
   asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
   return r;
+}
+
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// A kernel launched with launch_dependent() may be placed on the SMs while the kernel ahead of it in the stream is
+// still finishing, which hides its launch latency. Such a kernel calls wait_for_prior_grid() before it reads anything
+// an earlier kernel wrote and before it writes anything; the call returns once the earlier kernel has completed and
+// its writes are visible (a no-op for an ordinary launch).
+__device__ __forceinline__ void wait_for_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Called early by short kernels: lets the next kernel of the stream, if it was launched with launch_dependent(), move
+// onto the SMs and run up to its own wait_for_prior_grid() while this one is still working.
+__device__ __forceinline__ void let_next_grid_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    Args&&... args) {
+  static const bool off = std::getenv("ADORE_NO_DEPENDENT_LAUNCH") != nullptr;   // A/B switch
+  cudaLaunchConfig_t lc{};
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.gridDim = grid; lc.blockDim = block; lc.dynamicSmemBytes = smem; lc.stream = stream;
+  lc.attrs = at; lc.numAttrs = off ? 0 : 1;
+  return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
 }
 
 }  // namespace adore

@@ -130,6 +130,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) gather_rows_kernel(const T* x_table, long long seq_stride, int d, const int* row_b,
                                                           const int* row_tok, const int* row_total, int row_base,
                                                           int row_limit, T* a_out) {
+  let_next_grid_start();
+  wait_for_prior_grid();
   const int M = min(max(*row_total - row_base, 0), row_limit);
   for (int r = blockIdx.x; r < M; r += gridDim.x) {
     const uint4* src = reinterpret_cast<const uint4*>(x_table + (static_cast<long long>(row_b[r]) * seq_stride + row_tok[r]) * d);
@@ -302,10 +304,6 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int M = min(max(*p.row_total - p.row_base, 0), p.row_limit);
-  const int m_tiles = (M + kTcBM - 1) / kTcBM, n_tiles = p.N / BN;
-  const int total_tiles = m_tiles * n_tiles * p.ksplit;      // work units: (tile, part of K), parts of a tile adjacent
-  const int k_blocks = p.K / kTcBK;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { tc_mbar_init(&full[s], 1u); tc_mbar_init(&empty[s], 1u); }
@@ -319,6 +317,13 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+
+  // barriers and tensor memory are set up; from here on the kernel touches what earlier kernels wrote
+  wait_for_prior_grid();
+  const int M = min(max(*p.row_total - p.row_base, 0), p.row_limit);
+  const int m_tiles = (M + kTcBM - 1) / kTcBM, n_tiles = p.N / BN;
+  const int total_tiles = m_tiles * n_tiles * p.ksplit;      // work units: (tile, part of K), parts of a tile adjacent
+  const int k_blocks = p.K / kTcBK;
 
   if (warp == 0) {
     // ---------------- producer ----------------
@@ -538,22 +543,35 @@ inline adore_status_t tc_set_weights(TcState& s, int layer, const void* w_kv) {
 
 // Gathers the rows and runs the GEMM, in chunks of at most a_rows rows. Returns the launches made.
 template <typename T>
-inline cudaError_t launch_rebuild_tc(TcState&, const RebuildParams<T>&, int, int, cudaStream_t, int*) { return cudaErrorNotSupported; }
+inline cudaError_t launch_rebuild_tc(TcState&, const RebuildParams<T>&, int, int, cudaStream_t, int*, bool) { return cudaErrorNotSupported; }
+template <typename T>
+inline cudaError_t launch_gather_tc(TcState&, const RebuildParams<T>&, int, cudaStream_t) { return cudaErrorNotSupported; }
+
+// Gathers rows [0, m_max) of the row table into the compact A buffer (m_max <= a_rows).
+template <>
+inline cudaError_t launch_gather_tc<__nv_bfloat16>(TcState& s, const RebuildParams<__nv_bfloat16>& rp, int m_max, cudaStream_t stream) {
+  const int gather_grid = std::min(m_max, 8 * s.sms);
+  return launch_dependent(gather_rows_kernel<__nv_bfloat16>, dim3(gather_grid), dim3(256), 0, stream, rp.x_table, rp.seq_stride,
+                          rp.d, rp.row_b, rp.row_tok, rp.row_total, 0, m_max, s.a_buf);
+}
 
 template <>
 inline cudaError_t launch_rebuild_tc<__nv_bfloat16>(TcState& s, const RebuildParams<__nv_bfloat16>& rp, int layer, int m_max,
-                                                    cudaStream_t stream, int* launched) {
+                                                    cudaStream_t stream, int* launched, bool rows_in_place) {
+  // rows_in_place: the A buffer already holds the listed rows (gathered earlier for this row table; one chunk only)
   *launched = 0;
   if (!s.has_w[layer]) return cudaErrorInvalidValue;
   // the table may hold more rows than the gather buffer: go through it in chunks
   for (int base = 0; base < m_max; base += int(s.a_rows)) {
     const int limit = std::min(m_max - base, int(s.a_rows));
-    const int gather_grid = std::min(limit, 8 * s.sms);
-    gather_rows_kernel<__nv_bfloat16><<<gather_grid, 256, 0, stream>>>(rp.x_table, rp.seq_stride, rp.d, rp.row_b + base,
-                                                                    rp.row_tok + base, rp.row_total, base, limit, s.a_buf);
-    ++*launched;
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    if (!(rows_in_place && base == 0 && m_max <= int(s.a_rows))) {
+      const int gather_grid = std::min(limit, 8 * s.sms);
+      e = launch_dependent(gather_rows_kernel<__nv_bfloat16>, dim3(gather_grid), dim3(256), 0, stream, rp.x_table, rp.seq_stride,
+                           rp.d, rp.row_b + base, rp.row_tok + base, rp.row_total, base, limit, s.a_buf);
+      ++*launched;
+      if (e != cudaSuccess) return e;
+    }
     TcGemmParams g{};
     g.Kc = rp.Kc; g.Vc = rp.Vc; g.row_b = rp.row_b + base; g.row_tok = rp.row_tok + base; g.row_slot = rp.row_slot + base;
     g.row_total = rp.row_total; g.row_base = base; g.row_limit = limit;
@@ -563,20 +581,26 @@ inline cudaError_t launch_rebuild_tc<__nv_bfloat16>(TcState& s, const RebuildPar
     g.ksplit = plan.ksplit; g.partial = s.partial; g.unit_cnt = s.unit_cnt;
     if (plan.kind == 2) {
       cudaLaunchConfig_t lc{};
-      cudaLaunchAttribute at[1];
+      cudaLaunchAttribute at[2];
       at[0].id = cudaLaunchAttributeClusterDimension;
       at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      at[1].val.programmaticStreamSerializationAllowed = 1;
+      static const bool no_dep = std::getenv("ADORE_NO_DEPENDENT_LAUNCH") != nullptr;
       lc.gridDim = dim3(unsigned(plan.grid)); lc.blockDim = dim3(kTcThreads); lc.dynamicSmemBytes = kPairSmemBytes;
-      lc.stream = stream; lc.attrs = at; lc.numAttrs = 1;
+      lc.stream = stream; lc.attrs = at; lc.numAttrs = no_dep ? 1 : 2;
       e = cudaLaunchKernelEx(&lc, rebuild_tc_pair_kernel, s.map_a, s.map_w128[layer], g);
       ++*launched;
       if (e != cudaSuccess) return e;
       continue;
     }
-    if (plan.kind == 1) rebuild_tc_kernel<256><<<plan.grid, kTcThreads, TcSmem<256>::kTotal, stream>>>(s.map_a, s.map_w256[layer], g);
-    else rebuild_tc_kernel<128><<<plan.grid, kTcThreads, TcSmem<128>::kTotal, stream>>>(s.map_a, s.map_w128[layer], g);
+    if (plan.kind == 1)
+      e = launch_dependent(rebuild_tc_kernel<256>, dim3(plan.grid), dim3(kTcThreads), TcSmem<256>::kTotal, stream, s.map_a,
+                           s.map_w256[layer], g);
+    else
+      e = launch_dependent(rebuild_tc_kernel<128>, dim3(plan.grid), dim3(kTcThreads), TcSmem<128>::kTotal, stream, s.map_a,
+                           s.map_w128[layer], g);
     ++*launched;
-    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();

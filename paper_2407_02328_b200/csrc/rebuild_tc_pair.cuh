@@ -87,10 +87,6 @@ rebuild_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster.block_rank();             // 0: issues the MMAs, owns full[] and acc_empty[]
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int M = min(max(*p.row_total - p.row_base, 0), p.row_limit);
-  const int m_tiles = (M + 2 * kTcBM - 1) / (2 * kTcBM), n_tiles = p.N / BN;
-  const int total_tiles = m_tiles * n_tiles;
-  const int k_blocks = p.K / kTcBK;
   volatile int* partner_abort = cluster.map_shared_rank(const_cast<int*>(abort_flag), rank ^ 1u);
   auto give_up = [&]() {                                   // a wait ran out (or the partner's did)
     if (!*abort_flag) { set_error(p.err, ERRW_TIMEOUT); *abort_flag = 1; *partner_abort = 1; }
@@ -110,6 +106,13 @@ rebuild_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   cluster.sync();                                          // both CTAs' barriers exist before anything crosses over
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+
+  // barriers and tensor memory are set up; from here on the kernel touches what earlier kernels wrote
+  wait_for_prior_grid();
+  const int M = min(max(*p.row_total - p.row_base, 0), p.row_limit);
+  const int m_tiles = (M + 2 * kTcBM - 1) / (2 * kTcBM), n_tiles = p.N / BN;
+  const int total_tiles = m_tiles * n_tiles;
+  const int k_blocks = p.K / kTcBK;
 
   if (warp == 0) {
     // ---------------- producer: this CTA's half of every stage ----------------

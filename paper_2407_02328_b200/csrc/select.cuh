@@ -268,6 +268,8 @@ __global__ void __launch_bounds__(128) row_table_kernel(const int* rebuild_tok, 
                                                         int* row_slot, int* row_total, unsigned long long* rows_accum) {
   __shared__ int tmp[64];
   const int b = blockIdx.x, tid = threadIdx.x;
+  let_next_grid_start();
+  wait_for_prior_grid();
   int before = 0, all = 0;
   for (int i = tid; i < B; i += blockDim.x) {
     const int c = rebuild_count[i];
