@@ -67,6 +67,11 @@ typedef enum { ADORE_REBUILD_POLICY = 0, ADORE_REBUILD_EXPLICIT = 1 } adore_rebu
 /* Slot roles in the slot map. */
 enum { ADORE_SLOT_EMPTY = 0, ADORE_SLOT_RETAINED = 1, ADORE_SLOT_REBUILT = 2 };
 
+/* Controller ablation "w/o GRU" (Section 3.5.3, Table 5): the cell keeps no memory. Every token is scored
+ * from its own embedding alone, z_i = GRU(x_i, 0), then the same MLP. The paper does not say how the embedding
+ * reaches the MLP without the GRU; applying the cell to a zero state needs no extra parameters. */
+#define ADORE_FLAG_NO_RECURRENCE 1u
+
 typedef struct {
   uint32_t struct_size;  /* sizeof(adore_config_t), for versioning                               */
   int32_t batch;         /* B  sequences                                                        */
@@ -83,7 +88,7 @@ typedef struct {
   adore_rebuild_mode_t rebuild_mode;
   float rope_theta;      /* rotary base; 0 disables the rotation                                 */
   float pos_scale;       /* position feature of the controller is n / pos_scale                  */
-  uint32_t flags;        /* reserved, must be 0                                                  */
+  uint32_t flags;        /* ADORE_FLAG_* bits; unknown bits are rejected                         */
 } adore_config_t;
 
 /* Controller parameters (Section 2.2 Eq. 2 and Appendix B), float32, HOST pointers, copied at

@@ -222,6 +222,7 @@ class OracleConfig:
     rebuild_mode: str = "policy"
     rope_theta: float = 1.0e4
     pos_scale: float = 4096.0
+    no_recurrence: bool = False    # Section 3.5.3 "w/o GRU": z_i = GRU(x_i, 0), no memory of earlier tokens
 
     @property
     def retained_max(self) -> int:
@@ -275,7 +276,8 @@ class AdoreOracle:
         """z_n, score_n, sigma_n for the token at position self.n of every sequence."""
         c, n = self.cfg, self.n
         self.x[:, n, :] = x_new
-        self.z = gru_step(x_new, self.z, self.ctrl)
+        z_prev = np.zeros_like(self.z) if c.no_recurrence else self.z
+        self.z = gru_step(x_new, z_prev, self.ctrl)
         s = controller_score(self.z, n, c.pos_scale, self.ctrl)
         self.score[:, n] = s.astype(np.float32)
         self.sigma[:, n] = _sigm(s).astype(np.float32)

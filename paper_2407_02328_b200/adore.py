@@ -22,6 +22,9 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "OOM", 3: "TOKEN_TABLE_FULL", 4: "
                 6: "DEVICE_FLAG", 7: "TIMEOUT", 8: "UNSUPPORTED"}
 
 
+ADORE_FLAG_NO_RECURRENCE = 1
+
+
 class AdoreError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -256,10 +259,11 @@ def device_view(ptr: int, shape, dtype):
 
 
 def make_config(*, batch, n_layers, n_heads, head_dim, hidden, capacity, rebuild_max, topk, max_tokens,
-                ctrl_hidden=128, dtype="bf16", rebuild_mode="policy", rope_theta=1.0e4, pos_scale=4096.0) -> adore_config_t:
+                ctrl_hidden=128, dtype="bf16", rebuild_mode="policy", rope_theta=1.0e4, pos_scale=4096.0,
+                flags=0) -> adore_config_t:
     return adore_config_t(struct_size=C.sizeof(adore_config_t), batch=batch, n_layers=n_layers, n_heads=n_heads,
                           head_dim=head_dim, hidden=hidden, capacity=capacity, rebuild_max=rebuild_max, topk=topk,
                           max_tokens=max_tokens, ctrl_hidden=ctrl_hidden,
                           dtype=ADORE_F32 if dtype == "f32" else ADORE_BF16,
                           rebuild_mode=ADORE_REBUILD_POLICY if rebuild_mode == "policy" else ADORE_REBUILD_EXPLICIT,
-                          rope_theta=rope_theta, pos_scale=pos_scale, flags=0)
+                          rope_theta=rope_theta, pos_scale=pos_scale, flags=flags)

@@ -233,6 +233,7 @@ RecurParams recur_params(adore_cache* c, int rows, int tc, int ksplit, int n0) {
   r.w1 = c->w1; r.b1 = c->b1; r.w2 = c->w2; r.b2 = c->b2;
   r.z = c->z; r.score = c->score; r.sigma = c->sigma; r.max_tokens = c->cfg.max_tokens; r.n0 = n0;
   r.pos_scale = double(c->cfg.pos_scale);
+  r.no_recurrence = (c->cfg.flags & ADORE_FLAG_NO_RECURRENCE) ? 1 : 0;
   return r;
 }
 
@@ -357,7 +358,7 @@ adore_status_t fill_layer_impl(adore_cache* c, int layer, const void* x_table) {
 adore_status_t check_config(const adore_config_t* f) {
   if (f->struct_size != sizeof(adore_config_t)) return ADORE_ERR_INVALID_ARG;
   if (f->batch < 1 || f->n_layers < 1 || f->n_heads < 1 || f->hidden < 1 || f->capacity < 1 || f->topk < 1 ||
-      f->max_tokens < 1 || f->ctrl_hidden < 1 || f->rebuild_max < 0 || f->rebuild_max >= f->capacity || f->flags != 0 ||
+      f->max_tokens < 1 || f->ctrl_hidden < 1 || f->rebuild_max < 0 || f->rebuild_max >= f->capacity || (f->flags & ~uint32_t(ADORE_FLAG_NO_RECURRENCE)) != 0 ||
       !(f->pos_scale > 0.f) || f->rope_theta < 0.f)
     return ADORE_ERR_INVALID_ARG;
   if (f->dtype != ADORE_F32 && f->dtype != ADORE_BF16) return ADORE_ERR_INVALID_ARG;

@@ -135,6 +135,7 @@ struct RecurParams {
   int max_tokens;
   int n0;                // position of the first token of this call
   double pos_scale;
+  int no_recurrence;     // 1: every token sees a zero state (the ablation without the GRU's memory, Section 3.5.3)
 };
 
 
@@ -157,6 +158,11 @@ __device__ __forceinline__ void controller_tokens_impl(const RecurParams& p, int
   __syncthreads();
   for (int t = 0; t < p.tc; ++t) {
     const int row = b * p.tc + t;
+    if (p.no_recurrence) {
+      __syncthreads();
+      for (int i = tid; i < h; i += blockDim.x) s_z[i] = 0.0;
+      __syncthreads();
+    }
     // four output rows per warp at a time: all their loads are issued before the first is used
     for (int g0 = warp * 4; g0 < G; g0 += nw * 4) {
       float w[4][kCtrlJ];
@@ -310,6 +316,11 @@ __device__ __forceinline__ void controller_tokens_resident(const RecurParams& p,
   bool have_w = false;
   for (int t = 0; t < p.tc; ++t) {
     const int row = b * p.tc + t;
+    if (p.no_recurrence) {
+      __syncthreads();
+      for (int i = tid; i < h; i += blockDim.x) s_z[i] = 0.0;
+      __syncthreads();
+    }
     // input-side sums: the k-slices are added in a fixed order
     for (int g = tid; g < G; g += blockDim.x) {
       double gi = double(__ldg(p.b_ih + g));

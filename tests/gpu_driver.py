@@ -55,7 +55,8 @@ class GpuCache:
             lib.make_config(batch=self.B, n_layers=c.n_layers, n_heads=c.n_heads, head_dim=c.head_dim,
                             hidden=c.hidden, capacity=c.capacity, rebuild_max=c.rebuild_max, topk=c.topk,
                             max_tokens=c.max_tokens, ctrl_hidden=c.ctrl_hidden, dtype=c.dtype,
-                            rebuild_mode=c.rebuild_mode, rope_theta=c.rope_theta, pos_scale=c.pos_scale),
+                            rebuild_mode=c.rebuild_mode, rope_theta=c.rope_theta, pos_scale=c.pos_scale,
+                            flags=lib.ADORE_FLAG_NO_RECURRENCE if c.ctrl_no_recurrence else 0),
             w.ctrl, torch.cuda.current_stream().cuda_stream)
         self.w_kv_dev = [to_dev(m, c) for m in w.w_kv]
         for l, m in enumerate(self.w_kv_dev):

@@ -118,3 +118,11 @@ def test_controller_widths_off_the_default():
     shared-memory-resident one with partly filled warps."""
     _run(SMALL.scaled(name="ctrl160", ctrl_hidden=160, steps=25, seed=115))
     _run(SMALL.scaled(name="ctrl96", ctrl_hidden=96, steps=25, seed=116))
+
+
+def test_controller_ablations_width_64_and_no_recurrence():
+    """Section 3.5.3's variants: d' = 64, and the controller whose cell sees a zero state at every token (prompt scan
+    and decode steps both take the flag)."""
+    _run(SMALL.scaled(name="ctrl64", ctrl_hidden=64, steps=25, seed=121))
+    _run(SMALL.scaled(name="norecurrence", ctrl_no_recurrence=True, steps=25, seed=122))
+    _run(SMALL.scaled(name="norecurrence160", ctrl_no_recurrence=True, ctrl_hidden=160, steps=12, seed=123))

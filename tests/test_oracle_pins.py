@@ -376,6 +376,32 @@ def test_occupancy_never_exceeds_capacity_on_config_one():
     assert sum(len(l) for l in orc.info.rebuild_tok) >= 0
 
 
+def test_controller_without_recurrence_forgets_earlier_tokens():
+    """Section 3.5.3 "w/o GRU": the score of a token depends on its own embedding and position only, so shuffling the
+    tokens before it changes nothing; with the recurrence the same shuffle moves the score."""
+    cfg = wl.WorkloadConfig(name="norec", dtype="f32", n_layers=1, batch=2, n_heads=2, head_dim=64, hidden=128,
+                            capacity=16, topk=8, rebuild_max=2, prompt=0, steps=12, rope_theta=0.0,
+                            rebuild_mode="policy", rebuild_p=0.0, seed=77, ctrl_hidden=32)
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((2, 9, 128)).astype(np.float32)
+    perm = np.array([3, 0, 6, 1, 7, 5, 2, 4, 8])                 # the last token stays last
+    last = {}
+    for norec in (True, False):
+        for name, xs in (("plain", x), ("shuffled", x[:, perm])):
+            w = Workload(cfg.scaled(ctrl_no_recurrence=norec))
+            orc = make_oracle(w)
+            orc.append_tokens(xs)
+            last[norec, name] = orc.score[:, 8].copy()
+    assert np.array_equal(last[True, "plain"], last[True, "shuffled"])
+    assert not np.allclose(last[False, "plain"], last[False, "shuffled"], rtol=0, atol=1e-7)
+    # and it is the cell applied to a zero state: one token alone in an empty cache scores the same
+    w = Workload(cfg.scaled(ctrl_no_recurrence=True))
+    alone = make_oracle(w)
+    alone.n = 8                                                   # same position, nothing before it
+    alone._score_new_token(x[:, 8])
+    assert np.array_equal(alone.score[:, 8], last[True, "plain"])
+
+
 # ------------------------------------------------------------------ planted mistakes
 def test_pins_notice_planted_mistakes(monkeypatch):
     """Each plausible slip, planted in the oracle, must make one of the pins above fail."""

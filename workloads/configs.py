@@ -36,6 +36,7 @@ class WorkloadConfig:
     pos_scale: float = 4096.0
     identity_projection: bool = False   # W_k = W_v = I (needs hidden == n_heads*head_dim)
     per_layer_inputs: bool = False      # every layer has its own RMS-normalised input rows
+    ctrl_no_recurrence: bool = False    # controller ablation without the GRU's memory: every token sees a zero state
 
     @property
     def retained_max(self) -> int:
