@@ -86,20 +86,21 @@ def topk_keep(logits: np.ndarray, valid: np.ndarray, k: int) -> np.ndarray:
 
 
 def sparse_attention(q: np.ndarray, Kc: np.ndarray, Vc: np.ndarray, occupied: np.ndarray,
-                     k_new: np.ndarray, v_new: np.ndarray, topk: int
+                     k_new: np.ndarray, v_new: np.ndarray, topk: int, own_row: bool = True
                      ) -> Tuple[np.ndarray, np.ndarray]:
     """Target / rebuild attention for one sequence, all heads (Section 2.1, Section 2.3).
 
     q, k_new, v_new: [H, dh]; Kc, Vc: [H, C, dh]; occupied: [C] bool (same for all heads).
     Candidates are the occupied slots followed by the current token's own row (index C).
     Only the `topk` largest logits keep a weight. Returns out [H, dh] and weights
-    [H, C+1] (float64; zero for empty or masked rows).
+    [H, C+1] (float64; zero for empty or masked rows). own_row=False drops the row at index C from the
+    candidates (a rebuilt token's query must not see the current token, which comes after it).
     """
     H, C, dh = Kc.shape
     q = np.asarray(q, np.float64)
     Kall = np.concatenate([np.asarray(Kc, np.float64), np.asarray(k_new, np.float64)[:, None, :]], 1)
     Vall = np.concatenate([np.asarray(Vc, np.float64), np.asarray(v_new, np.float64)[:, None, :]], 1)
-    valid = np.concatenate([np.asarray(occupied, bool), [True]])[None, :].repeat(H, 0)
+    valid = np.concatenate([np.asarray(occupied, bool), [bool(own_row)]])[None, :].repeat(H, 0)
     logit = np.einsum("hd,hcd->hc", q, Kall) / np.sqrt(dh)
     keep = topk_keep(logit, valid, topk)
     lg = np.where(keep, logit, -np.inf)
@@ -433,6 +434,56 @@ class AdoreOracle:
             s = int(self.info.admit_slot[b])
             self.Kc[layer, b, :, s, :] = round_store(k_new[b], c.dtype)
             self.Vc[layer, b, :, s, :] = round_store(v_new[b], c.dtype)
+        return out, wts
+
+    # -- the step in the order Section 2.3 prints it: select, rebuild, then attend with R+1 query rows ----
+    def step_begin(self, x_new: np.ndarray, explicit: Optional[List[np.ndarray]] = None) -> None:
+        """Controller and selection for token n before any attention of the step: afterwards the map holds the
+        retained tokens, the slots of this step's rebuild list and the slot token n will be written to."""
+        c = self.cfg
+        if self.n >= c.max_tokens:
+            raise IndexError("token table full")
+        self._score_new_token(x_new)
+        admit = np.zeros(c.batch, np.int32)
+        evict = np.zeros(c.batch, np.int32)
+        lists, slots = [], []
+        for b in range(c.batch):
+            a, e, lst, sl = self._select_one(b, None if explicit is None else explicit[b])
+            admit[b], evict[b] = a, e
+            lists.append(lst)
+            slots.append(sl)
+        self.info = StepInfo(admit, evict, lists, slots)
+        self.n += 1
+
+    def attend_rows(self, layer: int, q_rows: np.ndarray, k_new: np.ndarray, v_new: np.ndarray
+                    ) -> Tuple[np.ndarray, np.ndarray]:
+        """The attention of Section 2.3 for `layer`, after step_begin() and rebuild(layer): R_max + 1 query rows per
+        sequence, row i < R_max for the i-th token of the rebuild list (rows past the list's end are padding and
+        return zeros), the last row for the current token. Keys and values are the cached rows, the rebuilt rows
+        (already in their slots) and the current token's own row; a query sees only tokens at positions up to its
+        own, and keeps the `topk` largest logits. Then the current token's row is stored in its slot.
+
+        q_rows: [B, H, R_max+1, dh]; returns out [B, H, R_max+1, dh] and weights [B, H, R_max+1, C+1].
+        """
+        c = self.cfg
+        B, H, C, dh, R1 = c.batch, c.n_heads, c.capacity, c.head_dim, c.rebuild_max + 1
+        n = self.n - 1                                        # position of the current token
+        out = np.zeros((B, H, R1, dh), np.float64)
+        wts = np.zeros((B, H, R1, C + 1), np.float64)
+        for b in range(B):
+            lst = self.info.rebuild_tok[b]
+            for i in range(R1):
+                tok = n if i == R1 - 1 else (int(lst[i]) if i < len(lst) else -1)
+                if tok < 0:
+                    continue
+                st = self.slot_tok[b]
+                seen = (st >= 0) & (st <= tok) & (st != n)     # token n's slot is reserved, its row not written yet
+                out[b, :, i], wts[b, :, i] = sparse_attention(q_rows[b, :, i], self.Kc[layer, b], self.Vc[layer, b], seen,
+                                                              k_new[b], v_new[b], c.topk, own_row=(tok == n))
+        for b in range(B):
+            s_ = int(self.info.admit_slot[b])
+            self.Kc[layer, b, :, s_, :] = round_store(k_new[b], c.dtype)
+            self.Vc[layer, b, :, s_, :] = round_store(v_new[b], c.dtype)
         return out, wts
 
     def rebuild(self, layer: int, x_table: Optional[np.ndarray] = None) -> int:

@@ -66,6 +66,25 @@ class Workload:
             q = ao.round_store(ao.rope_rotate(yq.reshape(B, c.n_heads, c.head_dim), n, c.rope_theta), c.dtype)
         return q, k, v
 
+    def q_rows(self, n: int, layer: int, x_table: np.ndarray, lists) -> np.ndarray:
+        """Query rows [B, H, R_max+1, dh] of the step in the order of Section 2.3: row i < R_max for the i-th token of
+        sequence b's rebuild list (zeros past the list's end), the last row for the current token n; each row is
+        projected from that token's layer input x_table[b, tok] and rotated to the token's own position."""
+        c = self.cfg
+        R1 = c.rebuild_max + 1
+        out = np.zeros((self.batch, c.n_heads, R1, c.head_dim), np.float32)
+        for b in range(self.batch):
+            toks = [int(t) for t in lists[b]] + [-1] * (c.rebuild_max - len(lists[b])) + [n]
+            for i, tok in enumerate(toks):
+                if tok < 0:
+                    continue
+                if c.identity_projection:
+                    out[b, :, i] = wl.gaussian(c.seed, "q", (c.n_heads, c.head_dim), 1.0, c.dtype, idx=(layer, tok, b))
+                else:
+                    out[b, :, i] = ao.project_q(self.w_q64[layer], x_table[b, tok], tok, c.n_heads, c.head_dim,
+                                                c.rope_theta, c.dtype)
+        return out
+
     def explicit(self, step: int, n: int) -> Tuple[Optional[np.ndarray], Optional[np.ndarray]]:
         if self.cfg.rebuild_mode != "explicit":
             return None, None

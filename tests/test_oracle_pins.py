@@ -260,6 +260,81 @@ def test_path_equals_full_attention_when_every_token_is_resident(rebuild_max, pr
                 assert np.allclose(out[b, h], ref, rtol=0, atol=1e-12)
 
 
+def run_rebuild_first(cfg, steps=None):
+    """The step in the order Section 2.3 prints it: select, rebuild, attend with R_max + 1 query rows."""
+    w = Workload(cfg)
+    orc = make_oracle(w)
+    if cfg.prompt:
+        orc.append_tokens(w.prompt())
+    hist = []
+    for s in range(cfg.steps if steps is None else steps):
+        n = orc.n
+        x = w.x_new(n)
+        _, k, v = w.qkv(n, 0, x)
+        lists, counts = w.explicit(s, n)
+        orc.step_begin(x, explicit_as_lists(lists, counts))
+        orc.rebuild(0)
+        q_rows = w.q_rows(n, 0, orc.x, orc.info.rebuild_tok)
+        out, wts = orc.attend_rows(0, q_rows, k, v)
+        orc.check_invariants()
+        hist.append((n, [list(map(int, l)) for l in orc.info.rebuild_tok], q_rows, out, wts))
+    return w, orc, hist
+
+
+@pytest.mark.parametrize("rebuild_max,prompt", [(20, 0), (27, 6)])
+def test_rebuilt_query_rows_equal_causal_full_attention_when_every_token_is_resident(rebuild_max, prompt):
+    """Section 2.3: with every token either retained or rebuilt, query row i must be Eq. 1 for its own token over the
+    tokens up to its own position, and the last row Eq. 1 for the current token; rows past the list are zero."""
+    cfg = TINY.scaled(capacity=32, topk=64, rebuild_max=rebuild_max, prompt=prompt, steps=30 - prompt)
+    w, orc, hist = run_rebuild_first(cfg)
+    K, V = history_kv(w, orc, orc.n)
+    rows_checked = 0
+    for n, lists, q_rows, out, _ in hist:
+        for b in range(w.batch):
+            toks = lists[b] + [-1] * (rebuild_max - len(lists[b])) + [n]
+            for i, tok in enumerate(toks):
+                for h in range(cfg.n_heads):
+                    if tok < 0:
+                        assert not out[b, h, i].any()
+                        continue
+                    ref = brute_attention(q_rows[b, h, i].astype(np.float64), K[b, h, : tok + 1], V[b, h, : tok + 1])
+                    assert np.allclose(out[b, h, i], ref, rtol=0, atol=1e-12)
+                    rows_checked += 1
+    assert rows_checked > 200
+
+
+def test_rebuilt_query_rows_do_not_see_later_tokens():
+    """A row's output must not move when the cache row of a LATER token changes, and must move when an earlier one does."""
+    cfg = TINY.scaled(capacity=32, topk=64, rebuild_max=20, prompt=0, steps=20)
+    w, orc, hist = run_rebuild_first(cfg, steps=19)
+    n = orc.n
+    x = w.x_new(n)
+    _, k, v = w.qkv(n, 0, x)
+    orc.step_begin(x, None)
+    orc.rebuild(0)
+    lst = [int(t) for t in orc.info.rebuild_tok[0]]
+    assert len(lst) >= 3
+    q_rows = w.q_rows(n, 0, orc.x, orc.info.rebuild_tok)
+    import copy
+    base, _ = copy.deepcopy(orc).attend_rows(0, q_rows, k, v)
+    i = int(np.argmin(lst))                                  # the oldest rebuilt token's row
+    later = [s for s in range(cfg.capacity) if orc.slot_tok[0, s] > lst[i] and orc.slot_tok[0, s] != n]
+    earlier = [s for s in range(cfg.capacity) if 0 <= orc.slot_tok[0, s] <= lst[i]]
+    assert later and earlier
+    o2 = copy.deepcopy(orc)
+    o2.Vc[0, 0, :, later[0], :] += 1.0
+    moved, _ = o2.attend_rows(0, q_rows, k, v)
+    assert np.array_equal(moved[0, :, i], base[0, :, i])
+    o3 = copy.deepcopy(orc)
+    o3.Vc[0, 0, :, earlier[0], :] += 1.0
+    moved, _ = o3.attend_rows(0, q_rows, k, v)
+    assert not np.allclose(moved[0, :, i], base[0, :, i])
+    # the current token's own row reaches the last query only
+    o4 = copy.deepcopy(orc)
+    moved, _ = o4.attend_rows(0, q_rows, k, v + 1.0)
+    assert np.array_equal(moved[0, :, :-1], base[0, :, :-1]) and not np.allclose(moved[0, :, -1], base[0, :, -1])
+
+
 def brute_select(score, slot_tok, slot_role, n, m, r_max, explicit):
     """Section 2.2 release rule and Section 2.3 list choice with Python sorts on (score, tok)."""
     slot_tok, slot_role = list(slot_tok), list(slot_role)
