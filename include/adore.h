@@ -250,6 +250,27 @@ adore_status_t adore_controller_score_static(const adore_controller_weights_t *w
                                              double *z, int32_t position, float pos_scale, float *score,
                                              float *sigma, void *cuda_stream);
 
+/* The step in the order Section 2.3 prints it: select first, then rebuild, then one attention in which the rebuilt
+ * tokens' query rows and the current token's share the key and value rows.
+ *
+ * adore_step_begin: controller + selection for the new token n (Section 2.2 Eq. 2 and release rule, Section 2.3
+ *   first sentence); x_new [B, d] DEVICE and the explicit list as for adore_decode_step at layer 0. Afterwards the
+ *   slot map holds the retained tokens, the slots of this step's rebuild list and the slot token n will get.
+ * Then per layer: adore_rebuild(cache, layer, x_table) writes the listed tokens' K/V rows, and
+ * adore_attend_rows runs Section 2.3's attention: q_rows [B, H, R_max+1, dh] DEVICE, row i < R_max for the i-th
+ *   token of adore_cache_rebuild_list() (rows past a sequence's count are ignored and produce zeros), the last row
+ *   for token n; k_new, v_new [B, H, dh] DEVICE are token n's own rows. Row i attends over the occupied slots
+ *   whose token position is at most its own (the cached and the rebuilt rows), the last row over token n's own
+ *   row too; each row keeps its topk largest logits. out [B, H, R_max+1, dh] DEVICE; weights
+ *   [B, H, R_max+1, C+1] float DEVICE or NULL. The call then stores k_new, v_new in token n's slot.
+ *   Needs head_dim 64 or 128 (ADORE_ERR_UNSUPPORTED otherwise).
+ * A step opened by adore_step_begin must be finished with these calls; adore_decode_step at layer 0 opens a
+ * step of the other kind. Mixing the two within a step returns ADORE_ERR_STATE. */
+adore_status_t adore_step_begin(adore_cache_t *cache, const void *x_new, const int32_t *explicit_list,
+                                const int32_t *explicit_count, int32_t r_in);
+adore_status_t adore_attend_rows(adore_cache_t *cache, int32_t layer, const void *q_rows, const void *k_new,
+                                 const void *v_new, void *out, float *weights);
+
 /* Snapshot of the small per-sequence state that scoring and selection carry from step to step
  * (Section 2.2: which tokens hold which slots, every token's controller score and the GRU state z;
  * Section 2.3: the step's rebuild list): both slot-map buffers, the token-to-slot table, score and sigma

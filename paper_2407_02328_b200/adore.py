@@ -53,7 +53,7 @@ EXPORTS = ["adore_cache_create", "adore_cache_destroy", "adore_cache_set_project
            "adore_cache_launch_count", "adore_cache_sync_status", "adore_status_string",
            "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows",
            "adore_controller_score_static", "adore_probe_read_bandwidth",
-           "adore_cache_export_state", "adore_cache_import_state"]
+           "adore_cache_export_state", "adore_cache_import_state", "adore_step_begin", "adore_attend_rows"]
 
 
 def _lib():
@@ -74,6 +74,8 @@ def _lib():
         lib.adore_decode_step.argtypes = step
         lib.adore_decode_step_host.argtypes = step
         lib.adore_rebuild.argtypes = [vp, i32, vp]
+        lib.adore_step_begin.argtypes = [vp, vp, vp, vp, i32]
+        lib.adore_attend_rows.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         lib.adore_cache_slot_map.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
         lib.adore_cache_rebuild_list.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
         lib.adore_cache_step_info.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
@@ -150,6 +152,15 @@ def adore_decode_step_host(cache: int, layer: int, q, k_new, v_new, x_new, expli
     _check(_lib().adore_decode_step_host(cache, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(x_new),
                                          _ptr(explicit_list), _ptr(explicit_count), r_in, _ptr(out), _ptr(weights)),
            "adore_decode_step_host")
+
+
+def adore_step_begin(cache: int, x_new, explicit_list, explicit_count, r_in: int) -> None:
+    _check(_lib().adore_step_begin(cache, _ptr(x_new), _ptr(explicit_list), _ptr(explicit_count), r_in), "adore_step_begin")
+
+
+def adore_attend_rows(cache: int, layer: int, q_rows, k_new, v_new, out, weights=None) -> None:
+    _check(_lib().adore_attend_rows(cache, layer, _ptr(q_rows), _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(weights)),
+           "adore_attend_rows")
 
 
 def adore_rebuild(cache: int, layer: int, x_table=None) -> None:

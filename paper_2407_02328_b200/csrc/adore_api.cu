@@ -266,7 +266,7 @@ adore_status_t launch_gates(adore_cache* c, const T* x, long long seq_stride, in
 
 template <typename T>
 adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const void* k_new, const void* v_new,
-                                void* out, float* weights, bool fused_admit) {
+                                void* out, float* weights, bool fused_admit, int rows_q = 1) {
   const adore_config_t& f = c->cfg;
   AttnParams<T> p{};
   const size_t layer_elems = size_t(f.batch) * f.n_heads * f.capacity * f.head_dim;
@@ -274,10 +274,11 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
   p.out = static_cast<T*>(out); p.weights = weights;
   p.Kc = static_cast<T*>(c->Kc) + layer * layer_elems; p.Vc = static_cast<T*>(c->Vc) + layer * layer_elems;
   p.slot_tok = c->slot_tok[c->attn]; p.admit_slot = fused_admit ? c->admit_slot : nullptr;
+  p.rows_q = rows_q; p.row_tok = c->rebuild_tok; p.r_max = f.rebuild_max; p.n_cur = c->n - 1;
   p.B = f.batch; p.H = f.n_heads; p.C = f.capacity; p.topk = f.topk;
   p.scale = float(1.0 / std::sqrt(double(f.head_dim)));
   p.err = c->err;
-  const int grid = f.batch * f.n_heads;
+  const int grid = f.batch * f.n_heads * rows_q;
   StageScope scope(c, 0);
   cudaError_t e;
   // ADORE_ATTN_DIRECT=1 selects the variant without shared-memory staging (for A/B timing)
@@ -285,6 +286,13 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
   // Few (b, h) pairs: a cluster of CTAs shares each of them. Not at layer 0: there the controller's
   // one-CTA-per-sequence kernel (200 KB of shared memory each) runs beside the attention and needs
   // SMs that the extra CTAs would occupy; measured at batch 1 the step got slower, not faster.
+  if (rows_q > 1) {            // several query rows per pair: the staged kernel only
+    if (!attn_tma_usable<T>(f.capacity, f.head_dim)) return ADORE_ERR_UNSUPPORTED;
+    cudaError_t er = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
+    ++c->launches;
+    CUDA_OK(er);
+    return ADORE_OK;
+  }
   const int split = (direct || layer == 0) ? 1 : attn_split_factor(grid, f.capacity, c->sms);
   if (split > 1) e = launch_attention_split<T>(p, f.head_dim, grid, split, c->stream);
   else if (!direct && attn_tma_usable<T>(f.capacity, f.head_dim)) e = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
@@ -366,6 +374,49 @@ adore_status_t check_config(const adore_config_t* f) {
   if (f->head_dim != 64 && f->head_dim != 128) return ADORE_ERR_UNSUPPORTED;
   if (f->capacity > 4096 || f->max_tokens > 8192 || f->ctrl_hidden > 256 || f->hidden % 64 != 0)
     return ADORE_ERR_UNSUPPORTED;
+  return ADORE_OK;
+}
+
+}  // namespace
+
+namespace {
+
+// Launches the controller of token n (gates, then GRU + MLP + score) on the controller stream and the step's
+// selection and row table on `sel`. Both streams must already wait for everything they depend on in the main stream.
+adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new, const int32_t* explicit_list,
+                                             const int32_t* explicit_count, int32_t r_in, cudaStream_t sel) {
+  const adore_config_t& f = c->cfg;
+  const bool ex = f.rebuild_mode == ADORE_REBUILD_EXPLICIT;
+  adore_status_t st;
+  StageScope scope(c, 1);
+  if (c->ctrl_pending) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_ctrl, 0));   // scores of token n-1
+  if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit, c->ctl);
+  else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit, c->ctl);
+  if (st != ADORE_OK) return st;
+  CUDA_OK(cudaEventRecord(c->ev_gates, c->ctl));
+  const int P = ex ? pow2_at_least(r_in) : pow2_at_least(c->n);
+  SelectParams sp = select_params(c, c->n, P, c->cur, 1 - c->cur);
+  sp.explicit_list = ex && r_in > 0 ? explicit_list : nullptr;
+  sp.explicit_count = ex && r_in > 0 ? explicit_count : nullptr;
+  sp.r_in = r_in;
+  const size_t smem = select_smem_bytes(f.capacity, P);
+  if (f.dtype == ADORE_F32)
+    select_kernel<float><<<f.batch, select_threads(c), smem, sel>>>(
+        sp, static_cast<const float*>(x_new), static_cast<float*>(c->x_store), f.hidden);
+  else
+    select_kernel<__nv_bfloat16><<<f.batch, select_threads(c), smem, sel>>>(
+        sp, static_cast<const __nv_bfloat16*>(x_new), static_cast<__nv_bfloat16*>(c->x_store), f.hidden);
+  ++c->launches;
+  CUDA_OK(cudaGetLastError());
+  st = launch_row_table(c, true, sel);
+  if (st != ADORE_OK) return st;
+  RecurParams rp = recur_params(c, f.batch, 1, c->ksplit, c->n);
+  ctrl_recur_kernel<<<f.batch, select_threads(c), ctrl_smem(c), c->ctl>>>(rp, ctrl_resident_ok(f.ctrl_hidden) ? 1 : 0, c->err);
+  ++c->launches;
+  CUDA_OK(cudaGetLastError());
+  CUDA_OK(cudaEventRecord(c->ev_ctrl, c->ctl));
+  c->ctrl_pending = true;
+  if (c->timing) { CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_ctrl, 0)); c->ctrl_pending = false; }
   return ADORE_OK;
 }
 
@@ -615,37 +666,8 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     if (c->timing) CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
     if (sel != c->stream) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_fork, 0));
     CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
-    {
-      StageScope scope(c, 1);
-      if (c->ctrl_pending) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_ctrl, 0));   // scores of token n-1
-      if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit, c->ctl);
-      else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit, c->ctl);
-      if (st != ADORE_OK) return st;
-      CUDA_OK(cudaEventRecord(c->ev_gates, c->ctl));
-      const int P = ex ? pow2_at_least(r_in) : pow2_at_least(c->n);
-      SelectParams sp = select_params(c, c->n, P, c->cur, 1 - c->cur);
-      sp.explicit_list = ex && r_in > 0 ? explicit_list : nullptr;
-      sp.explicit_count = ex && r_in > 0 ? explicit_count : nullptr;
-      sp.r_in = r_in;
-      const size_t smem = select_smem_bytes(f.capacity, P);
-      if (f.dtype == ADORE_F32)
-        select_kernel<float><<<f.batch, select_threads(c), smem, sel>>>(
-            sp, static_cast<const float*>(x_new), static_cast<float*>(c->x_store), f.hidden);
-      else
-        select_kernel<__nv_bfloat16><<<f.batch, select_threads(c), smem, sel>>>(
-            sp, static_cast<const __nv_bfloat16*>(x_new), static_cast<__nv_bfloat16*>(c->x_store), f.hidden);
-      ++c->launches;
-      CUDA_OK(cudaGetLastError());
-      st = launch_row_table(c, true, sel);
-      if (st != ADORE_OK) return st;
-      RecurParams rp = recur_params(c, f.batch, 1, c->ksplit, c->n);
-      ctrl_recur_kernel<<<f.batch, select_threads(c), ctrl_smem(c), c->ctl>>>(rp, ctrl_resident_ok(f.ctrl_hidden) ? 1 : 0, c->err);
-      ++c->launches;
-      CUDA_OK(cudaGetLastError());
-      CUDA_OK(cudaEventRecord(c->ev_ctrl, c->ctl));
-      c->ctrl_pending = true;
-      if (c->timing) { CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_ctrl, 0)); c->ctrl_pending = false; }
-    }
+    st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel);
+    if (st != ADORE_OK) return st;
     // A short list's rows are copied out of the token store into the GEMM's compact input right away, beside the
     // attention, so that the rebuild that follows starts with its GEMM. Long lists are copied after the attention:
     // side by side the two slow each other down by more than the copy takes (measured at 15k rows: attention
@@ -669,8 +691,8 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     c->cur = 1 - c->cur;
     c->n += 1;
     c->step_layer0_done = 1;
-  } else if (!c->step_layer0_done) {
-    return ADORE_ERR_STATE;
+  } else if (c->step_layer0_done != 1) {
+    return ADORE_ERR_STATE;       // no step open, or one opened by adore_step_begin
   }
   if (layer != 0)
     return f.dtype == ADORE_F32 ? launch_attention<float>(c, layer, q, k_new, v_new, out, weights, true)
@@ -688,6 +710,46 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     CUDA_OK(cudaGetLastError());
   }
   return ADORE_OK;
+}
+
+adore_status_t adore_step_begin(adore_cache_t* c, const void* x_new, const int32_t* explicit_list,
+                                const int32_t* explicit_count, int32_t r_in) {
+  if (!c || !x_new) return ADORE_ERR_INVALID_ARG;
+  const adore_config_t& f = c->cfg;
+  if (c->n >= f.max_tokens) return ADORE_ERR_TOKEN_TABLE_FULL;
+  const bool ex = f.rebuild_mode == ADORE_REBUILD_EXPLICIT;
+  if (r_in < 0 || (ex && r_in > 0 && (!explicit_list || !explicit_count))) return ADORE_ERR_INVALID_ARG;
+  if (ex && r_in > 8192) return ADORE_ERR_UNSUPPORTED;
+  // nothing of this step has run yet: selection and controller start side by side, the main stream waits for the
+  // selection (the rebuild and the attention of the step read its map) and for the kernel that reads x_new
+  cudaStream_t sel = c->timing ? c->stream : c->aux;
+  CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
+  if (sel != c->stream) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_fork, 0));
+  CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
+  adore_status_t st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel);
+  if (st != ADORE_OK) return st;
+  c->rows_gathered = false;
+  if (sel != c->stream) {
+    CUDA_OK(cudaEventRecord(c->ev_join, sel));
+    CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
+  }
+  c->joined = true;
+  CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_gates, 0));
+  c->cur = 1 - c->cur;
+  c->attn = c->cur;             // this step's attention reads the NEW map
+  c->n += 1;
+  c->step_layer0_done = 2;      // a rebuild-first step is open
+  return ADORE_OK;
+}
+
+adore_status_t adore_attend_rows(adore_cache_t* c, int32_t layer, const void* q_rows, const void* k_new, const void* v_new,
+                                 void* out, float* weights) {
+  if (!c || !q_rows || !k_new || !v_new || !out || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (c->step_layer0_done != 2) return ADORE_ERR_STATE;
+  const adore_config_t& f = c->cfg;
+  const int rows_q = f.rebuild_max + 1;
+  return f.dtype == ADORE_F32 ? launch_attention<float>(c, layer, q_rows, k_new, v_new, out, weights, true, rows_q)
+                              : launch_attention<__nv_bfloat16>(c, layer, q_rows, k_new, v_new, out, weights, true, rows_q);
 }
 
 adore_status_t adore_decode_step_host(adore_cache_t* c, int32_t layer, const void* q, const void* k_new,

@@ -30,6 +30,14 @@ struct AttnParams {
   int B, H, C, topk;
   float scale;           // 1/sqrt(DH)
   unsigned* err;
+  // Several query rows per (b, h) (Section 2.3: the rebuilt tokens' rows and the current token's; 1 = the plain
+  // decode step). q, out and weights then hold rows_q rows per pair, item = (b*H + h) * rows_q + i. Row i < rows_q-1
+  // belongs to token row_tok[b*r_max + i] (< 0: padding, the row's output is zero), the last row to token n_cur. A row
+  // sees the slots whose token position is at most its own, never the slot reserved for n_cur (not written yet), and
+  // the current token's own row (index C) only if it is the last row.
+  int rows_q;
+  const int* row_tok;    // [B, r_max] or nullptr
+  int r_max, n_cur;
 };
 
 constexpr int kAttnThreads = 256;
@@ -91,7 +99,7 @@ struct AttnSmem {
 // builds the ordered list of kept row indices. Returns the number of kept rows. Every thread of the
 // block calls it after a __syncthreads(); the results are published by a final __syncthreads().
 template <typename T, int DH, int NT = kAttnThreads>
-__device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh) {
+__device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh /* row of out/weights */) {
   constexpr int NW = NT / 32;
   float* s_logit = sm.logit;
   int* s_list = sm.list;
@@ -247,7 +255,8 @@ __device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, 
 // row into its slot (append of the most recent state, Section 2.2 third bullet).
 template <typename T, int DH, int NT = kAttnThreads>
 __device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh,
-                                                 float (&acc)[Elem<T>::kPer16B]) {
+                                                 float (&acc)[Elem<T>::kPer16B], int out_row = -1, bool admit = true) {
+  if (out_row < 0) out_row = bh;
   constexpr int NW = NT / 32;
   constexpr int EPL = Elem<T>::kPer16B;
   constexpr int LPR = DH / EPL;
@@ -279,11 +288,11 @@ __device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const A
     float s = 0.f;
 #pragma unroll
     for (int w = 0; w < NW; ++w) s += s_red[w * DH + e];
-    p.out[size_t(bh) * DH + e] = Elem<T>::from_float(s);
+    p.out[size_t(out_row) * DH + e] = Elem<T>::from_float(s);
   }
 
   // ---- admit: the current token's row goes into its slot (all reads of this block are done) --
-  if (p.admit_slot != nullptr) {
+  if (admit && p.admit_slot != nullptr) {
     const int s = p.admit_slot[b];
     if (s >= 0 && s < C) {
       constexpr int V16 = int(sizeof(T)) * DH / 16;

@@ -48,12 +48,26 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane / LPR, li = lane % LPR;
-  const int bh = blockIdx.x, b = bh / p.H;
+  // item = one query row; with rows_q > 1 the rows of a (b, h) pair sit next to each other in the grid, so that the
+  // pair's key and value blocks are fetched from HBM once and served to the other rows out of L2
+  const int item = blockIdx.x, qi = item % p.rows_q, bh = item / p.rows_q, b = bh / p.H;
+  const bool last_row = qi == p.rows_q - 1;
   const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * ROW_BYTES;
   const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * ROW_BYTES;
   const int* map = p.slot_tok + size_t(b) * C;
   const int n_chunks = (C + CHUNK_ROWS - 1) / CHUNK_ROWS;
 
+  wait_for_prior_grid();     // the cache rows, the slot map and q, k, v come from earlier kernels
+  // position bound of this query row (plain decode step: everything occupied is visible)
+  int q_tok = 0x7fffffff;
+  if (p.rows_q > 1) {
+    q_tok = last_row ? p.n_cur : p.row_tok[size_t(b) * p.r_max + qi];
+    if (q_tok < 0) {                                          // padding row: zeros, nothing else
+      for (int e = tid; e < DH; e += NT) p.out[size_t(item) * DH + e] = Elem<T>::from_float(0.f);
+      if (p.weights) for (int i = tid; i < rows; i += NT) p.weights[size_t(item) * rows + i] = 0.f;
+      return;
+    }
+  }
   if (tid == 0) {
 #pragma unroll
     for (int s = 0; s < kRingStages; ++s) mbar_init(&full[s], 1u);
@@ -62,7 +76,6 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
-  wait_for_prior_grid();     // the cache rows, the slot map and q, k, v come from earlier kernels
   auto issue = [&](int chunk) {
     const int stage = chunk % kRingStages;
     const int r0 = chunk * CHUNK_ROWS;
@@ -76,7 +89,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
   float qf[EPL];
   {
     const uint4 qr = *reinterpret_cast<const uint4*>(
-        reinterpret_cast<const unsigned char*>(p.q) + size_t(bh) * ROW_BYTES + li * 16);
+        reinterpret_cast<const unsigned char*>(p.q) + size_t(item) * ROW_BYTES + li * 16);
     Elem<T>::unpack(qr, qf);
   }
   // the current token's own key (row index C) does not go through the ring
@@ -88,7 +101,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kf[e], dot);
 #pragma unroll
     for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu >> (32 - LPR), dot, o);
-    if (li == 0) s_logit[C] = dot * p.scale;
+    if (li == 0) s_logit[C] = (p.rows_q == 1 || last_row) ? dot * p.scale : -INFINITY;
   }
 
   bool failed = false;
@@ -105,7 +118,8 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     for (int ps = 0; ps < PASSES; ++ps) {
       const int lr = ps * NW * RPW + warp * RPW + sub;      // row inside the chunk
       const int row = r0 + lr;
-      const bool ok = row < C && map[row] >= 0;
+      const int row_tok = row < C ? map[row] : -1;
+      const bool ok = row_tok >= 0 && row_tok <= q_tok && (p.rows_q == 1 || row_tok != p.n_cur);
       float kf[EPL];
       // rows past C in a ragged last chunk hold stale bytes of an earlier chunk: read, not used
       Elem<T>::unpack(*reinterpret_cast<const uint4*>(src + size_t(lr) * ROW_BYTES + li * 16), kf);
@@ -121,7 +135,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     if (tid == 0 && !failed && c + kRingStages < n_chunks) issue(c + kRingStages);
   }
   // (the loop's last __syncthreads also publishes the logits)
-  const int n_kept = attention_keep_and_weights<T, DH, NT>(p, sm, bh);
+  const int n_kept = attention_keep_and_weights<T, DH, NT>(p, sm, item);
 
   // ---- phase 4: only the kept value rows, gathered with direct 16-byte loads (one bulk copy per
   // 256-byte row was measured slower than the loads: the copy engine's per-operation cost dominates)
@@ -129,7 +143,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
   attention_values_direct<T, DH, NT>(p, sm, bh, n_kept, acc);
-  attention_finish<T, DH, NT>(p, sm, bh, acc);
+  attention_finish<T, DH, NT>(p, sm, bh, acc, item, last_row);
 }
 
 template <typename T>

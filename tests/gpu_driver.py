@@ -116,7 +116,7 @@ def _ulp(ref: np.ndarray, dtype: str) -> np.ndarray:
 
 
 def compare_attention(rep: Report, cfg, q, orc: ao.AdoreOracle, layer, k_new, attn_map, out_g, w_g, out_o, w_o,
-                      Kc_before, gpu_k=None, admit_slot=None):
+                      Kc_before, gpu_k=None, admit_slot=None, own_row=True):
     tol = TOL[cfg.dtype]
     err = np.abs(out_g - out_o)
     bound = tol["out_abs"] + tol["out_rel"] * np.abs(out_o)
@@ -129,7 +129,7 @@ def compare_attention(rep: Report, cfg, q, orc: ao.AdoreOracle, layer, k_new, at
     for b, h in bad:
         Kall = np.concatenate([Kc_before[b, h].astype(np.float64), k_new[b, h][None].astype(np.float64)])
         logit = Kall @ q[b, h].astype(np.float64) / np.sqrt(cfg.head_dim)
-        valid = np.concatenate([attn_map[b] >= 0, [True]])
+        valid = np.concatenate([attn_map[b] >= 0, [own_row]])
         scale = max(1.0, float(np.abs(logit[valid]).max()))
         diff = np.nonzero(keep_g[b, h] != keep_o[b, h])[0]
         assert keep_g[b, h].sum() == keep_o[b, h].sum(), "kept count differs"
@@ -263,6 +263,67 @@ def run_parity(cfg: wl.WorkloadConfig, batch: Optional[int] = None, steps: Optio
                 lib.adore_cache_sync_status(g.handle)
                 orc.check_invariants()
                 compare_state(rep, g, orc, range(L))
+        lib.adore_cache_sync_status(g.handle)
+    finally:
+        g.close()
+    return rep
+
+
+def run_parity_rebuild_first(cfg: wl.WorkloadConfig, steps: Optional[int] = None) -> Report:
+    """Free-running parity of the step in the order Section 2.3 prints it: adore_step_begin, then per layer
+    adore_rebuild and adore_attend_rows (R_max + 1 query rows per sequence), against the oracle's same three calls.
+    Every layer rebuilds from the token store."""
+    assert not cfg.per_layer_inputs
+    w = Workload(cfg, None)
+    orc = make_oracle(w)
+    g = GpuCache(w)
+    rep = Report()
+    L, R1 = cfg.n_layers, cfg.rebuild_max + 1
+    out_dev = torch.empty((g.B, cfg.n_heads, R1, cfg.head_dim), dtype=torch_dtype(cfg), device="cuda")
+    w_dev = torch.empty((g.B, cfg.n_heads, R1, cfg.capacity + 1), dtype=torch.float32, device="cuda")
+    try:
+        if cfg.prompt:
+            xp = w.prompt()
+            orc.append_tokens(xp)
+            lib.adore_cache_append_tokens(g.handle, to_dev(xp, cfg), cfg.prompt)
+            lib.adore_cache_sync_status(g.handle)
+            compare_state(rep, g, orc, range(L))
+        n_steps = cfg.steps if steps is None else steps
+        for s in range(n_steps):
+            n = orc.n
+            lists, counts = w.explicit(s, n)
+            dl = torch.from_numpy(lists).cuda() if lists is not None else None
+            dc = torch.from_numpy(counts).cuda() if counts is not None else None
+            x = w.x_new(n, 0)
+            orc.step_begin(x, explicit_as_lists(lists, counts))
+            lib.adore_step_begin(g.handle, to_dev(x, cfg), dl, dc, w.r_in)
+            for l in range(L):
+                _, k, v = w.qkv(n, l, x)
+                orc.rebuild(l)
+                lib.adore_rebuild(g.handle, l, None)
+                q_rows = w.q_rows(n, l, orc.x, orc.info.rebuild_tok)
+                K_before = orc.Kc[l].copy()
+                st = orc.slot_tok.copy()
+                out_o, w_o = orc.attend_rows(l, q_rows, k, v)
+                lib.adore_attend_rows(g.handle, l, to_dev(q_rows, cfg), to_dev(k, cfg), to_dev(v, cfg), out_dev, w_dev)
+                out_g, w_g = out_dev.float().cpu().numpy(), w_dev.cpu().numpy()
+                for i in range(R1):
+                    toks = np.array([n if i == R1 - 1 else (int(orc.info.rebuild_tok[b][i]) if i < len(orc.info.rebuild_tok[b]) else -1)
+                                     for b in range(g.B)])
+                    pad = toks < 0
+                    assert not out_g[pad, :, i].any() and not w_g[pad, :, i].any(), "padding rows must be zero"
+                    idx = np.nonzero(~pad)[0]
+                    if idx.size == 0:
+                        continue
+                    seen = np.where((st[idx] >= 0) & (st[idx] <= toks[idx, None]) & (st[idx] != n), st[idx], -1)
+                    compare_attention(rep, cfg, q_rows[idx, :, i], orc, l, k[idx], seen, out_g[idx, :, i], w_g[idx, :, i],
+                                      out_o[idx, :, i], w_o[idx, :, i], K_before[idx],
+                                      gpu_k=lambda l=l, idx=idx: g.kv(l)[0][idx], admit_slot=orc.info.admit_slot[idx],
+                                      own_row=(i == R1 - 1))
+            rep.steps += 1
+            lib.adore_cache_sync_status(g.handle)
+            orc.check_invariants()
+            compare_state(rep, g, orc, range(L))
         lib.adore_cache_sync_status(g.handle)
     finally:
         g.close()

@@ -126,3 +126,25 @@ def test_controller_ablations_width_64_and_no_recurrence():
     _run(SMALL.scaled(name="ctrl64", ctrl_hidden=64, steps=25, seed=121))
     _run(SMALL.scaled(name="norecurrence", ctrl_no_recurrence=True, steps=25, seed=122))
     _run(SMALL.scaled(name="norecurrence160", ctrl_no_recurrence=True, ctrl_hidden=160, steps=12, seed=123))
+
+
+def _run_rebuild_first(cfg, **kw):
+    from tests.gpu_driver import run_parity_rebuild_first
+    rep = run_parity_rebuild_first(cfg, **kw)
+    print(f"\n[{cfg.name}] steps={rep.steps} near_ties={rep.near_ties}+{rep.rounding_ties}r/{rep.topk_rows} rows "
+          f"max_out_err={rep.max_out_err:.3e} max_w_err={rep.max_w_err:.3e} max_kv_ulp={rep.max_kv_ulp:.2f}")
+    assert rep.near_ties <= max(2, rep.topk_rows // 1000)
+    assert rep.rounding_ties <= max(2, rep.topk_rows // 50)
+    return rep
+
+
+def test_rebuild_first_step_with_query_rows_of_the_rebuilt_tokens():
+    """Section 2.3 as printed: select, rebuild, then one attention with R_max + 1 query rows per sequence under a
+    causal bound (policy lists are full, explicit lists leave padding rows; fp32 and two layers as well)."""
+    _run_rebuild_first(SMALL.scaled(name="rows_policy", steps=30, seed=124))
+    _run_rebuild_first(SMALL.scaled(name="rows_explicit", rebuild_mode="explicit", rebuild_p=0.3, rebuild_max=20, capacity=48,
+                                    topk=24, prompt=0, steps=60, seed=125))
+    _run_rebuild_first(SMALL.scaled(name="rows_f32_dh64", dtype="f32", head_dim=64, n_heads=3, hidden=192, capacity=33, topk=7,
+                                    steps=20, seed=126))
+    _run_rebuild_first(SMALL.scaled(name="rows_two_layers_c300", n_layers=2, batch=2, capacity=300, topk=100, rebuild_max=9,
+                                    prompt=400, steps=8, seed=127))
