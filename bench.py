@@ -185,10 +185,11 @@ class ClockSampler:
 class DeviceRun:
     """Cache + pre-generated per-step inputs on the GPU for `total_steps` decode steps."""
 
-    def __init__(self, cfg: wl.WorkloadConfig, total_steps: int, rank: int):
+    def __init__(self, cfg: wl.WorkloadConfig, total_steps: int, rank: int, order: str = "attend-first"):
         import torch
         from paper_2407_02328_b200 import adore as lib
         self.torch, self.lib, self.cfg = torch, lib, cfg
+        self.order = order
         c = cfg
         assert total_steps <= c.steps, f"{total_steps} steps asked, the workload has {c.steps}"
         self.dt = torch.float32 if c.dtype == "f32" else torch.bfloat16
@@ -291,6 +292,12 @@ class DeviceRun:
         self.pc = None if self.counts is None else [self.counts[s].data_ptr() for s in range(self.counts.shape[0])]
         self.pt = None if self.tables is None else [t.data_ptr() for t in self.tables]
         self.pout, self.pw = self.out.data_ptr(), self.weights.data_ptr()
+        if order == "rebuild-first":
+            # R_max + 1 query rows per sequence (Section 2.3); the same random rows serve every step
+            R1 = c.rebuild_max + 1
+            self.q_rows = torch.randn((B, H, R1, dh), generator=g, device=dev, dtype=torch.float32).to(self.dt)
+            self.out_rows = torch.empty((B, H, R1, dh), dtype=self.dt, device=dev)
+            self.pqr, self.por = self.q_rows.data_ptr(), self.out_rows.data_ptr()
         lib.adore_cache_sync_status(self.handle)
 
     def _rope(self, y, n):
@@ -310,6 +317,13 @@ class DeviceRun:
         lib, c, s = self.lib, self.cfg, self.next
         pl = None if self.pl is None else self.pl[s]
         pc = None if self.pc is None else self.pc[s]
+        if self.order == "rebuild-first":
+            lib.adore_step_begin(self.handle, self.px[s], pl, pc, self.r_in)
+            for l in range(c.n_layers):
+                lib.adore_rebuild(self.handle, l, self.pt[l] if (self.pt is not None and l > 0) else None)
+                lib.adore_attend_rows(self.handle, l, self.pqr, self.pk[s][l], self.pv[s][l], self.por, None)
+            self.next += 1
+            return
         for l in range(c.n_layers):
             lib.adore_decode_step(self.handle, l, self.pq[s][l], self.pk[s][l], self.pv[s][l], self.px[s], pl, pc, self.r_in,
                                   self.pout, self.pw)
@@ -482,6 +496,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--order", default="attend-first", choices=["attend-first", "rebuild-first"],
+                    help="rebuild-first: select, rebuild, then one attention with R_max+1 query rows per sequence "
+                         "(adore_step_begin / adore_attend_rows); no end-to-end pass in that order")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
@@ -511,9 +528,9 @@ def main():
     from paper_2407_02328_b200 import adore as lib
 
     K, W = args.steps, args.warmup
-    with_e2e = not args.no_e2e
+    with_e2e = not args.no_e2e and args.order == "attend-first"
     total = W + K + (K if with_e2e else 0) + K          # warm-up, timed, end-to-end, per-stage pass
-    run = DeviceRun(cfg, total, rank)
+    run = DeviceRun(cfg, total, rank, args.order)
     flush = None
     if kv_bytes(cfg) <= 2.5e8:
         flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
@@ -639,7 +656,7 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
                 "ms_per_step": ms_total / K, "steps_per_s": K / (ms_total * 1e-3), "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-                "config": workload_desc(cfg), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+                "config": dict(workload_desc(cfg), step_order=args.order), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
                 "roofline": roofline, "stages": stages, "cpu_baseline": cpu}
         # the plain read kernel's time for the same bytes: what the access pattern allows on this GPU
         ideal_us = ceiling["stream_us"] + ceiling["gather_us"]
