@@ -205,6 +205,49 @@ def project_q(w_q: np.ndarray, x_row: np.ndarray, position: int, n_heads: int, h
 
 
 # --------------------------------------------------------------------------------------
+# labels for training the controller (Section 2.2 last paragraph, Appendix B, Appendix C)
+# --------------------------------------------------------------------------------------
+def attention_labels(weights: np.ndarray, topk: int):
+    """Uniform token set of one decode step from its per-slot attention weights.
+
+    weights: [L, B, H, S] (what the step emits; zero = masked or empty). For every (layer, head) the set of the
+    topk // 2 slots with the largest positive weight is taken (equal weights: lower slot first; fewer if fewer are
+    positive). count[b, s] is the number of these sets that contain slot s; the label is 1 for the `topk` slots of
+    a sequence with the largest positive count (equal counts: lower slot first), 0 for all others.
+    Also the two statistics of Appendix C (Figure 7): coverage[l, b], the share of layer l's set members that carry
+    the label, and mass[l, b], the attention weight of the labelled slots at layer l averaged over heads.
+
+    Returns sets [L, B, H, topk // 2] int32 (-1 padded, in descending weight order), count [B, S] int32,
+    label [B, S] uint8, coverage [L, B] float64, mass [L, B] float64.
+    """
+    w = np.asarray(weights)
+    L, B, H, S = w.shape
+    half = topk // 2
+    sets = np.full((L, B, H, half), -1, np.int32)
+    count = np.zeros((B, S), np.int32)
+    for l in range(L):
+        for b in range(B):
+            for h in range(H):
+                row = w[l, b, h]
+                order = sorted((s for s in range(S) if row[s] > 0), key=lambda s: (-float(row[s]), s))[:half]
+                sets[l, b, h, : len(order)] = order
+                for s in order:
+                    count[b, s] += 1
+    label = np.zeros((B, S), np.uint8)
+    for b in range(B):
+        order = sorted((s for s in range(S) if count[b, s] > 0), key=lambda s: (-int(count[b, s]), s))[:topk]
+        label[b, order] = 1
+    coverage = np.zeros((L, B), np.float64)
+    mass = np.zeros((L, B), np.float64)
+    for l in range(L):
+        for b in range(B):
+            members = sets[l, b][sets[l, b] >= 0]
+            coverage[l, b] = float(label[b, members].sum()) / members.size if members.size else 0.0
+            mass[l, b] = float(np.asarray(w[l, b], np.float64)[:, label[b] == 1].sum()) / H
+    return sets, count, label, coverage, mass
+
+
+# --------------------------------------------------------------------------------------
 # the stateful path
 # --------------------------------------------------------------------------------------
 @dataclass

@@ -477,6 +477,42 @@ def test_controller_without_recurrence_forgets_earlier_tokens():
     assert np.array_equal(alone.score[:, 8], last[True, "plain"])
 
 
+def test_labels_equal_counter_brute_force_and_invariants():
+    """Section 2.2 / Appendix C: the label set is the top-K of the membership counts of the per-(layer, head) top-K/2
+    sets; checked with collections.Counter and Python sets on seeded weights, plus what must always hold."""
+    from collections import Counter
+    L, B, H, S, K = 3, 2, 4, 41, 12
+    w = wl.slot_weights(9, L, B, H, S, nonzero=K, empty_frac=0.2)
+    sets, count, label, coverage, mass = ao.attention_labels(w, K)
+    for b in range(B):
+        c = Counter()
+        per_layer = []
+        for l in range(L):
+            members = []
+            for h in range(H):
+                pos = [(float(w[l, b, h, s]), -s) for s in range(S) if w[l, b, h, s] > 0]
+                top = [-i for _, i in sorted(pos, reverse=True)[: K // 2]]
+                assert list(sets[l, b, h][sets[l, b, h] >= 0]) == top
+                members += top
+            c.update(members)
+            per_layer.append(members)
+        assert all(count[b, s] == c.get(s, 0) for s in range(S))
+        ranked = sorted(c, key=lambda s: (-c[s], s))[:K]
+        assert set(np.nonzero(label[b])[0]) == set(ranked)
+        for l in range(L):
+            assert coverage[l, b] == pytest.approx(sum(s in ranked for s in per_layer[l]) / len(per_layer[l]))
+            assert mass[l, b] == pytest.approx(sum(float(w[l, b, h, s]) for h in range(H) for s in ranked) / H)
+    assert count.sum() == sum(min(K // 2, int((w[l, b, h] > 0).sum())) for l in range(L) for b in range(B) for h in range(H))
+    assert (label.sum(-1) <= K).all() and ((mass >= 0) & (mass <= 1 + 1e-6)).all()
+    # the same row in every layer and head: the labelled set contains every set, so coverage is one
+    same = np.broadcast_to(w[0, :, 0][None, :, None, :], w.shape).copy()
+    _, _, lab, cov, _ = ao.attention_labels(same, K)
+    assert (cov == 1.0).all() and (lab.sum(-1) == K // 2).all()
+    # the order of the layers does not matter to the labels
+    _, cnt2, lab2, _, _ = ao.attention_labels(w[::-1].copy(), K)
+    assert np.array_equal(cnt2, count) and np.array_equal(lab2, label)
+
+
 # ------------------------------------------------------------------ planted mistakes
 def test_pins_notice_planted_mistakes(monkeypatch):
     """Each plausible slip, planted in the oracle, must make one of the pins above fail."""

@@ -15,4 +15,5 @@ from .generate import (  # noqa: F401
     query_weights,
     gaussian,
     rebuild_flags,
+    slot_weights,
 )

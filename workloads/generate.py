@@ -115,3 +115,23 @@ def rebuild_flags(cfg: WorkloadConfig, step: int, n_tokens: int, r_in: int,
         lists[i, : idx.size] = idx
         counts[i] = idx.size
     return lists, counts
+
+
+def slot_weights(seed: int, n_layers: int, batch: int, n_heads: int, n_slots: int, nonzero: int,
+                 empty_frac: float = 0.1) -> np.ndarray:
+    """Per-slot weights with the shape of what a decode step emits: float32 [L, B, H, n_slots], at most `nonzero`
+    positive entries per (layer, sequence, head) row, rows summing to one, empty slots zero everywhere, long-tailed
+    values, and a per-sequence set of slots that every layer and head tends to favour."""
+    out = np.zeros((n_layers, batch, n_heads, n_slots), np.float32)
+    for b in range(batch):
+        rng = substream(seed, "slot_weights", b)
+        occupied = np.nonzero(rng.random(n_slots) >= empty_frac)[0]
+        favour = rng.random(n_slots) ** 4                      # a few slots matter to every head
+        for l in range(n_layers):
+            for h in range(n_heads):
+                k = min(nonzero, occupied.size)
+                pick_score = favour[occupied] + 0.3 * rng.random(occupied.size)
+                chosen = occupied[np.argsort(-pick_score, kind="stable")[:k]]
+                vals = rng.exponential(1.0, k) ** 3
+                out[l, b, h, chosen] = (vals / vals.sum()).astype(np.float32)
+    return out
