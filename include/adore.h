@@ -271,6 +271,22 @@ adore_status_t adore_step_begin(adore_cache_t *cache, const void *x_new, const i
 adore_status_t adore_attend_rows(adore_cache_t *cache, int32_t layer, const void *q_rows, const void *k_new,
                                  const void *v_new, void *out, float *weights);
 
+/* Labels for training the controller and the uniform-token-set statistics (Section 2.2 last paragraph, Appendix B
+ * "training data collection", Appendix C / Figure 7) from the per-slot weights one decode step emitted for all layers.
+ * Needs no cache; runs on the given CUDA stream (NULL = default stream) and allocates nothing.
+ *   weights  [n_layers, batch, n_heads, n_slots] float DEVICE (n_slots = C + 1 for weights of adore_decode_step;
+ *            zero = masked or empty), n_slots <= 4096 (else ADORE_ERR_UNSUPPORTED)
+ *   sets     [n_layers, batch, n_heads, topk/2] int32 DEVICE out: per layer and head the topk/2 slots with the
+ *            largest positive weight, descending, equal weights lower slot first, -1 padded
+ *   count    [batch, n_slots] int32 DEVICE out: how many of those sets contain the slot
+ *   label    [batch, n_slots] uint8 DEVICE out: 1 for the topk slots with the largest positive count (equal counts:
+ *            lower slot first), else 0
+ *   coverage [n_layers, batch] float DEVICE out: share of the layer's set members that carry the label
+ *   mass     [n_layers, batch] float DEVICE out: weight of the labelled slots at that layer, averaged over heads */
+adore_status_t adore_label_tokens(const float *weights, int32_t n_layers, int32_t batch, int32_t n_heads, int32_t n_slots,
+                                  int32_t topk, void *cuda_stream, int32_t *sets, int32_t *count, uint8_t *label,
+                                  float *coverage, float *mass);
+
 /* Snapshot of the small per-sequence state that scoring and selection carry from step to step
  * (Section 2.2: which tokens hold which slots, every token's controller score and the GRU state z;
  * Section 2.3: the step's rebuild list): both slot-map buffers, the token-to-slot table, score and sigma

@@ -53,7 +53,8 @@ EXPORTS = ["adore_cache_create", "adore_cache_destroy", "adore_cache_set_project
            "adore_cache_launch_count", "adore_cache_sync_status", "adore_status_string",
            "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows",
            "adore_controller_score_static", "adore_probe_read_bandwidth",
-           "adore_cache_export_state", "adore_cache_import_state", "adore_step_begin", "adore_attend_rows"]
+           "adore_cache_export_state", "adore_cache_import_state", "adore_step_begin", "adore_attend_rows",
+           "adore_label_tokens"]
 
 
 def _lib():
@@ -75,6 +76,7 @@ def _lib():
         lib.adore_decode_step_host.argtypes = step
         lib.adore_rebuild.argtypes = [vp, i32, vp]
         lib.adore_step_begin.argtypes = [vp, vp, vp, vp, i32]
+        lib.adore_label_tokens.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         lib.adore_attend_rows.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         lib.adore_cache_slot_map.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
         lib.adore_cache_rebuild_list.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
@@ -161,6 +163,12 @@ def adore_step_begin(cache: int, x_new, explicit_list, explicit_count, r_in: int
 def adore_attend_rows(cache: int, layer: int, q_rows, k_new, v_new, out, weights=None) -> None:
     _check(_lib().adore_attend_rows(cache, layer, _ptr(q_rows), _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(weights)),
            "adore_attend_rows")
+
+
+def adore_label_tokens(weights, n_layers: int, batch: int, n_heads: int, n_slots: int, topk: int, cuda_stream: int,
+                       sets, count, label, coverage, mass) -> None:
+    _check(_lib().adore_label_tokens(_ptr(weights), n_layers, batch, n_heads, n_slots, topk, cuda_stream or None, _ptr(sets),
+                                     _ptr(count), _ptr(label), _ptr(coverage), _ptr(mass)), "adore_label_tokens")
 
 
 def adore_rebuild(cache: int, layer: int, x_table=None) -> None:

@@ -15,6 +15,7 @@
 #include "rebuild_simt.cuh"
 #include "rebuild_tc.cuh"
 #include "select.cuh"
+#include "labels.cuh"
 
 using namespace adore;
 
@@ -963,6 +964,25 @@ adore_status_t adore_cache_import_state(adore_cache_t* c, const void* host_buf, 
   c->n = hd.n; c->cur = hd.cur; c->attn = hd.attn; c->step_layer0_done = hd.step_open;
   c->joined = true;
   c->rows_gathered = false;
+  return ADORE_OK;
+}
+
+adore_status_t adore_label_tokens(const float* weights, int32_t n_layers, int32_t batch, int32_t n_heads, int32_t n_slots,
+                                  int32_t topk, void* cuda_stream, int32_t* sets, int32_t* count, uint8_t* label,
+                                  float* coverage, float* mass) {
+  if (!weights || !sets || !count || !label || !coverage || !mass) return ADORE_ERR_INVALID_ARG;
+  if (n_layers < 1 || batch < 1 || n_heads < 1 || n_slots < 1 || topk < 2) return ADORE_ERR_INVALID_ARG;
+  if (n_slots > kLabelMaxSlots) return ADORE_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int half = topk / 2;
+  const size_t smem = size_t(label_pow2(n_slots)) * sizeof(unsigned long long);
+  CUDA_OK(cudaMemsetAsync(count, 0, size_t(batch) * n_slots * sizeof(int), st));
+  label_sets_kernel<<<n_layers * batch * n_heads, kLabelThreads, smem, st>>>(weights, batch, n_heads, n_slots, half, sets, count);
+  CUDA_OK(cudaGetLastError());
+  label_pick_kernel<<<batch, kLabelThreads, smem, st>>>(count, n_slots, topk, label);
+  CUDA_OK(cudaGetLastError());
+  label_stats_kernel<<<n_layers * batch, kLabelThreads, 0, st>>>(weights, sets, label, batch, n_heads, n_slots, half, coverage, mass);
+  CUDA_OK(cudaGetLastError());
   return ADORE_OK;
 }
 
