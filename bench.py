@@ -482,6 +482,49 @@ def probe_pattern_ceiling(run, flush):
     return out
 
 
+def run_labels(args):
+    """Times adore_label_tokens on weights of config 4's shape (32 layers x 32 sequences x 32 heads x 1025 slots, K = 512):
+    one JSON line with the time per call and the rate at which the weights are read."""
+    import torch
+    from paper_2407_02328_b200 import build
+    build.build()
+    from paper_2407_02328_b200 import adore as lib
+    cfg = wl.get_config(4)
+    L, B, H, S, K = cfg.n_layers, cfg.batch, cfg.n_heads, cfg.capacity + 1, cfg.topk
+    g = torch.Generator(device="cuda")
+    g.manual_seed(cfg.seed)
+    w = torch.rand((L, B, H, S), generator=g, device="cuda") ** 8          # long-tailed
+    keep = torch.rand((L, B, H, S), generator=g, device="cuda") < 0.5      # about K positive entries per row
+    w = torch.where(keep, w, torch.zeros_like(w))
+    w = (w / w.sum(-1, keepdim=True).clamp_min(1e-30)).contiguous()
+    sets = torch.empty((L, B, H, K // 2), dtype=torch.int32, device="cuda")
+    count = torch.empty((B, S), dtype=torch.int32, device="cuda")
+    label = torch.empty((B, S), dtype=torch.uint8, device="cuda")
+    cov = torch.empty((L, B), dtype=torch.float32, device="cuda")
+    mass = torch.empty_like(cov)
+    st = torch.cuda.current_stream().cuda_stream
+    call = lambda: lib.adore_label_tokens(w, L, B, H, S, K, st, sets, count, label, cov, mass)
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    n = args.steps or 20
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(n):
+        call()
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / n
+    peaks, kind = measured_peaks()
+    gbs = 2 * w.numel() * 4 / (ms * 1e-3) / 1e9                             # the weights are read twice (sets, statistics)
+    print(json.dumps({"metric": "label construction, calls/s", "value": 1e3 / ms, "unit": "calls/s", "ms_per_call": ms,
+                      "config": {"workload": "labels_cfg4_shape", "layers": L, "batch": B, "heads": H, "slots": S, "topk": K,
+                                 "l2": "weights 134 MB > L2"},
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": gbs / peaks["hbm_gbs"], "peak_source": f"{kind} (copy)", "traffic": None},
+                      "gpu_launches": 3 * n, "data": "synthetic"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -496,12 +539,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--labels", action="store_true", help="time the label-construction entry point instead of the decode step")
     ap.add_argument("--order", default="attend-first", choices=["attend-first", "rebuild-first"],
                     help="rebuild-first: select, rebuild, then one attention with R_max+1 query rows per sequence "
                          "(adore_step_begin / adore_attend_rows); no end-to-end pass in that order")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.labels:
+        run_labels(args)
         return
     cfg = sweep_point(args.capacity, args.batch) if args.config == 5 else wl.get_config(args.config)
     if args.steps is None:

@@ -267,6 +267,7 @@ class OracleConfig:
     rope_theta: float = 1.0e4
     pos_scale: float = 4096.0
     no_recurrence: bool = False    # Section 3.5.3 "w/o GRU": z_i = GRU(x_i, 0), no memory of earlier tokens
+    score_from_attention: bool = False   # Section 3.1 baselines 6 and 7: a token's value is its cumulative attention
 
     @property
     def retained_max(self) -> int:
@@ -320,6 +321,10 @@ class AdoreOracle:
         """z_n, score_n, sigma_n for the token at position self.n of every sequence."""
         c, n = self.cfg, self.n
         self.x[:, n, :] = x_new
+        if c.score_from_attention:          # no controller: the token starts at zero and earns weight when attended
+            self.score[:, n] = 0.0
+            self.sigma[:, n] = 0.0
+            return
         z_prev = np.zeros_like(self.z) if c.no_recurrence else self.z
         self.z = gru_step(x_new, z_prev, self.ctrl)
         s = controller_score(self.z, n, c.pos_scale, self.ctrl)
@@ -477,7 +482,25 @@ class AdoreOracle:
             s = int(self.info.admit_slot[b])
             self.Kc[layer, b, :, s, :] = round_store(k_new[b], c.dtype)
             self.Vc[layer, b, :, s, :] = round_store(v_new[b], c.dtype)
+        if c.score_from_attention:
+            self._add_attention(wts, self.attn_slot_tok, self.n - 1)
         return out, wts
+
+    def _add_attention(self, wts: np.ndarray, slot_tok: np.ndarray, n_cur: int) -> None:
+        """Cumulative attention as the tokens' value: every attended token gains the weight its row received, summed
+        over the heads (float32, heads in ascending order, as the ranking is done on float32); the selection of the
+        NEXT step is the first to see it."""
+        B, H, C1 = wts.shape
+        w32 = wts.astype(np.float32)
+        for b in range(B):
+            for s in range(C1):
+                tok = n_cur if s == C1 - 1 else int(slot_tok[b, s])
+                if tok < 0:
+                    continue
+                acc = np.float32(0.0)
+                for h in range(H):
+                    acc = np.float32(acc + w32[b, h, s])
+                self.score[b, tok] = np.float32(self.score[b, tok] + acc)
 
     # -- the step in the order Section 2.3 prints it: select, rebuild, then attend with R+1 query rows ----
     def step_begin(self, x_new: np.ndarray, explicit: Optional[List[np.ndarray]] = None) -> None:
@@ -509,6 +532,7 @@ class AdoreOracle:
         q_rows: [B, H, R_max+1, dh]; returns out [B, H, R_max+1, dh] and weights [B, H, R_max+1, C+1].
         """
         c = self.cfg
+        assert not c.score_from_attention, "the cumulative-attention score source is defined for the attend-first step"
         B, H, C, dh, R1 = c.batch, c.n_heads, c.capacity, c.head_dim, c.rebuild_max + 1
         n = self.n - 1                                        # position of the current token
         out = np.zeros((B, H, R1, dh), np.float64)

@@ -513,6 +513,40 @@ def test_labels_equal_counter_brute_force_and_invariants():
     assert np.array_equal(cnt2, count) and np.array_equal(lab2, label)
 
 
+def test_cumulative_attention_scores_equal_column_sums_of_the_causal_attention_matrix():
+    """Section 3.1 baseline 6 as a score source: with every token resident and no top-K mask, a token's value after S
+    steps is the sum, over the steps that saw it and over the heads, of its softmax weight, i.e. a column sum of the
+    dense causal attention matrix built from scratch; and every step hands out exactly one unit per head."""
+    cfg = TINY.scaled(capacity=40, topk=100, rebuild_max=0, prompt=0, steps=30, score_from_attention=True)
+    w, orc, hist = run_free(cfg)
+    K, _ = history_kv(w, orc, orc.n)
+    expect = np.zeros((w.batch, orc.n))
+    for i, (q, _, _) in enumerate(hist):
+        for b in range(w.batch):
+            for h in range(cfg.n_heads):
+                logit = np.array([float(np.dot(q[b, h].astype(np.float64), K[b, h, j])) / math.sqrt(cfg.head_dim) for j in range(i + 1)])
+                e = np.exp(logit - logit.max())
+                expect[b, : i + 1] += e / e.sum()
+    assert np.allclose(orc.score[:, : orc.n], expect, rtol=1e-5, atol=1e-6)
+    assert np.allclose(orc.score[:, : orc.n].sum(-1), len(hist) * cfg.n_heads, rtol=1e-5)
+    # with a small cache the least attended retained token is the one that leaves
+    small = TINY.scaled(capacity=8, topk=100, rebuild_max=2, prompt=0, steps=20, score_from_attention=True)
+    w2 = Workload(small)
+    o2 = make_oracle(w2)
+    for s_ in range(small.steps):
+        n = o2.n
+        x = w2.x_new(n)
+        q, k, v = w2.qkv(n, 0, x)
+        before_tok, before_role, before_score = o2.slot_tok.copy(), o2.slot_role.copy(), o2.score.copy()
+        o2.decode_step(0, q, k, v, x, None)
+        o2.rebuild(0)
+        for b in range(w2.batch):
+            ev = int(o2.info.evicted_tok[b])
+            if ev >= 0:
+                ret = [int(t) for t, r in zip(before_tok[b], before_role[b]) if r == ao.RETAINED]
+                assert ev == min(ret, key=lambda t: (float(before_score[b, t]), t))
+
+
 # ------------------------------------------------------------------ planted mistakes
 def test_pins_notice_planted_mistakes(monkeypatch):
     """Each plausible slip, planted in the oracle, must make one of the pins above fail."""

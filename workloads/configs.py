@@ -37,6 +37,7 @@ class WorkloadConfig:
     identity_projection: bool = False   # W_k = W_v = I (needs hidden == n_heads*head_dim)
     per_layer_inputs: bool = False      # every layer has its own RMS-normalised input rows
     ctrl_no_recurrence: bool = False    # controller ablation without the GRU's memory: every token sees a zero state
+    score_from_attention: bool = False  # tokens ranked by cumulative attention weight instead of the controller's score
 
     @property
     def retained_max(self) -> int:
