@@ -185,7 +185,8 @@ class ClockSampler:
 class DeviceRun:
     """Cache + pre-generated per-step inputs on the GPU for `total_steps` decode steps."""
 
-    def __init__(self, cfg: wl.WorkloadConfig, total_steps: int, rank: int, order: str = "attend-first"):
+    def __init__(self, cfg: wl.WorkloadConfig, total_steps: int, rank: int, order: str = "attend-first",
+                 score_source: str = "controller"):
         import torch
         from paper_2407_02328_b200 import adore as lib
         self.torch, self.lib, self.cfg = torch, lib, cfg
@@ -203,7 +204,8 @@ class DeviceRun:
             lib.make_config(batch=B, n_layers=L, n_heads=H, head_dim=dh, hidden=d, capacity=c.capacity,
                             rebuild_max=c.rebuild_max, topk=c.topk, max_tokens=c.max_tokens,
                             ctrl_hidden=c.ctrl_hidden, dtype=c.dtype, rebuild_mode=c.rebuild_mode,
-                            rope_theta=c.rope_theta, pos_scale=c.pos_scale),
+                            rope_theta=c.rope_theta, pos_scale=c.pos_scale,
+                            flags=lib.ADORE_FLAG_SCORE_FROM_ATTENTION if score_source == "attention" else 0),
             wl.controller_weights(c), self.stream)
 
         def randn(*shape, std=1.0):
@@ -539,6 +541,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--score-source", default="controller", choices=["controller", "attention"],
+                    help="attention: tokens ranked by cumulative attention weight (the H2O baselines' score), no controller")
     ap.add_argument("--labels", action="store_true", help="time the label-construction entry point instead of the decode step")
     ap.add_argument("--order", default="attend-first", choices=["attend-first", "rebuild-first"],
                     help="rebuild-first: select, rebuild, then one attention with R_max+1 query rows per sequence "
@@ -577,7 +581,7 @@ def main():
     K, W = args.steps, args.warmup
     with_e2e = not args.no_e2e and args.order == "attend-first"
     total = W + K + (K if with_e2e else 0) + K          # warm-up, timed, end-to-end, per-stage pass
-    run = DeviceRun(cfg, total, rank, args.order)
+    run = DeviceRun(cfg, total, rank, args.order, args.score_source)
     flush = None
     if kv_bytes(cfg) <= 2.5e8:
         flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
@@ -703,7 +707,7 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
                 "ms_per_step": ms_total / K, "steps_per_s": K / (ms_total * 1e-3), "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-                "config": dict(workload_desc(cfg), step_order=args.order), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+                "config": dict(workload_desc(cfg), step_order=args.order, score_source=args.score_source), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
                 "roofline": roofline, "stages": stages, "cpu_baseline": cpu}
         # the plain read kernel's time for the same bytes: what the access pattern allows on this GPU
         ideal_us = ceiling["stream_us"] + ceiling["gather_us"]

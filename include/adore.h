@@ -71,6 +71,12 @@ enum { ADORE_SLOT_EMPTY = 0, ADORE_SLOT_RETAINED = 1, ADORE_SLOT_REBUILT = 2 };
  * from its own embedding alone, z_i = GRU(x_i, 0), then the same MLP. The paper does not say how the embedding
  * reaches the MLP without the GRU; applying the cell to a zero state needs no extra parameters. */
 #define ADORE_FLAG_NO_RECURRENCE 1u
+/* Score source of the H2O and H2O(Rebuilt) baselines (Section 3.1, items 6 and 7) on the same kernels: no controller;
+ * a token's value is the attention weight it has received so far, summed over heads, layers and steps (float32). The
+ * weights of a step count from the next step's selection on; prompt tokens start at zero, so a prompt is cut to its
+ * most recent tokens. adore_decode_step then accumulates after every layer's attention (weights == NULL is fine: an
+ * internal buffer is used); adore_step_begin returns ADORE_ERR_UNSUPPORTED. */
+#define ADORE_FLAG_SCORE_FROM_ATTENTION 2u
 
 typedef struct {
   uint32_t struct_size;  /* sizeof(adore_config_t), for versioning                               */

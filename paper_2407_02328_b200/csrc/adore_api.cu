@@ -65,6 +65,21 @@ __global__ void admit_rows_kernel(unsigned char* Kc, unsigned char* Vc, const un
   }
 }
 
+// Cumulative attention as the tokens' value (Section 3.1, baselines 6 and 7): every attended token gains the weight its
+// row received in this launch, summed over the heads in ascending order. One thread per (sequence, slot).
+__global__ void add_attention_kernel(const float* weights, const int* slot_tok, int H, int C, int n_cur, int max_tokens,
+                                     float* score) {
+  const int b = blockIdx.x, s = blockIdx.y * blockDim.x + threadIdx.x;
+  let_next_grid_start();
+  wait_for_prior_grid();
+  if (s > C) return;
+  const int tok = s == C ? n_cur : slot_tok[size_t(b) * C + s];
+  if (tok < 0) return;
+  float acc = 0.f;
+  for (int h = 0; h < H; ++h) acc += weights[(size_t(b) * H + h) * (C + 1) + s];
+  score[size_t(b) * max_tokens + tok] += acc;
+}
+
 __global__ void fill_i32_kernel(int* p, int v, size_t n) {
   for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < n; i += size_t(gridDim.x) * blockDim.x) p[i] = v;
 }
@@ -140,6 +155,7 @@ struct adore_cache {
   bool joined = true;
   std::vector<const void*> w_kv;
   TcState tc;                   // tensor-core rebuild path (tensor maps, gather buffer)
+  float* w_internal = nullptr;  // [B,H,C+1] weights when the caller passes none but the scores need them
   bool rows_gathered = false;   // the gather buffer holds this step's listed rows, taken from the token store
   // staging for the host-buffer entry point
   void *h_q = nullptr, *h_k = nullptr, *h_v = nullptr, *h_x = nullptr, *h_out = nullptr;
@@ -342,6 +358,16 @@ adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, co
   return ADORE_OK;
 }
 
+// Adds the weights of the attention launch that just ran (caller's buffer or the internal one) to the tokens' scores.
+adore_status_t launch_add_attention(adore_cache* c, const float* weights) {
+  const adore_config_t& f = c->cfg;
+  StageScope scope(c, 1);
+  CUDA_OK(launch_dependent(add_attention_kernel, dim3(f.batch, (f.capacity + 1 + 127) / 128), dim3(128), 0, c->stream, weights,
+                           c->slot_tok[c->attn], f.n_heads, f.capacity, c->n - 1, f.max_tokens, c->score));
+  ++c->launches;
+  return ADORE_OK;
+}
+
 adore_status_t launch_row_table(adore_cache* c, bool count_rows, cudaStream_t stream) {
   const adore_config_t& f = c->cfg;
   if (f.rebuild_max == 0) return ADORE_OK;          // row_total stays 0
@@ -367,7 +393,7 @@ adore_status_t fill_layer_impl(adore_cache* c, int layer, const void* x_table) {
 adore_status_t check_config(const adore_config_t* f) {
   if (f->struct_size != sizeof(adore_config_t)) return ADORE_ERR_INVALID_ARG;
   if (f->batch < 1 || f->n_layers < 1 || f->n_heads < 1 || f->hidden < 1 || f->capacity < 1 || f->topk < 1 ||
-      f->max_tokens < 1 || f->ctrl_hidden < 1 || f->rebuild_max < 0 || f->rebuild_max >= f->capacity || (f->flags & ~uint32_t(ADORE_FLAG_NO_RECURRENCE)) != 0 ||
+      f->max_tokens < 1 || f->ctrl_hidden < 1 || f->rebuild_max < 0 || f->rebuild_max >= f->capacity || (f->flags & ~uint32_t(ADORE_FLAG_NO_RECURRENCE | ADORE_FLAG_SCORE_FROM_ATTENTION)) != 0 ||
       !(f->pos_scale > 0.f) || f->rope_theta < 0.f)
     return ADORE_ERR_INVALID_ARG;
   if (f->dtype != ADORE_F32 && f->dtype != ADORE_BF16) return ADORE_ERR_INVALID_ARG;
@@ -390,10 +416,13 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
   const bool ex = f.rebuild_mode == ADORE_REBUILD_EXPLICIT;
   adore_status_t st;
   StageScope scope(c, 1);
+  const bool controller = !(f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION);   // else the scores come from the attention
   if (c->ctrl_pending) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_ctrl, 0));   // scores of token n-1
-  if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit, c->ctl);
-  else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit, c->ctl);
-  if (st != ADORE_OK) return st;
+  if (controller) {
+    if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit, c->ctl);
+    else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit, c->ctl);
+    if (st != ADORE_OK) return st;
+  }
   CUDA_OK(cudaEventRecord(c->ev_gates, c->ctl));
   const int P = ex ? pow2_at_least(r_in) : pow2_at_least(c->n);
   SelectParams sp = select_params(c, c->n, P, c->cur, 1 - c->cur);
@@ -411,6 +440,7 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
   CUDA_OK(cudaGetLastError());
   st = launch_row_table(c, true, sel);
   if (st != ADORE_OK) return st;
+  if (!controller) return ADORE_OK;
   RecurParams rp = recur_params(c, f.batch, 1, c->ksplit, c->n);
   ctrl_recur_kernel<<<f.batch, select_threads(c), ctrl_smem(c), c->ctl>>>(rp, ctrl_resident_ok(f.ctrl_hidden) ? 1 : 0, c->err);
   ++c->launches;
@@ -492,6 +522,8 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, dev);
   }
   TRY(dev_alloc(c, &c->err, sizeof(unsigned), true));
+  if (f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION)
+    TRY(dev_alloc(c, &c->w_internal, B * f.n_heads * (C + 1) * sizeof(float), true));
   // decode splits the d-long dot products so that roughly one wave of CTAs is busy
   {
     const int tiles = int((G + kGateTileG - 1) / kGateTileG) * int((B + kGateTileR - 1) / kGateTileR);
@@ -598,7 +630,8 @@ adore_status_t adore_cache_append_tokens(adore_cache_t* c, const void* x, int32_
                             cudaMemcpyDeviceToDevice, c->stream));
   int chunk = int(c->part_doubles / (size_t(3) * f.ctrl_hidden) / f.batch);
   if (chunk < 1) chunk = 1;
-  for (int t0 = 0; t0 < T; t0 += chunk) {
+  // with the attention as the score source a prompt token has earned nothing yet: all scores stay zero
+  for (int t0 = 0; t0 < T && !(f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION); t0 += chunk) {
     const int tc = std::min(chunk, T - t0);
     adore_status_t st;
     if (f.dtype == ADORE_F32)
@@ -642,6 +675,8 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
                                  int32_t r_in, void* out, float* weights) {
   if (!c || !q || !k_new || !v_new || !out || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
   const adore_config_t& f = c->cfg;
+  const bool from_attention = (f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION) != 0;
+  if (from_attention && !weights) weights = c->w_internal;
   if (layer == 0) {
     if (!x_new) return ADORE_ERR_INVALID_ARG;
     if (c->n >= f.max_tokens) return ADORE_ERR_TOKEN_TABLE_FULL;
@@ -695,9 +730,12 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
   } else if (c->step_layer0_done != 1) {
     return ADORE_ERR_STATE;       // no step open, or one opened by adore_step_begin
   }
-  if (layer != 0)
-    return f.dtype == ADORE_F32 ? launch_attention<float>(c, layer, q, k_new, v_new, out, weights, true)
-                                : launch_attention<__nv_bfloat16>(c, layer, q, k_new, v_new, out, weights, true);
+  if (layer != 0) {
+    adore_status_t st = f.dtype == ADORE_F32 ? launch_attention<float>(c, layer, q, k_new, v_new, out, weights, true)
+                                             : launch_attention<__nv_bfloat16>(c, layer, q, k_new, v_new, out, weights, true);
+    if (st != ADORE_OK || !from_attention) return st;
+    return launch_add_attention(c, weights);
+  }
   if (!c->joined) CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
   c->joined = true;
   CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_gates, 0));   // x_new is borrowed only until the main stream passes the call
@@ -710,6 +748,8 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     ++c->launches;
     CUDA_OK(cudaGetLastError());
   }
+  // after the join: this step's selection has read the scores it ranks by, the weights count from the next step on
+  if (from_attention) return launch_add_attention(c, weights);
   return ADORE_OK;
 }
 
@@ -717,6 +757,7 @@ adore_status_t adore_step_begin(adore_cache_t* c, const void* x_new, const int32
                                 const int32_t* explicit_count, int32_t r_in) {
   if (!c || !x_new) return ADORE_ERR_INVALID_ARG;
   const adore_config_t& f = c->cfg;
+  if (f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION) return ADORE_ERR_UNSUPPORTED;   // defined for the attend-first step
   if (c->n >= f.max_tokens) return ADORE_ERR_TOKEN_TABLE_FULL;
   const bool ex = f.rebuild_mode == ADORE_REBUILD_EXPLICIT;
   if (r_in < 0 || (ex && r_in > 0 && (!explicit_list || !explicit_count))) return ADORE_ERR_INVALID_ARG;

@@ -56,7 +56,8 @@ class GpuCache:
                             hidden=c.hidden, capacity=c.capacity, rebuild_max=c.rebuild_max, topk=c.topk,
                             max_tokens=c.max_tokens, ctrl_hidden=c.ctrl_hidden, dtype=c.dtype,
                             rebuild_mode=c.rebuild_mode, rope_theta=c.rope_theta, pos_scale=c.pos_scale,
-                            flags=lib.ADORE_FLAG_NO_RECURRENCE if c.ctrl_no_recurrence else 0),
+                            flags=(lib.ADORE_FLAG_NO_RECURRENCE if c.ctrl_no_recurrence else 0) |
+                            (lib.ADORE_FLAG_SCORE_FROM_ATTENTION if c.score_from_attention else 0)),
             w.ctrl, torch.cuda.current_stream().cuda_stream)
         self.w_kv_dev = [to_dev(m, c) for m in w.w_kv]
         for l, m in enumerate(self.w_kv_dev):
@@ -162,7 +163,7 @@ def compare_attention(rep: Report, cfg, q, orc: ao.AdoreOracle, layer, k_new, at
     assert np.allclose(s, 1.0, atol=1e-4), "weights do not sum to one"
 
 
-def compare_state(rep: Report, g: GpuCache, orc: ao.AdoreOracle, layers, check_scores=True):
+def compare_state(rep: Report, g: GpuCache, orc: ao.AdoreOracle, layers, check_scores=True, score_rtol=1e-6):
     cfg = g.cfg
     st, sr = g.slot_map()
     assert np.array_equal(st, orc.slot_tok), f"slot map differs at step {rep.steps}"
@@ -178,7 +179,7 @@ def compare_state(rep: Report, g: GpuCache, orc: ao.AdoreOracle, layers, check_s
         sc, sg = g.scores(orc.n)
         mism = int((sc != orc.score[:, : orc.n]).sum())
         rep.score_mismatch += mism
-        assert np.allclose(sc, orc.score[:, : orc.n], rtol=1e-6, atol=1e-9)
+        assert np.allclose(sc, orc.score[:, : orc.n], rtol=score_rtol, atol=1e-9)
         assert np.allclose(sg, orc.sigma[:, : orc.n], rtol=1e-6, atol=1e-9)
     occ = orc.slot_tok >= 0
     for l in layers:
@@ -259,7 +260,16 @@ def run_parity(cfg: wl.WorkloadConfig, batch: Optional[int] = None, steps: Optio
                 orc.rebuild(l, otab[l] if (cfg.per_layer_inputs and l > 0) else None)
                 lib.adore_rebuild(g.handle, l, tables[l] if (cfg.per_layer_inputs and l > 0) else None)
             rep.steps += 1
-            if (s + 1) % state_every == 0 or s == n_steps - 1:
+            if cfg.score_from_attention:
+                # The values that rank the tokens are float32 sums of attention weights, which the two sides compute to
+                # within a few units in the last place of each other. They are compared every step, and once they agree
+                # to 1e-5 the oracle continues from the library's values, so that a difference in the last bits
+                # cannot grow into a different eviction many steps later.
+                lib.adore_cache_sync_status(g.handle)
+                orc.check_invariants()
+                compare_state(rep, g, orc, range(L), score_rtol=1e-5)
+                orc.score[:, : orc.n] = g.scores(orc.n)[0]
+            elif (s + 1) % state_every == 0 or s == n_steps - 1:
                 lib.adore_cache_sync_status(g.handle)
                 orc.check_invariants()
                 compare_state(rep, g, orc, range(L))

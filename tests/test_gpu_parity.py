@@ -148,3 +148,12 @@ def test_rebuild_first_step_with_query_rows_of_the_rebuilt_tokens():
                                     steps=20, seed=126))
     _run_rebuild_first(SMALL.scaled(name="rows_two_layers_c300", n_layers=2, batch=2, capacity=300, topk=100, rebuild_max=9,
                                     prompt=400, steps=8, seed=127))
+
+
+def test_cumulative_attention_as_the_score_source():
+    """The H2O / H2O(Rebuilt) score source on the same kernels: no controller, tokens ranked by the attention weight
+    they have received (policy lists = the released tokens with the most cumulative attention)."""
+    _run(SMALL.scaled(name="h2o_policy", score_from_attention=True, steps=40, seed=128))
+    _run(SMALL.scaled(name="h2o_no_rebuild", score_from_attention=True, rebuild_max=0, steps=30, seed=129))
+    _run(SMALL.scaled(name="h2o_two_layers_f32", score_from_attention=True, dtype="f32", n_layers=2, batch=2, n_heads=2,
+                      hidden=128, capacity=33, topk=7, steps=25, seed=130))
