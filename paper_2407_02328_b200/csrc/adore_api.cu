@@ -16,6 +16,7 @@
 #include "rebuild_tc.cuh"
 #include "select.cuh"
 #include "labels.cuh"
+#include "attention_rows.cuh"
 
 using namespace adore;
 
@@ -155,6 +156,7 @@ struct adore_cache {
   bool joined = true;
   std::vector<const void*> w_kv;
   TcState tc;                   // tensor-core rebuild path (tensor maps, gather buffer)
+  std::vector<CUtensorMap> map_k, map_v;   // per layer: the cache as [B*H*C, dh] tiles of 64 x 64 (bf16, dh 64 or 128)
   float* w_internal = nullptr;  // [B,H,C+1] weights when the caller passes none but the scores need them
   bool rows_gathered = false;   // the gather buffer holds this step's listed rows, taken from the token store
   // staging for the host-buffer entry point
@@ -282,6 +284,31 @@ adore_status_t launch_gates(adore_cache* c, const T* x, long long seq_stride, in
 }
 
 template <typename T>
+bool launch_attention_rows(adore_cache*, int, const AttnParams<T>&, int) { return false; }
+
+template <>
+bool launch_attention_rows<__nv_bfloat16>(adore_cache* c, int layer, const AttnParams<__nv_bfloat16>& p, int rows_q) {
+  const adore_config_t& f = c->cfg;
+  static const bool off = std::getenv("ADORE_ROWS_SIMT") != nullptr;     // A/B switch
+  const size_t smem = rows_smem_bytes(f.capacity, f.head_dim, rows_q);
+  if (off || c->map_k.empty() || rows_q > kRowsMaxQ || smem > 200 * 1024) return false;
+  static bool opted[2] = {false, false};
+  const int which = f.head_dim == 128 ? 1 : 0;
+  if (!opted[which]) {
+    cudaError_t e = which ? cudaFuncSetAttribute(attention_rows_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
+                          : cudaFuncSetAttribute(attention_rows_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) { cudaGetLastError(); return false; }
+    opted[which] = true;
+  }
+  const dim3 grid(unsigned(f.batch * f.n_heads)), block(kRowsThreads);
+  cudaError_t e = which ? launch_dependent(attention_rows_kernel<128>, grid, block, smem, c->stream, c->map_k[layer], c->map_v[layer], p)
+                        : launch_dependent(attention_rows_kernel<64>, grid, block, smem, c->stream, c->map_k[layer], c->map_v[layer], p);
+  ++c->launches;
+  if (e != cudaSuccess) { cudaGetLastError(); return false; }
+  return true;
+}
+
+template <typename T>
 adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const void* k_new, const void* v_new,
                                 void* out, float* weights, bool fused_admit, int rows_q = 1) {
   const adore_config_t& f = c->cfg;
@@ -303,7 +330,10 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
   // Few (b, h) pairs: a cluster of CTAs shares each of them. Not at layer 0: there the controller's
   // one-CTA-per-sequence kernel (200 KB of shared memory each) runs beside the attention and needs
   // SMs that the extra CTAs would occupy; measured at batch 1 the step got slower, not faster.
-  if (rows_q > 1) {            // several query rows per pair: the staged kernel only
+  if (rows_q > 1) {
+    // up to 16 rows on bfloat16 caches: the tensor-core kernel, one pass over the pair's keys and values for all rows
+    if (launch_attention_rows<T>(c, layer, p, rows_q)) return ADORE_OK;
+    // otherwise the staged kernel once per row (rows of a pair adjacent in the grid, sharing the blocks through L2)
     if (!attn_tma_usable<T>(f.capacity, f.head_dim)) return ADORE_ERR_UNSUPPORTED;
     cudaError_t er = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
     ++c->launches;
@@ -584,6 +614,26 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   if (f.dtype == ADORE_BF16) {
     st = tc_init(c->tc, f, c->owned, c->stream);
     if (st != ADORE_OK) { adore_cache_destroy(c); return st; }
+    if (c->tc.encode != nullptr && (f.head_dim == 64 || f.head_dim == 128)) {
+      // tensor maps over each layer's key and value cache for the kernel with several query rows per pair
+      const size_t layer_elems = B * f.n_heads * C * f.head_dim;
+      c->map_k.resize(f.n_layers);
+      c->map_v.resize(f.n_layers);
+      bool ok = true;
+      for (int l = 0; l < f.n_layers && ok; ++l) {
+        const cuuint64_t dims[2] = {cuuint64_t(f.head_dim), cuuint64_t(B * f.n_heads * C)};
+        const cuuint64_t strides[1] = {cuuint64_t(f.head_dim) * 2};
+        const cuuint32_t box[2] = {64u, uint32_t(kRowsTile)};
+        const cuuint32_t estr[2] = {1, 1};
+        void* bases[2] = {static_cast<__nv_bfloat16*>(c->Kc) + l * layer_elems, static_cast<__nv_bfloat16*>(c->Vc) + l * layer_elems};
+        CUtensorMap* maps[2] = {&c->map_k[l], &c->map_v[l]};
+        for (int j = 0; j < 2; ++j)
+          ok = ok && c->tc.encode(maps[j], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, bases[j], dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+      }
+      if (!ok) { c->map_k.clear(); c->map_v.clear(); }
+    }
   }
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) { adore_cache_destroy(c); return ADORE_ERR_CUDA; }
 #undef TRY

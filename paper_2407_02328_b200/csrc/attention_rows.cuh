@@ -1,0 +1,347 @@
+// Attention of Section 2.3 with several query rows per (sequence, head) on the tensor cores (bfloat16 caches).
+//
+// The R_max + 1 query rows of a pair (the rebuilt tokens' rows and the current token's; at most 16) share ONE pass
+// over the pair's key rows and ONE over its value rows:
+//   phase 1  S = Q K^T. The key block streams through shared memory in tiles of 64 rows (TMA, 128-byte swizzle);
+//            the 16 x dh query block sits in registers as the A operand of mma.sync.m16n8k16, each of the 8 warps
+//            takes 8 keys of a tile (B operand via ldmatrix). Logits go to shared memory, masked by each row's
+//            position bound (a row sees tokens up to its own position; the slot reserved for the current token
+//            is not written yet and is skipped).
+//   phase 2  one warp per row: K-th largest logit by a 4-pass radix select on a warp-private histogram, softmax,
+//            weights in place (and to global memory if asked for).
+//   phase 3  O = P V. The value block streams through the same ring; P is split into a bfloat16 head and a
+//            bfloat16 remainder (two MMAs per step) so that the weights enter with ~2^-17 relative error;
+//            each warp owns dh/8 output columns. The current token's own value row is added for the last row.
+// Then the current token's rows are stored in their slot. Every mbarrier wait is bounded.
+#pragma once
+
+#include <cuda.h>
+
+#include "attention.cuh"
+#include "mbarrier.cuh"
+
+namespace adore {
+
+constexpr int kRowsThreads = 256;
+constexpr int kRowsWarps = kRowsThreads / 32;
+constexpr int kRowsTile = 64;            // key / value rows per tile
+constexpr int kRowsStages = 3;
+constexpr int kRowsMaxQ = 16;
+
+__host__ __device__ inline int rows_logit_stride(int C) {
+  int sp = (C + 1 + 3) & ~3;
+  if (sp % 32 == 0) sp += 4;
+  return sp;
+}
+__host__ __device__ inline size_t rows_smem_bytes(int C, int DH, int rows_q) {
+  return 1024 + size_t(kRowsStages) * kRowsTile * DH * 2 + 64 + 64 + sizeof(unsigned) * kRowsWarps * 256 +
+         sizeof(float) * size_t(rows_q) * rows_logit_stride(C);
+}
+
+__device__ __forceinline__ void rows_tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void rows_ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void rows_ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void rows_mma(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t rows_pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&t);
+}
+// Byte offset of element (row, 16-byte chunk `c16` of the 128-byte line) inside a 64-row x 128-byte tile stored with the
+// 128-byte swizzle (tile base 1024-byte aligned): the chunk index is XORed with the row's low three bits.
+__device__ __forceinline__ uint32_t rows_swz(int row, int c16) { return uint32_t(row) * 128u + (uint32_t(c16 ^ (row & 7)) << 4); }
+
+template <int DH>
+__global__ void __launch_bounds__(kRowsThreads)
+attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                      const AttnParams<__nv_bfloat16> p) {
+  using T = __nv_bfloat16;
+  constexpr int HALVES = DH / 64;                       // 64-column (128-byte) boxes per tile
+  constexpr int TILE_BYTES = kRowsTile * DH * 2;
+  constexpr int KSTEPS = DH / 16;
+  extern __shared__ __align__(1024) unsigned char rows_smem_raw[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(rows_smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* ring = base;
+  uint64_t* full = reinterpret_cast<uint64_t*>(base + size_t(kRowsStages) * TILE_BYTES);
+  int* s_qtok = reinterpret_cast<int*>(full + 8);       // [16] position bound per row (< 0: padding)
+  unsigned* s_hist = reinterpret_cast<unsigned*>(s_qtok + 16);
+  float* S = reinterpret_cast<float*>(s_hist + kRowsWarps * 256);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int bh = blockIdx.x, b = bh / p.H;
+  const int C = p.C, R1 = p.rows_q, SP = rows_logit_stride(C);
+  const int n_tiles = (C + kRowsTile - 1) / kRowsTile;
+  const int* map = p.slot_tok + size_t(b) * C;
+
+  if (tid == 0) {
+    for (int s = 0; s < kRowsStages; ++s) mbar_init(&full[s], 1u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  wait_for_prior_grid();
+  if (tid < kRowsMaxQ) s_qtok[tid] = tid < R1 - 1 ? p.row_tok[size_t(b) * p.r_max + tid] : (tid == R1 - 1 ? p.n_cur : -1);
+  __syncthreads();
+
+  // loads are numbered 0 .. 2 n_tiles - 1 (keys first, then values); load i uses stage i % kRowsStages
+  auto issue = [&](int i) {
+    const bool is_v = i >= n_tiles;
+    const int t = is_v ? i - n_tiles : i;
+    const int stage = i % kRowsStages;
+    unsigned char* dst = ring + size_t(stage) * TILE_BYTES;
+    mbar_expect_tx(&full[stage], uint32_t(TILE_BYTES));
+#pragma unroll
+    for (int hlf = 0; hlf < HALVES; ++hlf)
+      rows_tma_load_2d(dst + hlf * (kRowsTile * 128), is_v ? &map_v : &map_k, hlf * 64, bh * C + t * kRowsTile, &full[stage]);
+  };
+  const int n_loads = 2 * n_tiles;
+  if (tid == 0)
+    for (int i = 0; i < min(kRowsStages, n_loads); ++i) issue(i);
+
+  // ---- query block as A fragments: rows lane/4 and lane/4 + 8, columns 16 ks + (lane % 4) * 2 (+8) ----
+  uint32_t qa[KSTEPS][4];
+  {
+    const T* qb = p.q + size_t(bh) * R1 * DH;
+    const int r0 = lane >> 2, r1 = r0 + 8, c0 = (lane & 3) * 2;
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks) {
+      const int col = ks * 16 + c0;
+      qa[ks][0] = r0 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r0) * DH + col) : 0u;
+      qa[ks][1] = r1 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r1) * DH + col) : 0u;
+      qa[ks][2] = r0 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r0) * DH + col + 8) : 0u;
+      qa[ks][3] = r1 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r1) * DH + col + 8) : 0u;
+    }
+  }
+  // the current token's own key: last row only (index C); every other row does not see it
+  if (warp == kRowsWarps - 1) {
+    const T* ql = p.q + (size_t(bh) * R1 + (R1 - 1)) * DH;
+    const T* kn = p.k_new + size_t(bh) * DH;
+    float dot = 0.f;
+    for (int e = lane; e < DH; e += 32) dot = fmaf(__bfloat162float(ql[e]), __bfloat162float(kn[e]), dot);
+    dot = warp_sum(dot);
+    for (int r = lane; r < R1; r += 32) S[size_t(r) * SP + C] = (r == R1 - 1) ? dot * p.scale : -INFINITY;
+  }
+
+  bool failed = false;
+  // ---- phase 1: logits ----
+  for (int t = 0; t < n_tiles; ++t) {
+    const int stage = t % kRowsStages;
+    const uint32_t parity = uint32_t(t / kRowsStages) & 1u;
+    if (!mbar_wait_bounded(&full[stage], parity, failed ? kDrainPolls : kWaitPolls)) {
+      if (!failed) set_error(p.err, ERRW_TIMEOUT);
+      failed = true;
+    }
+    const uint32_t tile = smem_u32(ring + size_t(stage) * TILE_BYTES);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    // ldmatrix.x4: matrix j holds keys warp*8 .. +7 (rows) x 8 columns starting at 8 * (4 q + j)
+    const int krow = warp * 8 + (lane & 7), mj = lane >> 3;
+#pragma unroll
+    for (int q4 = 0; q4 < DH / 32; ++q4) {
+      const int c16 = q4 * 4 + mj;                      // 16-byte chunk along dh (0 .. DH/8 - 1)
+      uint32_t bf[4];
+      rows_ldmatrix_x4(tile + uint32_t(c16 >> 3) * (kRowsTile * 128) + rows_swz(krow, c16 & 7), bf);
+      rows_mma(acc, qa[2 * q4], bf[0], bf[1]);
+      rows_mma(acc, qa[2 * q4 + 1], bf[2], bf[3]);
+    }
+    // accumulator: rows lane/4 (+8), keys (lane % 4) * 2 (+1) of this warp's 8
+    const int key0 = t * kRowsTile + warp * 8 + (lane & 3) * 2;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int r = (lane >> 2) + (e >> 1) * 8, key = key0 + (e & 1);
+      if (r < R1 && key < C) {
+        const int tok = map[key], qt = s_qtok[r];
+        const bool ok = tok >= 0 && tok <= qt && tok != p.n_cur;
+        S[size_t(r) * SP + key] = ok ? acc[e] * p.scale : -INFINITY;
+      }
+    }
+    __syncthreads();                                    // everyone is done with this stage
+    if (tid == 0 && !failed && t + kRowsStages < n_loads) issue(t + kRowsStages);
+  }
+
+  // ---- phase 2: per row, which logits are kept, softmax, weights (one warp per row) ----
+  const int rows_n = C + 1;
+  for (int r = warp; r < R1; r += kRowsWarps) {
+    float* row = S + size_t(r) * SP;
+    unsigned* hist = s_hist + warp * 256;
+    float* wout = p.weights ? p.weights + (size_t(bh) * R1 + r) * rows_n : nullptr;
+    int cnt = 0;
+    for (int i = lane; i < rows_n; i += 32) cnt += row[i] > -INFINITY ? 1 : 0;
+    cnt = warp_sum(cnt);
+    uint32_t thr_key = 0u;
+    if (cnt > p.topk) {
+      uint32_t prefix = 0u, mask = 0u;
+      int need = p.topk, n_eq = 0;
+      for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = lane; i < 256; i += 32) hist[i] = 0u;
+        __syncwarp();
+        for (int i = lane; i < rows_n; i += 32) {
+          const uint32_t key = float_key(row[i]);
+          if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+        __syncwarp();
+        int c8[8], tot = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c8[j] = int(hist[lane * 8 + j]); tot += c8[j]; }
+        int incl = tot;                                 // this lane's bins and all higher ones
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += v;
+        }
+        const int above = incl - tot;
+        int sel_bin = -1, sel_need = 0, sel_cnt = 0;
+        if (above < need && need <= above + tot) {
+          int a = above;
+#pragma unroll
+          for (int j = 7; j >= 0; --j) {
+            if (a < need && need <= a + c8[j]) { sel_bin = lane * 8 + j; sel_need = need - a; sel_cnt = c8[j]; }
+            a += c8[j];
+          }
+        }
+        const unsigned who = __ballot_sync(0xffffffffu, sel_bin >= 0);
+        const int src = __ffs(who) - 1;
+        sel_bin = __shfl_sync(0xffffffffu, sel_bin, src);
+        need = __shfl_sync(0xffffffffu, sel_need, src);
+        n_eq = __shfl_sync(0xffffffffu, sel_cnt, src);
+        prefix |= uint32_t(sel_bin) << shift;
+        mask |= 255u << shift;
+        __syncwarp();
+      }
+      thr_key = prefix;
+      if (n_eq != need) {                               // equal logits at the threshold: the lowest indices stay
+        if (lane == 0) {
+          int left = need;
+          for (int i = 0; i < rows_n; ++i)
+            if (float_key(row[i]) == thr_key) { if (left > 0) --left; else row[i] = -INFINITY; }
+        }
+        __syncwarp();
+      }
+    }
+    float mx = -INFINITY;
+    for (int i = lane; i < rows_n; i += 32) {
+      const float l = row[i];
+      if (l > -INFINITY && float_key(l) >= thr_key) mx = fmaxf(mx, l);
+    }
+    mx = warp_max(mx);
+    float part = 0.f;
+    for (int i = lane; i < rows_n; i += 32) {
+      const float l = row[i];
+      const bool keep = l > -INFINITY && float_key(l) >= thr_key;
+      const float e = keep ? expf(l - mx) : 0.f;
+      row[i] = e;
+      part += e;
+    }
+    part = warp_sum(part);
+    const float inv = part > 0.f ? 1.f / part : 0.f;    // a padding row (nothing visible) keeps all-zero weights
+    for (int i = lane; i < rows_n; i += 32) {
+      const float w = row[i] * inv;
+      row[i] = w;
+      if (wout) wout[i] = w;
+    }
+  }
+  __syncthreads();
+
+  // ---- phase 3: O = P V; warp w owns output columns [w * DH/8, (w + 1) * DH/8) ----
+  constexpr int NT = DH / 64;                           // 8-column n-tiles per warp (2 for dh 128, 1 for dh 64)
+  float o[NT][4];
+#pragma unroll
+  for (int j = 0; j < NT; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+  for (int t = 0; t < n_tiles; ++t) {
+    const int li = n_tiles + t;
+    const int stage = li % kRowsStages;
+    const uint32_t parity = uint32_t(li / kRowsStages) & 1u;
+    if (!mbar_wait_bounded(&full[stage], parity, failed ? kDrainPolls : kWaitPolls)) {
+      if (!failed) set_error(p.err, ERRW_TIMEOUT);
+      failed = true;
+    }
+    const uint32_t tile = smem_u32(ring + size_t(stage) * TILE_BYTES);
+#pragma unroll
+    for (int ks = 0; ks < kRowsTile / 16; ++ks) {
+      // A: weights of rows lane/4 (+8) for keys 16 ks + (lane % 4) * 2 (+1, +8, +9) of this tile, head + remainder
+      const int key = t * kRowsTile + ks * 16 + (lane & 3) * 2;
+      const int r0 = lane >> 2, r1 = r0 + 8;
+      float w[4][2];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int r = (e & 1) ? r1 : r0, k = key + (e >> 1) * 8;
+        w[e][0] = (r < R1 && k < C) ? S[size_t(r) * SP + k] : 0.f;
+        w[e][1] = (r < R1 && k + 1 < C) ? S[size_t(r) * SP + k + 1] : 0.f;
+      }
+      uint32_t ah[4], al[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(w[e][0]), h1 = __float2bfloat16_rn(w[e][1]);
+        ah[e] = rows_pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
+        al[e] = rows_pack_bf16(w[e][0] - __bfloat162float(h0), w[e][1] - __bfloat162float(h1));
+      }
+      // B (transposed load): matrix j: keys 16 ks + 8 (j % 2) .. +7 (rows of the tile) x columns of n-tile j / 2
+      const int vrow = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+      for (int nt = 0; nt < NT; nt += 2) {
+        const int ntile = nt + (lane >> 4);             // which of the warp's n-tiles this lane addresses
+        const int c16 = warp * NT + (ntile < NT ? ntile : 0);
+        uint32_t bf[4];
+        rows_ldmatrix_x4_trans(tile + uint32_t(c16 >> 3) * (kRowsTile * 128) + rows_swz(vrow, c16 & 7), bf);
+        rows_mma(o[nt], ah, bf[0], bf[1]);
+        rows_mma(o[nt], al, bf[0], bf[1]);
+        if (nt + 1 < NT) {
+          rows_mma(o[nt + 1], ah, bf[2], bf[3]);
+          rows_mma(o[nt + 1], al, bf[2], bf[3]);
+        }
+      }
+    }
+    __syncthreads();
+    if (tid == 0 && !failed && li + kRowsStages < n_loads) issue(li + kRowsStages);
+  }
+
+  // ---- output: rows lane/4 (+8), columns warp * DH/8 + 8 nt + (lane % 4) * 2 (+1); last row gets the own value row ----
+  {
+    const T* vn = p.v_new + size_t(bh) * DH;
+    const float w_own = S[size_t(R1 - 1) * SP + C];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int col = warp * (DH / 8) + nt * 8 + (lane & 3) * 2;
+#pragma unroll
+      for (int hrow = 0; hrow < 2; ++hrow) {
+        const int r = (lane >> 2) + hrow * 8;
+        if (r >= R1) continue;
+        float a0 = o[nt][hrow * 2], a1 = o[nt][hrow * 2 + 1];
+        if (r == R1 - 1) {
+          a0 = fmaf(w_own, __bfloat162float(vn[col]), a0);
+          a1 = fmaf(w_own, __bfloat162float(vn[col + 1]), a1);
+        }
+        *reinterpret_cast<uint32_t*>(p.out + (size_t(bh) * R1 + r) * DH + col) = rows_pack_bf16(a0, a1);
+      }
+    }
+  }
+  // ---- admit: the current token's rows go into their slot (all tiles of this pair have been consumed) ----
+  if (p.admit_slot != nullptr) {
+    const int s = p.admit_slot[b];
+    if (s >= 0 && s < C) {
+      constexpr int V16 = DH * 2 / 16;
+      unsigned char* kd = reinterpret_cast<unsigned char*>(p.Kc) + (size_t(bh) * C + s) * DH * 2;
+      unsigned char* vd = reinterpret_cast<unsigned char*>(p.Vc) + (size_t(bh) * C + s) * DH * 2;
+      const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * DH * 2;
+      const unsigned char* vnew = reinterpret_cast<const unsigned char*>(p.v_new) + size_t(bh) * DH * 2;
+      if (tid < V16) reinterpret_cast<uint4*>(kd)[tid] = reinterpret_cast<const uint4*>(knew)[tid];
+      else if (tid < 2 * V16) reinterpret_cast<uint4*>(vd)[tid - V16] = reinterpret_cast<const uint4*>(vnew)[tid - V16];
+    } else if (tid == 0) {
+      set_error(p.err, ERRW_BOUNDS);
+    }
+  }
+}
+
+}  // namespace adore

@@ -150,6 +150,15 @@ def test_rebuild_first_step_with_query_rows_of_the_rebuilt_tokens():
                                     prompt=400, steps=8, seed=127))
 
 
+def test_rebuild_first_step_on_the_tensor_core_kernel_shapes():
+    """Up to 16 query rows on bfloat16 caches take the kernel that passes once over the pair's keys and values for all
+    rows (mma.sync on TMA-staged, swizzled tiles): head dim 64, a capacity of several ragged tiles, 15 + 1 rows."""
+    _run_rebuild_first(SMALL.scaled(name="rows_dh64_bf16", head_dim=64, n_heads=3, hidden=192, steps=25, seed=131))
+    _run_rebuild_first(SMALL.scaled(name="rows_c517_r15", capacity=517, topk=200, rebuild_max=15, prompt=700, steps=8, batch=2,
+                                    seed=132))
+    _run_rebuild_first(SMALL.scaled(name="rows_topk_off", topk=1000, rebuild_max=7, capacity=70, prompt=90, steps=12, seed=133))
+
+
 def test_cumulative_attention_as_the_score_source():
     """The H2O / H2O(Rebuilt) score source on the same kernels: no controller, tokens ranked by the attention weight
     they have received (policy lists = the released tokens with the most cumulative attention)."""
