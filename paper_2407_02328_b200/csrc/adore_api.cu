@@ -286,26 +286,38 @@ adore_status_t launch_gates(adore_cache* c, const T* x, long long seq_stride, in
 template <typename T>
 bool launch_attention_rows(adore_cache*, int, const AttnParams<T>&, int) { return false; }
 
+template <int DH, int KPL>
+bool launch_attention_rows_as(adore_cache* c, int layer, const AttnParams<__nv_bfloat16>& p, size_t smem) {
+  static bool opted = false;                                // per instantiation
+  if (!opted) {
+    if (cudaFuncSetAttribute(attention_rows_kernel<DH, KPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    opted = true;
+  }
+  const dim3 grid(unsigned(c->cfg.batch * c->cfg.n_heads)), block(kRowsThreads);
+  cudaError_t e = launch_dependent(attention_rows_kernel<DH, KPL>, grid, block, smem, c->stream, c->map_k[layer], c->map_v[layer], p);
+  ++c->launches;
+  if (e != cudaSuccess) { cudaGetLastError(); return false; }
+  return true;
+}
+
 template <>
 bool launch_attention_rows<__nv_bfloat16>(adore_cache* c, int layer, const AttnParams<__nv_bfloat16>& p, int rows_q) {
   const adore_config_t& f = c->cfg;
   static const bool off = std::getenv("ADORE_ROWS_SIMT") != nullptr;     // A/B switch
   const size_t smem = rows_smem_bytes(f.capacity, f.head_dim, rows_q);
-  if (off || c->map_k.empty() || rows_q > kRowsMaxQ || smem > 200 * 1024) return false;
-  static bool opted[2] = {false, false};
-  const int which = f.head_dim == 128 ? 1 : 0;
-  if (!opted[which]) {
-    cudaError_t e = which ? cudaFuncSetAttribute(attention_rows_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
-                          : cudaFuncSetAttribute(attention_rows_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) { cudaGetLastError(); return false; }
-    opted[which] = true;
+  const int per_lane = (f.capacity + 1 + 31) / 32;
+  if (off || c->map_k.empty() || rows_q > kRowsMaxQ || per_lane > kRowsKeysPerLaneMax || smem > 200 * 1024) return false;
+  if (f.head_dim == 128) {
+    if (per_lane <= 9) return launch_attention_rows_as<128, 9>(c, layer, p, smem);
+    if (per_lane <= 17) return launch_attention_rows_as<128, 17>(c, layer, p, smem);
+    return launch_attention_rows_as<128, 33>(c, layer, p, smem);
   }
-  const dim3 grid(unsigned(f.batch * f.n_heads)), block(kRowsThreads);
-  cudaError_t e = which ? launch_dependent(attention_rows_kernel<128>, grid, block, smem, c->stream, c->map_k[layer], c->map_v[layer], p)
-                        : launch_dependent(attention_rows_kernel<64>, grid, block, smem, c->stream, c->map_k[layer], c->map_v[layer], p);
-  ++c->launches;
-  if (e != cudaSuccess) { cudaGetLastError(); return false; }
-  return true;
+  if (per_lane <= 9) return launch_attention_rows_as<64, 9>(c, layer, p, smem);
+  if (per_lane <= 17) return launch_attention_rows_as<64, 17>(c, layer, p, smem);
+  return launch_attention_rows_as<64, 33>(c, layer, p, smem);
 }
 
 template <typename T>

@@ -7,8 +7,8 @@
 //            takes 8 keys of a tile (B operand via ldmatrix). Logits go to shared memory, masked by each row's
 //            position bound (a row sees tokens up to its own position; the slot reserved for the current token
 //            is not written yet and is skipped).
-//   phase 2  one warp per row: K-th largest logit by a 4-pass radix select on a warp-private histogram, softmax,
-//            weights in place (and to global memory if asked for).
+//   phase 2  one warp per row: K-th largest logit by bisection on the bits of an order-preserving key (counting with
+//            compares and warp sums, no atomics), softmax, weights in place (and to global memory if asked for).
 //   phase 3  O = P V. The value block streams through the same ring; P is split into a bfloat16 head and a
 //            bfloat16 remainder (two MMAs per step) so that the weights enter with ~2^-17 relative error;
 //            each warp owns dh/8 output columns. The current token's own value row is added for the last row.
@@ -25,8 +25,9 @@ namespace adore {
 constexpr int kRowsThreads = 256;
 constexpr int kRowsWarps = kRowsThreads / 32;
 constexpr int kRowsTile = 64;            // key / value rows per tile
-constexpr int kRowsStages = 3;
+constexpr int kRowsStages = 4;
 constexpr int kRowsMaxQ = 16;
+constexpr int kRowsKeysPerLaneMax = 33;  // logits of a row per lane: C + 1 <= 1056
 
 __host__ __device__ inline int rows_logit_stride(int C) {
   int sp = (C + 1 + 3) & ~3;
@@ -34,7 +35,7 @@ __host__ __device__ inline int rows_logit_stride(int C) {
   return sp;
 }
 __host__ __device__ inline size_t rows_smem_bytes(int C, int DH, int rows_q) {
-  return 1024 + size_t(kRowsStages) * kRowsTile * DH * 2 + 64 + 64 + sizeof(unsigned) * kRowsWarps * 256 +
+  return 1024 + size_t(kRowsStages) * kRowsTile * DH * 2 + 64 + 64 + sizeof(int) * size_t((C + 3) & ~3) +
          sizeof(float) * size_t(rows_q) * rows_logit_stride(C);
 }
 
@@ -65,7 +66,9 @@ __device__ __forceinline__ uint32_t rows_pack_bf16(float lo, float hi) {
 // 128-byte swizzle (tile base 1024-byte aligned): the chunk index is XORed with the row's low three bits.
 __device__ __forceinline__ uint32_t rows_swz(int row, int c16) { return uint32_t(row) * 128u + (uint32_t(c16 ^ (row & 7)) << 4); }
 
-template <int DH>
+// KPL: logits of a row held per lane during the selection (C + 1 <= 32 KPL); the counting loops run over all KPL
+// registers without guards (slots past the row hold key 0, which never counts).
+template <int DH, int KPL>
 __global__ void __launch_bounds__(kRowsThreads)
 attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                       const AttnParams<__nv_bfloat16> p) {
@@ -78,8 +81,8 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   unsigned char* ring = base;
   uint64_t* full = reinterpret_cast<uint64_t*>(base + size_t(kRowsStages) * TILE_BYTES);
   int* s_qtok = reinterpret_cast<int*>(full + 8);       // [16] position bound per row (< 0: padding)
-  unsigned* s_hist = reinterpret_cast<unsigned*>(s_qtok + 16);
-  float* S = reinterpret_cast<float*>(s_hist + kRowsWarps * 256);
+  int* s_tok = s_qtok + 16;                             // [C] the pair's slot map row (token position per slot)
+  float* S = reinterpret_cast<float*>(s_tok + ((p.C + 3) & ~3));
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int bh = blockIdx.x, b = bh / p.H;
@@ -94,6 +97,7 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   }
   wait_for_prior_grid();
   if (tid < kRowsMaxQ) s_qtok[tid] = tid < R1 - 1 ? p.row_tok[size_t(b) * p.r_max + tid] : (tid == R1 - 1 ? p.n_cur : -1);
+  for (int i = tid; i < C; i += kRowsThreads) s_tok[i] = map[i];
   __syncthreads();
 
   // loads are numbered 0 .. 2 n_tiles - 1 (keys first, then values); load i uses stage i % kRowsStages
@@ -162,7 +166,7 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     for (int e = 0; e < 4; ++e) {
       const int r = (lane >> 2) + (e >> 1) * 8, key = key0 + (e & 1);
       if (r < R1 && key < C) {
-        const int tok = map[key], qt = s_qtok[r];
+        const int tok = s_tok[key], qt = s_qtok[r];
         const bool ok = tok >= 0 && tok <= qt && tok != p.n_cur;
         S[size_t(r) * SP + key] = ok ? acc[e] * p.scale : -INFINITY;
       }
@@ -175,53 +179,56 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   const int rows_n = C + 1;
   for (int r = warp; r < R1; r += kRowsWarps) {
     float* row = S + size_t(r) * SP;
-    unsigned* hist = s_hist + warp * 256;
     float* wout = p.weights ? p.weights + (size_t(bh) * R1 + r) * rows_n : nullptr;
+    // this lane's logits as order-preserving keys, in registers (masked and out-of-range entries rank lowest)
+    constexpr uint32_t kMasked = 0x007FFFFFu;           // key of -inf
+    uint32_t kk[KPL];
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) {
+      const int i = j * 32 + lane;
+      kk[j] = i < rows_n ? float_key(row[i]) : 0u;
+    }
     int cnt = 0;
-    for (int i = lane; i < rows_n; i += 32) cnt += row[i] > -INFINITY ? 1 : 0;
-    cnt = warp_sum(cnt);
+#pragma unroll
+    for (int j = 0; j < KPL; ++j)
+      cnt += __popc(__ballot_sync(0xffffffffu, kk[j] > kMasked));
     uint32_t thr_key = 0u;
     if (cnt > p.topk) {
-      uint32_t prefix = 0u, mask = 0u;
-      int need = p.topk, n_eq = 0;
-      for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int i = lane; i < 256; i += 32) hist[i] = 0u;
-        __syncwarp();
-        for (int i = lane; i < rows_n; i += 32) {
-          const uint32_t key = float_key(row[i]);
-          if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-        }
-        __syncwarp();
-        int c8[8], tot = 0;
+      // K-th largest key by bisection on the key's bits, most significant first: thr is the largest value with at
+      // least K keys >= thr. A count is a compare and a ballot per 32 keys, all in registers: no atomics, no
+      // shared-memory traffic, no dependence on how the logits are distributed. Bits above the highest bit in which
+      // the candidates differ are taken as given.
+      uint32_t kmin = 0xffffffffu, kmax = 0u;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { c8[j] = int(hist[lane * 8 + j]); tot += c8[j]; }
-        int incl = tot;                                 // this lane's bins and all higher ones
+      for (int j = 0; j < KPL; ++j)
+        if (kk[j] > kMasked) { kmin = min(kmin, kk[j]); kmax = max(kmax, kk[j]); }
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int v = __shfl_down_sync(0xffffffffu, incl, o);
-          if (lane + o < 32) incl += v;
-        }
-        const int above = incl - tot;
-        int sel_bin = -1, sel_need = 0, sel_cnt = 0;
-        if (above < need && need <= above + tot) {
-          int a = above;
-#pragma unroll
-          for (int j = 7; j >= 0; --j) {
-            if (a < need && need <= a + c8[j]) { sel_bin = lane * 8 + j; sel_need = need - a; sel_cnt = c8[j]; }
-            a += c8[j];
-          }
-        }
-        const unsigned who = __ballot_sync(0xffffffffu, sel_bin >= 0);
-        const int src = __ffs(who) - 1;
-        sel_bin = __shfl_sync(0xffffffffu, sel_bin, src);
-        need = __shfl_sync(0xffffffffu, sel_need, src);
-        n_eq = __shfl_sync(0xffffffffu, sel_cnt, src);
-        prefix |= uint32_t(sel_bin) << shift;
-        mask |= 255u << shift;
-        __syncwarp();
+      for (int o = 16; o > 0; o >>= 1) {
+        kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+        kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
       }
-      thr_key = prefix;
-      if (n_eq != need) {                               // equal logits at the threshold: the lowest indices stay
+      const uint32_t diff = kmin ^ kmax;
+      const int top = diff ? 31 - __clz(diff) : -1;
+      uint32_t thr = top >= 31 ? 0u : (kmax & ~((2u << (top < 0 ? 0 : top)) - 1u));
+      if (top < 0) thr = kmax;
+      for (int bit = top; bit >= 0; --bit) {
+        const uint32_t cand = thr | (1u << bit);
+        int c = 0;
+#pragma unroll
+        for (int j = 0; j < KPL; ++j)
+          c += __popc(__ballot_sync(0xffffffffu, kk[j] >= cand));
+        if (c >= p.topk) thr = cand;
+      }
+      thr_key = thr;
+      int gt = 0, eq = 0;
+#pragma unroll
+      for (int j = 0; j < KPL; ++j)
+      {
+        gt += __popc(__ballot_sync(0xffffffffu, kk[j] > thr));
+        eq += __popc(__ballot_sync(0xffffffffu, kk[j] == thr));
+      }
+      const int need = p.topk - gt;                     // how many of the keys equal to the threshold stay
+      if (eq != need) {                                 // equal logits at the threshold: the lowest indices stay
         if (lane == 0) {
           int left = need;
           for (int i = 0; i < rows_n; ++i)
