@@ -211,6 +211,7 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
       const int top = diff ? 31 - __clz(diff) : -1;
       uint32_t thr = top >= 31 ? 0u : (kmax & ~((2u << (top < 0 ? 0 : top)) - 1u));
       if (top < 0) thr = kmax;
+      bool exact = false;
       for (int bit = top; bit >= 0; --bit) {
         const uint32_t cand = thr | (1u << bit);
         int c = 0;
@@ -218,17 +219,19 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
         for (int j = 0; j < KPL; ++j)
           c += __popc(__ballot_sync(0xffffffffu, kk[j] >= cand));
         if (c >= p.topk) thr = cand;
+        if (c == p.topk) { exact = true; break; }       // exactly K keys are >= thr: that is the kept set
       }
       thr_key = thr;
       int gt = 0, eq = 0;
+      if (!exact) {
 #pragma unroll
-      for (int j = 0; j < KPL; ++j)
-      {
-        gt += __popc(__ballot_sync(0xffffffffu, kk[j] > thr));
-        eq += __popc(__ballot_sync(0xffffffffu, kk[j] == thr));
+        for (int j = 0; j < KPL; ++j) {
+          gt += __popc(__ballot_sync(0xffffffffu, kk[j] > thr));
+          eq += __popc(__ballot_sync(0xffffffffu, kk[j] == thr));
+        }
       }
       const int need = p.topk - gt;                     // how many of the keys equal to the threshold stay
-      if (eq != need) {                                 // equal logits at the threshold: the lowest indices stay
+      if (!exact && eq != need) {                       // equal logits at the threshold: the lowest indices stay
         if (lane == 0) {
           int left = need;
           for (int i = 0; i < rows_n; ++i)
