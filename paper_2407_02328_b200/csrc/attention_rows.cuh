@@ -11,7 +11,8 @@
 //            compares and warp sums, no atomics), softmax, weights in place (and to global memory if asked for).
 //   phase 3  O = P V. The value block streams through the same ring; P is split into a bfloat16 head and a
 //            bfloat16 remainder (two MMAs per step) so that the weights enter with ~2^-17 relative error;
-//            each warp owns dh/8 output columns. The current token's own value row is added for the last row.
+//            each warp takes one of a tile's four k-steps and half of the output columns, the partial outputs are
+//            added through shared memory. The current token's own value row is added for the last row.
 // Then the current token's rows are stored in their slot. Every mbarrier wait is bounded.
 #pragma once
 
@@ -177,7 +178,12 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
 
   // ---- phase 2: per row, which logits are kept, softmax, weights (one warp per row) ----
   const int rows_n = C + 1;
-  for (int r = warp; r < R1; r += kRowsWarps) {
+  // The current token's row always needs a selection (it sees every slot) and goes alone to warp 0; the other rows
+  // follow on warps 1..7, the ninth and later ones are stacked from warp 7 downwards.
+  for (int pass = 0; pass < 2; ++pass) {
+    const int e = pass == 0 ? warp : 15 - warp;          // entry 0: last row; entry e > 0: row e - 1
+    if (e >= R1) continue;
+    const int r = e == 0 ? R1 - 1 : e - 1;
     float* row = S + size_t(r) * SP;
     float* wout = p.weights ? p.weights + (size_t(bh) * R1 + r) * rows_n : nullptr;
     // this lane's logits as order-preserving keys, in registers (masked and out-of-range entries rank lowest)
@@ -264,11 +270,13 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   }
   __syncthreads();
 
-  // ---- phase 3: O = P V; warp w owns output columns [w * DH/8, (w + 1) * DH/8) ----
-  constexpr int NT = DH / 64;                           // 8-column n-tiles per warp (2 for dh 128, 1 for dh 64)
-  float o[NT][4];
+  // ---- phase 3: O = P V. Warp w takes k-step w % 4 (16 keys) of every tile and column half w / 4, so the weight
+  // fragments of a k-step are built by two warps instead of all eight; the partial outputs meet in shared memory ----
+  constexpr int NTW = DH / 16;                          // 8-column n-tiles per warp (8 for dh 128, 4 for dh 64)
+  const int my_ks = warp & 3, col_half = warp >> 2;
+  float o[NTW][4];
 #pragma unroll
-  for (int j = 0; j < NT; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+  for (int j = 0; j < NTW; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
   for (int t = 0; t < n_tiles; ++t) {
     const int li = n_tiles + t;
     const int stage = li % kRowsStages;
@@ -278,63 +286,69 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
       failed = true;
     }
     const uint32_t tile = smem_u32(ring + size_t(stage) * TILE_BYTES);
-#pragma unroll
-    for (int ks = 0; ks < kRowsTile / 16; ++ks) {
-      // A: weights of rows lane/4 (+8) for keys 16 ks + (lane % 4) * 2 (+1, +8, +9) of this tile, head + remainder
-      const int key = t * kRowsTile + ks * 16 + (lane & 3) * 2;
+    {
+      // A: weights of rows lane/4 (+8) for keys 16 my_ks + (lane % 4) * 2 (+1, +8, +9) of this tile, head + remainder
+      const int key = t * kRowsTile + my_ks * 16 + (lane & 3) * 2;
       const int r0 = lane >> 2, r1 = r0 + 8;
-      float w[4][2];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int r = (e & 1) ? r1 : r0, k = key + (e >> 1) * 8;
-        w[e][0] = (r < R1 && k < C) ? S[size_t(r) * SP + k] : 0.f;
-        w[e][1] = (r < R1 && k + 1 < C) ? S[size_t(r) * SP + k + 1] : 0.f;
-      }
       uint32_t ah[4], al[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const __nv_bfloat16 h0 = __float2bfloat16_rn(w[e][0]), h1 = __float2bfloat16_rn(w[e][1]);
+        const int r = (e & 1) ? r1 : r0, k = key + (e >> 1) * 8;
+        const float w0 = (r < R1 && k < C) ? S[size_t(r) * SP + k] : 0.f;
+        const float w1 = (r < R1 && k + 1 < C) ? S[size_t(r) * SP + k + 1] : 0.f;
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(w0), h1 = __float2bfloat16_rn(w1);
         ah[e] = rows_pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
-        al[e] = rows_pack_bf16(w[e][0] - __bfloat162float(h0), w[e][1] - __bfloat162float(h1));
+        al[e] = rows_pack_bf16(w0 - __bfloat162float(h0), w1 - __bfloat162float(h1));
       }
-      // B (transposed load): matrix j: keys 16 ks + 8 (j % 2) .. +7 (rows of the tile) x columns of n-tile j / 2
-      const int vrow = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+      // B (transposed load): matrix j: keys 16 my_ks + 8 (j % 2) .. +7 (rows of the tile) x the columns of n-tile j / 2
+      const int vrow = my_ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-      for (int nt = 0; nt < NT; nt += 2) {
-        const int ntile = nt + (lane >> 4);             // which of the warp's n-tiles this lane addresses
-        const int c16 = warp * NT + (ntile < NT ? ntile : 0);
+      for (int nt = 0; nt < NTW; nt += 2) {
+        const int c16 = col_half * NTW + nt + (lane >> 4);
         uint32_t bf[4];
         rows_ldmatrix_x4_trans(tile + uint32_t(c16 >> 3) * (kRowsTile * 128) + rows_swz(vrow, c16 & 7), bf);
         rows_mma(o[nt], ah, bf[0], bf[1]);
         rows_mma(o[nt], al, bf[0], bf[1]);
-        if (nt + 1 < NT) {
-          rows_mma(o[nt + 1], ah, bf[2], bf[3]);
-          rows_mma(o[nt + 1], al, bf[2], bf[3]);
-        }
+        rows_mma(o[nt + 1], ah, bf[2], bf[3]);
+        rows_mma(o[nt + 1], al, bf[2], bf[3]);
       }
     }
     __syncthreads();
     if (tid == 0 && !failed && li + kRowsStages < n_loads) issue(li + kRowsStages);
   }
 
-  // ---- output: rows lane/4 (+8), columns warp * DH/8 + 8 nt + (lane % 4) * 2 (+1); last row gets the own value row ----
+  // ---- the four k-step warps of a column half add up through shared memory (the ring is free now), then rows < R1
+  // go out; the last row also gets the current token's own value row ----
   {
-    const T* vn = p.v_new + size_t(bh) * DH;
-    const float w_own = S[size_t(R1 - 1) * SP + C];
+    float* part = reinterpret_cast<float*>(ring);       // [4 k-steps][16 rows][DH] floats: at most 32 KB
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const int col = warp * (DH / 8) + nt * 8 + (lane & 3) * 2;
+    for (int nt = 0; nt < NTW; ++nt) {
+      const int col = col_half * (DH / 2) + nt * 8 + (lane & 3) * 2;
 #pragma unroll
       for (int hrow = 0; hrow < 2; ++hrow) {
         const int r = (lane >> 2) + hrow * 8;
-        if (r >= R1) continue;
-        float a0 = o[nt][hrow * 2], a1 = o[nt][hrow * 2 + 1];
-        if (r == R1 - 1) {
-          a0 = fmaf(w_own, __bfloat162float(vn[col]), a0);
-          a1 = fmaf(w_own, __bfloat162float(vn[col + 1]), a1);
-        }
-        *reinterpret_cast<uint32_t*>(p.out + (size_t(bh) * R1 + r) * DH + col) = rows_pack_bf16(a0, a1);
+        float* d = part + (size_t(my_ks) * 16 + r) * DH + col;
+        d[0] = o[nt][hrow * 2];
+        d[1] = o[nt][hrow * 2 + 1];
       }
+    }
+    __syncthreads();
+    const T* vn = p.v_new + size_t(bh) * DH;
+    const float w_own = S[size_t(R1 - 1) * SP + C];
+    for (int i = tid; i < R1 * (DH / 2); i += kRowsThreads) {
+      const int r = i / (DH / 2), col = (i % (DH / 2)) * 2;
+      float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        const float* d = part + (size_t(q4) * 16 + r) * DH + col;
+        a0 += d[0];
+        a1 += d[1];
+      }
+      if (r == R1 - 1) {
+        a0 = fmaf(w_own, __bfloat162float(vn[col]), a0);
+        a1 = fmaf(w_own, __bfloat162float(vn[col + 1]), a1);
+      }
+      *reinterpret_cast<uint32_t*>(p.out + (size_t(bh) * R1 + r) * DH + col) = rows_pack_bf16(a0, a1);
     }
   }
   // ---- admit: the current token's rows go into their slot (all tiles of this pair have been consumed) ----
