@@ -27,7 +27,9 @@ __host__ __device__ inline size_t attn_tma_smem_bytes(int C, int DH, int threads
 // NT threads per CTA and kRingStages ring stages are chosen per launch: 128 threads / 2 stages put
 // 8-10 CTAs on an SM (fewer, shorter waves when there are many (b, h) pairs), 256 threads / 4 stages
 // give each pair more threads (better when there are few pairs or very long key blocks).
-template <typename T, int DH, int NT, int kRingStages>
+// MULTI: several query rows per pair (Section 2.3's rebuilt tokens' rows); the plain decode step compiles without any
+// of that logic.
+template <typename T, int DH, int NT, int kRingStages, bool MULTI>
 __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p) {
   constexpr int NW = NT / 32;
   constexpr int EPL = Elem<T>::kPer16B;
@@ -50,17 +52,18 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
   const int sub = lane / LPR, li = lane % LPR;
   // item = one query row; with rows_q > 1 the rows of a (b, h) pair sit next to each other in the grid, so that the
   // pair's key and value blocks are fetched from HBM once and served to the other rows out of L2
-  const int item = blockIdx.x, qi = item % p.rows_q, bh = item / p.rows_q, b = bh / p.H;
-  const bool last_row = qi == p.rows_q - 1;
+  const int rows_q = MULTI ? p.rows_q : 1;
+  const int item = blockIdx.x, qi = MULTI ? item % rows_q : 0, bh = MULTI ? item / rows_q : item, b = bh / p.H;
+  const bool last_row = !MULTI || qi == rows_q - 1;
   const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * ROW_BYTES;
   const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * ROW_BYTES;
   const int* map = p.slot_tok + size_t(b) * C;
   const int n_chunks = (C + CHUNK_ROWS - 1) / CHUNK_ROWS;
 
-  wait_for_prior_grid();     // the cache rows, the slot map and q, k, v come from earlier kernels
   // position bound of this query row (plain decode step: everything occupied is visible)
   int q_tok = 0x7fffffff;
-  if (p.rows_q > 1) {
+  if (MULTI) {
+    wait_for_prior_grid();   // the row table comes from an earlier kernel
     q_tok = last_row ? p.n_cur : p.row_tok[size_t(b) * p.r_max + qi];
     if (q_tok < 0) {                                          // padding row: zeros, nothing else
       for (int e = tid; e < DH; e += NT) p.out[size_t(item) * DH + e] = Elem<T>::from_float(0.f);
@@ -76,6 +79,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+  if (!MULTI) wait_for_prior_grid();   // the cache rows, the slot map and q, k, v come from earlier kernels
   auto issue = [&](int chunk) {
     const int stage = chunk % kRingStages;
     const int r0 = chunk * CHUNK_ROWS;
@@ -101,7 +105,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kf[e], dot);
 #pragma unroll
     for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu >> (32 - LPR), dot, o);
-    if (li == 0) s_logit[C] = (p.rows_q == 1 || last_row) ? dot * p.scale : -INFINITY;
+    if (li == 0) s_logit[C] = last_row ? dot * p.scale : -INFINITY;
   }
 
   bool failed = false;
@@ -118,8 +122,13 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     for (int ps = 0; ps < PASSES; ++ps) {
       const int lr = ps * NW * RPW + warp * RPW + sub;      // row inside the chunk
       const int row = r0 + lr;
-      const int row_tok = row < C ? map[row] : -1;
-      const bool ok = row_tok >= 0 && row_tok <= q_tok && (p.rows_q == 1 || row_tok != p.n_cur);
+      bool ok;
+      if (MULTI) {
+        const int row_tok = row < C ? map[row] : -1;
+        ok = row_tok >= 0 && row_tok <= q_tok && row_tok != p.n_cur;
+      } else {
+        ok = row < C && map[row] >= 0;
+      }
       float kf[EPL];
       // rows past C in a ragged last chunk hold stale bytes of an earlier chunk: read, not used
       Elem<T>::unpack(*reinterpret_cast<const uint4*>(src + size_t(lr) * ROW_BYTES + li * 16), kf);
@@ -149,16 +158,21 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
 template <typename T>
 inline bool attn_tma_usable(int /*C*/, int DH) { return DH == 64 || DH == 128; }
 
-template <typename T, int DH, int NT, int STAGES>
-inline cudaError_t launch_attention_tma_cfg(const AttnParams<T>& p, int grid, cudaStream_t stream) {
+template <typename T, int DH, int NT, int STAGES, bool MULTI>
+inline cudaError_t launch_attention_tma_as(const AttnParams<T>& p, int grid, cudaStream_t stream) {
   const size_t smem = attn_tma_smem_bytes(p.C, DH, NT, STAGES);
   static bool opted_in = false;            // per instantiation; the attribute is per function
   if (!opted_in) {
-    cudaError_t e = cudaFuncSetAttribute(attention_tma_kernel<T, DH, NT, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(attention_tma_kernel<T, DH, NT, STAGES, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
     if (e != cudaSuccess) return e;
     opted_in = true;
   }
-  return launch_dependent(attention_tma_kernel<T, DH, NT, STAGES>, dim3(grid), dim3(NT), smem, stream, p);
+  return launch_dependent(attention_tma_kernel<T, DH, NT, STAGES, MULTI>, dim3(grid), dim3(NT), smem, stream, p);
+}
+template <typename T, int DH, int NT, int STAGES>
+inline cudaError_t launch_attention_tma_cfg(const AttnParams<T>& p, int grid, cudaStream_t stream) {
+  return p.rows_q > 1 ? launch_attention_tma_as<T, DH, NT, STAGES, true>(p, grid, stream)
+                      : launch_attention_tma_as<T, DH, NT, STAGES, false>(p, grid, stream);
 }
 
 // Many (b, h) pairs with key blocks of moderate length: small CTAs; otherwise large ones (measured on the
