@@ -342,15 +342,25 @@ class DeviceRun:
                       counts=None if self.counts is None else pin(self.counts[sl]),
                       out=t.empty(self.out.shape, dtype=self.dt).pin_memory())
         self.h_first = first
+        # host addresses taken once: the timed loop passes integers only
+        h = self.h
+        self.hp = dict(q=[[h["q"][i, l].data_ptr() for l in range(h["q"].shape[1])] for i in range(count)],
+                       k=[[h["k"][i, l].data_ptr() for l in range(h["k"].shape[1])] for i in range(count)],
+                       v=[[h["v"][i, l].data_ptr() for l in range(h["v"].shape[1])] for i in range(count)],
+                       x=[h["x"][i, 0].data_ptr() for i in range(count)],
+                       lists=None if h["lists"] is None else [h["lists"][i].data_ptr() for i in range(count)],
+                       counts=None if h["counts"] is None else [h["counts"][i].data_ptr() for i in range(count)],
+                       out=h["out"].data_ptr())
 
     def step_host(self):
         lib, c, s = self.lib, self.cfg, self.next
-        i, h = s - self.h_first, self.h
+        i, hp = s - self.h_first, self.hp
+        pl = None if hp["lists"] is None else hp["lists"][i]
+        pc = None if hp["counts"] is None else hp["counts"][i]
         for l in range(c.n_layers):
-            lib.adore_decode_step_host(self.handle, l, h["q"][i, l], h["k"][i, l], h["v"][i, l], h["x"][i, 0],
-                                       None if h["lists"] is None else h["lists"][i],
-                                       None if h["counts"] is None else h["counts"][i], self.r_in, h["out"], self.weights)
-            lib.adore_rebuild(self.handle, l, self.tables[l] if (self.tables is not None and l > 0) else None)
+            lib.adore_decode_step_host(self.handle, l, hp["q"][i][l], hp["k"][i][l], hp["v"][i][l], hp["x"][i], pl, pc, self.r_in,
+                                       hp["out"], self.pw)
+            lib.adore_rebuild(self.handle, l, self.pt[l] if (self.pt is not None and l > 0) else None)
         self.next += 1
 
     def host_bytes_per_step(self):

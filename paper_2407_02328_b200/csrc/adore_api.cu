@@ -275,7 +275,15 @@ adore_status_t launch_gates(adore_cache* c, const T* x, long long seq_stride, in
   g.x = x; g.seq_stride = seq_stride; g.tc = tc; g.rows = c->cfg.batch * tc; g.d = c->cfg.hidden; g.G = 3 * c->cfg.ctrl_hidden;
   g.w_ih = c->w_ih; g.part = c->part; g.ksplit = ksplit;
   const int per = (c->cfg.hidden + ksplit - 1) / ksplit;
-  g.kslice = ((per + kGateKChunk - 1) / kGateKChunk) * kGateKChunk;
+  g.kslice = ((per + kGateKInner - 1) / kGateKInner) * kGateKInner;
+  static const bool narrow_only = std::getenv("ADORE_GATES_NARROW") != nullptr;   // A/B switch
+  if (g.rows >= kGateWideMinRows && !narrow_only) {
+    dim3 grid((g.G + kGateWideG - 1) / kGateWideG, (g.rows + kGateWideR - 1) / kGateWideR, ksplit);
+    ctrl_gates_wide_kernel<T><<<grid, kGateWideThreads, kGateWideSmem, stream>>>(g);
+    ++c->launches;
+    CUDA_OK(cudaGetLastError());
+    return ADORE_OK;
+  }
   dim3 grid((g.G + kGateTileG - 1) / kGateTileG, (g.rows + kGateTileR - 1) / kGateTileR, ksplit);
   ctrl_gates_kernel<T><<<grid, kGateThreads, 0, stream>>>(g);
   ++c->launches;
@@ -568,9 +576,14 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
     TRY(dev_alloc(c, &c->w_internal, B * f.n_heads * (C + 1) * sizeof(float), true));
   // decode splits the d-long dot products so that roughly one wave of CTAs is busy
   {
-    const int tiles = int((G + kGateTileG - 1) / kGateTileG) * int((B + kGateTileR - 1) / kGateTileR);
     int ks = 1;
-    while (ks < 16 && tiles * ks * 2 <= 296 && int(d) / (ks * 2) >= kGateKChunk) ks *= 2;
+    if (int(B) >= kGateWideMinRows) {     // decode uses the 128 x 64 tile kernel: one CTA per SM at most
+      const int tiles = int((G + kGateWideG - 1) / kGateWideG) * int((B + kGateWideR - 1) / kGateWideR);
+      while (ks < 32 && tiles * ks * 2 <= 192 && int(d) / (ks * 2) >= 2 * kGateKInner) ks *= 2;
+    } else {
+      const int tiles = int((G + kGateTileG - 1) / kGateTileG) * int((B + kGateTileR - 1) / kGateTileR);
+      while (ks < 16 && tiles * ks * 2 <= 296 && int(d) / (ks * 2) >= kGateKChunk) ks *= 2;
+    }
     c->ksplit = ks;
     const size_t rows_prefill = std::min<size_t>(B * MT, std::max<size_t>(kMaxPrefillRows, B));
     c->part_doubles = std::max<size_t>(size_t(ks) * B, rows_prefill) * G;
@@ -603,6 +616,8 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   {
     const int big = 227 * 1024;
     cudaFuncSetAttribute(ctrl_recur_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    cudaFuncSetAttribute(ctrl_gates_wide_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGateWideSmem));
+    cudaFuncSetAttribute(ctrl_gates_wide_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGateWideSmem));
     cudaFuncSetAttribute(select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     cudaFuncSetAttribute(select_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     cudaFuncSetAttribute(bulk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);

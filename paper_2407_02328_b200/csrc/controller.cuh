@@ -29,7 +29,7 @@ struct GateParams {
   int d, G;              // input width (multiple of 64), 3*d'
   const float* w_ih;     // [G, d]
   double* part;          // [ksplit, rows, G]
-  int ksplit, kslice;    // kslice is a multiple of kGateKChunk
+  int ksplit, kslice;    // kslice is a multiple of kGateKInner
 };
 
 // 64 gates x 32 rows per CTA, 4 x 2 outputs per thread, float64 FMA, k in chunks of 32. The next
@@ -114,6 +114,126 @@ __global__ void __launch_bounds__(kGateThreads) ctrl_gates_kernel(const GatePara
       const int g = g0 + 2 * tx + (a & 1) + 32 * (a >> 1), r = r0 + 2 * ty + c;
       if (g < p.G && r < p.rows) p.part[(size_t(ks) * p.rows + r) * p.G + g] = acc[a][c];
     }
+}
+
+// Same product for many rows (prompt chunks, decode at batch >= 48): 128 gates x 64 rows per CTA of 128 threads, 8 x 8
+// outputs per thread. Per k the thread reads 8 + 8 operands for 64 FMAs (2 bytes of shared memory per FMA instead of 6
+// with the 4 x 2 tile above), which is what the float64 pipe needs to stay busy.
+constexpr int kGateWideG = 128;
+constexpr int kGateWideR = 64;
+constexpr int kGateWideThreads = 128;
+constexpr int kGateWideMinRows = 48;     // fewer rows: the 64 x 32 tile kernel wastes less
+constexpr int kGateWideWS = kGateWideG + 2, kGateWideXS = kGateWideR + 2;   // padded row lengths (doubles)
+constexpr size_t kGateWideSmem = sizeof(double) * kGateKInner * (kGateWideWS + kGateWideXS);
+
+template <typename T>
+__global__ void __launch_bounds__(kGateWideThreads) ctrl_gates_wide_kernel(const GateParams<T> p) {
+  extern __shared__ __align__(16) double gw_smem[];
+  double (*Ws)[kGateWideWS] = reinterpret_cast<double (*)[kGateWideWS]>(gw_smem);
+  double (*Xs)[kGateWideXS] = reinterpret_cast<double (*)[kGateWideXS]>(gw_smem + kGateKInner * kGateWideWS);
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int g0 = blockIdx.x * kGateWideG, r0 = blockIdx.y * kGateWideR, ks = blockIdx.z;
+  const int k_begin = ks * p.kslice, k_end = min(p.d, k_begin + p.kslice);
+  // fetch roles: 8 float4 of W (gate (tid + 128 q) / 8, k offset 4 * ((tid + 128 q) % 8)) and 2 x 8 elements of x
+  // (row (tid + 128 q) / 4, k offset 8 * ((tid + 128 q) % 4)) per chunk of 32 k
+  const float* wsrc[8];
+  bool wok[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const int idx = tid + kGateWideThreads * q, g = g0 + (idx >> 3);
+    wok[q] = g < p.G;
+    wsrc[q] = p.w_ih + size_t(wok[q] ? g : 0) * p.d + 4 * (idx & 7);
+  }
+  const T* xsrc[2];
+  bool xok[2];
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    const int idx = tid + kGateWideThreads * q;
+    const long long r = r0 + (idx >> 2);
+    xok[q] = r < p.rows;
+    xsrc[q] = p.x;
+    if (xok[q]) xsrc[q] = p.x + ((r / p.tc) * p.seq_stride + (r % p.tc)) * p.d + 8 * (idx & 3);
+  }
+  float4 wreg[8];
+  float xreg[2][8];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q)
+      wreg[q] = wok[q] ? __ldg(reinterpret_cast<const float4*>(wsrc[q] + k0)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      if (!xok[q]) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) xreg[q][e] = 0.f;
+      } else if (sizeof(T) == 2) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(xsrc[q] + k0));
+        const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          xreg[q][2 * e] = __uint_as_float(u[e] << 16);
+          xreg[q][2 * e + 1] = __uint_as_float(u[e] & 0xffff0000u);
+        }
+      } else {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(xsrc[q] + k0));
+        const float4 b = __ldg(reinterpret_cast<const float4*>(xsrc[q] + k0) + 1);
+        xreg[q][0] = a.x; xreg[q][1] = a.y; xreg[q][2] = a.z; xreg[q][3] = a.w;
+        xreg[q][4] = b.x; xreg[q][5] = b.y; xreg[q][6] = b.z; xreg[q][7] = b.w;
+      }
+    }
+  };
+  double acc[4][4][2][2];       // [gate pair j][row pair i][gate within pair][row within pair]
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { acc[j][i][0][0] = acc[j][i][0][1] = acc[j][i][1][0] = acc[j][i][1][1] = 0.0; }
+  if (k_begin < k_end) fetch(k_begin);
+  for (int k0 = k_begin; k0 < k_end; k0 += kGateKInner) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int idx = tid + kGateWideThreads * q, g = idx >> 3, kk = 4 * (idx & 7);
+      Ws[kk + 0][g] = double(wreg[q].x);
+      Ws[kk + 1][g] = double(wreg[q].y);
+      Ws[kk + 2][g] = double(wreg[q].z);
+      Ws[kk + 3][g] = double(wreg[q].w);
+    }
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int idx = tid + kGateWideThreads * q, r = idx >> 2, kk = 8 * (idx & 3);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) Xs[kk + e][r] = double(xreg[q][e]);
+    }
+    __syncthreads();
+    if (k0 + kGateKInner < k_end) fetch(k0 + kGateKInner);
+#pragma unroll 4
+    for (int kk = 0; kk < kGateKInner; ++kk) {
+      double2 wv[4], xv[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) wv[j] = *reinterpret_cast<const double2*>(&Ws[kk][2 * tx + 32 * j]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) xv[i] = *reinterpret_cast<const double2*>(&Xs[kk][2 * ty + 16 * i]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          acc[j][i][0][0] = fma(wv[j].x, xv[i].x, acc[j][i][0][0]);
+          acc[j][i][0][1] = fma(wv[j].x, xv[i].y, acc[j][i][0][1]);
+          acc[j][i][1][0] = fma(wv[j].y, xv[i].x, acc[j][i][1][0]);
+          acc[j][i][1][1] = fma(wv[j].y, xv[i].y, acc[j][i][1][1]);
+        }
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+          const int g = g0 + 2 * tx + 32 * j + a, r = r0 + 2 * ty + 16 * i + b;
+          if (g < p.G && r < p.rows) p.part[(size_t(ks) * p.rows + r) * p.G + g] = acc[j][i][a][b];
+        }
 }
 
 struct RecurParams {
