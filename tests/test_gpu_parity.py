@@ -157,6 +157,8 @@ def test_rebuild_first_step_on_the_tensor_core_kernel_shapes():
     _run_rebuild_first(SMALL.scaled(name="rows_c517_r15", capacity=517, topk=200, rebuild_max=15, prompt=700, steps=8, batch=2,
                                     seed=132))
     _run_rebuild_first(SMALL.scaled(name="rows_topk_off", topk=1000, rebuild_max=7, capacity=70, prompt=90, steps=12, seed=133))
+    _run_rebuild_first(wl.get_config(4).scaled(name="rows_cfg4_shape", n_layers=1, batch=2, per_layer_inputs=False, steps=3))
+    _run_rebuild_first(wl.get_config(2).scaled(name="rows_cfg2_shape", batch=2, steps=4))
 
 
 def test_cumulative_attention_as_the_score_source():
