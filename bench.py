@@ -262,7 +262,7 @@ class DeviceRun:
                 if c.identity_projection:
                     self.q[s, l] = randn(B, H, dh).to(self.dt)
                 else:
-                    self.q[s, l] = self._rope((xl @ self.w_q[l].float().t()).reshape(B, H, dh), n).to(self.dt)
+                    self.q[s, l] = (c.q_scale * self._rope((xl @ self.w_q[l].float().t()).reshape(B, H, dh), n)).to(self.dt)
                 if c.per_layer_inputs:
                     self.tables[l][:, n] = self.x[s, l]
         self.r_in = 0

@@ -64,7 +64,7 @@ class Workload:
                           for b in range(B)])
         else:
             yq = x64 @ self.w_q64[layer].T
-            q = ao.round_store(ao.rope_rotate(yq.reshape(B, c.n_heads, c.head_dim), n, c.rope_theta), c.dtype)
+            q = ao.round_store(c.q_scale * ao.rope_rotate(yq.reshape(B, c.n_heads, c.head_dim), n, c.rope_theta), c.dtype)
         return q, k, v
 
     def q_rows(self, n: int, layer: int, x_table: np.ndarray, lists) -> np.ndarray:

@@ -168,3 +168,12 @@ def test_cumulative_attention_as_the_score_source():
     _run(SMALL.scaled(name="h2o_no_rebuild", score_from_attention=True, rebuild_max=0, steps=30, seed=129))
     _run(SMALL.scaled(name="h2o_two_layers_f32", score_from_attention=True, dtype="f32", n_layers=2, batch=2, n_heads=2,
                       hidden=128, capacity=33, topk=7, steps=25, seed=130))
+
+
+def test_peaked_logits_as_in_real_attention():
+    """Appendix C, Figure 8: real softmax rows are long-tailed. Queries scaled by 8 give logits of several tens, a few
+    slots holding nearly all the weight, and kept sets decided far out in the tail."""
+    _run(SMALL.scaled(name="peaked_q8", q_scale=8.0, steps=30, seed=134))
+    _run(SMALL.scaled(name="peaked_q8_c517", q_scale=8.0, capacity=517, topk=200, rebuild_max=37, prompt=700, steps=8, batch=2,
+                      seed=135))
+    _run_rebuild_first(SMALL.scaled(name="peaked_rows", q_scale=8.0, rebuild_max=7, capacity=70, prompt=90, steps=10, seed=136))
