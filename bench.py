@@ -358,9 +358,8 @@ class DeviceRun:
         pl = None if hp["lists"] is None else hp["lists"][i]
         pc = None if hp["counts"] is None else hp["counts"][i]
         for l in range(c.n_layers):
-            lib.adore_decode_step_host(self.handle, l, hp["q"][i][l], hp["k"][i][l], hp["v"][i][l], hp["x"][i], pl, pc, self.r_in,
-                                       hp["out"], self.pw)
-            lib.adore_rebuild(self.handle, l, self.pt[l] if (self.pt is not None and l > 0) else None)
+            lib.adore_decode_rebuild_host(self.handle, l, hp["q"][i][l], hp["k"][i][l], hp["v"][i][l], hp["x"][i], pl, pc,
+                                          self.r_in, self.pt[l] if (self.pt is not None and l > 0) else None, hp["out"], self.pw)
         self.next += 1
 
     def host_bytes_per_step(self):

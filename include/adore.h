@@ -16,7 +16,7 @@
  * Conventions
  *   - Every function returns an adore_status_t. Nothing throws, aborts or traps the device.
  *   - All device work is queued on the CUDA stream given at create time and is asynchronous;
- *     only adore_cache_sync_status, adore_decode_step_host (at its end), the state snapshot
+ *     only adore_cache_sync_status, the host-buffer step calls (for their output), the state snapshot
  *     calls and adore_cache_destroy wait for the device.
  *   - "device" pointers are CUDA device addresses of the cache's GPU; "host" pointers are
  *     ordinary (ideally pinned) host memory. The library borrows per-call buffers until the
@@ -165,6 +165,16 @@ adore_status_t adore_decode_step(adore_cache_t *cache, int32_t layer, const void
 adore_status_t adore_decode_step_host(adore_cache_t *cache, int32_t layer, const void *q, const void *k_new,
                                       const void *v_new, const void *x_new, const int32_t *explicit_list,
                                       const int32_t *explicit_count, int32_t r_in, void *out, float *weights);
+
+/* adore_decode_step_host followed by adore_rebuild(cache, layer, x_table) (Sections 2.1-2.3), with one difference in
+ * what the host waits for: the rebuild is queued before the wait, and the call returns as soon as `out` has reached
+ * the host, so the GPU runs from the attention straight into the rebuild while the caller consumes `out` and hands in
+ * the next inputs. x_table as for adore_rebuild (DEVICE or NULL); everything else as for adore_decode_step_host.
+ * Errors as for the two calls (STATE if the layer has no projection). */
+adore_status_t adore_decode_rebuild_host(adore_cache_t *cache, int32_t layer, const void *q, const void *k_new,
+                                         const void *v_new, const void *x_new, const int32_t *explicit_list,
+                                         const int32_t *explicit_count, int32_t r_in, const void *x_table, void *out,
+                                         float *weights);
 
 /* Rebuild for one layer (Section 2.3): Y = X_L [W_k ; W_v]^T for the rows of this step's rebuild
  * list, rotary embedding on the key half at each token's original position, rounding to T and

@@ -55,7 +55,7 @@ EXPORTS = ["adore_cache_create", "adore_cache_destroy", "adore_cache_set_project
            "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows",
            "adore_controller_score_static", "adore_probe_read_bandwidth",
            "adore_cache_export_state", "adore_cache_import_state", "adore_step_begin", "adore_attend_rows",
-           "adore_label_tokens"]
+           "adore_label_tokens", "adore_decode_rebuild_host"]
 
 
 def _lib():
@@ -75,6 +75,7 @@ def _lib():
         step = [vp, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp]
         lib.adore_decode_step.argtypes = step
         lib.adore_decode_step_host.argtypes = step
+        lib.adore_decode_rebuild_host.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         lib.adore_rebuild.argtypes = [vp, i32, vp]
         lib.adore_step_begin.argtypes = [vp, vp, vp, vp, i32]
         lib.adore_label_tokens.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
@@ -155,6 +156,13 @@ def adore_decode_step_host(cache: int, layer: int, q, k_new, v_new, x_new, expli
     _check(_lib().adore_decode_step_host(cache, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(x_new),
                                          _ptr(explicit_list), _ptr(explicit_count), r_in, _ptr(out), _ptr(weights)),
            "adore_decode_step_host")
+
+
+def adore_decode_rebuild_host(cache: int, layer: int, q, k_new, v_new, x_new, explicit_list, explicit_count, r_in: int,
+                              x_table, out, weights=None) -> None:
+    _check(_lib().adore_decode_rebuild_host(cache, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(x_new),
+                                            _ptr(explicit_list), _ptr(explicit_count), r_in, _ptr(x_table), _ptr(out),
+                                            _ptr(weights)), "adore_decode_rebuild_host")
 
 
 def adore_step_begin(cache: int, x_new, explicit_list, explicit_count, r_in: int) -> None:

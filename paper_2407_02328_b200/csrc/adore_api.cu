@@ -153,6 +153,7 @@ struct adore_cache {
   // uploads of the host-buffer entry point run on their own stream, beside the previous rebuild
   cudaStream_t copy = nullptr;
   cudaEvent_t ev_copy = nullptr;
+  cudaEvent_t ev_out = nullptr;     // `out` has reached the host (host-buffer entry point that also queues the rebuild)
   bool joined = true;
   std::vector<const void*> w_kv;
   TcState tc;                   // tensor-core rebuild path (tensor maps, gather buffer)
@@ -634,7 +635,8 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
       cudaEventCreateWithFlags(&c->ev_gates, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_ctrl, cudaEventDisableTiming) != cudaSuccess ||
       cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess ||
-      cudaEventCreateWithFlags(&c->ev_copy, cudaEventDisableTiming) != cudaSuccess) {
+      cudaEventCreateWithFlags(&c->ev_copy, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_out, cudaEventDisableTiming) != cudaSuccess) {
     adore_cache_destroy(c);
     return ADORE_ERR_CUDA;
   }
@@ -677,6 +679,7 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (c->ev_ctrl) cudaEventDestroy(c->ev_ctrl);
   if (c->copy) { cudaStreamSynchronize(c->copy); cudaStreamDestroy(c->copy); }
   if (c->ev_copy) cudaEventDestroy(c->ev_copy);
+  if (c->ev_out) cudaEventDestroy(c->ev_out);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   for (void* p : c->owned) cudaFree(p);
@@ -871,9 +874,12 @@ adore_status_t adore_attend_rows(adore_cache_t* c, int32_t layer, const void* q_
                               : launch_attention<__nv_bfloat16>(c, layer, q_rows, k_new, v_new, out, weights, true, rows_q);
 }
 
-adore_status_t adore_decode_step_host(adore_cache_t* c, int32_t layer, const void* q, const void* k_new,
-                                      const void* v_new, const void* x_new, const int32_t* explicit_list,
-                                      const int32_t* explicit_count, int32_t r_in, void* out, float* weights) {
+namespace {
+
+adore_status_t decode_step_host_impl(adore_cache_t* c, int32_t layer, const void* q, const void* k_new,
+                                     const void* v_new, const void* x_new, const int32_t* explicit_list,
+                                     const int32_t* explicit_count, int32_t r_in, void* out, float* weights,
+                                     bool then_rebuild, const void* x_table) {
   if (!c || !q || !k_new || !v_new || !out) return ADORE_ERR_INVALID_ARG;
   const adore_config_t& f = c->cfg;
   const size_t qb = size_t(f.batch) * f.n_heads * f.head_dim * c->esz, xb = size_t(f.batch) * f.hidden * c->esz;
@@ -904,8 +910,34 @@ adore_status_t adore_decode_step_host(adore_cache_t* c, int32_t layer, const voi
                                         lists ? c->h_count : nullptr, lists ? r_in : 0, c->h_out, weights);
   if (st != ADORE_OK) return st;
   CUDA_OK(cudaMemcpyAsync(out, c->h_out, qb, cudaMemcpyDeviceToHost, c->stream));
-  CUDA_OK(cudaStreamSynchronize(c->stream));
+  if (!then_rebuild) {
+    CUDA_OK(cudaStreamSynchronize(c->stream));
+    return ADORE_OK;
+  }
+  // The rebuild is queued BEFORE the host waits, and the host waits for the copy of `out` only: the GPU goes from the
+  // attention straight into the GEMM while the caller already works on `out` (and uploads the next step's inputs).
+  // Every kernel that reads the staging buffers has finished by the time `out` has arrived.
+  CUDA_OK(cudaEventRecord(c->ev_out, c->stream));
+  st = adore_rebuild(c, layer, x_table);
+  if (st != ADORE_OK) return st;
+  CUDA_OK(cudaEventSynchronize(c->ev_out));
   return ADORE_OK;
+}
+
+}  // namespace
+
+adore_status_t adore_decode_step_host(adore_cache_t* c, int32_t layer, const void* q, const void* k_new,
+                                      const void* v_new, const void* x_new, const int32_t* explicit_list,
+                                      const int32_t* explicit_count, int32_t r_in, void* out, float* weights) {
+  return decode_step_host_impl(c, layer, q, k_new, v_new, x_new, explicit_list, explicit_count, r_in, out, weights, false, nullptr);
+}
+
+adore_status_t adore_decode_rebuild_host(adore_cache_t* c, int32_t layer, const void* q, const void* k_new,
+                                         const void* v_new, const void* x_new, const int32_t* explicit_list,
+                                         const int32_t* explicit_count, int32_t r_in, const void* x_table, void* out,
+                                         float* weights) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || !c->w_kv[layer]) return c ? ADORE_ERR_STATE : ADORE_ERR_INVALID_ARG;
+  return decode_step_host_impl(c, layer, q, k_new, v_new, x_new, explicit_list, explicit_count, r_in, out, weights, true, x_table);
 }
 
 adore_status_t adore_rebuild(adore_cache_t* c, int32_t layer, const void* x_table) {

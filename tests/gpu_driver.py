@@ -247,8 +247,13 @@ def run_parity(cfg: wl.WorkloadConfig, batch: Optional[int] = None, steps: Optio
                     ho = np.zeros((g.B, cfg.n_heads, cfg.head_dim), np.float32)
                     hq, hk, hv, hx = (to_dev(a, cfg).cpu() for a in (q, k, v, x))
                     hout = torch.zeros((g.B, cfg.n_heads, cfg.head_dim), dtype=torch_dtype(cfg))
-                    lib.adore_decode_step_host(g.handle, l, hq, hk, hv, hx, lists if l == 0 else None,
-                                               counts if l == 0 else None, w.r_in if l == 0 else 0, hout, g.weights)
+                    if host_entry == "with_rebuild":     # the call that also queues the layer's rebuild
+                        lib.adore_decode_rebuild_host(g.handle, l, hq, hk, hv, hx, lists if l == 0 else None,
+                                                      counts if l == 0 else None, w.r_in if l == 0 else 0,
+                                                      tables[l] if (cfg.per_layer_inputs and l > 0) else None, hout, g.weights)
+                    else:
+                        lib.adore_decode_step_host(g.handle, l, hq, hk, hv, hx, lists if l == 0 else None,
+                                                   counts if l == 0 else None, w.r_in if l == 0 else 0, hout, g.weights)
                     out_g, w_g = hout.float().numpy(), g.weights.cpu().numpy()
                 else:
                     lib.adore_decode_step(g.handle, l, to_dev(q, cfg), to_dev(k, cfg), to_dev(v, cfg), to_dev(x, cfg),
@@ -258,7 +263,8 @@ def run_parity(cfg: wl.WorkloadConfig, batch: Optional[int] = None, steps: Optio
                 compare_attention(rep, cfg, q, orc, l, k, attn_map, out_g, w_g, out_o, w_o, K_before,
                                   gpu_k=lambda l=l: g.kv(l)[0], admit_slot=orc.info.admit_slot)
                 orc.rebuild(l, otab[l] if (cfg.per_layer_inputs and l > 0) else None)
-                lib.adore_rebuild(g.handle, l, tables[l] if (cfg.per_layer_inputs and l > 0) else None)
+                if host_entry != "with_rebuild":
+                    lib.adore_rebuild(g.handle, l, tables[l] if (cfg.per_layer_inputs and l > 0) else None)
             rep.steps += 1
             if cfg.score_from_attention:
                 # The values that rank the tokens are float32 sums of attention weights, which the two sides compute to

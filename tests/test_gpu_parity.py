@@ -62,6 +62,9 @@ def test_three_layers_with_their_own_inputs():
 def test_host_buffer_entry_point():
     _run(SMALL.scaled(name="host_entry", steps=12, seed=110), host_entry=True)
     _run(wl.get_config(1).scaled(steps=40), host_entry=True)
+    _run(SMALL.scaled(name="host_entry_rebuild", steps=12, seed=137), host_entry="with_rebuild")
+    _run(SMALL.scaled(name="host_entry_rebuild_L3", n_layers=3, batch=2, per_layer_inputs=True, seed=138, steps=10),
+         host_entry="with_rebuild")
 
 
 def test_capacity_spanning_several_tiles_with_ragged_tail():
