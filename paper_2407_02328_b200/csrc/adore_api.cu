@@ -1127,7 +1127,17 @@ adore_status_t adore_label_tokens(const float* weights, int32_t n_layers, int32_
   const int half = topk / 2;
   const size_t smem = size_t(label_pow2(n_slots)) * sizeof(unsigned long long);
   CUDA_OK(cudaMemsetAsync(count, 0, size_t(batch) * n_slots * sizeof(int), st));
-  label_sets_kernel<<<n_layers * batch * n_heads, kLabelThreads, smem, st>>>(weights, batch, n_heads, n_slots, half, sets, count);
+  const int n_rows = n_layers * batch * n_heads;
+  static const bool full_sort = std::getenv("ADORE_LABELS_FULL_SORT") != nullptr;   // A/B switch
+  if (!full_sort && half <= kLabelWarpMaxHalf && n_slots <= 32 * kLabelWarpKeysPerLane) {
+    int P = 32;
+    while (P < half) P <<= 1;
+    label_sets_warp_kernel<<<(n_rows + kLabelRowsPerCta - 1) / kLabelRowsPerCta, kLabelThreads,
+                             size_t(kLabelRowsPerCta) * P * sizeof(unsigned long long), st>>>(weights, n_rows, batch, n_heads,
+                                                                                              n_slots, half, sets, count);
+  } else {
+    label_sets_kernel<<<n_rows, kLabelThreads, smem, st>>>(weights, batch, n_heads, n_slots, half, sets, count);
+  }
   CUDA_OK(cudaGetLastError());
   label_pick_kernel<<<batch, kLabelThreads, smem, st>>>(count, n_slots, topk, label);
   CUDA_OK(cudaGetLastError());

@@ -56,6 +56,79 @@ __global__ void __launch_bounds__(kLabelThreads) label_sets_kernel(const float* 
   }
 }
 
+// Same result with one warp per row and no full sort, for K/2 <= 512 and S <= 1056: the row's keys stay in registers,
+// the (K/2)-th largest key is found by bisection on the key's bits (a count is a compare, a ballot and a popc; the
+// 64-bit keys are all different, so the search ends with exactly K/2 keys at or above the threshold), the kept keys
+// are compacted in slot order into shared memory and only those are sorted. grid = ceil(L*B*H / 8), 8 rows per CTA.
+constexpr int kLabelRowsPerCta = kLabelThreads / 32;
+constexpr int kLabelWarpMaxHalf = 512;
+constexpr int kLabelWarpKeysPerLane = 33;
+
+__global__ void __launch_bounds__(kLabelThreads) label_sets_warp_kernel(const float* weights, int n_rows, int B, int H, int S,
+                                                                        int half, int* sets, int* count) {
+  extern __shared__ __align__(16) unsigned long long lab_keys[];        // [8 warps][pow2 >= half]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lbh = blockIdx.x * kLabelRowsPerCta + warp;
+  if (lbh >= n_rows) return;                                             // whole warps leave; no block barrier below
+  const int b = (lbh / H) % B;
+  const float* row = weights + size_t(lbh) * S;
+  int P = 32;
+  while (P < half) P <<= 1;
+  unsigned long long* mine = lab_keys + size_t(warp) * P;
+  unsigned long long kk[kLabelWarpKeysPerLane];
+  int positive = 0;
+#pragma unroll
+  for (int j = 0; j < kLabelWarpKeysPerLane; ++j) {
+    const int i = j * 32 + lane;
+    const float w = i < S ? row[i] : 0.f;
+    kk[j] = w > 0.f ? ((static_cast<unsigned long long>(__float_as_uint(w)) << 32) | (0xFFFFFFFFu - unsigned(i))) : 0ull;
+    positive += __popc(__ballot_sync(0xffffffffu, kk[j] != 0ull));
+  }
+  unsigned long long thr = 1ull;                                         // fewer than K/2 positive weights: keep them all
+  if (positive > half) {
+    thr = 0ull;
+    for (int bit = 63; bit >= 0; --bit) {
+      const unsigned long long cand = thr | (1ull << bit);
+      int c = 0;
+#pragma unroll
+      for (int j = 0; j < kLabelWarpKeysPerLane; ++j) c += __popc(__ballot_sync(0xffffffffu, kk[j] >= cand));
+      if (c >= half) thr = cand;
+      if (c == half) break;
+    }
+  }
+  // compaction of the kept keys, then a bitonic sort of P keys by this warp alone
+  int n_kept = 0;
+#pragma unroll
+  for (int j = 0; j < kLabelWarpKeysPerLane; ++j) {
+    const bool keep = kk[j] >= thr;                                      // thr >= 1: zero keys never pass
+    const unsigned m = __ballot_sync(0xffffffffu, keep);
+    if (keep) mine[n_kept + __popc(m & ((1u << lane) - 1u))] = kk[j];
+    n_kept += __popc(m);
+  }
+  for (int i = n_kept + lane; i < P; i += 32) mine[i] = 0ull;
+  __syncwarp();
+  for (int k = 2; k <= P; k <<= 1)
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int t = lane; t < (P >> 1); t += 32) {
+        const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+        const int l = i | j;
+        const unsigned long long a = mine[i], c = mine[l];
+        const bool desc = (i & k) == 0;
+        if (desc ? (a < c) : (a > c)) { mine[i] = c; mine[l] = a; }
+      }
+      __syncwarp();
+    }
+  for (int j = lane; j < half; j += 32) {
+    const unsigned long long k = j < P ? mine[j] : 0ull;
+    int slot = -1;
+    if (k != 0ull) {
+      slot = int(0xFFFFFFFFu - unsigned(k & 0xFFFFFFFFull));
+      atomicAdd(&count[size_t(b) * S + slot], 1);
+    }
+    sets[size_t(lbh) * half + j] = slot;
+  }
+}
+
 // grid = B
 __global__ void __launch_bounds__(kLabelThreads) label_pick_kernel(const int* count, int S, int topk, unsigned char* label) {
   extern __shared__ __align__(16) unsigned long long lab_keys[];
