@@ -81,7 +81,6 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(rows_smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* ring = base;
   uint64_t* full = reinterpret_cast<uint64_t*>(base + size_t(kRowsStages) * TILE_BYTES);
-  uint64_t* empty = full + 4;                           // per stage: all 8 warps have read the tile (kRowsStages <= 4)
   int* s_qtok = reinterpret_cast<int*>(full + 8);       // [16] position bound per row (< 0: padding)
   int* s_tok = s_qtok + 16;                             // [C] the pair's slot map row (token position per slot)
   float* S = reinterpret_cast<float*>(s_tok + ((p.C + 3) & ~3));
@@ -93,7 +92,7 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   const int* map = p.slot_tok + size_t(b) * C;
 
   if (tid == 0) {
-    for (int s = 0; s < kRowsStages; ++s) { mbar_init(&full[s], 1u); mbar_init(&empty[s], uint32_t(kRowsWarps)); }
+    for (int s = 0; s < kRowsStages; ++s) mbar_init(&full[s], 1u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -116,22 +115,6 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   const int n_loads = 2 * n_tiles;
   if (tid == 0)
     for (int i = 0; i < min(kRowsStages, n_loads); ++i) issue(i);
-  // No block barrier per tile: a warp that is done with load j arrives on the stage's `empty` barrier and goes on; the
-  // warp whose turn it is (they rotate) waits until all eight have arrived and refills the stage with load j + stages.
-  bool failed = false;
-  auto done_with = [&](int j) {
-    const int stage = j % kRowsStages;
-    __syncwarp();
-    if (lane == 0) {
-      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&empty[stage])) : "memory");
-      const int next = j + kRowsStages;
-      if (next < n_loads && warp == (j % kRowsWarps)) {
-        const uint32_t par = uint32_t(j / kRowsStages) & 1u;
-        if (mbar_wait_bounded(&empty[stage], par, kWaitPolls)) issue(next);
-        else set_error(p.err, ERRW_TIMEOUT);            // the consumers of `next` time out on their own wait
-      }
-    }
-  };
 
   // ---- query block as A fragments: rows lane/4 and lane/4 + 8, columns 16 ks + (lane % 4) * 2 (+8) ----
   uint32_t qa[KSTEPS][4];
@@ -157,6 +140,7 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     for (int r = lane; r < R1; r += 32) S[size_t(r) * SP + C] = (r == R1 - 1) ? dot * p.scale : -INFINITY;
   }
 
+  bool failed = false;
   // ---- phase 1: logits ----
   for (int t = 0; t < n_tiles; ++t) {
     const int stage = t % kRowsStages;
@@ -188,9 +172,9 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
         S[size_t(r) * SP + key] = ok ? acc[e] * p.scale : -INFINITY;
       }
     }
-    done_with(t);
+    __syncthreads();                                    // everyone is done with this stage
+    if (tid == 0 && !failed && t + kRowsStages < n_loads) issue(t + kRowsStages);
   }
-  __syncthreads();                                      // all logits are in shared memory
 
   // ---- phase 2: per row, which logits are kept, softmax, weights (one warp per row) ----
   const int rows_n = C + 1;
@@ -329,9 +313,9 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
         rows_mma(o[nt + 1], al, bf[2], bf[3]);
       }
     }
-    done_with(li);
+    __syncthreads();
+    if (tid == 0 && !failed && li + kRowsStages < n_loads) issue(li + kRowsStages);
   }
-  __syncthreads();                                      // every warp is done with the ring: it becomes the partial-output buffer
 
   // ---- the four k-step warps of a column half add up through shared memory (the ring is free now), then rows < R1
   // go out; the last row also gets the current token's own value row ----
