@@ -88,7 +88,9 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int bh = blockIdx.x, b = bh / p.H;
   const int C = p.C, R1 = p.rows_q, SP = rows_logit_stride(C);
-  const int n_tiles = (C + kRowsTile - 1) / kRowsTile;
+  // tiles are consumed two at a time (one block barrier and one round of refills per 128 rows): an even count, the
+  // tile past the end, if any, holds rows of the next pair or zeros and is masked like every row >= C
+  const int n_tiles = (((C + kRowsTile - 1) / kRowsTile) + 1) & ~1;
   const int* map = p.slot_tok + size_t(b) * C;
 
   if (tid == 0) {
@@ -98,7 +100,10 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   }
   wait_for_prior_grid();
   if (tid < kRowsMaxQ) s_qtok[tid] = tid < R1 - 1 ? p.row_tok[size_t(b) * p.r_max + tid] : (tid == R1 - 1 ? p.n_cur : -1);
-  for (int i = tid; i < C; i += kRowsThreads) s_tok[i] = map[i];
+  for (int i = tid; i < C; i += kRowsThreads) {         // the slot reserved for the current token is not written yet
+    const int tok = map[i];
+    s_tok[i] = tok == p.n_cur ? -1 : tok;
+  }
   __syncthreads();
 
   // loads are numbered 0 .. 2 n_tiles - 1 (keys first, then values); load i uses stage i % kRowsStages
@@ -141,39 +146,50 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   }
 
   bool failed = false;
-  // ---- phase 1: logits ----
-  for (int t = 0; t < n_tiles; ++t) {
+  // ---- phase 1: logits, two tiles (two independent accumulator chains per warp) per block barrier ----
+  const int qt0 = s_qtok[lane >> 2], qt1 = s_qtok[(lane >> 2) + 8];
+  for (int t = 0; t < n_tiles; t += 2) {
     const int stage = t % kRowsStages;
     const uint32_t parity = uint32_t(t / kRowsStages) & 1u;
-    if (!mbar_wait_bounded(&full[stage], parity, failed ? kDrainPolls : kWaitPolls)) {
-      if (!failed) set_error(p.err, ERRW_TIMEOUT);
-      failed = true;
-    }
+#pragma unroll
+    for (int h2 = 0; h2 < 2; ++h2)
+      if (!mbar_wait_bounded(&full[stage + h2], parity, failed ? kDrainPolls : kWaitPolls)) {
+        if (!failed) set_error(p.err, ERRW_TIMEOUT);
+        failed = true;
+      }
     const uint32_t tile = smem_u32(ring + size_t(stage) * TILE_BYTES);
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     // ldmatrix.x4: matrix j holds keys warp*8 .. +7 (rows) x 8 columns starting at 8 * (4 q + j)
     const int krow = warp * 8 + (lane & 7), mj = lane >> 3;
 #pragma unroll
     for (int q4 = 0; q4 < DH / 32; ++q4) {
       const int c16 = q4 * 4 + mj;                      // 16-byte chunk along dh (0 .. DH/8 - 1)
-      uint32_t bf[4];
-      rows_ldmatrix_x4(tile + uint32_t(c16 >> 3) * (kRowsTile * 128) + rows_swz(krow, c16 & 7), bf);
-      rows_mma(acc, qa[2 * q4], bf[0], bf[1]);
-      rows_mma(acc, qa[2 * q4 + 1], bf[2], bf[3]);
-    }
-    // accumulator: rows lane/4 (+8), keys (lane % 4) * 2 (+1) of this warp's 8
-    const int key0 = t * kRowsTile + warp * 8 + (lane & 3) * 2;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int r = (lane >> 2) + (e >> 1) * 8, key = key0 + (e & 1);
-      if (r < R1 && key < C) {
-        const int tok = s_tok[key], qt = s_qtok[r];
-        const bool ok = tok >= 0 && tok <= qt && tok != p.n_cur;
-        S[size_t(r) * SP + key] = ok ? acc[e] * p.scale : -INFINITY;
+      for (int h2 = 0; h2 < 2; ++h2) {
+        uint32_t bf[4];
+        rows_ldmatrix_x4(tile + uint32_t(h2) * TILE_BYTES + uint32_t(c16 >> 3) * (kRowsTile * 128) + rows_swz(krow, c16 & 7), bf);
+        rows_mma(acc[h2], qa[2 * q4], bf[0], bf[1]);
+        rows_mma(acc[h2], qa[2 * q4 + 1], bf[2], bf[3]);
       }
     }
-    __syncthreads();                                    // everyone is done with this stage
-    if (tid == 0 && !failed && t + kRowsStages < n_loads) issue(t + kRowsStages);
+    // accumulator: rows lane/4 (+8), keys (lane % 4) * 2 (+1) of this warp's 8 in each tile
+#pragma unroll
+    for (int h2 = 0; h2 < 2; ++h2) {
+      const int key0 = (t + h2) * kRowsTile + warp * 8 + (lane & 3) * 2;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int r = (lane >> 2) + (e >> 1) * 8, key = key0 + (e & 1);
+        if (r < R1 && key < C) {
+          const int tok = s_tok[key], qt = (e >> 1) ? qt1 : qt0;
+          S[size_t(r) * SP + key] = (tok >= 0 && tok <= qt) ? acc[h2][e] * p.scale : -INFINITY;
+        }
+      }
+    }
+    __syncthreads();                                    // everyone is done with these two stages
+    if (tid == 0 && !failed) {
+      if (t + kRowsStages < n_loads) issue(t + kRowsStages);
+      if (t + kRowsStages + 1 < n_loads) issue(t + kRowsStages + 1);
+    }
   }
 
   // ---- phase 2: per row, which logits are kept, softmax, weights (one warp per row) ----
@@ -277,18 +293,21 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   float o[NTW][4];
 #pragma unroll
   for (int j = 0; j < NTW; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
-  for (int t = 0; t < n_tiles; ++t) {
+  for (int t = 0; t < n_tiles; t += 2) {
     const int li = n_tiles + t;
     const int stage = li % kRowsStages;
     const uint32_t parity = uint32_t(li / kRowsStages) & 1u;
-    if (!mbar_wait_bounded(&full[stage], parity, failed ? kDrainPolls : kWaitPolls)) {
-      if (!failed) set_error(p.err, ERRW_TIMEOUT);
-      failed = true;
-    }
-    const uint32_t tile = smem_u32(ring + size_t(stage) * TILE_BYTES);
-    {
+#pragma unroll
+    for (int h2 = 0; h2 < 2; ++h2)
+      if (!mbar_wait_bounded(&full[stage + h2], parity, failed ? kDrainPolls : kWaitPolls)) {
+        if (!failed) set_error(p.err, ERRW_TIMEOUT);
+        failed = true;
+      }
+#pragma unroll
+    for (int h2 = 0; h2 < 2; ++h2) {
+      const uint32_t tile = smem_u32(ring + size_t(stage + h2) * TILE_BYTES);
       // A: weights of rows lane/4 (+8) for keys 16 my_ks + (lane % 4) * 2 (+1, +8, +9) of this tile, head + remainder
-      const int key = t * kRowsTile + my_ks * 16 + (lane & 3) * 2;
+      const int key = (t + h2) * kRowsTile + my_ks * 16 + (lane & 3) * 2;
       const int r0 = lane >> 2, r1 = r0 + 8;
       uint32_t ah[4], al[4];
 #pragma unroll
@@ -314,7 +333,10 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
       }
     }
     __syncthreads();
-    if (tid == 0 && !failed && li + kRowsStages < n_loads) issue(li + kRowsStages);
+    if (tid == 0 && !failed) {
+      if (li + kRowsStages < n_loads) issue(li + kRowsStages);
+      if (li + kRowsStages + 1 < n_loads) issue(li + kRowsStages + 1);
+    }
   }
 
   // ---- the four k-step warps of a column half add up through shared memory (the ring is free now), then rows < R1
