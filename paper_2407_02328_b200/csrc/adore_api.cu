@@ -462,19 +462,15 @@ namespace {
 // Launches the controller of token n (gates, then GRU + MLP + score) on the controller stream and the step's
 // selection and row table on `sel`. Both streams must already wait for everything they depend on in the main stream.
 adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new, const int32_t* explicit_list,
-                                             const int32_t* explicit_count, int32_t r_in, cudaStream_t sel) {
+                                             const int32_t* explicit_count, int32_t r_in, cudaStream_t sel,
+                                             bool early_gather) {
   const adore_config_t& f = c->cfg;
   const bool ex = f.rebuild_mode == ADORE_REBUILD_EXPLICIT;
   adore_status_t st;
   StageScope scope(c, 1);
   const bool controller = !(f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION);   // else the scores come from the attention
   if (c->ctrl_pending) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_ctrl, 0));   // scores of token n-1
-  if (controller) {
-    if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit, c->ctl);
-    else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit, c->ctl);
-    if (st != ADORE_OK) return st;
-  }
-  CUDA_OK(cudaEventRecord(c->ev_gates, c->ctl));
+  // The selection chain is what the step waits for, so it is queued first; the controller's launches follow.
   const int P = ex ? pow2_at_least(r_in) : pow2_at_least(c->n);
   SelectParams sp = select_params(c, c->n, P, c->cur, 1 - c->cur);
   sp.explicit_list = ex && r_in > 0 ? explicit_list : nullptr;
@@ -491,6 +487,30 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
   CUDA_OK(cudaGetLastError());
   st = launch_row_table(c, true, sel);
   if (st != ADORE_OK) return st;
+  // A short list's rows are copied out of the token store into the GEMM's compact input right away, beside the
+  // attention, so that the rebuild that follows starts with its GEMM. Long lists are copied after the attention:
+  // side by side the two slow each other down by more than the copy takes (measured at 15k rows: attention
+  // 104 -> 193 us beside a copy that takes 35 us alone). (Not with per-stage timing on: there the copy stays
+  // with the rebuild stage.)
+  c->rows_gathered = false;
+  {
+    const int m_max = f.batch * f.rebuild_max;
+    if (early_gather && !c->timing && f.dtype == ADORE_BF16 && tc_usable<__nv_bfloat16>(c->tc) && m_max > 0 && m_max <= 2048 &&
+        size_t(m_max) <= c->tc.a_rows) {
+      RebuildParams<__nv_bfloat16> gp{};
+      gp.x_table = static_cast<const __nv_bfloat16*>(c->x_store); gp.seq_stride = f.max_tokens; gp.d = f.hidden;
+      gp.row_b = c->row_b; gp.row_tok = c->row_tok; gp.row_total = c->row_total;
+      CUDA_OK(launch_gather_tc<__nv_bfloat16>(c->tc, gp, m_max, sel));
+      ++c->launches;
+      c->rows_gathered = true;
+    }
+  }
+  if (controller) {
+    if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit, c->ctl);
+    else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit, c->ctl);
+    if (st != ADORE_OK) return st;
+  }
+  CUDA_OK(cudaEventRecord(c->ev_gates, c->ctl));
   if (!controller) return ADORE_OK;
   RecurParams rp = recur_params(c, f.batch, 1, c->ksplit, c->n);
   ctrl_recur_kernel<<<f.batch, select_threads(c), ctrl_smem(c), c->ctl>>>(rp, ctrl_resident_ok(f.ctrl_hidden) ? 1 : 0, c->err);
@@ -782,26 +802,8 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     if (c->timing) CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
     if (sel != c->stream) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_fork, 0));
     CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
-    st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel);
+    st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel, true);
     if (st != ADORE_OK) return st;
-    // A short list's rows are copied out of the token store into the GEMM's compact input right away, beside the
-    // attention, so that the rebuild that follows starts with its GEMM. Long lists are copied after the attention:
-    // side by side the two slow each other down by more than the copy takes (measured at 15k rows: attention
-    // 104 -> 193 us beside a copy that takes 35 us alone). (Not with per-stage timing on: there the copy stays
-    // with the rebuild stage.)
-    c->rows_gathered = false;
-    {
-      const int m_max = f.batch * f.rebuild_max;
-      if (!c->timing && f.dtype == ADORE_BF16 && tc_usable<__nv_bfloat16>(c->tc) && m_max > 0 && m_max <= 2048 &&
-          size_t(m_max) <= c->tc.a_rows) {
-        RebuildParams<__nv_bfloat16> gp{};
-        gp.x_table = static_cast<const __nv_bfloat16*>(c->x_store); gp.seq_stride = f.max_tokens; gp.d = f.hidden;
-        gp.row_b = c->row_b; gp.row_tok = c->row_tok; gp.row_total = c->row_total;
-        CUDA_OK(launch_gather_tc<__nv_bfloat16>(c->tc, gp, m_max, sel));
-        ++c->launches;
-        c->rows_gathered = true;
-      }
-    }
     c->joined = sel == c->stream;
     if (!c->joined) CUDA_OK(cudaEventRecord(c->ev_join, sel));
     c->cur = 1 - c->cur;
@@ -848,9 +850,8 @@ adore_status_t adore_step_begin(adore_cache_t* c, const void* x_new, const int32
   CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
   if (sel != c->stream) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_fork, 0));
   CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
-  adore_status_t st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel);
+  adore_status_t st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel, false);
   if (st != ADORE_OK) return st;
-  c->rows_gathered = false;
   if (sel != c->stream) {
     CUDA_OK(cudaEventRecord(c->ev_join, sel));
     CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
