@@ -27,7 +27,8 @@ standard three-gate GRU with the reset gate applied to the hidden-side candidate
 position feature u = i / pos_scale; the mask keeps the K largest logits with the lower
 index winning ties; sqrt of the head dimension; newer token wins score ties; rebuilt
 states live for one step; rotary embedding at the token's original position on adjacent
-pairs (2j, 2j+1).
+pairs (2j, 2j+1). A second reading of the position feature, u = (n - i) / pos_scale with every token
+scored anew at every step (controller_rescore), is kept beside the first as an option.
 """
 from __future__ import annotations
 
@@ -143,6 +144,23 @@ def controller_score(z: np.ndarray, position: float, pos_scale: float,
     p = np.asarray(w["pos_w"], np.float64) * u + np.asarray(w["pos_b"], np.float64)
     t = np.tanh((p + z) @ np.asarray(w["mlp_w1"], np.float64).T + np.asarray(w["mlp_b1"], np.float64))
     return t @ np.asarray(w["mlp_w2"], np.float64) + float(np.asarray(w["mlp_b2"]).reshape(-1)[0])
+
+
+def controller_rescore(z_rows: np.ndarray, n: int, pos_scale: float, w: Dict[str, np.ndarray]) -> np.ndarray:
+    """Scores of tokens 0..n as seen from the current token n. Section 1 and the caption of Figure 2 describe the
+    controller's importance as one taken with respect to the token being decoded, over all earlier tokens, cached
+    or released. Read that way, sigma_i = Sigmoid(MLP(p + z_i)) of Eq. 2 takes its position feature RELATIVE to
+    the current token, u = (n - i) / pos_scale: a token's score moves as the sequence grows, while its GRU state
+    z_i stays what it was when the token arrived.
+
+    z_rows: [..., n+1, d'] states of tokens 0..n. Returns the pre-sigmoid scores [..., n+1] (float64).
+    """
+    z_rows = np.asarray(z_rows, np.float64)
+    assert z_rows.shape[-2] == n + 1
+    out = np.zeros(z_rows.shape[:-1], np.float64)
+    for i in range(n + 1):
+        out[..., i] = controller_score(z_rows[..., i, :], n - i, pos_scale, w)
+    return out
 
 
 def controller_param_count(d: int, h: int) -> int:
@@ -268,6 +286,7 @@ class OracleConfig:
     pos_scale: float = 4096.0
     no_recurrence: bool = False    # Section 3.5.3 "w/o GRU": z_i = GRU(x_i, 0), no memory of earlier tokens
     score_from_attention: bool = False   # Section 3.1 baselines 6 and 7: a token's value is its cumulative attention
+    relative_position: bool = False      # every token is re-scored at every step with its distance to the current token
 
     @property
     def retained_max(self) -> int:
@@ -299,6 +318,9 @@ class AdoreOracle:
         self.n = 0                                             # tokens seen per sequence
         self.x = np.zeros((B, T, cfg.hidden), np.float32)
         self.z = np.zeros((B, cfg.ctrl_hidden), np.float64)    # z_{-1} = 0
+        if cfg.relative_position and cfg.score_from_attention:
+            raise ValueError("relative positions belong to the controller's score")
+        self.z_rows = np.zeros((B, T, cfg.ctrl_hidden), np.float64) if cfg.relative_position else None
         self.score = np.zeros((B, T), np.float32)
         self.sigma = np.zeros((B, T), np.float32)
         self.tok_slot = np.full((B, T), -1, np.int32)
@@ -317,8 +339,9 @@ class AdoreOracle:
         self.w_kv[layer] = np.asarray(w_kv, np.float64)
 
     # -- controller --------------------------------------------------------------------
-    def _score_new_token(self, x_new: np.ndarray) -> None:
-        """z_n, score_n, sigma_n for the token at position self.n of every sequence."""
+    def _score_new_token(self, x_new: np.ndarray, rescore: bool = True) -> None:
+        """z_n, score_n, sigma_n for the token at position self.n of every sequence. With relative positions
+        the states of all tokens are kept and (unless `rescore` is off) tokens 0..n are all scored anew."""
         c, n = self.cfg, self.n
         self.x[:, n, :] = x_new
         if c.score_from_attention:          # no controller: the token starts at zero and earns weight when attended
@@ -327,6 +350,13 @@ class AdoreOracle:
             return
         z_prev = np.zeros_like(self.z) if c.no_recurrence else self.z
         self.z = gru_step(x_new, z_prev, self.ctrl)
+        if c.relative_position:
+            self.z_rows[:, n, :] = self.z
+            if rescore:
+                s = controller_rescore(self.z_rows[:, : n + 1, :], n, c.pos_scale, self.ctrl)
+                self.score[:, : n + 1] = s.astype(np.float32)
+                self.sigma[:, : n + 1] = _sigm(s).astype(np.float32)
+            return
         s = controller_score(self.z, n, c.pos_scale, self.ctrl)
         self.score[:, n] = s.astype(np.float32)
         self.sigma[:, n] = _sigm(s).astype(np.float32)
@@ -414,12 +444,16 @@ class AdoreOracle:
         set that token-by-token release would reach, because a token's score does not
         change after it arrives. The rebuild list follows as in a decode step (empty in
         explicit mode). Every layer with a projection is filled from these rows.
+
+        With relative positions the prompt is given at once, so its tokens are scored
+        once, as seen from the last prompt token, and the same selection is made on those
+        scores (token-by-token release would differ here: scores move with the position).
         """
         c = self.cfg
         assert self.n == 0, "bulk load needs an empty cache"
         B, T, _ = x.shape
         for t in range(T):
-            self._score_new_token(x[:, t, :])
+            self._score_new_token(x[:, t, :], rescore=(t == T - 1))
             self.n += 1
         last = T - 1
         lists, slots = [], []

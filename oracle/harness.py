@@ -22,7 +22,8 @@ def oracle_config(cfg: wl.WorkloadConfig, batch: Optional[int] = None) -> ao.Ora
                            max_tokens=cfg.max_tokens, ctrl_hidden=cfg.ctrl_hidden, dtype=cfg.dtype,
                            rebuild_mode=cfg.rebuild_mode, rope_theta=cfg.rope_theta,
                            pos_scale=cfg.pos_scale, no_recurrence=cfg.ctrl_no_recurrence,
-                           score_from_attention=cfg.score_from_attention)
+                           score_from_attention=cfg.score_from_attention,
+                           relative_position=cfg.ctrl_relative_position)
 
 
 class Workload:

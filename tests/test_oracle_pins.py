@@ -547,6 +547,129 @@ def test_cumulative_attention_scores_equal_column_sums_of_the_causal_attention_m
                 assert ev == min(ret, key=lambda t: (float(before_score[b, t]), t))
 
 
+# ------------------------------------------------------ relative positions (re-scoring every step)
+def test_relative_rescoring_equals_torch_modules_on_the_distance_to_the_current_token():
+    """Scores as seen from token n: the Appendix B modules fed with (n - i) / pos_scale and the state of token i."""
+    d, h, n = 10, 6, 9
+    w = _ctrl(d, h)
+    pos, fc1, fc2 = torch.nn.Linear(1, h).double(), torch.nn.Linear(h, h).double(), torch.nn.Linear(h, 1).double()
+    z = np.random.default_rng(21).standard_normal((3, n + 1, h))
+    with torch.no_grad():
+        pos.weight.copy_(torch.tensor(w["pos_w"], dtype=torch.float64)[:, None])
+        pos.bias.copy_(torch.tensor(w["pos_b"], dtype=torch.float64))
+        fc1.weight.copy_(torch.tensor(w["mlp_w1"], dtype=torch.float64))
+        fc1.bias.copy_(torch.tensor(w["mlp_b1"], dtype=torch.float64))
+        fc2.weight.copy_(torch.tensor(w["mlp_w2"], dtype=torch.float64)[None, :])
+        fc2.bias.copy_(torch.tensor(w["mlp_b2"], dtype=torch.float64))
+        dist = torch.tensor([[float(n - i)] for i in range(n + 1)], dtype=torch.float64) / 64.0     # [n+1, 1]
+        ref = fc2(torch.tanh(fc1(pos(dist)[None] + torch.tensor(z))))[..., 0]
+    got = ao.controller_rescore(z, n, 64.0, w)
+    assert got.shape == (3, n + 1) and np.allclose(got, ref.numpy(), atol=1e-14)
+    assert not np.allclose(got[:, :-1], got[:, 1:], atol=1e-6)          # the position feature does move the scores
+
+
+REL = wl.WorkloadConfig(name="rel", dtype="f32", n_layers=1, batch=2, n_heads=2, head_dim=8, hidden=16, capacity=8,
+                        topk=4, rebuild_max=2, prompt=0, steps=24, rope_theta=1.0e4, rebuild_mode="policy",
+                        rebuild_p=0.0, seed=31, ctrl_hidden=8, pos_scale=16.0, ctrl_relative_position=True)
+
+
+def test_relative_scores_shift_with_the_sequence_and_meet_the_absolute_score_at_the_same_distance():
+    """Without the GRU's memory and with one and the same embedding for every token all states are equal, so the
+    score as seen from token n depends on the distance n - i alone: the scores of step n + 1 are those of step n
+    moved by one position, and a token at distance k scores what a token at ABSOLUTE position k scores under the
+    absolute reading (which is pinned above)."""
+    cfg = REL.scaled(ctrl_no_recurrence=True)
+    w = Workload(cfg)
+    x = np.tile(w.x_new(0)[:1, None, :], (cfg.batch, 1, 1))[:, 0]       # the same row for every sequence and token
+    rel, ab = make_oracle(w), make_oracle(Workload(cfg.scaled(ctrl_relative_position=False)))
+    prev = None
+    for n in range(12):
+        rel._score_new_token(x)
+        ab._score_new_token(x)
+        rel.n += 1
+        ab.n += 1
+        cur = rel.score[:, : n + 1].copy()
+        assert np.array_equal(cur[:, ::-1], ab.score[:, : n + 1])      # distance k  <->  absolute position k
+        if prev is not None:
+            assert np.array_equal(cur[:, 1:], prev)
+        prev = cur
+    assert len(np.unique(prev[0])) == prev.shape[1]                    # the scores are not all alike
+
+
+def test_relative_rescoring_with_a_zero_position_weight_is_the_absolute_path():
+    """If the position layer ignores its input, the reading of the position cannot matter: same maps, same lists."""
+    runs = []
+    for relative in (True, False):
+        w = Workload(REL.scaled(ctrl_relative_position=relative))
+        w.ctrl = dict(w.ctrl, pos_w=np.zeros_like(w.ctrl["pos_w"]))
+        orc = make_oracle(w)
+        trace = []
+        for s in range(REL.steps):
+            x = w.x_new(orc.n)
+            q, k, v = w.qkv(orc.n, 0, x)
+            orc.decode_step(0, q, k, v, x, None)
+            orc.rebuild(0)
+            orc.check_invariants()
+            trace.append((orc.slot_tok.copy(), orc.info.evicted_tok.copy(), [l.copy() for l in orc.info.rebuild_tok]))
+        runs.append(trace)
+    for (st_a, ev_a, l_a), (st_b, ev_b, l_b) in zip(*runs):
+        assert np.array_equal(st_a, st_b) and np.array_equal(ev_a, ev_b)
+        assert all(np.array_equal(a, b) for a, b in zip(l_a, l_b))
+    assert any((ev >= 0).any() for _, ev, _ in runs[0])
+
+
+@pytest.mark.parametrize("mode", ["policy", "explicit"])
+def test_relative_selection_ranks_by_the_scores_of_the_current_step(mode):
+    """Release rule and list choice with Python sorts, on the scores as seen from the token that was just added;
+    over the run the order of two tokens must actually change (else the re-scoring would not be exercised)."""
+    cfg = REL.scaled(rebuild_mode=mode, rebuild_p=0.3, steps=40, rebuild_max=3)
+    w = Workload(cfg)
+    # weights of order one instead of 0.02: the Tanh layer leaves its linear range, where a change of position would
+    # move every token's score by the same amount and never change an order
+    w.ctrl = {k: (v * 50.0 if k in ("pos_w", "pos_b", "mlp_w1", "mlp_b1", "gru_w_hh") else v) for k, v in w.ctrl.items()}
+    orc = make_oracle(w)
+    flips, before_scores = 0, None
+    for s in range(cfg.steps):
+        n = orc.n
+        x = w.x_new(n)
+        q, k, v = w.qkv(n, 0, x)
+        ex = explicit_as_lists(*w.explicit(s, n))
+        before = (orc.slot_tok.copy(), orc.slot_role.copy())
+        orc.decode_step(0, q, k, v, x, ex)
+        orc.check_invariants()
+        assert np.allclose(orc.score[:, : n + 1], ao.controller_rescore(orc.z_rows[:, : n + 1], n, cfg.pos_scale, w.ctrl),
+                           rtol=1e-6, atol=1e-9)
+        for b in range(w.batch):
+            st, sr, admit, ev, lst = brute_select(orc.score[b], before[0][b], before[1][b], n, cfg.retained_max,
+                                                  cfg.rebuild_max, None if ex is None else ex[b])
+            assert st == orc.slot_tok[b].tolist() and sr == orc.slot_role[b].tolist()
+            assert admit == orc.info.admit_slot[b] and ev == orc.info.evicted_tok[b]
+            assert lst == orc.info.rebuild_tok[b].tolist()
+        if before_scores is not None:
+            a, c = before_scores[0, :n], orc.score[0, :n]
+            flips += int((np.sign(a[:, None] - a[None, :]) * np.sign(c[:, None] - c[None, :]) < 0).sum())
+        before_scores = orc.score.copy()
+        orc.rebuild(0)
+    assert flips > 0
+
+
+@pytest.mark.parametrize("prompt", [1, 5, 19])
+def test_relative_bulk_load_selects_on_the_scores_seen_from_the_last_prompt_token(prompt):
+    cfg = REL.scaled(prompt=prompt, steps=2)
+    w = Workload(cfg)
+    orc = make_oracle(w)
+    orc.append_tokens(w.prompt())
+    orc.check_invariants()
+    want = ao.controller_rescore(orc.z_rows[:, :prompt], prompt - 1, cfg.pos_scale, w.ctrl).astype(np.float32)
+    assert np.array_equal(orc.score[:, :prompt], want)
+    for b in range(w.batch):
+        ranked = sorted(range(prompt - 1), key=lambda t: (float(want[b, t]), t), reverse=True)
+        keep = sorted(ranked[: cfg.retained_max - 1] + [prompt - 1])
+        ret = orc.slot_tok[b][orc.slot_role[b] == ao.RETAINED].tolist()
+        assert ret == keep
+        assert orc.info.rebuild_tok[b].tolist() == ranked[cfg.retained_max - 1:][: cfg.rebuild_max]
+
+
 # ------------------------------------------------------------------ planted mistakes
 def test_pins_notice_planted_mistakes(monkeypatch):
     """Each plausible slip, planted in the oracle, must make one of the pins above fail."""
@@ -595,3 +718,12 @@ def test_pins_notice_planted_mistakes(monkeypatch):
     monkeypatch.setattr(ao, "sparse_attention", attn_no_scale)
     assert fails(test_path_equals_full_attention_when_every_token_is_resident, 0, 0)
     monkeypatch.setattr(ao, "sparse_attention", real_attn)
+
+    real_rescore = ao.controller_rescore
+    monkeypatch.setattr(ao, "controller_rescore",                      # distance counted from the wrong end
+                        lambda z, n, ps, w: real_rescore(np.asarray(z)[..., ::-1, :], n, ps, w)[..., ::-1])
+    assert fails(test_relative_rescoring_equals_torch_modules_on_the_distance_to_the_current_token)
+    assert fails(test_relative_scores_shift_with_the_sequence_and_meet_the_absolute_score_at_the_same_distance)
+    monkeypatch.setattr(ao, "controller_rescore", lambda z, n, ps, w: real_rescore(z, n, ps / 2, w))   # wrong scale
+    assert fails(test_relative_scores_shift_with_the_sequence_and_meet_the_absolute_score_at_the_same_distance)
+    monkeypatch.setattr(ao, "controller_rescore", real_rescore)
