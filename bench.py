@@ -205,7 +205,8 @@ class DeviceRun:
                             rebuild_max=c.rebuild_max, topk=c.topk, max_tokens=c.max_tokens,
                             ctrl_hidden=c.ctrl_hidden, dtype=c.dtype, rebuild_mode=c.rebuild_mode,
                             rope_theta=c.rope_theta, pos_scale=c.pos_scale,
-                            flags=lib.ADORE_FLAG_SCORE_FROM_ATTENTION if score_source == "attention" else 0),
+                            flags={"attention": lib.ADORE_FLAG_SCORE_FROM_ATTENTION,
+                                   "controller-relative": lib.ADORE_FLAG_RELATIVE_POSITION}.get(score_source, 0)),
             wl.controller_weights(c), self.stream)
 
         def randn(*shape, std=1.0):
@@ -550,8 +551,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--score-source", default="controller", choices=["controller", "attention"],
-                    help="attention: tokens ranked by cumulative attention weight (the H2O baselines' score), no controller")
+    ap.add_argument("--score-source", default="controller", choices=["controller", "attention", "controller-relative"],
+                    help="attention: tokens ranked by cumulative attention weight (the H2O baselines' score), no controller; "
+                         "controller-relative: position feature = distance to the current token, every token re-scored every step")
     ap.add_argument("--labels", action="store_true", help="time the label-construction entry point instead of the decode step")
     ap.add_argument("--order", default="attend-first", choices=["attend-first", "rebuild-first"],
                     help="rebuild-first: select, rebuild, then one attention with R_max+1 query rows per sequence "

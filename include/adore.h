@@ -77,6 +77,13 @@ enum { ADORE_SLOT_EMPTY = 0, ADORE_SLOT_RETAINED = 1, ADORE_SLOT_REBUILT = 2 };
  * most recent tokens. adore_decode_step then accumulates after every layer's attention (weights == NULL is fine: an
  * internal buffer is used); adore_step_begin returns ADORE_ERR_UNSUPPORTED. */
 #define ADORE_FLAG_SCORE_FROM_ATTENTION 2u
+/* Position feature of the controller read as the distance to the token being decoded (Section 1 and the caption of
+ * Figure 2 speak of importance with respect to the current token, for all earlier tokens, cached or released; Eq. 2
+ * itself only says "position embedding"): u = (n - i) / pos_scale, so every earlier token is scored anew at every
+ * step, from the GRU state it had when it arrived, and the step's release and rebuild list rank by those fresh scores.
+ * A prompt is scored once, as seen from its last token. adore_cache_scores() then shows tokens 0..n-1 as seen from
+ * token n-1. Needs max_tokens * ctrl_hidden * 8 bytes per sequence more; not with ADORE_FLAG_SCORE_FROM_ATTENTION. */
+#define ADORE_FLAG_RELATIVE_POSITION 4u
 
 typedef struct {
   uint32_t struct_size;  /* sizeof(adore_config_t), for versioning                               */

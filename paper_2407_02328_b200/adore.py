@@ -24,6 +24,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "OOM", 3: "TOKEN_TABLE_FULL", 4: "
 
 ADORE_FLAG_NO_RECURRENCE = 1
 ADORE_FLAG_SCORE_FROM_ATTENTION = 2
+ADORE_FLAG_RELATIVE_POSITION = 4
 
 
 class AdoreError(RuntimeError):

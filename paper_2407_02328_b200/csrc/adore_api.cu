@@ -106,6 +106,8 @@ struct adore_cache {
   void* Vc = nullptr;
   void* x_store = nullptr;
   double* z = nullptr;
+  double* a_tab = nullptr;      // relative positions: per token the input of the controller's Tanh layer at distance 0
+  double* c_vec = nullptr;      // relative positions: W1 pos_w
   float* score = nullptr;
   float* sigma = nullptr;
   int* tok_slot = nullptr;
@@ -254,6 +256,7 @@ RecurParams recur_params(adore_cache* c, int rows, int tc, int ksplit, int n0) {
   r.z = c->z; r.score = c->score; r.sigma = c->sigma; r.max_tokens = c->cfg.max_tokens; r.n0 = n0;
   r.pos_scale = double(c->cfg.pos_scale);
   r.no_recurrence = (c->cfg.flags & ADORE_FLAG_NO_RECURRENCE) ? 1 : 0;
+  r.a_tab = c->a_tab;
   return r;
 }
 
@@ -419,6 +422,19 @@ adore_status_t launch_add_attention(adore_cache* c, const float* weights) {
   return ADORE_OK;
 }
 
+// Relative positions: tokens 0 .. n-1 scored as seen from token n. Needs the controller launches of all of them.
+adore_status_t launch_rescore(adore_cache* c, int n, cudaStream_t stream) {
+  if (!c->a_tab || n < 1) return ADORE_OK;
+  RescoreParams p{};
+  p.a_tab = c->a_tab; p.c_vec = c->c_vec; p.w2 = c->w2; p.b2 = c->b2; p.score = c->score; p.sigma = c->sigma;
+  p.h = c->cfg.ctrl_hidden; p.max_tokens = c->cfg.max_tokens; p.n = n; p.pos_scale = double(c->cfg.pos_scale);
+  dim3 grid((n + kRescoreTokens - 1) / kRescoreTokens, c->cfg.batch);
+  ctrl_rescore_kernel<<<grid, kRescoreThreads, 0, stream>>>(p);
+  ++c->launches;
+  CUDA_OK(cudaGetLastError());
+  return ADORE_OK;
+}
+
 adore_status_t launch_row_table(adore_cache* c, bool count_rows, cudaStream_t stream) {
   const adore_config_t& f = c->cfg;
   if (f.rebuild_max == 0) return ADORE_OK;          // row_total stays 0
@@ -444,7 +460,8 @@ adore_status_t fill_layer_impl(adore_cache* c, int layer, const void* x_table) {
 adore_status_t check_config(const adore_config_t* f) {
   if (f->struct_size != sizeof(adore_config_t)) return ADORE_ERR_INVALID_ARG;
   if (f->batch < 1 || f->n_layers < 1 || f->n_heads < 1 || f->hidden < 1 || f->capacity < 1 || f->topk < 1 ||
-      f->max_tokens < 1 || f->ctrl_hidden < 1 || f->rebuild_max < 0 || f->rebuild_max >= f->capacity || (f->flags & ~uint32_t(ADORE_FLAG_NO_RECURRENCE | ADORE_FLAG_SCORE_FROM_ATTENTION)) != 0 ||
+      f->max_tokens < 1 || f->ctrl_hidden < 1 || f->rebuild_max < 0 || f->rebuild_max >= f->capacity || (f->flags & ~uint32_t(ADORE_FLAG_NO_RECURRENCE | ADORE_FLAG_SCORE_FROM_ATTENTION | ADORE_FLAG_RELATIVE_POSITION)) != 0 ||
+      ((f->flags & ADORE_FLAG_SCORE_FROM_ATTENTION) && (f->flags & ADORE_FLAG_RELATIVE_POSITION)) ||
       !(f->pos_scale > 0.f) || f->rope_theta < 0.f)
     return ADORE_ERR_INVALID_ARG;
   if (f->dtype != ADORE_F32 && f->dtype != ADORE_BF16) return ADORE_ERR_INVALID_ARG;
@@ -471,6 +488,8 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
   const bool controller = !(f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION);   // else the scores come from the attention
   if (c->ctrl_pending) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_ctrl, 0));   // scores of token n-1
   // The selection chain is what the step waits for, so it is queued first; the controller's launches follow.
+  st = launch_rescore(c, c->n, sel);            // relative positions: the ranking below is the one seen from token n
+  if (st != ADORE_OK) return st;
   const int P = ex ? pow2_at_least(r_in) : pow2_at_least(c->n);
   SelectParams sp = select_params(c, c->n, P, c->cur, 1 - c->cur);
   sp.explicit_list = ex && r_in > 0 ? explicit_list : nullptr;
@@ -620,6 +639,13 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   TRY(upload(c, &c->b1, w->mlp_b1, h));
   TRY(upload(c, &c->w2, w->mlp_w2, h));
   TRY(upload(c, &c->b2, w->mlp_b2, 1));
+  if (f.flags & ADORE_FLAG_RELATIVE_POSITION) {
+    TRY(dev_alloc(c, &c->a_tab, B * MT * h * sizeof(double), true));
+    TRY(dev_alloc(c, &c->c_vec, h * sizeof(double), false));
+    ctrl_position_direction_kernel<<<int((h + 127) / 128), 128, 0, c->stream>>>(c->w1, c->pos_w, c->c_vec, int(h));
+    ++c->launches;
+    if (cudaGetLastError() != cudaSuccess) { adore_cache_destroy(c); return ADORE_ERR_CUDA; }
+  }
   if (f.rope_theta != 0.f) {   // rotation angle of pair j at position p: p * theta^(-2j/dh)
     const size_t half = f.head_dim / 2;
     std::vector<float> cs(MT * half), sn(MT * half);
@@ -744,6 +770,10 @@ adore_status_t adore_cache_append_tokens(adore_cache_t* c, const void* x, int32_
     ctrl_recur_kernel<<<f.batch, select_threads(c), ctrl_smem(c), c->stream>>>(rp, ctrl_resident_ok(f.ctrl_hidden) ? 1 : 0, c->err);
     ++c->launches;
     CUDA_OK(cudaGetLastError());
+  }
+  {                                             // relative positions: the prompt as seen from its last token
+    adore_status_t st = launch_rescore(c, T - 1, c->stream);
+    if (st != ADORE_OK) return st;
   }
   const int P = pow2_at_least(T);
   SelectParams sp = select_params(c, T, P, c->cur, c->cur);
@@ -1056,13 +1086,18 @@ std::vector<StateSection> state_sections(adore_cache* c) {
       {c->row_total, sizeof(int)},
   };
 }
+// with relative positions the per-token Tanh inputs are state too (they are what later steps score from)
+void add_relative_state(adore_cache* c, std::vector<StateSection>& sec) {
+  if (c->a_tab) sec.push_back({c->a_tab, size_t(c->cfg.batch) * c->cfg.max_tokens * c->cfg.ctrl_hidden * sizeof(double)});
+}
 inline size_t pad8(size_t v) { return (v + 7) & ~size_t(7); }
 
 }  // namespace
 
 adore_status_t adore_cache_export_state(adore_cache_t* c, void* host_buf, size_t* bytes) {
   if (!c || !bytes) return ADORE_ERR_INVALID_ARG;
-  const std::vector<StateSection> sec = state_sections(c);
+  std::vector<StateSection> sec = state_sections(c);
+  add_relative_state(c, sec);
   size_t need = sizeof(StateHeader);
   for (const StateSection& s : sec) need += pad8(s.bytes);
   if (!host_buf) { *bytes = need; return ADORE_OK; }
@@ -1078,6 +1113,7 @@ adore_status_t adore_cache_export_state(adore_cache_t* c, void* host_buf, size_t
   hd.batch = c->cfg.batch; hd.capacity = c->cfg.capacity; hd.rebuild_max = c->cfg.rebuild_max;
   hd.max_tokens = c->cfg.max_tokens; hd.ctrl_hidden = c->cfg.ctrl_hidden;
   hd.n = c->n; hd.cur = c->cur; hd.attn = c->attn; hd.step_open = c->step_layer0_done;
+  hd.reserved[0] = c->cfg.flags & ADORE_FLAG_RELATIVE_POSITION;   // decides whether the last section is present
   unsigned char* dst = static_cast<unsigned char*>(host_buf);
   std::memset(dst, 0, need);
   std::memcpy(dst, &hd, sizeof(hd));
@@ -1096,9 +1132,10 @@ adore_status_t adore_cache_import_state(adore_cache_t* c, const void* host_buf, 
   const adore_config_t& f = c->cfg;
   if (hd.magic != kStateMagic || hd.version != 1 || hd.batch != f.batch || hd.capacity != f.capacity ||
       hd.rebuild_max != f.rebuild_max || hd.max_tokens != f.max_tokens || hd.ctrl_hidden != f.ctrl_hidden ||
-      hd.n < 0 || hd.n > f.max_tokens || (hd.cur != 0 && hd.cur != 1) || (hd.attn != 0 && hd.attn != 1))
+      hd.reserved[0] != (f.flags & ADORE_FLAG_RELATIVE_POSITION) || hd.n < 0 || hd.n > f.max_tokens || (hd.cur != 0 && hd.cur != 1) || (hd.attn != 0 && hd.attn != 1))
     return ADORE_ERR_INVALID_ARG;
-  const std::vector<StateSection> sec = state_sections(c);
+  std::vector<StateSection> sec = state_sections(c);
+  add_relative_state(c, sec);
   size_t need = sizeof(StateHeader);
   for (const StateSection& s : sec) need += pad8(s.bytes);
   if (bytes < need) return ADORE_ERR_INVALID_ARG;

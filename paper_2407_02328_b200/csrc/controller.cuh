@@ -256,6 +256,8 @@ struct RecurParams {
   int n0;                // position of the first token of this call
   double pos_scale;
   int no_recurrence;     // 1: every token sees a zero state (the ablation without the GRU's memory, Section 3.5.3)
+  double* a_tab;         // [B, max_tokens, h] or null. Set: positions are relative to the current token; the token is
+                         // scored at distance 0 and the input of its Tanh layer is kept for later re-scoring
 };
 
 
@@ -325,7 +327,7 @@ __device__ __forceinline__ void controller_tokens_impl(const RecurParams& p, int
       const double c = tanh(s_gi[2 * h + tid] + r * s_gh[tid]);
       const double zn = (1.0 - u) * c + u * s_z[tid];
       s_z[tid] = zn;
-      const double upos = double(pos) / p.pos_scale;
+      const double upos = p.a_tab ? 0.0 : double(pos) / p.pos_scale;
       s_pz[tid] = double(p.pos_w[tid]) * upos + double(p.pos_b[tid]) + zn;
     }
     __syncthreads();
@@ -353,7 +355,11 @@ __device__ __forceinline__ void controller_tokens_impl(const RecurParams& p, int
           if (j < h) acc = fma(double(w[a][jj]), s_pz[j], acc);
         }
         acc = warp_sum(acc);
-        if (lane == 0 && i < h) s_t[i] = double(ww[a]) * tanh(acc + double(bb[a]));
+        if (lane == 0 && i < h) {
+          const double pre = acc + double(bb[a]);
+          s_t[i] = double(ww[a]) * tanh(pre);
+          if (p.a_tab) p.a_tab[(size_t(b) * p.max_tokens + pos) * h + i] = pre;
+        }
       }
     }
     __syncthreads();
@@ -498,7 +504,7 @@ __device__ __forceinline__ void controller_tokens_resident(const RecurParams& p,
       const double c = tanh(s_gi[2 * h + tid] + r * s_gh[tid]);
       const double zn = (1.0 - u) * c + u * s_z[tid];
       s_z[tid] = zn;
-      s_pz[tid] = double(s_posw[tid]) * (double(pos) / p.pos_scale) + double(s_posb[tid]) + zn;
+      s_pz[tid] = double(s_posw[tid]) * (p.a_tab ? 0.0 : double(pos) / p.pos_scale) + double(s_posb[tid]) + zn;
     }
     __syncthreads();
     {
@@ -522,7 +528,11 @@ __device__ __forceinline__ void controller_tokens_resident(const RecurParams& p,
 #pragma unroll
         for (int a = 1; a < RW; ++a) if (lane == a) mine = acc[a];
         const int i = warp * rw + lane;
-        if (lane < rw && i < h) s_t[i] = double(s_w2[i]) * tanh(mine + double(s_b1[i]));
+        if (lane < rw && i < h) {
+          const double pre = mine + double(s_b1[i]);
+          s_t[i] = double(s_w2[i]) * tanh(pre);
+          if (p.a_tab) p.a_tab[(size_t(b) * p.max_tokens + pos) * h + i] = pre;
+        }
       }
     }
     __syncthreads();
@@ -539,6 +549,73 @@ __device__ __forceinline__ void controller_tokens_resident(const RecurParams& p,
     __syncthreads();
   }
   if (tid < h) p.z[size_t(b) * h + tid] = s_z[tid];
+}
+
+// ---- relative positions: every earlier token scored anew at every step ---------------------------
+// Section 1 and Figure 2 describe the controller's importance as taken with respect to the token being decoded,
+// over all earlier tokens, cached or released. With the position feature read as the distance to the current
+// token, u = (n - i) / pos_scale, the score of token i at step n is
+//   w2 . tanh(W1 (pos_w u + pos_b + z_i) + b1) + b2  =  w2 . tanh(a_i + u c) + b2,
+// with a_i = W1 (pos_b + z_i) + b1 kept from the step the token arrived in (a_tab above) and c = W1 pos_w
+// computed once. A step then costs d' tanh per token instead of a d' x d' product, in float64 like the rest of
+// the controller (the score decides which token leaves the cache).
+struct RescoreParams {
+  const double* a_tab;   // [B, max_tokens, h]
+  const double* c_vec;   // [h]  W1 pos_w
+  const float* w2;       // [h]
+  const float* b2;       // [1]
+  float* score;          // [B, max_tokens]
+  float* sigma;          // [B, max_tokens]
+  int h, max_tokens;
+  int n;                 // current token; tokens 0 .. n-1 are re-scored
+  double pos_scale;
+};
+
+constexpr int kRescoreThreads = 256;
+constexpr int kRescoreTokens = 32;     // per CTA: one warp per token, four rounds
+
+// c[i] = sum_j W1[i][j] pos_w[j], j ascending. One thread per row; runs once per cache.
+static __global__ void ctrl_position_direction_kernel(const float* __restrict__ w1, const float* __restrict__ pos_w, double* c_vec, int h) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= h) return;
+  double acc = 0.0;
+  for (int j = 0; j < h; ++j) acc = fma(double(w1[size_t(i) * h + j]), double(pos_w[j]), acc);
+  c_vec[i] = acc;
+}
+
+// grid (ceil(n / kRescoreTokens), B). A warp owns a token: lanes split the d' terms, a shuffle tree adds them in a
+// fixed order.
+static __global__ void __launch_bounds__(kRescoreThreads) ctrl_rescore_kernel(const RescoreParams p) {
+  const int b = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int kWarps = kRescoreThreads / 32;
+  constexpr int JMAX = 8;                      // d' <= 256
+  double cj[JMAX];
+  float wj[JMAX];
+#pragma unroll
+  for (int jj = 0; jj < JMAX; ++jj) {
+    const int j = lane + 32 * jj;
+    cj[jj] = j < p.h ? p.c_vec[j] : 0.0;
+    wj[jj] = j < p.h ? __ldg(p.w2 + j) : 0.f;
+  }
+  const double b2 = double(__ldg(p.b2));
+  for (int k = warp; k < kRescoreTokens; k += kWarps) {
+    const int i = blockIdx.x * kRescoreTokens + k;
+    if (i >= p.n) break;                       // warp-uniform
+    const double u = double(p.n - i) / p.pos_scale;
+    const double* a = p.a_tab + (size_t(b) * p.max_tokens + i) * p.h;
+    double acc = 0.0;
+#pragma unroll
+    for (int jj = 0; jj < JMAX; ++jj) {
+      const int j = lane + 32 * jj;
+      if (j < p.h) acc += double(wj[jj]) * tanh(fma(u, cj[jj], a[j]));
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) {
+      const double sc = acc + b2;
+      p.score[size_t(b) * p.max_tokens + i] = float(sc);
+      p.sigma[size_t(b) * p.max_tokens + i] = float(1.0 / (1.0 + exp(-sc)));
+    }
+  }
 }
 
 __device__ inline void controller_tokens(const RecurParams& p, int b, double* sm) {

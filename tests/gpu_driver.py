@@ -57,7 +57,8 @@ class GpuCache:
                             max_tokens=c.max_tokens, ctrl_hidden=c.ctrl_hidden, dtype=c.dtype,
                             rebuild_mode=c.rebuild_mode, rope_theta=c.rope_theta, pos_scale=c.pos_scale,
                             flags=(lib.ADORE_FLAG_NO_RECURRENCE if c.ctrl_no_recurrence else 0) |
-                            (lib.ADORE_FLAG_SCORE_FROM_ATTENTION if c.score_from_attention else 0)),
+                            (lib.ADORE_FLAG_SCORE_FROM_ATTENTION if c.score_from_attention else 0) |
+                            (lib.ADORE_FLAG_RELATIVE_POSITION if c.ctrl_relative_position else 0)),
             w.ctrl, torch.cuda.current_stream().cuda_stream)
         self.w_kv_dev = [to_dev(m, c) for m in w.w_kv]
         for l, m in enumerate(self.w_kv_dev):

@@ -75,6 +75,15 @@ def test_full_token_table_and_bad_arguments():
                 call()
             assert e.value.status == 1
         lib.adore_cache_sync_status(g.handle)
+        # flags that exclude each other, and a flag bit that does not exist
+        for flags in (lib.ADORE_FLAG_SCORE_FROM_ATTENTION | lib.ADORE_FLAG_RELATIVE_POSITION, 1 << 9):
+            with pytest.raises(lib.AdoreError) as e:
+                lib.adore_cache_create(
+                    lib.make_config(batch=2, n_layers=1, n_heads=2, head_dim=64, hidden=128, capacity=16, rebuild_max=2, topk=4,
+                                    max_tokens=32, ctrl_hidden=32, dtype="f32", rebuild_mode="policy", rope_theta=0.0,
+                                    pos_scale=64.0, flags=flags),
+                    w.ctrl, torch.cuda.current_stream().cuda_stream)
+            assert e.value.status == 1
     finally:
         g.close()
 

@@ -180,3 +180,20 @@ def test_peaked_logits_as_in_real_attention():
     _run(SMALL.scaled(name="peaked_q8_c517", q_scale=8.0, capacity=517, topk=200, rebuild_max=37, prompt=700, steps=8, batch=2,
                       seed=135))
     _run_rebuild_first(SMALL.scaled(name="peaked_rows", q_scale=8.0, rebuild_max=7, capacity=70, prompt=90, steps=10, seed=136))
+
+
+
+def test_relative_positions_rescore_every_token_at_every_step():
+    """The controller's position feature read as the distance to the current token: tokens 0..n-1 are scored anew at
+    every step, from the Tanh-layer inputs kept when they arrived, and release and rebuild list follow the fresh scores
+    (prompt: scored once, as seen from its last token). Weights of order 0.3 and a short position scale take the Tanh
+    layer out of its linear range, so that the order of tokens really changes from step to step."""
+    rel = dict(ctrl_relative_position=True, pos_scale=32.0, ctrl_weight_std=0.3)
+    _run(SMALL.scaled(name="rel_policy", steps=40, seed=139, **rel))
+    _run(SMALL.scaled(name="rel_default_init", ctrl_relative_position=True, steps=20, seed=140))
+    _run(SMALL.scaled(name="rel_explicit_empty_f32", dtype="f32", n_heads=2, hidden=128, rebuild_mode="explicit", rebuild_p=0.3,
+                      rebuild_max=12, capacity=33, topk=7, prompt=0, steps=70, seed=141, **rel))
+    _run(SMALL.scaled(name="rel_ctrl160_norecurrence", ctrl_hidden=160, ctrl_no_recurrence=True, steps=15, seed=142, **rel))
+    _run(SMALL.scaled(name="rel_ctrl96_L2", ctrl_hidden=96, n_layers=2, batch=2, per_layer_inputs=True, steps=12, seed=143, **rel))
+    _run(SMALL.scaled(name="rel_host_entry", steps=10, seed=144, **rel), host_entry="with_rebuild")
+    _run_rebuild_first(SMALL.scaled(name="rel_rows", steps=20, seed=145, **rel))

@@ -32,7 +32,9 @@ def _steps(g, w, lib, torch, to_dev, first, count):
     return seen
 
 
-def test_export_import_rewinds_the_cache():
+@pytest.mark.parametrize("CFG", [CFG, CFG.scaled(name="snapshot_relative", ctrl_relative_position=True, pos_scale=32.0,
+                                                 ctrl_weight_std=0.3)], ids=["absolute", "relative"])
+def test_export_import_rewinds_the_cache(CFG):
     import torch
     from paper_2407_02328_b200 import adore as lib
     from oracle.harness import Workload
@@ -98,3 +100,16 @@ def test_import_rejects_a_snapshot_of_another_shape():
     finally:
         g1.close()
         g2.close()
+    # and of another reading of the position: the relative one carries a section more
+    g1 = GpuCache(Workload(CFG, None))
+    g3 = GpuCache(Workload(CFG.scaled(name="snapshot_rel", ctrl_relative_position=True), None))
+    try:
+        for src, dst in ((g1, g3), (g3, g1)):
+            snap = np.zeros(lib.adore_cache_export_state(src.handle, None), np.uint8)
+            lib.adore_cache_export_state(src.handle, snap)
+            with pytest.raises(lib.AdoreError) as e:
+                lib.adore_cache_import_state(dst.handle, snap)
+            assert e.value.status == 1
+    finally:
+        g1.close()
+        g3.close()

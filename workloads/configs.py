@@ -38,6 +38,7 @@ class WorkloadConfig:
     per_layer_inputs: bool = False      # every layer has its own RMS-normalised input rows
     ctrl_no_recurrence: bool = False    # controller ablation without the GRU's memory: every token sees a zero state
     score_from_attention: bool = False  # tokens ranked by cumulative attention weight instead of the controller's score
+    ctrl_weight_std: float = 0.02         # standard deviation of the random-init controller parameters
     ctrl_relative_position: bool = False  # controller re-scores every token at every step by its distance to the current one
     q_scale: float = 1.0                # factor on the queries: > 1 gives the peaked, long-tailed softmax of real attention
 

@@ -40,12 +40,14 @@ def gaussian(seed: int, name: str, shape: Tuple[int, ...], std: float = 1.0,
     return round_to_dtype(a, dtype)
 
 
-def controller_weights(cfg: WorkloadConfig, std: float = 0.02) -> Dict[str, np.ndarray]:
+def controller_weights(cfg: WorkloadConfig, std: float | None = None) -> Dict[str, np.ndarray]:
     """Random-init controller: GRU(d -> d'), position FC(1 -> d'), FC(d' -> d'), FC(d' -> 1).
 
-    Gate order of the stacked GRU matrices is reset, update, candidate. All fp32.
+    Gate order of the stacked GRU matrices is reset, update, candidate. All fp32. The standard deviation is the
+    config's `ctrl_weight_std` (0.02) unless given.
     """
     d, h, s = cfg.hidden, cfg.ctrl_hidden, cfg.seed
+    std = cfg.ctrl_weight_std if std is None else std
     return {
         "gru_w_ih": gaussian(s, "gru_w_ih", (3 * h, d), std),
         "gru_w_hh": gaussian(s, "gru_w_hh", (3 * h, h), std),
