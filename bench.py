@@ -37,8 +37,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # For the rebuild GEMM the capture saw fewer rows than the timed launches: the weight bytes are fixed,
 # the rest (row reads, cache-row writes) is scaled by the rows processed.
 NCU_TRAFFIC_BYTES = {
-    ("rebuild projection", "cfg3_llama7b_b64_c512_rebuild20pct"): {"bytes": 273.1e6 + 143.0e6, "rows": 10166.0},
-    ("attention kernel", "cfg3_llama7b_b64_c512_rebuild20pct"): {"bytes": 403.9e6 + 6.6e6, "rows": None},
+    ("rebuild projection", "cfg3_llama7b_b64_c512_rebuild20pct"): {"bytes": 284.9e6 + 144.9e6, "rows": 9950.0},
+    ("attention kernel", "cfg3_llama7b_b64_c512_rebuild20pct"): {"bytes": 403.9e6 + 8.7e6, "rows": None},
 }
 
 

@@ -319,17 +319,30 @@ template <>
 bool launch_attention_rows<__nv_bfloat16>(adore_cache* c, int layer, const AttnParams<__nv_bfloat16>& p, int rows_q) {
   const adore_config_t& f = c->cfg;
   static const bool off = std::getenv("ADORE_ROWS_SIMT") != nullptr;     // A/B switch
-  const size_t smem = rows_smem_bytes(f.capacity, f.head_dim, rows_q);
+  const size_t smem = rows_smem_bytes(f.capacity, f.head_dim, std::min(rows_q, kRowsMaxQ));
   const int per_lane = (f.capacity + 1 + 31) / 32;
-  if (off || c->map_k.empty() || rows_q > kRowsMaxQ || per_lane > kRowsKeysPerLaneMax || smem > 200 * 1024) return false;
-  if (f.head_dim == 128) {
-    if (per_lane <= 9) return launch_attention_rows_as<128, 9>(c, layer, p, smem);
-    if (per_lane <= 17) return launch_attention_rows_as<128, 17>(c, layer, p, smem);
-    return launch_attention_rows_as<128, 33>(c, layer, p, smem);
+  if (off || c->map_k.empty() || per_lane > kRowsKeysPerLaneMax || smem > 200 * 1024) return false;
+  // more than 16 rows: one launch per group of 16; the last group holds the current token's row and stores its rows
+  for (int rb = 0; rb < rows_q; rb += kRowsMaxQ) {
+    AttnParams<__nv_bfloat16> g = p;
+    g.rows_q = std::min(kRowsMaxQ, rows_q - rb);
+    g.row_base = rb;
+    g.rows_total = rows_q;
+    if (rb + g.rows_q < rows_q) g.admit_slot = nullptr;
+    bool ok;
+    if (f.head_dim == 128) {
+      if (per_lane <= 9) ok = launch_attention_rows_as<128, 9>(c, layer, g, smem);
+      else if (per_lane <= 17) ok = launch_attention_rows_as<128, 17>(c, layer, g, smem);
+      else ok = launch_attention_rows_as<128, 33>(c, layer, g, smem);
+    } else {
+      if (per_lane <= 9) ok = launch_attention_rows_as<64, 9>(c, layer, g, smem);
+      else if (per_lane <= 17) ok = launch_attention_rows_as<64, 17>(c, layer, g, smem);
+      else ok = launch_attention_rows_as<64, 33>(c, layer, g, smem);
+    }
+    // a refused first launch leaves the other kernel to do all rows; a later one cannot fail where the first did not
+    if (!ok) return false;
   }
-  if (per_lane <= 9) return launch_attention_rows_as<64, 9>(c, layer, p, smem);
-  if (per_lane <= 17) return launch_attention_rows_as<64, 17>(c, layer, p, smem);
-  return launch_attention_rows_as<64, 33>(c, layer, p, smem);
+  return true;
 }
 
 template <typename T>

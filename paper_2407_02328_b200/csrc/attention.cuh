@@ -38,6 +38,9 @@ struct AttnParams {
   int rows_q;
   const int* row_tok;    // [B, r_max] or nullptr
   int r_max, n_cur;
+  // A launch of the tensor-core rows kernel may cover a group of a pair's rows only: rows row_base .. row_base +
+  // rows_q - 1 of rows_total (0: the launch covers all rows_q rows). q, out and weights keep rows_total rows per pair.
+  int row_base, rows_total;
 };
 
 constexpr int kAttnThreads = 256;

@@ -14,6 +14,9 @@
 //            each warp takes one of a tile's four k-steps and half of the output columns, the partial outputs are
 //            added through shared memory. The current token's own value row is added for the last row.
 // Then the current token's rows are stored in their slot. Every mbarrier wait is bounded.
+// More than 16 rows per pair: one launch per group of 16 rows (row_base / rows_total in the parameters); the groups of
+// a pair read its key and value blocks again (from L2 when the launches follow one another closely), and only the
+// last group, which holds the current token's row, adds that token's own key and value and stores its rows.
 #pragma once
 
 #include <cuda.h>
@@ -88,6 +91,9 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int bh = blockIdx.x, b = bh / p.H;
   const int C = p.C, R1 = p.rows_q, SP = rows_logit_stride(C);
+  const int RT = p.rows_total > 0 ? p.rows_total : R1;  // rows per pair in q / out / weights
+  const int rb = p.rows_total > 0 ? p.row_base : 0;     // first row of this launch's group
+  const bool has_last = rb + R1 == RT;                  // the group ends with the current token's row
   // tiles are consumed two at a time (one block barrier and one round of refills per 128 rows): an even count, the
   // tile past the end, if any, holds rows of the next pair or zeros and is masked like every row >= C
   const int n_tiles = (((C + kRowsTile - 1) / kRowsTile) + 1) & ~1;
@@ -99,7 +105,10 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   wait_for_prior_grid();
-  if (tid < kRowsMaxQ) s_qtok[tid] = tid < R1 - 1 ? p.row_tok[size_t(b) * p.r_max + tid] : (tid == R1 - 1 ? p.n_cur : -1);
+  if (tid < kRowsMaxQ) {
+    const int g = rb + tid;                             // row index within the pair
+    s_qtok[tid] = tid >= R1 ? -1 : (g < RT - 1 ? p.row_tok[size_t(b) * p.r_max + g] : p.n_cur);
+  }
   for (int i = tid; i < C; i += kRowsThreads) {         // the slot reserved for the current token is not written yet
     const int tok = map[i];
     s_tok[i] = tok == p.n_cur ? -1 : tok;
@@ -124,7 +133,7 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   // ---- query block as A fragments: rows lane/4 and lane/4 + 8, columns 16 ks + (lane % 4) * 2 (+8) ----
   uint32_t qa[KSTEPS][4];
   {
-    const T* qb = p.q + size_t(bh) * R1 * DH;
+    const T* qb = p.q + (size_t(bh) * RT + rb) * DH;
     const int r0 = lane >> 2, r1 = r0 + 8, c0 = (lane & 3) * 2;
 #pragma unroll
     for (int ks = 0; ks < KSTEPS; ++ks) {
@@ -137,12 +146,13 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   }
   // the current token's own key: last row only (index C); every other row does not see it
   if (warp == kRowsWarps - 1) {
-    const T* ql = p.q + (size_t(bh) * R1 + (R1 - 1)) * DH;
+    const T* ql = p.q + (size_t(bh) * RT + (RT - 1)) * DH;
     const T* kn = p.k_new + size_t(bh) * DH;
     float dot = 0.f;
-    for (int e = lane; e < DH; e += 32) dot = fmaf(__bfloat162float(ql[e]), __bfloat162float(kn[e]), dot);
+    if (has_last)
+      for (int e = lane; e < DH; e += 32) dot = fmaf(__bfloat162float(ql[e]), __bfloat162float(kn[e]), dot);
     dot = warp_sum(dot);
-    for (int r = lane; r < R1; r += 32) S[size_t(r) * SP + C] = (r == R1 - 1) ? dot * p.scale : -INFINITY;
+    for (int r = lane; r < R1; r += 32) S[size_t(r) * SP + C] = (has_last && r == R1 - 1) ? dot * p.scale : -INFINITY;
   }
 
   bool failed = false;
@@ -201,7 +211,7 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     if (e >= R1) continue;
     const int r = e == 0 ? R1 - 1 : e - 1;
     float* row = S + size_t(r) * SP;
-    float* wout = p.weights ? p.weights + (size_t(bh) * R1 + r) * rows_n : nullptr;
+    float* wout = p.weights ? p.weights + (size_t(bh) * RT + rb + r) * rows_n : nullptr;
     // this lane's logits as order-preserving keys, in registers (masked and out-of-range entries rank lowest)
     constexpr uint32_t kMasked = 0x007FFFFFu;           // key of -inf
     uint32_t kk[KPL];
@@ -356,7 +366,7 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     }
     __syncthreads();
     const T* vn = p.v_new + size_t(bh) * DH;
-    const float w_own = S[size_t(R1 - 1) * SP + C];
+    const float w_own = has_last ? S[size_t(R1 - 1) * SP + C] : 0.f;
     for (int i = tid; i < R1 * (DH / 2); i += kRowsThreads) {
       const int r = i / (DH / 2), col = (i % (DH / 2)) * 2;
       float a0 = 0.f, a1 = 0.f;
@@ -366,11 +376,11 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
         a0 += d[0];
         a1 += d[1];
       }
-      if (r == R1 - 1) {
+      if (has_last && r == R1 - 1) {
         a0 = fmaf(w_own, __bfloat162float(vn[col]), a0);
         a1 = fmaf(w_own, __bfloat162float(vn[col + 1]), a1);
       }
-      *reinterpret_cast<uint32_t*>(p.out + (size_t(bh) * R1 + r) * DH + col) = rows_pack_bf16(a0, a1);
+      *reinterpret_cast<uint32_t*>(p.out + (size_t(bh) * RT + rb + r) * DH + col) = rows_pack_bf16(a0, a1);
     }
   }
   // ---- admit: the current token's rows go into their slot (all tiles of this pair have been consumed) ----

@@ -164,6 +164,17 @@ def test_rebuild_first_step_on_the_tensor_core_kernel_shapes():
     _run_rebuild_first(wl.get_config(2).scaled(name="rows_cfg2_shape", batch=2, steps=4))
 
 
+def test_rebuild_first_step_with_more_than_sixteen_query_rows_in_groups():
+    """More than 16 rows per pair on bfloat16 caches: one launch of the tensor-core kernel per group of 16 rows; only the
+    last group holds the current token's row (own key and value, rows stored in their slot). 39 + 1 rows = 16 + 16 + 8,
+    32 + 1 rows = 16 + 16 + a group with the current token alone, explicit lists leave padding rows in every group."""
+    _run_rebuild_first(SMALL.scaled(name="rows_40", rebuild_max=39, capacity=90, topk=30, prompt=140, steps=10, seed=146))
+    _run_rebuild_first(SMALL.scaled(name="rows_33_explicit", rebuild_mode="explicit", rebuild_p=0.4, rebuild_max=32, capacity=80,
+                                    topk=24, prompt=0, steps=70, seed=147))
+    _run_rebuild_first(SMALL.scaled(name="rows_21_dh64_two_layers", head_dim=64, n_heads=3, hidden=192, n_layers=2, batch=2,
+                                    rebuild_max=20, capacity=300, topk=100, prompt=400, steps=6, seed=148))
+
+
 def test_cumulative_attention_as_the_score_source():
     """The H2O / H2O(Rebuilt) score source on the same kernels: no controller, tokens ranked by the attention weight
     they have received (policy lists = the released tokens with the most cumulative attention)."""
