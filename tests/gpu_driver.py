@@ -122,11 +122,18 @@ def compare_attention(rep: Report, cfg, q, orc: ao.AdoreOracle, layer, k_new, at
     tol = TOL[cfg.dtype]
     err = np.abs(out_g - out_o)
     bound = tol["out_abs"] + tol["out_rel"] * np.abs(out_o)
-    assert (err <= bound).all(), f"attention output off by {err.max():.3e} (step {rep.steps}, layer {layer})"
-    rep.max_out_err = max(rep.max_out_err, float(err.max()))
     keep_g, keep_o = w_g > 0, w_o > 0
     rep.topk_rows += keep_o.shape[0] * keep_o.shape[1]
     bad = np.argwhere((keep_g != keep_o).any(-1))
+    # Where the two kept sets differ by a tie (each case is judged below), the outputs differ by the weight that moved
+    # times the value rows it moved between: |out_g - out_o| <= sum_s |w_g - w_o|_s * max|v|. Everywhere else the plain
+    # bound holds.
+    if len(bad):
+        vmax = float(np.abs(orc.Vc[layer]).max())
+        for b, h in bad:
+            bound[b, h] = bound[b, h] + np.abs(w_g[b, h] - w_o[b, h]).sum() * vmax
+    assert (err <= bound).all(), f"attention output off by {err.max():.3e} (step {rep.steps}, layer {layer})"
+    rep.max_out_err = max(rep.max_out_err, float(err.max()))
     w_ok = np.ones_like(keep_o)
     for b, h in bad:
         Kall = np.concatenate([Kc_before[b, h].astype(np.float64), k_new[b, h][None].astype(np.float64)])
