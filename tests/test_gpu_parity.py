@@ -99,6 +99,23 @@ def test_rebuild_with_the_reduction_dimension_split_over_work_units():
                       rebuild_mode="explicit", rebuild_p=0.7, prompt=160, steps=6, seed=120))   # 200 rows: 2 x 8 tiles x 2 parts
 
 
+def test_largest_capacity_and_token_table_the_library_accepts():
+    """C = 4096 slots and a token table of 8192 rows (the limits of adore_cache_create): the prompt fills the table up
+    to eight tokens short of its end, the decode steps take it to the last row. The selection sorts 8192 keys, the
+    attention covers 65 ring chunks per pair, the policy list has 512 rows per step."""
+    _run(SMALL.scaled(name="max_sizes", batch=1, n_heads=2, head_dim=64, hidden=128, capacity=4096, topk=2048, rebuild_max=512,
+                      prompt=8184, steps=8, seed=149), state_every=4)
+
+
+def test_capacity_batch_sweep_corner_shapes():
+    """Three points of the capacity x batch sweep (context 4096 = prompt 3840 + steps, K = C/2, R_max = C/4, explicit
+    flags at 10 %) with the sweep's own shapes per sequence and a sub-batch the oracle finishes in a minute."""
+    pts = {(cap, b): cfg for cap, b, cfg in wl.sweep_points()}
+    _run(pts[(128, 1)], steps=3)
+    _run(pts[(2048, 8)], batch=1, steps=2)
+    _run(pts[(1024, 32)], batch=2, steps=2)
+
+
 def test_config2_sub_batch():
     _run(wl.get_config(2), batch=2, steps=24, state_every=4)
 
