@@ -618,6 +618,7 @@ def main():
         ev0.record()
         for _ in range(K):
             run.step()
+        lib.adore_cache_join(run.handle)                # the last step's side-stream work counts too
         ev1.record()
         barrier()
         ms_local = ev0.elapsed_time(ev1)
@@ -628,6 +629,7 @@ def main():
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             run.step()
+            lib.adore_cache_join(run.handle)
             b.record()
             pairs.append((a, b))
         barrier()

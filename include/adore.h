@@ -187,8 +187,19 @@ adore_status_t adore_decode_rebuild_host(adore_cache_t *cache, int32_t layer, co
  * list, rotary embedding on the key half at each token's original position, rounding to T and
  * scatter into the list's slots. x_table: device T[B, max_tokens, d] rows indexed by token
  * position, or NULL for the cache's stored rows. Call after adore_decode_step of the same layer.
+ * In a cache of several layers (attend-first order) the work is queued on a stream of the library's own, behind
+ * everything the cache's stream holds at the time of the call, and runs beside the attention of the following
+ * layers: nothing reads this layer's rows before the next step's adore_decode_step of this layer, which waits for
+ * it, as does every other call that touches what the rebuild reads or writes. x_table is therefore borrowed until
+ * the next adore_decode_step of layer 0, adore_cache_join or adore_cache_sync_status.
  * Errors: STATE (no projection / no step), INVALID_ARG, CUDA. */
 adore_status_t adore_rebuild(adore_cache_t *cache, int32_t layer, const void *x_table);
+
+/* Makes the stream given at create wait for everything the library has queued on its own streams (the controller of
+ * the last token, rebuilds that run beside later layers), without waiting on the host: work queued on that stream
+ * afterwards, an event recorded on it for timing included, comes after all of the step (Sections 2.2-2.3).
+ * Errors: INVALID_ARG, CUDA. */
+adore_status_t adore_cache_join(adore_cache_t *cache);
 
 /* Read-only DEVICE views of the state of Sections 2.2-2.3 for checking; valid until the next
  * call that changes the cache. */

@@ -52,7 +52,7 @@ EXPORTS = ["adore_cache_create", "adore_cache_destroy", "adore_cache_set_project
            "adore_cache_append_tokens", "adore_cache_fill_layer", "adore_decode_step",
            "adore_decode_step_host", "adore_rebuild", "adore_cache_slot_map", "adore_cache_rebuild_list",
            "adore_cache_step_info", "adore_cache_scores", "adore_cache_kv", "adore_cache_num_tokens",
-           "adore_cache_launch_count", "adore_cache_sync_status", "adore_status_string",
+           "adore_cache_launch_count", "adore_cache_sync_status", "adore_cache_join", "adore_status_string",
            "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows",
            "adore_controller_score_static", "adore_probe_read_bandwidth",
            "adore_cache_export_state", "adore_cache_import_state", "adore_step_begin", "adore_attend_rows",
@@ -91,6 +91,7 @@ def _lib():
         lib.adore_cache_launch_count.argtypes = [vp]
         lib.adore_cache_launch_count.restype = C.c_int64
         lib.adore_cache_sync_status.argtypes = [vp]
+        lib.adore_cache_join.argtypes = [vp]
         lib.adore_cache_set_stage_timing.argtypes = [vp, i32]
         lib.adore_cache_stage_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         lib.adore_cache_rebuild_rows.argtypes = [vp, C.POINTER(C.c_int64)]
@@ -217,6 +218,10 @@ def adore_cache_num_tokens(cache: int) -> int:
 
 def adore_cache_launch_count(cache: int) -> int:
     return _lib().adore_cache_launch_count(cache)
+
+
+def adore_cache_join(cache: int) -> None:
+    _check(_lib().adore_cache_join(cache), "adore_cache_join")
 
 
 def adore_cache_sync_status(cache: int) -> None:

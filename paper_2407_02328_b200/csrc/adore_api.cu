@@ -157,6 +157,15 @@ struct adore_cache {
   cudaEvent_t ev_copy = nullptr;
   cudaEvent_t ev_out = nullptr;     // `out` has reached the host (host-buffer entry point that also queues the rebuild)
   bool joined = true;
+  // Caches of several layers, attend-first order: the rebuild of layer l writes layer l's rows only, which nothing reads
+  // before the NEXT step's attention of that layer, so it runs on a stream of its own beside the attention of the layers
+  // that follow. ev_rebuilt[l] marks its end; whoever next touches layer l's rows, the row table or the gather buffer
+  // waits for it.
+  cudaStream_t rb = nullptr;
+  cudaEvent_t ev_rb_fork = nullptr;
+  std::vector<cudaEvent_t> ev_rebuilt;
+  std::vector<char> rb_pending;
+  int rb_last = -1;             // layer of the most recent launch on `rb` that nobody has waited for yet
   std::vector<const void*> w_kv;
   TcState tc;                   // tensor-core rebuild path (tensor maps, gather buffer)
   std::vector<CUtensorMap> map_k, map_v;   // per layer: the cache as [B*H*C, dh] tiles of 64 x 64 (bf16, dh 64 or 128)
@@ -211,6 +220,21 @@ adore_status_t join_controller(adore_cache* c) {
     CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_ctrl, 0));
     c->ctrl_pending = false;
   }
+  return ADORE_OK;
+}
+
+// Makes `stream` wait for the rebuild of `layer` if it is still running beside the main stream.
+adore_status_t wait_rebuild(adore_cache* c, int layer, cudaStream_t stream) {
+  if (layer >= 0 && layer < int(c->rb_pending.size()) && c->rb_pending[layer])
+    CUDA_OK(cudaStreamWaitEvent(stream, c->ev_rebuilt[layer], 0));
+  return ADORE_OK;
+}
+// Makes the main stream wait for every rebuild that runs beside it. The side stream runs them in order, so the
+// event of the most recent one covers all.
+adore_status_t join_rebuilds(adore_cache* c) {
+  if (c->rb_last >= 0) CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_rebuilt[c->rb_last], 0));
+  c->rb_last = -1;
+  std::fill(c->rb_pending.begin(), c->rb_pending.end(), char(0));
   return ADORE_OK;
 }
 
@@ -396,9 +420,11 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
 
 template <typename T>
 adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, const int* row_b, const int* row_tok,
-                              const int* row_slot, const int* row_total, int m_max, bool step_table) {
+                              const int* row_slot, const int* row_total, int m_max, bool step_table,
+                              cudaStream_t stream = nullptr) {
   const adore_config_t& f = c->cfg;
   if (m_max <= 0) return ADORE_OK;
+  if (!stream) stream = c->stream;
   RebuildParams<T> p{};
   const size_t layer_elems = size_t(f.batch) * f.n_heads * f.capacity * f.head_dim;
   p.x_table = static_cast<const T*>(x_table ? x_table : c->x_store); p.seq_stride = f.max_tokens; p.d = f.hidden;
@@ -412,14 +438,14 @@ adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, co
     // Rows gathered from the token store for this step's table serve every layer that rebuilds from the store.
     const bool from_store = step_table && x_table == nullptr && size_t(m_max) <= c->tc.a_rows;
     int launched = 0;
-    cudaError_t e = launch_rebuild_tc(c->tc, p, layer, m_max, c->stream, &launched, from_store && c->rows_gathered);
+    cudaError_t e = launch_rebuild_tc(c->tc, p, layer, m_max, stream, &launched, from_store && c->rows_gathered);
     c->launches += launched;
     c->rows_gathered = from_store;
     CUDA_OK(e);
     return ADORE_OK;
   }
   dim3 grid(p.N / kSimtTile, (m_max + kSimtTile - 1) / kSimtTile);
-  rebuild_simt_kernel<T><<<grid, 256, 0, c->stream>>>(p);
+  rebuild_simt_kernel<T><<<grid, 256, 0, stream>>>(p);
   ++c->launches;
   CUDA_OK(cudaGetLastError());
   return ADORE_OK;
@@ -699,6 +725,17 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
     adore_cache_destroy(c);
     return ADORE_ERR_CUDA;
   }
+  if (f.n_layers > 1) {
+    bool ok = cudaStreamCreateWithFlags(&c->rb, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_rb_fork, cudaEventDisableTiming) == cudaSuccess;
+    c->rb_pending.assign(size_t(f.n_layers), char(0));
+    for (int l = 0; ok && l < f.n_layers; ++l) {
+      cudaEvent_t e = nullptr;
+      ok = cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+      if (ok) c->ev_rebuilt.push_back(e);
+    }
+    if (!ok) { adore_cache_destroy(c); return ADORE_ERR_CUDA; }
+  }
   if (f.dtype == ADORE_BF16) {
     st = tc_init(c->tc, f, c->owned, c->stream);
     if (st != ADORE_OK) { adore_cache_destroy(c); return st; }
@@ -734,6 +771,9 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   cudaStreamSynchronize(c->stream);
   if (c->aux) { cudaStreamSynchronize(c->aux); cudaStreamDestroy(c->aux); }
   if (c->ctl) { cudaStreamSynchronize(c->ctl); cudaStreamDestroy(c->ctl); }
+  if (c->rb) { cudaStreamSynchronize(c->rb); cudaStreamDestroy(c->rb); }
+  if (c->ev_rb_fork) cudaEventDestroy(c->ev_rb_fork);
+  for (cudaEvent_t e : c->ev_rebuilt) cudaEventDestroy(e);
   if (c->ev_gates) cudaEventDestroy(c->ev_gates);
   if (c->ev_ctrl) cudaEventDestroy(c->ev_ctrl);
   if (c->copy) { cudaStreamSynchronize(c->copy); cudaStreamDestroy(c->copy); }
@@ -752,6 +792,7 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
 
 adore_status_t adore_cache_set_projection(adore_cache_t* c, int32_t layer, const void* w_kv) {
   if (!c || !w_kv || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;   // a rebuild beside the main stream may still read the old weights
   if (reinterpret_cast<uintptr_t>(w_kv) % 16 != 0) return ADORE_ERR_INVALID_ARG;
   c->w_kv[layer] = w_kv;
   if (c->cfg.dtype == ADORE_BF16) return tc_set_weights(c->tc, layer, w_kv);
@@ -763,7 +804,7 @@ adore_status_t adore_cache_append_tokens(adore_cache_t* c, const void* x, int32_
   if (c->n != 0) return ADORE_ERR_STATE;
   const adore_config_t& f = c->cfg;
   if (T > f.max_tokens) return ADORE_ERR_TOKEN_TABLE_FULL;
-  if (join_controller(c) != ADORE_OK) return ADORE_ERR_CUDA;
+  if (join_controller(c) != ADORE_OK || join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   const size_t row = size_t(f.hidden) * c->esz;
   CUDA_OK(cudaMemcpy2DAsync(c->x_store, size_t(f.max_tokens) * row, x, size_t(T) * row, size_t(T) * row, f.batch,
                             cudaMemcpyDeviceToDevice, c->stream));
@@ -810,6 +851,7 @@ adore_status_t adore_cache_append_tokens(adore_cache_t* c, const void* x, int32_
 adore_status_t adore_cache_fill_layer(adore_cache_t* c, int32_t layer, const void* x_table) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
   if (!c->w_kv[layer]) return ADORE_ERR_STATE;
+  if (join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   return fill_layer_impl(c, layer, x_table);
 }
 
@@ -835,6 +877,17 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     // stage's closing event, so that the stage times add up.)
     cudaStream_t sel = c->timing ? c->stream : c->aux;
     adore_status_t st;
+    // Rebuilds of the previous step may still run beside the main stream: the attention below needs layer 0's, the
+    // selection chain (which rewrites the row table and the gather buffer they read) needs all of them.
+    if (c->timing) { if (join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA; }
+    else if (wait_rebuild(c, 0, c->stream) != ADORE_OK) return ADORE_ERR_CUDA;
+    if (!c->timing && c->rb_last >= 0) {
+      CUDA_OK(cudaStreamWaitEvent(sel, c->ev_rebuilt[c->rb_last], 0));
+      // the selection joins the main stream before this step's first rebuild: from then on the main stream is
+      // behind every earlier rebuild too
+      c->rb_last = -1;
+      std::fill(c->rb_pending.begin(), c->rb_pending.end(), char(0));
+    }
     // the attention is the longest of the three and is launched first; the side streams start from the same point
     // (with per-stage timing on: from the end of the attention, so that no stage overlaps another)
     if (!c->timing) CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
@@ -856,6 +909,7 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     return ADORE_ERR_STATE;       // no step open, or one opened by adore_step_begin
   }
   if (layer != 0) {
+    if (wait_rebuild(c, layer, c->stream) != ADORE_OK) return ADORE_ERR_CUDA;
     adore_status_t st = f.dtype == ADORE_F32 ? launch_attention<float>(c, layer, q, k_new, v_new, out, weights, true)
                                              : launch_attention<__nv_bfloat16>(c, layer, q, k_new, v_new, out, weights, true);
     if (st != ADORE_OK || !from_attention) return st;
@@ -890,6 +944,7 @@ adore_status_t adore_step_begin(adore_cache_t* c, const void* x_new, const int32
   // nothing of this step has run yet: selection and controller start side by side, the main stream waits for the
   // selection (the rebuild and the attention of the step read its map) and for the kernel that reads x_new
   cudaStream_t sel = c->timing ? c->stream : c->aux;
+  if (join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
   if (sel != c->stream) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_fork, 0));
   CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
@@ -988,10 +1043,38 @@ adore_status_t adore_rebuild(adore_cache_t* c, int32_t layer, const void* x_tabl
   if (!c || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
   if (!c->w_kv[layer] || !c->step_layer0_done) return ADORE_ERR_STATE;
   const adore_config_t& f = c->cfg;
-  if (f.dtype == ADORE_F32)
-    return launch_rebuild<float>(c, layer, x_table, c->row_b, c->row_tok, c->row_slot, c->row_total, f.batch * f.rebuild_max, true);
-  return launch_rebuild<__nv_bfloat16>(c, layer, x_table, c->row_b, c->row_tok, c->row_slot, c->row_total,
-                                       f.batch * f.rebuild_max, true);
+  // Attend-first order with several layers: this layer's rows are next read by the next step's attention of this
+  // layer, so the rebuild goes to its own stream, behind everything queued so far (this layer's attention, the
+  // selection, the new token's row), and the attention of the following layers runs beside it. (Not with per-stage
+  // timing on, where stages must not overlap, and not in the rebuild-first order, whose attention reads these rows.)
+  static const bool inline_only = std::getenv("ADORE_REBUILD_INLINE") != nullptr;   // A/B switch
+  const bool beside = c->rb && !c->timing && !inline_only && c->step_layer0_done == 1 && f.batch * f.rebuild_max > 0;
+  cudaStream_t stream = c->stream;
+  if (beside) {
+    CUDA_OK(cudaEventRecord(c->ev_rb_fork, c->stream));
+    CUDA_OK(cudaStreamWaitEvent(c->rb, c->ev_rb_fork, 0));
+    stream = c->rb;
+  } else if (join_rebuilds(c) != ADORE_OK) {
+    return ADORE_ERR_CUDA;
+  }
+  adore_status_t st =
+      f.dtype == ADORE_F32
+          ? launch_rebuild<float>(c, layer, x_table, c->row_b, c->row_tok, c->row_slot, c->row_total, f.batch * f.rebuild_max, true, stream)
+          : launch_rebuild<__nv_bfloat16>(c, layer, x_table, c->row_b, c->row_tok, c->row_slot, c->row_total,
+                                          f.batch * f.rebuild_max, true, stream);
+  if (beside) {
+    // recorded even after a failed launch: what did get queued on the side stream must be waited for all the same
+    if (cudaEventRecord(c->ev_rebuilt[layer], c->rb) != cudaSuccess) return ADORE_ERR_CUDA;
+    c->rb_pending[layer] = 1;
+    c->rb_last = layer;
+  }
+  return st;
+}
+
+adore_status_t adore_cache_join(adore_cache_t* c) {
+  if (!c) return ADORE_ERR_INVALID_ARG;
+  if (join_controller(c) != ADORE_OK || join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
+  return ADORE_OK;
 }
 
 adore_status_t adore_cache_slot_map(adore_cache_t* c, const int32_t** slot_tok, const uint8_t** slot_role) {
@@ -1025,6 +1108,7 @@ adore_status_t adore_cache_scores(adore_cache_t* c, const float** score, const f
 
 adore_status_t adore_cache_kv(adore_cache_t* c, int32_t layer, const void** k, const void** v) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;   // the rows may still be on their way on the side stream
   const size_t off = size_t(layer) * c->cfg.batch * c->cfg.n_heads * c->cfg.capacity * c->cfg.head_dim * c->esz;
   if (k) *k = static_cast<const unsigned char*>(c->Kc) + off;
   if (v) *v = static_cast<const unsigned char*>(c->Vc) + off;
@@ -1037,12 +1121,14 @@ int64_t adore_cache_launch_count(const adore_cache_t* c) { return c ? c->launche
 
 adore_status_t adore_cache_set_stage_timing(adore_cache_t* c, int32_t enable) {
   if (!c) return ADORE_ERR_INVALID_ARG;
+  if (join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   c->timing = enable != 0;
   return ADORE_OK;
 }
 
 adore_status_t adore_cache_stage_times(adore_cache_t* c, double* ms, int64_t* launches) {
   if (!c || !ms || !launches) return ADORE_ERR_INVALID_ARG;
+  if (join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
   for (size_t i = 0; i < c->ev_stage.size(); ++i) {
     float t = 0.f;
@@ -1063,6 +1149,7 @@ adore_status_t adore_cache_stage_times(adore_cache_t* c, double* ms, int64_t* la
 
 adore_status_t adore_cache_rebuild_rows(adore_cache_t* c, int64_t* rows) {
   if (!c || !rows) return ADORE_ERR_INVALID_ARG;
+  if (join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
   unsigned long long v = 0;
   if (cudaMemcpy(&v, c->rows_accum, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return ADORE_ERR_CUDA;
@@ -1117,7 +1204,7 @@ adore_status_t adore_cache_export_state(adore_cache_t* c, void* host_buf, size_t
   if (*bytes < need) { *bytes = need; return ADORE_ERR_INVALID_ARG; }
   *bytes = need;
   // the side stream's work is joined into the main stream by the calls that use it; wait for both anyway
-  if (join_controller(c) != ADORE_OK) return ADORE_ERR_CUDA;
+  if (join_controller(c) != ADORE_OK || join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
   if (c->aux && cudaStreamSynchronize(c->aux) != cudaSuccess) return ADORE_ERR_CUDA;
   if (c->ctl && cudaStreamSynchronize(c->ctl) != cudaSuccess) return ADORE_ERR_CUDA;
@@ -1152,7 +1239,7 @@ adore_status_t adore_cache_import_state(adore_cache_t* c, const void* host_buf, 
   size_t need = sizeof(StateHeader);
   for (const StateSection& s : sec) need += pad8(s.bytes);
   if (bytes < need) return ADORE_ERR_INVALID_ARG;
-  if (join_controller(c) != ADORE_OK) return ADORE_ERR_CUDA;
+  if (join_controller(c) != ADORE_OK || join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
   if (c->aux && cudaStreamSynchronize(c->aux) != cudaSuccess) return ADORE_ERR_CUDA;
   if (c->ctl && cudaStreamSynchronize(c->ctl) != cudaSuccess) return ADORE_ERR_CUDA;
@@ -1199,7 +1286,7 @@ adore_status_t adore_label_tokens(const float* weights, int32_t n_layers, int32_
 
 adore_status_t adore_cache_sync_status(adore_cache_t* c) {
   if (!c) return ADORE_ERR_INVALID_ARG;
-  if (join_controller(c) != ADORE_OK) return ADORE_ERR_CUDA;
+  if (join_controller(c) != ADORE_OK || join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
   unsigned word = 0;
   if (cudaMemcpy(&word, c->err, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return ADORE_ERR_CUDA;

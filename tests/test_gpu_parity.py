@@ -59,6 +59,16 @@ def test_three_layers_with_their_own_inputs():
     _run(SMALL.scaled(name="L3", n_layers=3, batch=2, per_layer_inputs=True, seed=109, steps=20))
 
 
+def test_rebuilds_beside_the_following_layers_without_a_host_wait_between_steps():
+    """In a cache of several layers the rebuild of a layer runs on the library's own stream beside the attention of the
+    layers after it (and of the next step's first layers). The state is only read every fifth step here, so nothing but
+    the library's own stream dependencies orders the rebuilds against the next step's selection, gather and attention."""
+    _run(SMALL.scaled(name="L4_free_running", n_layers=4, batch=2, per_layer_inputs=True, seed=150, steps=20), state_every=5)
+    _run(SMALL.scaled(name="L3_explicit_free_running", n_layers=3, batch=4, n_heads=8, per_layer_inputs=True, rebuild_mode="explicit",
+                      rebuild_p=0.5, rebuild_max=30, capacity=64, topk=20, prompt=100, seed=151, steps=15), state_every=5)
+    _run(SMALL.scaled(name="L2_store_rows_free_running", n_layers=2, batch=2, seed=152, steps=15), state_every=15)
+
+
 def test_host_buffer_entry_point():
     _run(SMALL.scaled(name="host_entry", steps=12, seed=110), host_entry=True)
     _run(wl.get_config(1).scaled(steps=40), host_entry=True)
