@@ -438,7 +438,9 @@ adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, co
     // Rows gathered from the token store for this step's table serve every layer that rebuilds from the store.
     const bool from_store = step_table && x_table == nullptr && size_t(m_max) <= c->tc.a_rows;
     int launched = 0;
-    cudaError_t e = launch_rebuild_tc(c->tc, p, layer, m_max, stream, &launched, from_store && c->rows_gathered);
+    static const int lean_mode = std::getenv("ADORE_REBUILD_LEAN") ? std::atoi(std::getenv("ADORE_REBUILD_LEAN")) : 1;   // A/B switch
+    cudaError_t e = launch_rebuild_tc(c->tc, p, layer, m_max, stream, &launched, from_store && c->rows_gathered,
+                                      lean_mode != 0 && stream != c->stream);
     c->launches += launched;
     c->rows_gathered = from_store;
     CUDA_OK(e);

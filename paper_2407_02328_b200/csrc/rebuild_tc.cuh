@@ -161,9 +161,13 @@ struct TcGemmParams {
   unsigned* unit_cnt;         // [tiles (x 2 CTAs of a pair)][4 lane quarters], zero between launches
 };
 
-template <int BN>
+// STAGES: 4 (256-wide tiles) or 6 (128-wide) fill the SM's shared memory; the 128-wide kernel also exists with 3
+// stages (97 KB), which leaves room for CTAs of another kernel on the same SM when a small rebuild runs beside the
+// attention of the following layers.
+constexpr int kTcLeanStages = 3;
+template <int BN, int STAGES = (BN == 256 ? 4 : 6)>
 struct TcSmem {
-  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static constexpr int kStages = STAGES;
   static constexpr int kABytes = kTcBM * kTcBK * 2;
   static constexpr int kBBytes = BN * kTcBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
@@ -287,10 +291,10 @@ __device__ __forceinline__ bool tc_split_arrive(const TcGemmParams& p, uint32_t 
   return last;
 }
 
-template <int BN>
+template <int BN, int STAGES = (BN == 256 ? 4 : 6)>
 __global__ void __launch_bounds__(kTcThreads, 1)
 rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const TcGemmParams p) {
-  using S = TcSmem<BN>;
+  using S = TcSmem<BN, STAGES>;
   constexpr int kStages = S::kStages;
   constexpr uint32_t kTmemCols = 2 * BN;                  // two fp32 accumulators of BN columns
   extern __shared__ __align__(1024) unsigned char tc_smem_raw[];
@@ -514,7 +518,9 @@ inline adore_status_t tc_init(TcState& s, const adore_config_t& f, std::vector<v
   s.map_w128.resize(f.n_layers);
   s.has_w.assign(f.n_layers, 0);
   if (cudaFuncSetAttribute(rebuild_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(TcSmem<256>::kTotal)) != cudaSuccess ||
-      cudaFuncSetAttribute(rebuild_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(TcSmem<128>::kTotal)) != cudaSuccess)
+      cudaFuncSetAttribute(rebuild_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(TcSmem<128>::kTotal)) != cudaSuccess ||
+      cudaFuncSetAttribute(rebuild_tc_kernel<128, kTcLeanStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(TcSmem<128, kTcLeanStages>::kTotal)) != cudaSuccess)
     return ADORE_ERR_CUDA;
   // the two-SM kernel needs pairs of SMs that can host a cluster of two 1-CTA-per-SM blocks
   if (s.N % kPairBN == 0 && std::getenv("ADORE_REBUILD_ONE_SM") == nullptr &&
@@ -543,7 +549,7 @@ inline adore_status_t tc_set_weights(TcState& s, int layer, const void* w_kv) {
 
 // Gathers the rows and runs the GEMM, in chunks of at most a_rows rows. Returns the launches made.
 template <typename T>
-inline cudaError_t launch_rebuild_tc(TcState&, const RebuildParams<T>&, int, int, cudaStream_t, int*, bool) { return cudaErrorNotSupported; }
+inline cudaError_t launch_rebuild_tc(TcState&, const RebuildParams<T>&, int, int, cudaStream_t, int*, bool, bool = false) { return cudaErrorNotSupported; }
 template <typename T>
 inline cudaError_t launch_gather_tc(TcState&, const RebuildParams<T>&, int, cudaStream_t) { return cudaErrorNotSupported; }
 
@@ -557,8 +563,9 @@ inline cudaError_t launch_gather_tc<__nv_bfloat16>(TcState& s, const RebuildPara
 
 template <>
 inline cudaError_t launch_rebuild_tc<__nv_bfloat16>(TcState& s, const RebuildParams<__nv_bfloat16>& rp, int layer, int m_max,
-                                                    cudaStream_t stream, int* launched, bool rows_in_place) {
+                                                    cudaStream_t stream, int* launched, bool rows_in_place, bool lean) {
   // rows_in_place: the A buffer already holds the listed rows (gathered earlier for this row table; one chunk only)
+  // lean: the launch runs beside another kernel; a weight-streaming (128-wide) launch then takes the small ring
   *launched = 0;
   if (!s.has_w[layer]) return cudaErrorInvalidValue;
   // the table may hold more rows than the gather buffer: go through it in chunks
@@ -597,6 +604,9 @@ inline cudaError_t launch_rebuild_tc<__nv_bfloat16>(TcState& s, const RebuildPar
     if (plan.kind == 1)
       e = launch_dependent(rebuild_tc_kernel<256>, dim3(plan.grid), dim3(kTcThreads), TcSmem<256>::kTotal, stream, s.map_a,
                            s.map_w256[layer], g);
+    else if (lean)
+      e = launch_dependent(rebuild_tc_kernel<128, kTcLeanStages>, dim3(plan.grid), dim3(kTcThreads),
+                           TcSmem<128, kTcLeanStages>::kTotal, stream, s.map_a, s.map_w128[layer], g);
     else
       e = launch_dependent(rebuild_tc_kernel<128>, dim3(plan.grid), dim3(kTcThreads), TcSmem<128>::kTotal, stream, s.map_a,
                            s.map_w128[layer], g);
