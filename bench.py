@@ -591,7 +591,7 @@ def main():
 
     K, W = args.steps, args.warmup
     with_e2e = not args.no_e2e and args.order == "attend-first"
-    total = W + K + (K if with_e2e else 0) + K          # warm-up, timed, end-to-end, per-stage pass
+    total = W + K                                       # warm-up and timed steps; the other passes replay the timed ones
     run = DeviceRun(cfg, total, rank, args.order, args.score_source)
     flush = None
     if kv_bytes(cfg) <= 2.5e8:
@@ -605,6 +605,24 @@ def main():
     for _ in range(W):
         run.step()
     lib.adore_cache_sync_status(run.handle)
+
+    # The end-to-end pass and the per-stage pass below replay the SAME K steps as the timed region: the small state
+    # (slot maps, token table, scores) is snapshotted here and put back before each of them, so that all three see the
+    # same list lengths and occupancy. The K/V rows are copied aside and put back too (on the device): on rows that do
+    # not belong to the restored maps the attention kernel measured ~4 % slower.
+    snap = np.zeros(lib.adore_cache_export_state(run.handle, None), np.uint8)
+    lib.adore_cache_export_state(run.handle, snap)
+    next0 = run.next
+    kv_shape = (cfg.n_layers, cfg.batch, cfg.n_heads, cfg.capacity, cfg.head_dim)
+    kv_live = [lib.device_view(p, kv_shape, run.dt) for p in lib.adore_cache_kv(run.handle, 0)]
+    kv_keep = [t.clone() for t in kv_live]
+
+    def rewind():
+        lib.adore_cache_import_state(run.handle, snap)
+        for live, keep in zip(kv_live, kv_keep):
+            live.copy_(keep)
+        torch.cuda.synchronize()
+        run.next = next0
 
     # ---- timed region: K steps, device time, max over ranks ----
     launches0 = lib.adore_cache_launch_count(run.handle)
@@ -642,6 +660,7 @@ def main():
     # ---- end to end through the host-buffer entry point ----
     e2e = None
     if with_e2e:
+        rewind()
         run.make_host_inputs(run.next, K)
         barrier()
         t0 = time.perf_counter()
@@ -654,6 +673,7 @@ def main():
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     # ---- per-stage pass (events around every launch) for the roofline figures ----
+    rewind()
     rows0 = lib.adore_cache_rebuild_rows(run.handle)
     lib.adore_cache_set_stage_timing(run.handle, True)
     lib.adore_cache_stage_times(run.handle)
