@@ -125,7 +125,7 @@ def compare_attention(rep: Report, cfg, q, orc: ao.AdoreOracle, layer, k_new, at
     keep_g, keep_o = w_g > 0, w_o > 0
     rep.topk_rows += keep_o.shape[0] * keep_o.shape[1]
     bad = np.argwhere((keep_g != keep_o).any(-1))
-    # Where the two kept sets differ by a tie (each case is judged below), the outputs differ by the weight that moved
+    # Where the two kept sets differ by a tie (each case is classified below), the outputs differ by the weight that moved
     # times the value rows it moved between: |out_g - out_o| <= sum_s |w_g - w_o|_s * max|v|. Everywhere else the plain
     # bound holds.
     if len(bad):
@@ -150,7 +150,7 @@ def compare_attention(rep: Report, cfg, q, orc: ao.AdoreOracle, layer, k_new, at
         else:
             # Rebuilt cache rows may differ from the oracle's by one unit in the last place (float32
             # against float64 accumulation before the rounding; checked by compare_state). Such a row
-            # moves its logit by far more than 1e-6, so the GPU's choice is judged on the rows it
+            # moves its logit by far more than 1e-6, so the GPU's choice is checked on the rows it
             # actually holds: with float64 logits of ITS cache bytes the kept set must be the top K.
             assert gpu_k is not None, f"top-K sets differ beyond a near-tie: gap {gap:.3e} scale {scale:.3e}"
             Kg = gpu_k()[b, h].astype(np.float64)
