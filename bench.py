@@ -341,7 +341,7 @@ class DeviceRun:
         self.h = dict(q=pin(self.q[sl]), k=pin(self.k[sl]), v=pin(self.v[sl]), x=pin(self.x[sl]),
                       lists=None if self.lists is None else pin(self.lists[sl]),
                       counts=None if self.counts is None else pin(self.counts[sl]),
-                      out=t.empty(self.out.shape, dtype=self.dt).pin_memory())
+                      out=t.empty((self.cfg.n_layers,) + tuple(self.out.shape), dtype=self.dt).pin_memory())
         self.h_first = first
         # host addresses taken once: the timed loop passes integers only
         h = self.h
@@ -351,16 +351,20 @@ class DeviceRun:
                        x=[h["x"][i, 0].data_ptr() for i in range(count)],
                        lists=None if h["lists"] is None else [h["lists"][i].data_ptr() for i in range(count)],
                        counts=None if h["counts"] is None else [h["counts"][i].data_ptr() for i in range(count)],
-                       out=h["out"].data_ptr())
+                       out=[h["out"][l].data_ptr() for l in range(self.cfg.n_layers)])
 
     def step_host(self):
         lib, c, s = self.lib, self.cfg, self.next
         i, hp = s - self.h_first, self.hp
         pl = None if hp["lists"] is None else hp["lists"][i]
         pc = None if hp["counts"] is None else hp["counts"][i]
+        # the calls of all layers are queued back to back (each layer has its own `out` buffer on the host), then the
+        # host waits once for the step's results
         for l in range(c.n_layers):
-            lib.adore_decode_rebuild_host(self.handle, l, hp["q"][i][l], hp["k"][i][l], hp["v"][i][l], hp["x"][i], pl, pc,
-                                          self.r_in, self.pt[l] if (self.pt is not None and l > 0) else None, hp["out"], self.pw)
+            lib.adore_decode_rebuild_host_queued(self.handle, l, hp["q"][i][l], hp["k"][i][l], hp["v"][i][l], hp["x"][i], pl, pc,
+                                                 self.r_in, self.pt[l] if (self.pt is not None and l > 0) else None,
+                                                 hp["out"][l], self.pw)
+        lib.adore_cache_wait_outputs(self.handle)
         self.next += 1
 
     def host_bytes_per_step(self):

@@ -183,6 +183,24 @@ adore_status_t adore_decode_rebuild_host(adore_cache_t *cache, int32_t layer, co
                                          const int32_t *explicit_count, int32_t r_in, const void *x_table, void *out,
                                          float *weights);
 
+/* The same step and rebuild (Sections 2.1-2.3) with HOST buffers, QUEUED: the call returns without waiting for
+ * anything, so the calls of all layers of a step (and of the next steps) can be issued back to back and the host
+ * waits once, with adore_cache_wait_outputs (or adore_cache_sync_status), before it reads the `out` buffers. Every layer has a staging set of its own
+ * on the device; its upload waits (on the device) for the previous step's use of that set. All host buffers must be
+ * pinned for the copies to be asynchronous and must stay valid and unchanged until that wait; `out` of different calls
+ * in flight must be different buffers. Arguments and errors as for adore_decode_rebuild_host. The first call
+ * allocates the staging sets. */
+adore_status_t adore_decode_rebuild_host_queued(adore_cache_t *cache, int32_t layer, const void *q, const void *k_new,
+                                                const void *v_new, const void *x_new, const int32_t *explicit_list,
+                                                const int32_t *explicit_count, int32_t r_in, const void *x_table,
+                                                void *out, float *weights);
+
+/* Host-side wait for the `out` buffers of every adore_decode_rebuild_host_queued call issued so far (Section 2.1's
+ * attention output of each layer), and for nothing else: the rebuilds queued by those calls may still be running,
+ * and the next step's calls can be issued beside them. By then the host input buffers of those calls have been read
+ * too. Does not report the device error word (adore_cache_sync_status does). Errors: INVALID_ARG, CUDA. */
+adore_status_t adore_cache_wait_outputs(adore_cache_t *cache);
+
 /* Rebuild for one layer (Section 2.3): Y = X_L [W_k ; W_v]^T for the rows of this step's rebuild
  * list, rotary embedding on the key half at each token's original position, rounding to T and
  * scatter into the list's slots. x_table: device T[B, max_tokens, d] rows indexed by token

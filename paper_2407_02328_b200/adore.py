@@ -56,7 +56,7 @@ EXPORTS = ["adore_cache_create", "adore_cache_destroy", "adore_cache_set_project
            "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows",
            "adore_controller_score_static", "adore_probe_read_bandwidth",
            "adore_cache_export_state", "adore_cache_import_state", "adore_step_begin", "adore_attend_rows",
-           "adore_label_tokens", "adore_decode_rebuild_host"]
+           "adore_label_tokens", "adore_decode_rebuild_host", "adore_decode_rebuild_host_queued", "adore_cache_wait_outputs"]
 
 
 def _lib():
@@ -77,6 +77,7 @@ def _lib():
         lib.adore_decode_step.argtypes = step
         lib.adore_decode_step_host.argtypes = step
         lib.adore_decode_rebuild_host.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
+        lib.adore_decode_rebuild_host_queued.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         lib.adore_rebuild.argtypes = [vp, i32, vp]
         lib.adore_step_begin.argtypes = [vp, vp, vp, vp, i32]
         lib.adore_label_tokens.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
@@ -92,6 +93,7 @@ def _lib():
         lib.adore_cache_launch_count.restype = C.c_int64
         lib.adore_cache_sync_status.argtypes = [vp]
         lib.adore_cache_join.argtypes = [vp]
+        lib.adore_cache_wait_outputs.argtypes = [vp]
         lib.adore_cache_set_stage_timing.argtypes = [vp, i32]
         lib.adore_cache_stage_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         lib.adore_cache_rebuild_rows.argtypes = [vp, C.POINTER(C.c_int64)]
@@ -167,6 +169,13 @@ def adore_decode_rebuild_host(cache: int, layer: int, q, k_new, v_new, x_new, ex
                                             _ptr(weights)), "adore_decode_rebuild_host")
 
 
+def adore_decode_rebuild_host_queued(cache: int, layer: int, q, k_new, v_new, x_new, explicit_list, explicit_count,
+                                     r_in: int, x_table, out, weights=None) -> None:
+    _check(_lib().adore_decode_rebuild_host_queued(cache, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(x_new),
+                                                   _ptr(explicit_list), _ptr(explicit_count), r_in, _ptr(x_table), _ptr(out),
+                                                   _ptr(weights)), "adore_decode_rebuild_host_queued")
+
+
 def adore_step_begin(cache: int, x_new, explicit_list, explicit_count, r_in: int) -> None:
     _check(_lib().adore_step_begin(cache, _ptr(x_new), _ptr(explicit_list), _ptr(explicit_count), r_in), "adore_step_begin")
 
@@ -222,6 +231,10 @@ def adore_cache_launch_count(cache: int) -> int:
 
 def adore_cache_join(cache: int) -> None:
     _check(_lib().adore_cache_join(cache), "adore_cache_join")
+
+
+def adore_cache_wait_outputs(cache: int) -> None:
+    _check(_lib().adore_cache_wait_outputs(cache), "adore_cache_wait_outputs")
 
 
 def adore_cache_sync_status(cache: int) -> None:

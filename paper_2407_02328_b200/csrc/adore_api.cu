@@ -175,6 +175,13 @@ struct adore_cache {
   void *h_q = nullptr, *h_k = nullptr, *h_v = nullptr, *h_x = nullptr, *h_out = nullptr;
   int* h_list = nullptr;
   int* h_count = nullptr;
+  // staging of the queued host-buffer entry point: one set per layer (several layers' calls are in flight at once)
+  unsigned char* hq_all = nullptr;              // [L][4][B*H*dh] elements: q, k, v, out
+  void* hq_x = nullptr;
+  int* hq_list = nullptr;
+  int* hq_count = nullptr;
+  std::vector<cudaEvent_t> ev_stage_free;       // per layer: every reader of the layer's staging set is done
+  cudaStream_t d2h = nullptr;                   // `out` goes back on its own stream, beside the next layer's attention
   std::vector<void*> owned;
 };
 
@@ -774,6 +781,7 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (c->aux) { cudaStreamSynchronize(c->aux); cudaStreamDestroy(c->aux); }
   if (c->ctl) { cudaStreamSynchronize(c->ctl); cudaStreamDestroy(c->ctl); }
   if (c->rb) { cudaStreamSynchronize(c->rb); cudaStreamDestroy(c->rb); }
+  if (c->d2h) { cudaStreamSynchronize(c->d2h); cudaStreamDestroy(c->d2h); }
   if (c->ev_rb_fork) cudaEventDestroy(c->ev_rb_fork);
   for (cudaEvent_t e : c->ev_rebuilt) cudaEventDestroy(e);
   if (c->ev_gates) cudaEventDestroy(c->ev_gates);
@@ -785,7 +793,8 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   for (void* p : c->owned) cudaFree(p);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
-  void* hosts[] = {c->h_q, c->h_k, c->h_v, c->h_x, c->h_out, c->h_list, c->h_count};
+  for (cudaEvent_t e : c->ev_stage_free) cudaEventDestroy(e);
+  void* hosts[] = {c->h_q, c->h_k, c->h_v, c->h_x, c->h_out, c->h_list, c->h_count, c->hq_all, c->hq_x, c->hq_list, c->hq_count};
   for (void* p : hosts) if (p) cudaFree(p);
   cudaGetLastError();
   delete c;
@@ -1041,6 +1050,65 @@ adore_status_t adore_decode_rebuild_host(adore_cache_t* c, int32_t layer, const 
   return decode_step_host_impl(c, layer, q, k_new, v_new, x_new, explicit_list, explicit_count, r_in, out, weights, true, x_table);
 }
 
+adore_status_t adore_decode_rebuild_host_queued(adore_cache_t* c, int32_t layer, const void* q, const void* k_new,
+                                                const void* v_new, const void* x_new, const int32_t* explicit_list,
+                                                const int32_t* explicit_count, int32_t r_in, const void* x_table, void* out,
+                                                float* weights) {
+  if (!c || !q || !k_new || !v_new || !out || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (!c->w_kv[layer]) return ADORE_ERR_STATE;
+  const adore_config_t& f = c->cfg;
+  const size_t qb = size_t(f.batch) * f.n_heads * f.head_dim * c->esz, xb = size_t(f.batch) * f.hidden * c->esz;
+  if (r_in < 0 || r_in > f.max_tokens) return ADORE_ERR_INVALID_ARG;
+  if (layer == 0 && !x_new) return ADORE_ERR_INVALID_ARG;
+  if (!c->hq_all) {
+    CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->hq_all), size_t(f.n_layers) * 4 * qb));
+    CUDA_OK(cudaMalloc(&c->hq_x, xb));
+    CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->hq_list), size_t(f.batch) * f.max_tokens * sizeof(int)));
+    CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->hq_count), size_t(f.batch) * sizeof(int)));
+    CUDA_OK(cudaStreamCreateWithFlags(&c->d2h, cudaStreamNonBlocking));
+    for (int l = 0; l < f.n_layers; ++l) {
+      cudaEvent_t e = nullptr;
+      CUDA_OK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+      c->ev_stage_free.push_back(e);
+      CUDA_OK(cudaEventRecord(e, c->stream));
+    }
+  }
+  unsigned char* set = c->hq_all + size_t(layer) * 4 * qb;
+  void *dq = set, *dk = set + qb, *dv = set + 2 * qb, *dout = set + 3 * qb;
+  // the layer's staging set is free once the previous step's kernels that read it (and the copy of its `out`) are done
+  CUDA_OK(cudaStreamWaitEvent(c->copy, c->ev_stage_free[layer], 0));
+  CUDA_OK(cudaMemcpyAsync(dq, q, qb, cudaMemcpyHostToDevice, c->copy));
+  CUDA_OK(cudaMemcpyAsync(dk, k_new, qb, cudaMemcpyHostToDevice, c->copy));
+  CUDA_OK(cudaMemcpyAsync(dv, v_new, qb, cudaMemcpyHostToDevice, c->copy));
+  const bool lists = layer == 0 && explicit_list && explicit_count && r_in > 0;
+  if (layer == 0) {
+    CUDA_OK(cudaMemcpyAsync(c->hq_x, x_new, xb, cudaMemcpyHostToDevice, c->copy));
+    if (lists) {
+      CUDA_OK(cudaMemcpyAsync(c->hq_list, explicit_list, size_t(f.batch) * r_in * sizeof(int), cudaMemcpyHostToDevice, c->copy));
+      CUDA_OK(cudaMemcpyAsync(c->hq_count, explicit_count, size_t(f.batch) * sizeof(int), cudaMemcpyHostToDevice, c->copy));
+    }
+  }
+  CUDA_OK(cudaEventRecord(c->ev_copy, c->copy));
+  CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_copy, 0));
+  adore_status_t st = adore_decode_step(c, layer, dq, dk, dv, c->hq_x, lists ? c->hq_list : nullptr,
+                                        lists ? c->hq_count : nullptr, lists ? r_in : 0, dout, weights);
+  if (st != ADORE_OK) return st;
+  // by now the main stream is behind every kernel of this call that reads the staging set (the side streams were
+  // joined inside adore_decode_step); `out` travels on its own stream, so that the next layer's attention follows
+  // this one directly
+  CUDA_OK(cudaEventRecord(c->ev_out, c->stream));
+  CUDA_OK(cudaStreamWaitEvent(c->d2h, c->ev_out, 0));
+  CUDA_OK(cudaMemcpyAsync(out, dout, qb, cudaMemcpyDeviceToHost, c->d2h));
+  CUDA_OK(cudaEventRecord(c->ev_stage_free[layer], c->d2h));
+  return adore_rebuild(c, layer, x_table);
+}
+
+adore_status_t adore_cache_wait_outputs(adore_cache_t* c) {
+  if (!c) return ADORE_ERR_INVALID_ARG;
+  if (c->d2h && cudaStreamSynchronize(c->d2h) != cudaSuccess) return ADORE_ERR_CUDA;
+  return ADORE_OK;
+}
+
 adore_status_t adore_rebuild(adore_cache_t* c, int32_t layer, const void* x_table) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
   if (!c->w_kv[layer] || !c->step_layer0_done) return ADORE_ERR_STATE;
@@ -1290,6 +1358,7 @@ adore_status_t adore_cache_sync_status(adore_cache_t* c) {
   if (!c) return ADORE_ERR_INVALID_ARG;
   if (join_controller(c) != ADORE_OK || join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
+  if (c->d2h && cudaStreamSynchronize(c->d2h) != cudaSuccess) return ADORE_ERR_CUDA;   // queued `out` copies
   unsigned word = 0;
   if (cudaMemcpy(&word, c->err, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return ADORE_ERR_CUDA;
   if (word != 0) {

@@ -293,6 +293,77 @@ def run_parity(cfg: wl.WorkloadConfig, batch: Optional[int] = None, steps: Optio
     return rep
 
 
+def run_parity_queued_host(cfg: wl.WorkloadConfig, steps: Optional[int] = None, sync_every: int = 1) -> Report:
+    """Parity of adore_decode_rebuild_host_queued: per step the calls of ALL layers are issued back to back from pinned
+    host buffers, the host waits once every `sync_every` steps, and only then are the outputs of those steps compared
+    with the oracle's, layer by layer (every call in flight has `out`, `weights` and input buffers of its own)."""
+    w = Workload(cfg, None)
+    orc = make_oracle(w)
+    g = GpuCache(w)
+    rep = Report()
+    L = cfg.n_layers
+    pin = lambda a: to_dev(a, cfg).cpu().pin_memory()
+    try:
+        tables = otab = None
+        if cfg.prompt:
+            xp = w.prompt()
+            orc.append_tokens(xp)
+            lib.adore_cache_append_tokens(g.handle, to_dev(xp, cfg), cfg.prompt)
+        if cfg.per_layer_inputs:
+            tables = [torch.zeros((g.B, cfg.max_tokens, cfg.hidden), dtype=torch_dtype(cfg), device="cuda") for _ in range(L)]
+            otab = [np.zeros((g.B, cfg.max_tokens, cfg.hidden), np.float32) for _ in range(L)]
+            # the tables hold every row of the run from the start: a queued rebuild reads them while later steps are issued
+            n_all = cfg.prompt + (cfg.steps if steps is None else steps)
+            for l in range(L):
+                for t0 in range(0, n_all, 64):
+                    rows = wl.hidden_rows(cfg, t0, min(64, n_all - t0), l, g.B)
+                    otab[l][:, t0:t0 + rows.shape[1]] = rows
+                tables[l].copy_(to_dev(otab[l], cfg))
+                if l > 0 and cfg.prompt:
+                    orc.fill_layer(l, otab[l])
+                    lib.adore_cache_fill_layer(g.handle, l, tables[l])
+        lib.adore_cache_sync_status(g.handle)
+        n_steps = cfg.steps if steps is None else steps
+        pending = []
+        for s in range(n_steps):
+            n = cfg.prompt + s
+            lists, counts = w.explicit(s, n)
+            hl = None if lists is None else torch.from_numpy(lists).pin_memory()
+            hc = None if counts is None else torch.from_numpy(counts).pin_memory()
+            calls = []
+            for l in range(L):
+                x = w.x_new(n, l if cfg.per_layer_inputs else 0)
+                q, k, v = w.qkv(n, l, x)
+                hq, hk, hv, hx = pin(q), pin(k), pin(v), pin(x)
+                hout = torch.zeros((g.B, cfg.n_heads, cfg.head_dim), dtype=torch_dtype(cfg)).pin_memory()
+                wts = torch.empty((g.B, cfg.n_heads, cfg.capacity + 1), dtype=torch.float32, device="cuda")
+                lib.adore_decode_rebuild_host_queued(g.handle, l, hq, hk, hv, hx if l == 0 else None, hl if l == 0 else None,
+                                                     hc if l == 0 else None, w.r_in if l == 0 else 0,
+                                                     tables[l] if (cfg.per_layer_inputs and l > 0) else None, hout, wts)
+                calls.append((q, k, v, x, hout, wts, (hq, hk, hv, hx, hl, hc)))
+            pending.append((lists, counts, calls))
+            if (s + 1) % sync_every and s != n_steps - 1:
+                continue
+            lib.adore_cache_wait_outputs(g.handle)      # the outputs are in; the rebuilds may still be running
+            for lists_p, counts_p, calls_p in pending:
+                ex = explicit_as_lists(lists_p, counts_p)
+                for l, (q, k, v, x, hout, wts, _keep) in enumerate(calls_p):
+                    attn_map = orc.slot_tok.copy() if l == 0 else orc.attn_slot_tok.copy()
+                    K_before = orc.Kc[l].copy()
+                    out_o, w_o = orc.decode_step(l, q, k, v, x if l == 0 else None, ex if l == 0 else None)
+                    compare_attention(rep, cfg, q, orc, l, k, attn_map, hout.float().numpy(), wts.cpu().numpy(), out_o, w_o,
+                                      K_before, gpu_k=None, admit_slot=orc.info.admit_slot)
+                    orc.rebuild(l, otab[l] if (cfg.per_layer_inputs and l > 0) else None)
+                rep.steps += 1
+            pending = []
+            orc.check_invariants()
+            compare_state(rep, g, orc, range(L))
+        lib.adore_cache_sync_status(g.handle)
+    finally:
+        g.close()
+    return rep
+
+
 def run_parity_rebuild_first(cfg: wl.WorkloadConfig, steps: Optional[int] = None) -> Report:
     """Free-running parity of the step in the order Section 2.3 prints it: adore_step_begin, then per layer
     adore_rebuild and adore_attend_rows (R_max + 1 query rows per sequence), against the oracle's same three calls.

@@ -77,6 +77,20 @@ def test_host_buffer_entry_point():
          host_entry="with_rebuild")
 
 
+def test_queued_host_buffer_entry_point():
+    """adore_decode_rebuild_host_queued: the calls of all layers (and of several steps) are issued without a host wait in
+    between, every layer through a staging set of its own; outputs are read after one sync."""
+    from tests.gpu_driver import run_parity_queued_host
+    for cfg, kw in ((SMALL.scaled(name="queued_L3", n_layers=3, batch=2, per_layer_inputs=True, seed=153, steps=12), dict(sync_every=1)),
+                    (SMALL.scaled(name="queued_L2_three_steps_in_flight", n_layers=2, batch=2, per_layer_inputs=True, seed=154, steps=12,
+                                  rebuild_mode="explicit", rebuild_p=0.4, rebuild_max=10), dict(sync_every=3)),
+                    (SMALL.scaled(name="queued_one_layer", seed=155, steps=10), dict(sync_every=2))):
+        rep = run_parity_queued_host(cfg, **kw)
+        print(f"\n[{cfg.name}] steps={rep.steps} near_ties={rep.near_ties}+{rep.rounding_ties}r/{rep.topk_rows} rows "
+              f"max_out_err={rep.max_out_err:.3e} max_w_err={rep.max_w_err:.3e} max_kv_ulp={rep.max_kv_ulp:.2f}")
+        assert rep.steps == cfg.steps and rep.near_ties <= 2
+
+
 def test_capacity_spanning_several_tiles_with_ragged_tail():
     _run(SMALL.scaled(name="c517", capacity=517, topk=200, rebuild_max=37, prompt=700, steps=12, batch=2,
                       n_heads=2, seed=111))
