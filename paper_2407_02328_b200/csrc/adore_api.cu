@@ -163,6 +163,7 @@ struct adore_cache {
   // waits for it.
   cudaStream_t rb = nullptr;
   cudaEvent_t ev_rb_fork = nullptr;
+  cudaEvent_t ev_step_open = nullptr;   // rebuild-first order: the main stream at the end of adore_step_begin
   std::vector<cudaEvent_t> ev_rebuilt;
   std::vector<char> rb_pending;
   int rb_last = -1;             // layer of the most recent launch on `rb` that nobody has waited for yet
@@ -736,7 +737,8 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   }
   if (f.n_layers > 1) {
     bool ok = cudaStreamCreateWithFlags(&c->rb, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaEventCreateWithFlags(&c->ev_rb_fork, cudaEventDisableTiming) == cudaSuccess;
+              cudaEventCreateWithFlags(&c->ev_rb_fork, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_step_open, cudaEventDisableTiming) == cudaSuccess;
     c->rb_pending.assign(size_t(f.n_layers), char(0));
     for (int l = 0; ok && l < f.n_layers; ++l) {
       cudaEvent_t e = nullptr;
@@ -783,6 +785,7 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (c->rb) { cudaStreamSynchronize(c->rb); cudaStreamDestroy(c->rb); }
   if (c->d2h) { cudaStreamSynchronize(c->d2h); cudaStreamDestroy(c->d2h); }
   if (c->ev_rb_fork) cudaEventDestroy(c->ev_rb_fork);
+  if (c->ev_step_open) cudaEventDestroy(c->ev_step_open);
   for (cudaEvent_t e : c->ev_rebuilt) cudaEventDestroy(e);
   if (c->ev_gates) cudaEventDestroy(c->ev_gates);
   if (c->ev_ctrl) cudaEventDestroy(c->ev_ctrl);
@@ -967,6 +970,7 @@ adore_status_t adore_step_begin(adore_cache_t* c, const void* x_new, const int32
   }
   c->joined = true;
   CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_gates, 0));
+  if (c->ev_step_open) CUDA_OK(cudaEventRecord(c->ev_step_open, c->stream));
   c->cur = 1 - c->cur;
   c->attn = c->cur;             // this step's attention reads the NEW map
   c->n += 1;
@@ -978,6 +982,7 @@ adore_status_t adore_attend_rows(adore_cache_t* c, int32_t layer, const void* q_
                                  void* out, float* weights) {
   if (!c || !q_rows || !k_new || !v_new || !out || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
   if (c->step_layer0_done != 2) return ADORE_ERR_STATE;
+  if (wait_rebuild(c, layer, c->stream) != ADORE_OK) return ADORE_ERR_CUDA;   // this layer's rows may come from the side stream
   const adore_config_t& f = c->cfg;
   const int rows_q = f.rebuild_max + 1;
   return f.dtype == ADORE_F32 ? launch_attention<float>(c, layer, q_rows, k_new, v_new, out, weights, true, rows_q)
@@ -1118,11 +1123,18 @@ adore_status_t adore_rebuild(adore_cache_t* c, int32_t layer, const void* x_tabl
   // selection, the new token's row), and the attention of the following layers runs beside it. (Not with per-stage
   // timing on, where stages must not overlap, and not in the rebuild-first order, whose attention reads these rows.)
   static const bool inline_only = std::getenv("ADORE_REBUILD_INLINE") != nullptr;   // A/B switch
-  const bool beside = c->rb && !c->timing && !inline_only && c->step_layer0_done == 1 && f.batch * f.rebuild_max > 0;
+  // In the rebuild-first order the attention of layer l reads what rebuild(l) writes, but rebuild(l + 1) needs only the
+  // step's selection: on the side stream it starts from the end of adore_step_begin and runs beside the attention of
+  // layer l; adore_attend_rows(l + 1) waits for it.
+  const bool beside = c->rb && !c->timing && !inline_only && c->step_layer0_done != 0 && f.batch * f.rebuild_max > 0;
   cudaStream_t stream = c->stream;
   if (beside) {
-    CUDA_OK(cudaEventRecord(c->ev_rb_fork, c->stream));
-    CUDA_OK(cudaStreamWaitEvent(c->rb, c->ev_rb_fork, 0));
+    if (c->step_layer0_done == 2) {
+      CUDA_OK(cudaStreamWaitEvent(c->rb, c->ev_step_open, 0));
+    } else {
+      CUDA_OK(cudaEventRecord(c->ev_rb_fork, c->stream));
+      CUDA_OK(cudaStreamWaitEvent(c->rb, c->ev_rb_fork, 0));
+    }
     stream = c->rb;
   } else if (join_rebuilds(c) != ADORE_OK) {
     return ADORE_ERR_CUDA;
