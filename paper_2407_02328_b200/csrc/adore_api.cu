@@ -1156,6 +1156,7 @@ adore_status_t adore_rebuild(adore_cache_t* c, int32_t layer, const void* x_tabl
 adore_status_t adore_cache_join(adore_cache_t* c) {
   if (!c) return ADORE_ERR_INVALID_ARG;
   if (join_controller(c) != ADORE_OK || join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
+  for (cudaEvent_t e : c->ev_stage_free) CUDA_OK(cudaStreamWaitEvent(c->stream, e, 0));   // queued `out` copies
   return ADORE_OK;
 }
 

@@ -249,3 +249,5 @@ def test_relative_positions_rescore_every_token_at_every_step():
     _run(SMALL.scaled(name="rel_ctrl96_L2", ctrl_hidden=96, n_layers=2, batch=2, per_layer_inputs=True, steps=12, seed=143, **rel))
     _run(SMALL.scaled(name="rel_host_entry", steps=10, seed=144, **rel), host_entry="with_rebuild")
     _run_rebuild_first(SMALL.scaled(name="rel_rows", steps=20, seed=145, **rel))
+    # config 2's shape (d = 4096, d' = 128, 512 prompt tokens re-scored every step), two of its sequences
+    _run(wl.get_config(2).scaled(name="rel_cfg2_shape", ctrl_relative_position=True), batch=2, steps=12, state_every=4)
