@@ -1,5 +1,5 @@
 """Error reporting of the C ABI on a GPU: call order, a full token table, a bad explicit entry (device error word),
-bad arguments. None of these cases faults or hangs the device: every one is caught on the host or turned into a no-op."""
+bad arguments, a cache that cannot fit. None of these cases faults or hangs the device: every one is caught on the host or turned into a no-op."""
 import numpy as np
 import pytest
 
@@ -109,5 +109,28 @@ def test_bad_explicit_entry_sets_the_device_error_word_and_is_ignored():
         with pytest.raises(lib.AdoreError) as e:              # more candidates than the selection kernel sorts
             lib.adore_decode_step(g.handle, 0, q, k, v, x, lists, counts, 9000, g.out, None)
         assert e.value.status == 8
+    finally:
+        g.close()
+
+
+def test_a_cache_that_cannot_fit_is_refused_with_out_of_memory_and_leaves_the_device_usable():
+    """One request far beyond the device's memory (several terabytes of K/V rows): the allocation itself is refused by
+    the driver, create reports OOM, frees what it had taken, and a normal cache can be made and used right after."""
+    torch, lib, w, g, to_dev = _setup()
+    try:
+        free0, _ = torch.cuda.mem_get_info()
+        with pytest.raises(lib.AdoreError) as e:
+            lib.adore_cache_create(
+                lib.make_config(batch=1024, n_layers=64, n_heads=128, head_dim=128, hidden=CFG.hidden, capacity=4096, rebuild_max=8,
+                                topk=64, max_tokens=4100, ctrl_hidden=CFG.ctrl_hidden, dtype="bf16", rebuild_mode="policy",
+                                rope_theta=1.0e4, pos_scale=4096.0),
+                w.ctrl, torch.cuda.current_stream().cuda_stream)
+        assert e.value.status == 2
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 >= free0 - (64 << 20), "the failed create kept device memory"
+        n = lib.adore_cache_num_tokens(g.handle)
+        q, k, v, x = _inputs(w, to_dev, n)
+        lib.adore_decode_step(g.handle, 0, q, k, v, x, None, None, 0, g.out, None)     # the existing cache still works
+        lib.adore_cache_sync_status(g.handle)
     finally:
         g.close()
