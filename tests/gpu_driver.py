@@ -164,8 +164,13 @@ def compare_attention(rep: Report, cfg, q, orc: ao.AdoreOracle, layer, k_new, at
             assert np.abs(lg - logit)[valid].max() <= 0.05 * scale
             rep.rounding_ties += 1
         w_ok[b, h, diff] = False
-    werr = np.abs(w_g - w_o)[w_ok]
-    assert (werr <= tol["w_abs"]).all(), f"attention weights off by {werr.max():.3e}"
+    # A cache row that sits one unit in the last place away from the oracle's (allowed by the row check in
+    # compare_state) moves its logit by |q_e| ulp(k_e) / sqrt(dh), up to ~2e-3 per element in bfloat16, and a weight w
+    # by that factor times w: the bound has a part relative to the weight, the same 1e-2 (1e-4) as for the output.
+    werr = np.abs(w_g - w_o)
+    wbound = tol["w_abs"] + tol["out_rel"] * np.abs(w_o)
+    assert (werr <= wbound)[w_ok].all(), f"attention weights off by {werr[w_ok].max():.3e}"
+    werr = werr[w_ok]
     rep.max_w_err = max(rep.max_w_err, float(werr.max()))
     s = w_g.sum(-1)
     assert np.allclose(s, 1.0, atol=1e-4), "weights do not sum to one"

@@ -144,6 +144,13 @@ def test_config2_sub_batch():
     _run(wl.get_config(2), batch=2, steps=24, state_every=4)
 
 
+def test_config2_full_length_two_sequences():
+    """All 512 decode steps of config 2 for two of its sequences (sequences are independent): 512 evictions per sequence,
+    4096 rebuilt rows, the token table filled to its last row; state compared every 32 steps."""
+    rep = _run(wl.get_config(2), batch=2, state_every=32)
+    assert rep.steps == 512
+
+
 def test_config3_full_size_in_the_benchmark_launch_configuration():
     """All 64 sequences, C=512, K=256, R_max=256, prompt 1024: the shapes and launch configurations
     `bench.py` times (persistent GEMM over ~10k rebuilt rows, 2048 attention items). Two decode steps,
