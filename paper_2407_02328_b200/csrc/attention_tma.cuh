@@ -47,6 +47,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
   const AttnSmem<DH, NT> sm(smem_raw + size_t(kRingStages) * kRingChunkBytes + 64, rows);
   float* s_logit = sm.logit;
   int* s_fail = sm.sel + 24;               // one word of the broadcast area
+  int* s_last = sm.sel + 25;               // highest occupied slot of the sequence (-1: none)
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane / LPR, li = lane % LPR;
@@ -75,6 +76,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
 #pragma unroll
     for (int s = 0; s < kRingStages; ++s) mbar_init(&full[s], 1u);
     *s_fail = 0;
+    *s_last = -1;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -89,6 +91,16 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
   };
   if (tid == 0)
     for (int c = 0; c < min(kRingStages, n_chunks); ++c) issue(c);
+  // Slots are handed out from the lowest index up, so the empty ones form a tail whenever the cache is not full: the
+  // key stream stops after the chunk that holds the highest occupied slot (found while the first chunks are on their way).
+  {
+    int last = -1;
+    for (int i = tid; i < C; i += NT)
+      if (map[i] >= 0) last = i;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+    if (lane == 0 && last >= 0) atomicMax(s_last, last);
+  }
 
   float qf[EPL];
   {
@@ -108,8 +120,12 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     if (li == 0) s_logit[C] = last_row ? dot * p.scale : -INFINITY;
   }
 
+  __syncthreads();                                           // s_last is complete
+  // chunks already issued are consumed in any case
+  const int n_used = max(min(kRingStages, n_chunks), min(n_chunks, (*s_last + CHUNK_ROWS) / CHUNK_ROWS));
+  for (int i = n_used * CHUNK_ROWS + tid; i < C; i += NT) s_logit[i] = -INFINITY;   // the empty tail is never loaded
   bool failed = false;
-  for (int c = 0; c < n_chunks; ++c) {
+  for (int c = 0; c < n_used; ++c) {
     const int stage = c % kRingStages;
     const uint32_t parity = uint32_t(c / kRingStages) & 1u;
     if (!mbar_wait_bounded(&full[stage], parity, failed ? kDrainPolls : kWaitPolls)) {
@@ -141,7 +157,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     }
     __syncthreads();                                         // everyone is done with this stage
     failed = failed || (*s_fail != 0);
-    if (tid == 0 && !failed && c + kRingStages < n_chunks) issue(c + kRingStages);
+    if (tid == 0 && !failed && c + kRingStages < n_used) issue(c + kRingStages);
   }
   // (the loop's last __syncthreads also publishes the logits)
   const int n_kept = attention_keep_and_weights<T, DH, NT>(p, sm, item);
