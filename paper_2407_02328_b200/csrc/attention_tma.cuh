@@ -95,8 +95,11 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
   // key stream stops after the chunk that holds the highest occupied slot (found while the first chunks are on their way).
   {
     int last = -1;
-    for (int i = tid; i < C; i += NT)
-      if (map[i] >= 0) last = i;
+    for (int i = tid; i < C; i += NT) {
+      const int t = map[i];
+      sm.list[i] = t;                      // the logit loop reads the map row from here (the list area is free until phase 2)
+      if (t >= 0) last = i;
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
     if (lane == 0 && last >= 0) atomicMax(s_last, last);
@@ -120,7 +123,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
     if (li == 0) s_logit[C] = last_row ? dot * p.scale : -INFINITY;
   }
 
-  __syncthreads();                                           // s_last is complete
+  __syncthreads();                                           // s_last and the staged map row are complete
   // chunks already issued are consumed in any case
   const int n_used = max(min(kRingStages, n_chunks), min(n_chunks, (*s_last + CHUNK_ROWS) / CHUNK_ROWS));
   for (int i = n_used * CHUNK_ROWS + tid; i < C; i += NT) s_logit[i] = -INFINITY;   // the empty tail is never loaded
@@ -140,10 +143,10 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
       const int row = r0 + lr;
       bool ok;
       if (MULTI) {
-        const int row_tok = row < C ? map[row] : -1;
+        const int row_tok = row < C ? sm.list[row] : -1;
         ok = row_tok >= 0 && row_tok <= q_tok && row_tok != p.n_cur;
       } else {
-        ok = row < C && map[row] >= 0;
+        ok = row < C && sm.list[row] >= 0;
       }
       float kf[EPL];
       // rows past C in a ragged last chunk hold stale bytes of an earlier chunk: read, not used
