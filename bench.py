@@ -38,10 +38,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # the rest (row reads, cache-row writes) is scaled by the rows processed.
 NCU_TRAFFIC_BYTES = {
     ("rebuild projection", "cfg3_llama7b_b64_c512_rebuild20pct"): {"bytes": 284.9e6 + 144.9e6, "rows": 9950.0},
-    ("attention kernel", "cfg3_llama7b_b64_c512_rebuild20pct"): {"bytes": 403.9e6 + 8.7e6, "rows": None},
+    ("attention kernel", "cfg3_llama7b_b64_c512_rebuild20pct"): {"bytes": 358.9e6 + 6.4e6, "rows": None},
     # config 4's per-layer launch, captured on a one-layer cache of the same shape (the sweep point C=1024, B=32)
-    ("attention kernel", "cfg4_llama7b_L32_b32_c1024"): {"bytes": 403.3e6 + 3.75e6, "rows": None},
-    ("attention kernel", "cfg5_sweep_c1024_b32"): {"bytes": 403.3e6 + 3.75e6, "rows": None},
+    ("attention kernel", "cfg4_llama7b_L32_b32_c1024"): {"bytes": 403.4e6 + 3.7e6, "rows": None},
+    ("attention kernel", "cfg5_sweep_c1024_b32"): {"bytes": 403.4e6 + 3.7e6, "rows": None},
 }
 
 
