@@ -63,13 +63,17 @@ __global__ void __launch_bounds__(kAttnThreads) attention_split_kernel(const Att
         reinterpret_cast<const unsigned char*>(p.q) + size_t(bh) * row_bytes + li * 16);
     Elem<T>::unpack(qr, qf);
   }
+  // this CTA's slice of the map row goes to shared memory first (the kept-list area is free until phase 2): a lookup in
+  // global memory in front of every key row's load would put two dependent loads in a row
+  for (int i = lo + tid; i < min(hi, C); i += NT) sm.list[i] = map[i];
+  __syncthreads();
   for (int r0 = lo + warp * RPW; r0 < hi; r0 += NW * RPW * U) {
     uint4 kv[U];
     bool ok[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int row = r0 + u * NW * RPW + sub;
-      ok[u] = row < hi && (row == C || map[row] >= 0);
+      ok[u] = row < hi && (row == C || sm.list[row] >= 0);
       kv[u] = make_uint4(0u, 0u, 0u, 0u);
       if (ok[u]) kv[u] = ldg_stream((row == C ? knew : Kb + size_t(row) * row_bytes) + li * 16);
     }
