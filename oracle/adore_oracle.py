@@ -205,16 +205,6 @@ def rope_rotate(v: np.ndarray, position: int, theta: float) -> np.ndarray:
     return out
 
 
-def project_kv(w_kv: np.ndarray, x_row: np.ndarray, position: int, n_heads: int, head_dim: int,
-               theta: float, dtype: str) -> Tuple[np.ndarray, np.ndarray]:
-    """K and V rows [H, dh] of one token from its layer-input row, as stored in the cache."""
-    y = np.asarray(w_kv, np.float64) @ np.asarray(x_row, np.float64)
-    n = n_heads * head_dim
-    k = rope_rotate(y[:n].reshape(n_heads, head_dim), position, theta)
-    v = y[n:].reshape(n_heads, head_dim)
-    return round_store(k, dtype), round_store(v, dtype)
-
-
 def project_q(w_q: np.ndarray, x_row: np.ndarray, position: int, n_heads: int, head_dim: int,
               theta: float, dtype: str) -> np.ndarray:
     """Query rows [H, dh] of the current token (harness side: same rotation as the keys)."""
@@ -420,6 +410,65 @@ class AdoreOracle:
             res = np.nonzero(self.tok_slot[b, : self.n] >= 0)[0]
             assert res.size == occ.size
             assert np.array_equal(self.slot_tok[b, self.tok_slot[b, res]], res)
+
+    # -- adopting a state from outside ---------------------------------------------------
+    def import_state(self, n: int, slot_tok: np.ndarray, slot_role: np.ndarray, score: np.ndarray, sigma: np.ndarray,
+                     z: np.ndarray, x_rows: np.ndarray, rebuild_tok: List[np.ndarray], rebuild_slot: List[np.ndarray],
+                     admit_slot: Optional[np.ndarray] = None, evicted_tok: Optional[np.ndarray] = None,
+                     z_rows: Optional[np.ndarray] = None) -> None:
+        """Continue from the small state of Sections 2.2-2.3 as somebody else left it after `n` tokens: which token
+        holds which slot in which role, every token's score and sigma, the GRU state z_{n-1}, the tokens' stored
+        embeddings and the last step's rebuild list. The token-to-slot table is the inverse of the slot map. The cache
+        rows are not taken over: by Section 2.3 a resident token's K/V state IS its recomputed state, so every layer
+        with a projection is filled from x_rows by definition.
+
+        slot_tok, slot_role: [B, C]; score, sigma: [B, >= n] float32; z: [B, d']; x_rows: [B, >= n, d];
+        rebuild_tok / rebuild_slot: per sequence, most valuable first. z_rows [B, >= n, d'] only with relative positions.
+        """
+        c = self.cfg
+        B, C = c.batch, c.capacity
+        slot_tok = np.asarray(slot_tok, np.int32)
+        slot_role = np.asarray(slot_role, np.uint8)
+        if slot_tok.shape != (B, C) or slot_role.shape != (B, C) or not (0 <= n <= c.max_tokens):
+            raise ValueError("state of another shape")
+        self.n = int(n)
+        self.slot_tok = slot_tok.copy()
+        self.slot_role = slot_role.copy()
+        self.tok_slot = np.full((B, c.max_tokens), -1, np.int32)
+        for b in range(B):
+            for s in range(C):
+                t = int(slot_tok[b, s])
+                if t >= 0:
+                    if not (t < n) or self.tok_slot[b, t] != -1 or slot_role[b, s] == EMPTY:
+                        raise ValueError("slot map is not a one-to-one map of tokens < n")
+                    self.tok_slot[b, t] = s
+                elif slot_role[b, s] != EMPTY:
+                    raise ValueError("an unoccupied slot carries a role")
+        self.score = np.zeros((B, c.max_tokens), np.float32)
+        self.sigma = np.zeros((B, c.max_tokens), np.float32)
+        self.score[:, :n] = np.asarray(score, np.float32)[:, :n]
+        self.sigma[:, :n] = np.asarray(sigma, np.float32)[:, :n]
+        self.z = np.asarray(z, np.float64).reshape(B, c.ctrl_hidden).copy()
+        self.x = np.zeros((B, c.max_tokens, c.hidden), np.float32)
+        self.x[:, :n] = np.asarray(x_rows, np.float32)[:, :n]
+        if c.relative_position:
+            self.z_rows = np.zeros((B, c.max_tokens, c.ctrl_hidden), np.float64)
+            self.z_rows[:, :n] = np.asarray(z_rows, np.float64)[:, :n]
+        lists = [np.asarray(t, np.int32).copy() for t in rebuild_tok]
+        slots = [np.asarray(s, np.int32).copy() for s in rebuild_slot]
+        for b in range(B):                                    # the list must be what the map shows as rebuilt
+            where = np.nonzero(self.slot_role[b] == REBUILT)[0]
+            if not (np.array_equal(np.sort(slots[b]), where) and np.array_equal(self.slot_tok[b, slots[b]], lists[b])):
+                raise ValueError("rebuild list and slot map disagree")
+        self.info = StepInfo(np.full(B, -1, np.int32) if admit_slot is None else np.asarray(admit_slot, np.int32).copy(),
+                             np.full(B, -1, np.int32) if evicted_tok is None else np.asarray(evicted_tok, np.int32).copy(),
+                             lists, slots)
+        self.attn_slot_tok = self.slot_tok.copy()
+        self.kept = None
+        self.check_invariants()
+        for layer in range(c.n_layers):
+            if self.w_kv[layer] is not None:
+                self.fill_layer(layer, None)
 
     # -- cache rows --------------------------------------------------------------------
     def _store_projections(self, layer: int, rows: List[Tuple[int, int, int]], src: np.ndarray) -> None:

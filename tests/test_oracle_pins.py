@@ -670,6 +670,76 @@ def test_relative_bulk_load_selects_on_the_scores_seen_from_the_last_prompt_toke
         assert orc.info.rebuild_tok[b].tolist() == ranked[cfg.retained_max - 1:][: cfg.rebuild_max]
 
 
+# ------------------------------------------------- query projection, adopting a state
+def test_query_projection_equals_explicit_loops():
+    """The harness's query rows: y = W_q x with explicit loops, adjacent pairs (2j, 2j+1) of every head turned by
+    position * theta^(-2j/dh) (the same rotation as the keys, so that q.k depends on the distance only), rounded to the
+    element type by torch."""
+    g = np.random.default_rng(21)
+    H, dh, d, pos, theta = 3, 8, 10, 37, 1.0e4
+    W = g.standard_normal((H * dh, d))
+    x = g.standard_normal(d)
+    y = [sum(float(W[i, j]) * float(x[j]) for j in range(d)) for i in range(H * dh)]
+    ref = np.zeros((H, dh))
+    for h in range(H):
+        for j in range(dh // 2):
+            ang = pos * theta ** (-2.0 * j / dh)
+            a, b = y[h * dh + 2 * j], y[h * dh + 2 * j + 1]
+            ref[h, 2 * j] = a * math.cos(ang) - b * math.sin(ang)
+            ref[h, 2 * j + 1] = a * math.sin(ang) + b * math.cos(ang)
+    got32 = ao.project_q(W, x, pos, H, dh, theta, "f32")
+    assert got32.shape == (H, dh) and np.allclose(got32, ref, rtol=1e-6, atol=1e-6)
+    got16 = ao.project_q(W, x, pos, H, dh, theta, "bf16")
+    assert np.array_equal(got16, torch.from_numpy(ref).to(torch.bfloat16).float().numpy())
+    # q.k of two rotated rows depends on the distance of their positions only
+    k = g.standard_normal(d)
+    dots = []
+    for p0 in (5, 100):
+        qq = ao.project_q(W, x, p0 + 9, H, dh, theta, "f32").astype(np.float64)
+        kk = ao.project_q(W, k, p0, H, dh, theta, "f32").astype(np.float64)
+        dots.append((qq * kk).sum(-1))
+    assert np.allclose(dots[0], dots[1], atol=1e-4)
+
+
+@pytest.mark.parametrize("mode", ["policy", "explicit"])
+def test_a_run_continued_from_an_imported_state_equals_the_uninterrupted_run(mode):
+    """Sections 2.2-2.3: the small state (slot map, roles, scores, z, stored embeddings, the last rebuild list) plus
+    "a resident token's K/V is its recomputed state" determine everything that follows. A fresh oracle that adopts
+    that state after 17 steps must produce, for the next 12 steps, the outputs and the state of the run that never
+    stopped; a state whose list contradicts its map, or whose map names a token twice, is refused."""
+    cfg = TINY.scaled(rebuild_mode=mode, rebuild_p=0.4, prompt=6, steps=40, capacity=8, rebuild_max=3, dtype="bf16")
+    w, orc, _ = run_free(cfg, steps=17)
+    other = make_oracle(w)
+    other.import_state(orc.n, orc.slot_tok, orc.slot_role, orc.score, orc.sigma, orc.z, orc.x, orc.info.rebuild_tok,
+                       orc.info.rebuild_slot, orc.info.admit_slot, orc.info.evicted_tok)
+    occ = orc.slot_tok >= 0
+    m = np.broadcast_to(occ[:, None, :, None], orc.Kc[0].shape)
+    assert np.array_equal(other.Kc[0][m], orc.Kc[0][m]) and np.array_equal(other.Vc[0][m], orc.Vc[0][m])
+    assert np.array_equal(other.tok_slot, orc.tok_slot)
+    for s in range(17, 29):
+        n = orc.n
+        x = w.x_new(n)
+        q, k, v = w.qkv(n, 0, x)
+        lists, counts = w.explicit(s, n)
+        ex = explicit_as_lists(lists, counts)
+        o1, w1 = orc.decode_step(0, q, k, v, x, ex)
+        o2, w2 = other.decode_step(0, q, k, v, x, ex)
+        orc.rebuild(0)
+        other.rebuild(0)
+        other.check_invariants()
+        assert np.array_equal(o1, o2) and np.array_equal(w1, w2)
+        assert np.array_equal(orc.slot_tok, other.slot_tok) and np.array_equal(orc.slot_role, other.slot_role)
+        assert np.array_equal(orc.score[:, : orc.n], other.score[:, : orc.n])
+    bad = make_oracle(w)
+    st = orc.slot_tok.copy()
+    st[0, 0] = st[0, 1]                                        # one token in two slots
+    with pytest.raises(ValueError):
+        bad.import_state(orc.n, st, orc.slot_role, orc.score, orc.sigma, orc.z, orc.x, orc.info.rebuild_tok, orc.info.rebuild_slot)
+    with pytest.raises(ValueError):                            # a list that the map does not show
+        bad.import_state(orc.n, orc.slot_tok, orc.slot_role, orc.score, orc.sigma, orc.z, orc.x,
+                         [l[:-1] for l in orc.info.rebuild_tok], [l[:-1] for l in orc.info.rebuild_slot])
+
+
 # ------------------------------------------------------------------ planted mistakes
 def test_pins_notice_planted_mistakes(monkeypatch):
     """Each plausible slip, planted in the oracle, must make one of the pins above fail."""
@@ -727,3 +797,17 @@ def test_pins_notice_planted_mistakes(monkeypatch):
     monkeypatch.setattr(ao, "controller_rescore", lambda z, n, ps, w: real_rescore(z, n, ps / 2, w))   # wrong scale
     assert fails(test_relative_scores_shift_with_the_sequence_and_meet_the_absolute_score_at_the_same_distance)
     monkeypatch.setattr(ao, "controller_rescore", real_rescore)
+
+    real_pq = ao.project_q
+    monkeypatch.setattr(ao, "project_q", lambda w, x, p, H, dh, t, dt: real_pq(w, x, p + 1, H, dh, t, dt))
+    assert fails(test_query_projection_equals_explicit_loops)          # rotated to the neighbouring position
+    monkeypatch.setattr(ao, "project_q", real_pq)
+
+    real_import = ao.AdoreOracle.import_state
+
+    def import_without_z(self, n, st, sr, sc, sg, z, *a, **k):          # forgets the GRU state
+        return real_import(self, n, st, sr, sc, sg, np.zeros_like(z), *a, **k)
+
+    monkeypatch.setattr(ao.AdoreOracle, "import_state", import_without_z)
+    assert fails(test_a_run_continued_from_an_imported_state_equals_the_uninterrupted_run, "policy")
+    monkeypatch.setattr(ao.AdoreOracle, "import_state", real_import)
