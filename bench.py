@@ -7,6 +7,9 @@ top-K attention over the slot cache (with weight emission and the in-place admit
 step the controller + selection, and for every layer the rebuild projection + RoPE + scatter.
 Inputs are synthetic (seeded Gaussians of the workload's shapes) and resident in HBM when the
 timed region starts; the `e2e` number repeats the steps through the host-buffer entry point.
+The K timed steps are replayed (the cache put back to the same state outside the events) until
+their device time adds up to about a second; `value` is the median over those repeats. The
+default run (config 3) also carries a short run of config 4, the largest one, in `largest_config`.
 One JSON line is printed by rank 0.
 """
 from __future__ import annotations
@@ -32,27 +35,28 @@ METRIC = "decode tokens/s (= batch x decode steps/s) at batch B, cache C"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries,
-# keyed by (kernel, workload); None until captured for the kernel as it stands.
-# For the rebuild GEMM the capture saw fewer rows than the timed launches: the weight bytes are fixed,
-# the rest (row reads, cache-row writes) is scaled by the rows processed.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, taken from the committed ncu summary
+# named beside it (one capture of the kernel as it stands; None once the kernel has changed since). For the rebuild GEMM
+# the capture saw fewer rows than the timed launches: the weight bytes are fixed, the rest (row reads, cache-row
+# writes) is scaled by the rows processed.
 NCU_TRAFFIC_BYTES = {
-    ("rebuild projection", "cfg3_llama7b_b64_c512_rebuild20pct"): {"bytes": 284.9e6 + 144.9e6, "rows": 9950.0},
-    ("attention kernel", "cfg3_llama7b_b64_c512_rebuild20pct"): {"bytes": 358.9e6 + 6.4e6, "rows": None},
-    # config 4's per-layer launch, captured on a one-layer cache of the same shape (the sweep point C=1024, B=32)
-    ("attention kernel", "cfg4_llama7b_L32_b32_c1024"): {"bytes": 403.4e6 + 3.7e6, "rows": None},
-    ("attention kernel", "cfg5_sweep_c1024_b32"): {"bytes": 403.4e6 + 3.7e6, "rows": None},
+    ("rebuild projection", "cfg3_llama7b_b64_c512_rebuild20pct"):
+        {"bytes": 284.9e6 + 144.9e6, "rows": 9950.0, "profile": "profiles/rebuild_tc_pair_kernel_cfg3.md"},
+    ("attention kernel", "cfg3_llama7b_b64_c512_rebuild20pct"): None,
+    ("attention kernel", "cfg4_llama7b_L32_b32_c1024"): None,
+    ("attention kernel", "cfg5_sweep_c1024_b32"): None,
 }
 
 
 def ncu_traffic(kernel, cfg, rows):
+    """(bytes per launch or None, the profile the figure comes from or None)"""
     t = NCU_TRAFFIC_BYTES.get((kernel, cfg.name))
     if t is None:
-        return None
+        return None, None
     if t["rows"] is None:
-        return t["bytes"]
+        return t["bytes"], t["profile"]
     fixed = 2 * cfg.n_heads * cfg.head_dim * cfg.hidden * cfg.elem_bytes
-    return fixed + (t["bytes"] - fixed) * rows / t["rows"]
+    return fixed + (t["bytes"] - fixed) * rows / t["rows"], t["profile"]
 
 
 def measured_peaks():
@@ -79,7 +83,7 @@ def run_sweep(args):
     """Capacity x batch sweep: every point in its own process (a fresh context per point)."""
     for cap, b, cfg in wl.sweep_points():
         cmd = [sys.executable, os.path.abspath(__file__), "--config", "5", "--capacity", str(cap), "--batch", str(b),
-               "--no-cpu-baseline", "--no-e2e", "--warmup", str(args.warmup)]
+               "--no-cpu-baseline", "--no-e2e", "--warmup", str(args.warmup), "--min-timed-ms", "300"]
         if args.steps is not None:
             cmd += ["--steps", str(args.steps)]
         res = subprocess.run(cmd, capture_output=True, text=True)
@@ -92,6 +96,7 @@ def run_sweep(args):
                           "tokens_per_s": d["value"], "ms_per_step": d["ms_per_step"],
                           "attention_hbm_frac": st["attention"]["frac"],
                           "attention_plus_selection_hbm_frac": st["attention_plus_selection"]["frac"],
+                          "attention_plus_selection_frac_is": st["attention_plus_selection"]["frac_is"],
                           "rebuild": {k: st.get("rebuild", {}).get(k) for k in ("bound", "frac", "rows_per_launch", "ms_per_launch")},
                           "clocks": d["clocks"]}), flush=True)
 
@@ -129,35 +134,36 @@ def whole_job_tokens_per_s(batch_per_rank: int, steps: int, world: int, ms_max: 
 # clocks
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
+    """nvidia-smi in the background, one sample every 20 ms; window() gives the median SM clock and the throttle reasons
+    seen between two time.time() stamps."""
     QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index: int):
         self.path = tempfile.mktemp(prefix="adore_clocks_", suffix=".csv")
         self.proc = None
+        self.rows = None
         try:
             self.f = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "50", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+                                          "-lms", "20", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self, t_begin: float, t_end: float):
-        """Median SM clock and throttle reasons of the samples taken between two time.time() stamps."""
+    def close(self):
+        """Stops the sampler and reads what it wrote: (time, sm MHz, max MHz, power W, [reason flags])."""
         import datetime
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0,
-               "window": "timed region + end-to-end pass + per-stage pass"}
+        self.rows = []
         if self.proc is None:
-            return out
+            return
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
         self.f.close()
-        sm, reasons, mx = [], set(), None
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         try:
             for line in open(self.path):
                 parts = [p.strip() for p in line.split(",")]
@@ -165,20 +171,23 @@ class ClockSampler:
                     continue
                 try:
                     ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
-                    if ts < t_begin - 0.05 or ts > t_end + 0.05:
-                        continue
-                    sm.append(float(parts[1]))
-                    mx = float(parts[2])
+                    self.rows.append((ts, float(parts[1]), float(parts[2]), float(parts[3]),
+                                      [v.lower().startswith("active") for v in parts[5:9]]))
                 except ValueError:
                     continue
-                for name, val in zip(names, parts[5:9]):
-                    if val.lower().startswith("active"):
-                        reasons.add(name)
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+
+    def window(self, t_begin: float, t_end: float, what: str):
+        if self.rows is None:
+            self.close()
+        sel = [r for r in self.rows if t_begin - 0.01 <= r[0] <= t_end + 0.01]
+        out = {"sm_mhz": None, "sm_max_mhz": None, "power_w": None, "reasons": [], "samples": len(sel), "window": what}
+        if sel:
+            reasons = sorted({n for r in sel for n, on in zip(self.NAMES, r[4]) if on})
+            out.update(sm_mhz=float(np.median([r[1] for r in sel])), sm_max_mhz=sel[-1][2],
+                       power_w=float(np.median([r[3] for r in sel])), reasons=reasons)
         return out
 
 
@@ -436,7 +445,8 @@ def run_reference(args, cfg):
     value, threads, desc, ms = time_oracle(cfg, args.steps, args.warmup, budget_s=120.0)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f64", "data": "synthetic", "config": workload_desc(cfg),
+            "dtype": "f64", "data": "synthetic",
+            "config": dict(workload_desc(cfg), step_order=args.order, score_source=args.score_source),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -472,33 +482,6 @@ def rebuild_flops_bytes_per_launch(cfg, rows: float):
     flops = 2.0 * rows * cfg.hidden * n_out
     bytes_ = (n_out * cfg.hidden + rows * cfg.hidden + rows * n_out) * cfg.elem_bytes
     return flops, bytes_
-
-
-def probe_pattern_ceiling(run, flush):
-    """Times a plain read kernel on the layer-0 cache with the attention's two access patterns: all key
-    blocks streamed, then `topk` of the C value rows of every (b, h) gathered. Returns GB/s of each."""
-    import torch
-    lib, c = run.lib, run.cfg
-    kptr, vptr = lib.adore_cache_kv(run.handle, 0)
-    n_blocks, row_bytes = c.batch * c.n_heads, c.head_dim * c.elem_bytes
-    sink = torch.zeros(4, dtype=torch.int32, device="cuda")
-    stream = torch.cuda.current_stream().cuda_stream
-    out = {}
-    for name, ptr, kept, gather in (("stream", kptr, c.capacity, False), ("gather", vptr, min(c.topk, c.capacity), True)):
-        best = None
-        for _ in range(5):
-            if flush is not None:
-                flush.zero_()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            lib.adore_probe_read_bandwidth(ptr, n_blocks, c.capacity, row_bytes, kept, gather, 148 * 8, sink, stream)
-            b.record()
-            torch.cuda.synchronize()
-            ms = a.elapsed_time(b)
-            best = ms if best is None else min(best, ms)
-        out[name + "_gbs"] = n_blocks * kept * row_bytes / (best * 1e-3) / 1e9
-        out[name + "_us"] = best * 1e3
-    return out
 
 
 def run_labels(args):
@@ -558,6 +541,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-largest", action="store_true", help="skip the config-4 run that the default (config 3) line carries")
+    ap.add_argument("--largest-steps", type=int, default=8, help="timed steps of that config-4 run")
+    ap.add_argument("--leg", action="store_true", help=argparse.SUPPRESS)      # this process IS that config-4 run
+    ap.add_argument("--min-timed-ms", type=float, default=1000.0,
+                    help="the timed steps are replayed (state put back outside the events) until their device time adds up to this")
+    ap.add_argument("--max-repeats", type=int, default=200)
     ap.add_argument("--score-source", default="controller", choices=["controller", "attention", "controller-relative"],
                     help="attention: tokens ranked by cumulative attention weight (the H2O baselines' score), no controller; "
                          "controller-relative: position feature = distance to the current token, every token re-scored every step")
@@ -598,7 +587,7 @@ def main():
 
     K, W = args.steps, args.warmup
     with_e2e = not args.no_e2e and args.order == "attend-first"
-    total = W + K                                       # warm-up and timed steps; the other passes replay the timed ones
+    total = W + K                                       # warm-up and timed steps; every other pass replays the timed ones
     run = DeviceRun(cfg, total, rank, args.order, args.score_source)
     flush = None
     if kv_bytes(cfg) <= 2.5e8:
@@ -613,10 +602,10 @@ def main():
         run.step()
     lib.adore_cache_sync_status(run.handle)
 
-    # The end-to-end pass and the per-stage pass below replay the SAME K steps as the timed region: the small state
-    # (slot maps, token table, scores) is snapshotted here and put back before each of them, so that all three see the
-    # same list lengths and occupancy. The K/V rows are copied aside and put back too (on the device): on rows that do
-    # not belong to the restored maps the attention kernel measured ~4 % slower.
+    # Every pass below replays the SAME K steps: the small state (slot maps, token table, scores) is snapshotted here and
+    # put back before each pass, so that all of them see the same list lengths and occupancy. The K/V rows are copied
+    # aside and put back too (on the device): on rows that do not belong to the restored maps the attention kernel
+    # measured ~4 % slower.
     snap = np.zeros(lib.adore_cache_export_state(run.handle, None), np.uint8)
     lib.adore_cache_export_state(run.handle, snap)
     next0 = run.next
@@ -631,24 +620,18 @@ def main():
         torch.cuda.synchronize()
         run.next = next0
 
-    # ---- timed region: K steps, device time, max over ranks ----
-    launches0 = lib.adore_cache_launch_count(run.handle)
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    if sampler:
-        time.sleep(0.5)                                 # let the sampler come up
-    barrier()
-    t_clock0 = time.time()
-    if flush is None:
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record()
-        for _ in range(K):
-            run.step()
-        lib.adore_cache_join(run.handle)                # the last step's side-stream work counts too
-        ev1.record()
-        barrier()
-        ms_local = ev0.elapsed_time(ev1)
-    else:                                               # small workloads: flush L2 between steps
-        pairs = []
+    def timed_pass():
+        """The K steps once, device time in ms on this rank (events on the stream the library launches on)."""
+        if flush is None:
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            for _ in range(K):
+                run.step()
+            lib.adore_cache_join(run.handle)            # the last step's side-stream work counts too
+            ev1.record()
+            barrier()
+            return ev0.elapsed_time(ev1)
+        pairs = []                                      # small workloads: flush L2 between steps
         for _ in range(K):
             flush.zero_()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -658,71 +641,147 @@ def main():
             b.record()
             pairs.append((a, b))
         barrier()
-        ms_local = sum(a.elapsed_time(b) for a, b in pairs)
+        return sum(a.elapsed_time(b) for a, b in pairs)
+
+    # ---- timed region: the K steps, replayed until the device time adds up to about a second; max over ranks per
+    # repeat, median over the repeats ----
+    launches0 = lib.adore_cache_launch_count(run.handle)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        time.sleep(0.3)                                 # let the sampler come up
+    barrier()
+    t_timed0 = time.time()
+    first = max_over_ranks(timed_pass(), world, dev)
     launches = lib.adore_cache_launch_count(run.handle) - launches0
+    repeats = int(min(args.max_repeats, max(1, math.ceil(args.min_timed_ms / max(first, 1e-3)))))
+    per_repeat = [first]
+    for _ in range(repeats - 1):
+        rewind()
+        barrier()
+        per_repeat.append(max_over_ranks(timed_pass(), world, dev))
+    t_timed1 = time.time()
     lib.adore_cache_sync_status(run.handle)
-    ms_total = max_over_ranks(ms_local, world, dev)
+    ms_total = float(np.median(per_repeat))
     value = whole_job_tokens_per_s(cfg.batch, K, world, ms_total)
 
-    # ---- end to end through the host-buffer entry point ----
+    # ---- end to end through the host-buffer entry point (same repeats, median) ----
     e2e = None
     if with_e2e:
         rewind()
         run.make_host_inputs(run.next, K)
-        barrier()
-        t0 = time.perf_counter()
-        for _ in range(K):
-            run.step_host()
-        torch.cuda.synchronize()
-        e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, world, dev)
+        e2e_runs = []
+        for r in range(max(1, min(repeats, args.max_repeats // 2))):
+            if r:
+                rewind()
+            barrier()
+            t0 = time.perf_counter()
+            for _ in range(K):
+                run.step_host()
+            torch.cuda.synchronize()
+            e2e_runs.append(max_over_ranks((time.perf_counter() - t0) * 1e3, world, dev))
+        e2e_ms = float(np.median(e2e_runs))
         h2d, d2h = run.host_bytes_per_step()
         e2e = {"value": whole_job_tokens_per_s(cfg.batch, K, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms / K,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "repeats": len(e2e_runs),
+               "excludes": "per-slot weights (emitted on the device for device-side consumers, not copied to the host)"}
 
-    # ---- per-stage pass (events around every launch) for the roofline figures ----
-    rewind()
-    rows0 = lib.adore_cache_rebuild_rows(run.handle)
-    lib.adore_cache_set_stage_timing(run.handle, True)
-    lib.adore_cache_stage_times(run.handle)
-    for _ in range(K):
-        if flush is not None:
-            flush.zero_()
-        run.step()
-    st_ms, st_n = lib.adore_cache_stage_times(run.handle)
-    lib.adore_cache_set_stage_timing(run.handle, False)
-    rows = (lib.adore_cache_rebuild_rows(run.handle) - rows0) / max(K, 1)      # rebuilt rows per step
+    # ---- per-stage pass (events around every launch, stages one after the other) for the roofline figures ----
+    st_ms, st_n, rows_sum, stage_steps = [0.0] * 4, [0] * 4, 0, 0
+    stage_repeats = max(1, min(repeats, args.max_repeats // 2))
+    t_stage0 = time.time()
+    for _ in range(stage_repeats):
+        rewind()
+        rows0 = lib.adore_cache_rebuild_rows(run.handle)
+        lib.adore_cache_set_stage_timing(run.handle, 1)
+        lib.adore_cache_stage_times(run.handle)
+        for _ in range(K):
+            if flush is not None:
+                flush.zero_()
+            run.step()
+        ms_i, n_i = lib.adore_cache_stage_times(run.handle)
+        lib.adore_cache_set_stage_timing(run.handle, 0)
+        rows_sum += lib.adore_cache_rebuild_rows(run.handle) - rows0
+        stage_steps += K
+        st_ms = [a + b for a, b in zip(st_ms, ms_i)]
+        st_n = [a + b for a, b in zip(st_n, n_i)]
+    t_stage1 = time.time()
+    rows = rows_sum / max(stage_steps, 1)                # rebuilt rows per step
     lib.adore_cache_sync_status(run.handle)
-    clocks = sampler.stop(t_clock0, time.time()) if sampler else None
 
-    ceiling = probe_pattern_ceiling(run, flush)
+    # ---- group pass: the step's own schedule (selection and controller beside the attention, rebuilds beside the
+    # following layers); device time from the start of the step's attention to the later of {last attention / new
+    # token's row written, controller chain done} ----
+    group_ms = group_steps = 0
+    if args.order == "attend-first":
+        for _ in range(stage_repeats):
+            rewind()
+            lib.adore_cache_set_stage_timing(run.handle, 2)
+            lib.adore_cache_group_times(run.handle)
+            for _ in range(K):
+                if flush is not None:
+                    flush.zero_()
+                run.step()
+            g_ms, g_n = lib.adore_cache_group_times(run.handle)
+            lib.adore_cache_set_stage_timing(run.handle, 0)
+            group_ms += g_ms
+            group_steps += g_n
+        lib.adore_cache_sync_status(run.handle)
+    clocks = clocks_stage = None
+    if sampler:
+        sampler.close()
+        clocks = sampler.window(t_timed0, t_timed1, "timed region (all repeats)")
+        clocks_stage = sampler.window(t_stage0, t_stage1, "per-stage pass")
 
     peaks, peak_kind = measured_peaks()
     occ = min(cfg.capacity, cfg.retained_max + rows / cfg.batch)
     att_ms = st_ms[0] / max(st_n[0], 1)
-    sel_ms = st_ms[1] / max(K, 1)
+    sel_ms = st_ms[1] / max(stage_steps, 1)
+    adm_ms = st_ms[3] / max(stage_steps, 1)
     reb_ms = st_ms[2] / max(st_n[2], 1)
     att_bytes = attention_bytes_per_launch(cfg, occ)
     reb_flops, reb_bytes = rebuild_flops_bytes_per_launch(cfg, rows)
     att_gbs = att_bytes / (att_ms * 1e-3) / 1e9 if att_ms > 0 else 0.0
     stages = {
-        "admit_layer0": {"ms_per_step": st_ms[3] / max(K, 1)},
+        "admit_layer0": {"ms_per_step": adm_ms},
         "attention": {"bound": "hbm", "ms_per_launch": att_ms, "launches_per_step": cfg.n_layers,
                       "algorithmic_bytes": att_bytes, "achieved": att_gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"],
                       "frac": att_gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": att_gbs / NOMINAL_HBM_GBS},
         "controller_select": {"ms_per_step": sel_ms},
     }
     sel_bytes = 4 * (3 * cfg.ctrl_hidden * (cfg.hidden + cfg.ctrl_hidden)) + cfg.batch * cfg.hidden * cfg.elem_bytes
-    both_ms = att_ms * cfg.n_layers + sel_ms + st_ms[3] / max(K, 1)
-    both_gbs = (att_bytes * cfg.n_layers + sel_bytes) / (both_ms * 1e-3) / 1e9 if both_ms > 0 else 0.0
-    stages["attention_plus_selection"] = {"bound": "hbm", "achieved": both_gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"],
-                                          "frac": both_gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": both_gbs / NOMINAL_HBM_GBS}
+    group_bytes = att_bytes * cfg.n_layers + sel_bytes
+    both_ms = att_ms * cfg.n_layers + sel_ms + adm_ms
+    both_gbs = group_bytes / (both_ms * 1e-3) / 1e9 if both_ms > 0 else 0.0
+    stages["attention_plus_selection"] = {
+        "bound": "hbm", "algorithmic_bytes": group_bytes, "unit": "GB/s", "peak": peaks["hbm_gbs"],
+        "stages_added": {"ms_per_step": both_ms, "achieved": both_gbs, "frac": both_gbs / peaks["hbm_gbs"],
+                         "note": "per-stage pass: the stages run one after the other and their times are added"}}
+    if group_steps:
+        ov_ms = group_ms / group_steps
+        ov_gbs = group_bytes / (ov_ms * 1e-3) / 1e9
+        stages["attention_plus_selection"]["overlapped"] = {
+            "ms_per_step": ov_ms, "achieved": ov_gbs, "frac": ov_gbs / peaks["hbm_gbs"],
+            "frac_of_nominal_8TBs": ov_gbs / NOMINAL_HBM_GBS,
+            "note": "the step's own schedule: device time from the start of the attention to the later of {last "
+                    "attention / new token's row written, controller chain done}"
+                    + ("; the rebuilds of the earlier layers run inside this window on their own stream" if cfg.n_layers > 1 else "")}
+        stages["attention_plus_selection"].update(achieved=ov_gbs, frac=ov_gbs / peaks["hbm_gbs"], frac_is="overlapped")
+    else:
+        stages["attention_plus_selection"].update(achieved=both_gbs, frac=both_gbs / peaks["hbm_gbs"], frac_is="stages_added")
     tensor_bound = cfg.dtype == "bf16" and rows >= 300
     if reb_ms > 0 and rows > 0:
         if tensor_bound:
             tf = reb_flops / (reb_ms * 1e-3) / 1e12
+            # which cuBLAS figure the launch is put against follows the clocks seen while it was timed: at (nearly) full
+            # clock the burst figure, under the power cap the sustained one
+            ck = clocks_stage or {}
+            full_clock = bool(ck.get("sm_mhz")) and ck["sm_mhz"] >= 0.95 * (ck.get("sm_max_mhz") or peaks.get("sm_max_mhz", 1965.0))
+            which = "burst" if (full_clock or not ck.get("sm_mhz")) else "sustained"
+            peak_tf = peaks["bf16_tflops"] if which == "burst" else peaks["bf16_tflops_sustained"]
             stages["rebuild"] = {"bound": "tensor", "ms_per_launch": reb_ms, "rows_per_launch": rows, "flops": reb_flops,
-                                 "achieved": tf, "unit": "TFLOP/s", "peak": peaks["bf16_tflops_sustained"],
-                                 "frac": tf / peaks["bf16_tflops_sustained"], "frac_of_burst": tf / peaks["bf16_tflops"]}
+                                 "achieved": tf, "unit": "TFLOP/s", "peak": peak_tf, "frac": tf / peak_tf, "frac_is": which,
+                                 "frac_of_burst": tf / peaks["bf16_tflops"], "frac_of_sustained": tf / peaks["bf16_tflops_sustained"],
+                                 "sm_mhz_while_timed": ck.get("sm_mhz")}
         else:
             gb = reb_bytes / (reb_ms * 1e-3) / 1e9
             stages["rebuild"] = {"bound": "hbm", "ms_per_launch": reb_ms, "rows_per_launch": rows,
@@ -731,12 +790,23 @@ def main():
     dominant = "rebuild" if ("rebuild" in stages and st_ms[2] > st_ms[0]) else "attention"
     d = stages[dominant]
     kernel_name = {"attention": "attention kernel", "rebuild": "rebuild projection"}[dominant]
+    traffic, traffic_from = ncu_traffic(kernel_name, cfg, rows)
     roofline = {"kernel": kernel_name, "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"], "unit": d["unit"],
-                "frac": d["frac"], "peak_source": f"{peak_kind} ({'sustained' if d['bound'] == 'tensor' else 'copy'})",
-                "traffic": ncu_traffic(kernel_name, cfg, rows),
+                "frac": d["frac"],
+                "peak_source": f"{peak_kind} ({d.get('frac_is', 'copy') if d['bound'] == 'tensor' else 'copy'})",
+                "traffic": traffic, "traffic_source": traffic_from,
                 "share_of_step": {"attention": (st_ms[0] + st_ms[3]) / max(sum(st_ms), 1e-9),
                                   "controller_select": st_ms[1] / max(sum(st_ms), 1e-9),
                                   "rebuild": st_ms[2] / max(sum(st_ms), 1e-9)}}
+
+    run.close()
+    del run, kv_live, kv_keep
+    torch.cuda.empty_cache()
+
+    # ---- the HBM target is stated for the largest configuration: its own short run, in a process of its own ----
+    largest = None
+    if rank == 0 and world == 1 and cfg_index(cfg) == 3 and not args.no_largest and not args.leg:
+        largest = run_largest_leg(args)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -745,18 +815,35 @@ def main():
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-                "ms_per_step": ms_total / K, "steps_per_s": K / (ms_total * 1e-3), "higher_is_better": True,
+                "ms_per_step": ms_total / K, "steps_per_s": K / (ms_total * 1e-3), "repeats": len(per_repeat),
+                "ms_per_step_min_max": [min(per_repeat) / K, max(per_repeat) / K],
+                "timed_ms_total": float(sum(per_repeat)), "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-                "config": dict(workload_desc(cfg), step_order=args.order, score_source=args.score_source), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-                "roofline": roofline, "stages": stages, "cpu_baseline": cpu}
-        # the plain read kernel's time for the same bytes: what the access pattern allows on this GPU
-        ideal_us = ceiling["stream_us"] + ceiling["gather_us"]
-        line["attention_pattern_ceiling"] = dict(ceiling, ideal_us=ideal_us, kernel_us=att_ms * 1e3,
-                                                 kernel_over_ideal=att_ms * 1e3 / ideal_us if ideal_us > 0 else None)
+                "config": dict(workload_desc(cfg), step_order=args.order, score_source=args.score_source), "clocks": clocks,
+                "clocks_stage_pass": clocks_stage, "e2e": e2e, "gpu_launches": int(launches),
+                "roofline": roofline, "stages": stages, "cpu_baseline": cpu, "largest_config": largest}
         print(json.dumps(line))
-    run.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_largest_leg(args):
+    """Config 4 (32 layers, B 32, C 1024: the configuration the HBM target is stated for) in a process of its own, a few
+    timed steps; returns the part of its line that the metric names."""
+    cmd = [sys.executable, os.path.abspath(__file__), "--config", "4", "--leg", "--no-cpu-baseline", "--no-e2e",
+           "--steps", str(args.largest_steps), "--warmup", "3", "--min-timed-ms", "400", "--max-repeats", "12"]
+    try:
+        res = subprocess.run(cmd, capture_output=True, text=True, timeout=900)
+    except subprocess.TimeoutExpired:
+        return {"error": "the config-4 run did not finish in 900 s"}
+    if res.returncode != 0:
+        return {"error": (res.stderr.strip().splitlines() or ["failed"])[-1][:300]}
+    d = json.loads(res.stdout.strip().splitlines()[-1])
+    st = d["stages"]
+    return {"workload": d["config"]["workload"], "steps": d["steps"], "repeats": d["repeats"], "ms_per_step": d["ms_per_step"],
+            "tokens_per_s": d["value"], "steps_per_s": d["steps_per_s"], "gpu_launches": d["gpu_launches"], "clocks": d["clocks"],
+            "attention": st["attention"], "attention_plus_selection": st["attention_plus_selection"],
+            "controller_select": st["controller_select"], "rebuild": st.get("rebuild")}
 
 
 if __name__ == "__main__":

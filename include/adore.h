@@ -243,26 +243,27 @@ int64_t adore_cache_launch_count(const adore_cache_t *cache);
  * adds up the elapsed milliseconds and launch counts per stage since the last call and resets
  * them. Stage index: 0 attention (with the fused admit of layers > 0), 1 controller + selection,
  * 2 rebuild projection (gather + GEMM), 3 the separate admit launch of layer 0.
- * ms and launches: HOST arrays of 4. While timing is enabled the controller runs on the main
+ * enable: 0 off, 1 per-stage timing, 2 group timing (see adore_cache_group_times).
+ * ms and launches: HOST arrays of 4. While per-stage timing is enabled the controller runs on the main
  * stream instead of beside the attention, so that the stage times add up. Event recording costs a few microseconds per launch, so
  * whole-step throughput should be measured with timing disabled. */
 adore_status_t adore_cache_set_stage_timing(adore_cache_t *cache, int32_t enable);
 adore_status_t adore_cache_stage_times(adore_cache_t *cache, double *ms, int64_t *launches);
 
+/* Device time of the attention + selection group as the step really runs it (no counterpart in the paper; Section 1
+ * and Section 3.2 name the attention's KV traffic as the cost that matters). With adore_cache_set_stage_timing(cache, 2)
+ * the schedule stays as it is: selection and controller on their side streams beside the attention, rebuilds beside
+ * the following layers. Per attend-first step three events are recorded: where the group starts (before the attention
+ * of layer 0), where its main-stream part ends (after the last layer's attention; in a one-layer cache after the new
+ * token's row has been written) and where the controller chain ends. adore_cache_group_times waits for the streams and
+ * returns, summed over the steps since the last call, the time from the first event to the later of the other two,
+ * and the number of steps; both are reset. ms, steps: HOST pointers. In a cache of several layers the rebuilds of
+ * layers 0..L-2 run inside that window, on their own stream. */
+adore_status_t adore_cache_group_times(adore_cache_t *cache, double *ms, int64_t *steps);
+
 /* Total number of rows rebuilt by decode steps so far (Section 2.3: sum over steps and sequences
  * of the rebuild-list lengths); waits for the stream. rows: HOST pointer. */
 adore_status_t adore_cache_rebuild_rows(adore_cache_t *cache, int64_t *rows);
-
-/* Measurement aid (no counterpart in the paper): reads `buffer`, laid out as n_blocks blocks of
- * block_rows rows of row_bytes (128, 256 or 512) bytes, with plain 16-byte loads and `ctas` CTAs of
- * 256 threads. gather == 0 streams every block whole (the key pass of the attention);
- * gather != 0 reads kept_rows rows per block, spread over the block with a pseudo-random jitter
- * (the kept value rows of a top-K mask). Nothing is written except possibly 4 bytes at scratch4
- * (device). The caller times the launch on cuda_stream; bytes read = n_blocks * rows * row_bytes.
- * buffer: DEVICE pointer, 16-byte aligned. Errors: INVALID_ARG, CUDA. */
-adore_status_t adore_probe_read_bandwidth(const void *buffer, int32_t n_blocks, int32_t block_rows,
-                                          int32_t row_bytes, int32_t kept_rows, int32_t gather,
-                                          int32_t ctas, void *scratch4, void *cuda_stream);
 
 /* Controller scoring for callers that cannot allocate device memory. (The paper has no
  * counterpart: this is a packaging of its controller, Section 2.2 Eq. 2, for a constrained
@@ -288,6 +289,8 @@ adore_status_t adore_probe_read_bandwidth(const void *buffer, int32_t n_blocks, 
  * Limits and rules:
  *   - batch * 3 * ctrl_hidden doubles must fit the 2 MiB array (batch <= 682 for d' = 128);
  *     larger requests return ADORE_ERR_UNSUPPORTED and launch nothing.
+ *   - hidden must be a multiple of 64 (as for adore_cache_create), x and w->gru_w_ih must be
+ *     16-byte aligned and z 8-byte aligned; otherwise ADORE_ERR_UNSUPPORTED, nothing is launched.
  *   - The array is part of the library image: every GPU on which the library runs holds
  *     these 2 MiB until the process exits.
  *   - The first call on each device looks up the array's device address (no allocation). Make
@@ -351,7 +354,20 @@ adore_status_t adore_label_tokens(const float *weights, int32_t n_layers, int32_
  *   import: host_buf is a snapshot taken from a cache created with the same batch, capacity,
  *           rebuild_max, max_tokens and ctrl_hidden; anything else returns ADORE_ERR_INVALID_ARG and
  *           changes nothing.
- * Both wait for the cache's streams before copying (synchronous calls). */
+ * Both wait for the cache's streams before copying (synchronous calls).
+ *
+ * Layout of a snapshot (version 1, little endian, every section padded to a multiple of 8 bytes):
+ *   header, 64 bytes: uint32 magic 0x54534441, uint32 version = 1, then int32 batch, capacity, rebuild_max, max_tokens,
+ *     ctrl_hidden, n, cur (which of the two slot-map buffers is the current one), attn (the one the cache rows follow),
+ *     step_open (0 none, 1 attend-first, 2 rebuild-first), uint32 flag word (ADORE_FLAG_RELATIVE_POSITION bit), 16 bytes zero;
+ *   sections, with B = batch, C = capacity, T = max_tokens, R = max(rebuild_max, 1):
+ *     int32 slot_tok[2][B][C] (as two sections), uint8 slot_role[2][B][C] (two sections), int32 tok_slot[B][T],
+ *     float score[B][T], float sigma[B][T], double z[B][ctrl_hidden], int32 admit_slot[B], int32 evicted_tok[B],
+ *     int32 rebuild_tok[B][R], int32 rebuild_slot[B][R], int32 rebuild_count[B], int32 row_b[B*R], int32 row_tok[B*R],
+ *     int32 row_slot[B*R], int32 row_total[1]; with ADORE_FLAG_RELATIVE_POSITION also double a[B][T][ctrl_hidden].
+ * import checks every index of the integer sections against the cache's shape before anything is copied to the
+ * device (token positions < n, slots < C, roles, counts within m and R_max, row table entries within the batch);
+ * a snapshot that fails returns ADORE_ERR_INVALID_ARG and changes nothing. */
 adore_status_t adore_cache_export_state(adore_cache_t *cache, void *host_buf, size_t *bytes);
 adore_status_t adore_cache_import_state(adore_cache_t *cache, const void *host_buf, size_t bytes);
 

@@ -415,12 +415,13 @@ class AdoreOracle:
     def import_state(self, n: int, slot_tok: np.ndarray, slot_role: np.ndarray, score: np.ndarray, sigma: np.ndarray,
                      z: np.ndarray, x_rows: np.ndarray, rebuild_tok: List[np.ndarray], rebuild_slot: List[np.ndarray],
                      admit_slot: Optional[np.ndarray] = None, evicted_tok: Optional[np.ndarray] = None,
-                     z_rows: Optional[np.ndarray] = None) -> None:
+                     z_rows: Optional[np.ndarray] = None, x_tables: Optional[List[np.ndarray]] = None) -> None:
         """Continue from the small state of Sections 2.2-2.3 as somebody else left it after `n` tokens: which token
         holds which slot in which role, every token's score and sigma, the GRU state z_{n-1}, the tokens' stored
         embeddings and the last step's rebuild list. The token-to-slot table is the inverse of the slot map. The cache
         rows are not taken over: by Section 2.3 a resident token's K/V state IS its recomputed state, so every layer
-        with a projection is filled from x_rows by definition.
+        with a projection is filled by definition, from x_rows or, for stacks whose layers have their own input rows,
+        from x_tables[layer].
 
         slot_tok, slot_role: [B, C]; score, sigma: [B, >= n] float32; z: [B, d']; x_rows: [B, >= n, d];
         rebuild_tok / rebuild_slot: per sequence, most valuable first. z_rows [B, >= n, d'] only with relative positions.
@@ -468,7 +469,7 @@ class AdoreOracle:
         self.check_invariants()
         for layer in range(c.n_layers):
             if self.w_kv[layer] is not None:
-                self.fill_layer(layer, None)
+                self.fill_layer(layer, None if (x_tables is None or layer == 0) else x_tables[layer])
 
     # -- cache rows --------------------------------------------------------------------
     def _store_projections(self, layer: int, rows: List[Tuple[int, int, int]], src: np.ndarray) -> None:

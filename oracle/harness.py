@@ -27,14 +27,20 @@ def oracle_config(cfg: wl.WorkloadConfig, batch: Optional[int] = None) -> ao.Ora
 
 
 class Workload:
-    """Seeded inputs of one config, restricted to the first `batch` sequences."""
+    """Seeded inputs of one config, restricted to the first `batch` sequences and, with `layers`, to some of its
+    layers: layer index l of this object (and of the oracle made from it) then stands for layer layers[l] of `cfg`."""
 
-    def __init__(self, cfg: wl.WorkloadConfig, batch: Optional[int] = None):
-        self.cfg = cfg
+    def __init__(self, cfg: wl.WorkloadConfig, batch: Optional[int] = None, layers: Optional[List[int]] = None):
         self.batch = cfg.batch if batch is None else batch
+        self.layers = list(range(cfg.n_layers)) if layers is None else list(layers)
+        self.full_cfg = cfg                                   # what the random streams are keyed by
+        self.cfg = cfg if layers is None else cfg.scaled(n_layers=len(self.layers))
+        # every random tensor is drawn row by row from one stream, so a generator asked for fewer sequences returns the
+        # same first rows: the numbers are drawn for `batch` sequences only
+        self.gen_cfg = cfg.scaled(batch=self.batch)
         self.ctrl = wl.controller_weights(cfg)
-        self.w_kv = [wl.projection_weights(cfg, l) for l in range(cfg.n_layers)]
-        self.w_q = [wl.query_weights(cfg, l) for l in range(cfg.n_layers)]
+        self.w_kv = [wl.projection_weights(cfg, l) for l in self.layers]
+        self.w_q = [wl.query_weights(cfg, l) for l in self.layers]
         self.w_kv64 = [w.astype(np.float64) for w in self.w_kv]
         self.w_q64 = [w.astype(np.float64) for w in self.w_q]
         self.r_in = self._r_in()
@@ -46,11 +52,16 @@ class Workload:
         mean = n * self.cfg.rebuild_p
         return int(min(n, np.ceil(mean + 6 * np.sqrt(mean) + 8)))
 
+    def rows(self, first: int, count: int, layer: int = 0) -> np.ndarray:
+        """Layer-input rows [batch, count, d] of tokens first .. first+count-1 for this object's layer `layer`."""
+        src = self.layers[layer] if self.cfg.per_layer_inputs else 0
+        return wl.hidden_rows(self.gen_cfg, first, count, src, self.batch)
+
     def prompt(self, layer: int = 0) -> np.ndarray:
-        return wl.hidden_rows(self.cfg, 0, self.cfg.prompt, layer, self.batch)
+        return self.rows(0, self.cfg.prompt, layer)
 
     def x_new(self, n: int, layer: int = 0) -> np.ndarray:
-        return wl.hidden_rows(self.cfg, n, 1, layer, self.batch)[:, 0, :]
+        return self.rows(n, 1, layer)[:, 0, :]
 
     def qkv(self, n: int, layer: int, x_row: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
         """q, k_new, v_new [B, H, dh] of the token at position n (all sequences in one product)."""
@@ -61,7 +72,7 @@ class Workload:
         k = ao.round_store(ao.rope_rotate(ykv[:, :hd].reshape(B, c.n_heads, c.head_dim), n, c.rope_theta), c.dtype)
         v = ao.round_store(ykv[:, hd:].reshape(B, c.n_heads, c.head_dim), c.dtype)
         if c.identity_projection:          # q, k, v i.i.d. N(0,1): q is its own draw
-            q = np.stack([wl.gaussian(c.seed, "q", (c.n_heads, c.head_dim), 1.0, c.dtype, idx=(layer, n, b))
+            q = np.stack([wl.gaussian(c.seed, "q", (c.n_heads, c.head_dim), 1.0, c.dtype, idx=(self.layers[layer], n, b))
                           for b in range(B)])
         else:
             yq = x64 @ self.w_q64[layer].T
@@ -81,7 +92,7 @@ class Workload:
                 if tok < 0:
                     continue
                 if c.identity_projection:
-                    out[b, :, i] = wl.gaussian(c.seed, "q", (c.n_heads, c.head_dim), 1.0, c.dtype, idx=(layer, tok, b))
+                    out[b, :, i] = wl.gaussian(c.seed, "q", (c.n_heads, c.head_dim), 1.0, c.dtype, idx=(self.layers[layer], tok, b))
                 else:
                     out[b, :, i] = ao.project_q(self.w_q64[layer], x_table[b, tok], tok, c.n_heads, c.head_dim,
                                                 c.rope_theta, c.dtype)
@@ -90,7 +101,7 @@ class Workload:
     def explicit(self, step: int, n: int) -> Tuple[Optional[np.ndarray], Optional[np.ndarray]]:
         if self.cfg.rebuild_mode != "explicit":
             return None, None
-        return wl.rebuild_flags(self.cfg, step, n, self.r_in, self.batch)
+        return wl.rebuild_flags(self.gen_cfg, step, n, self.r_in, self.batch)
 
 
 def make_oracle(w: Workload) -> ao.AdoreOracle:

@@ -13,8 +13,7 @@ from typing import Dict, Optional, Tuple
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# ADORE_LIB points at another build of the same library (e.g. an instrumented one)
-LIB_PATH = os.environ.get("ADORE_LIB") or os.path.join(_HERE, "libadore.so")
+LIB_PATH = os.path.join(_HERE, "libadore.so")
 
 ADORE_F32, ADORE_BF16 = 0, 1
 ADORE_REBUILD_POLICY, ADORE_REBUILD_EXPLICIT = 0, 1
@@ -53,8 +52,8 @@ EXPORTS = ["adore_cache_create", "adore_cache_destroy", "adore_cache_set_project
            "adore_decode_step_host", "adore_rebuild", "adore_cache_slot_map", "adore_cache_rebuild_list",
            "adore_cache_step_info", "adore_cache_scores", "adore_cache_kv", "adore_cache_num_tokens",
            "adore_cache_launch_count", "adore_cache_sync_status", "adore_cache_join", "adore_status_string",
-           "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_rebuild_rows",
-           "adore_controller_score_static", "adore_probe_read_bandwidth",
+           "adore_cache_set_stage_timing", "adore_cache_stage_times", "adore_cache_group_times", "adore_cache_rebuild_rows",
+           "adore_controller_score_static",
            "adore_cache_export_state", "adore_cache_import_state", "adore_step_begin", "adore_attend_rows",
            "adore_label_tokens", "adore_decode_rebuild_host", "adore_decode_rebuild_host_queued", "adore_cache_wait_outputs"]
 
@@ -96,10 +95,10 @@ def _lib():
         lib.adore_cache_wait_outputs.argtypes = [vp]
         lib.adore_cache_set_stage_timing.argtypes = [vp, i32]
         lib.adore_cache_stage_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+        lib.adore_cache_group_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         lib.adore_cache_rebuild_rows.argtypes = [vp, C.POINTER(C.c_int64)]
         lib.adore_cache_export_state.argtypes = [vp, vp, C.POINTER(C.c_size_t)]
         lib.adore_cache_import_state.argtypes = [vp, vp, C.c_size_t]
-        lib.adore_probe_read_bandwidth.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp]
         lib.adore_controller_score_static.argtypes = [C.POINTER(adore_controller_weights_t), C.c_int, i32, i32, i32, vp, vp,
                                                       i32, C.c_float, vp, vp, vp]
         _LIB = lib
@@ -252,8 +251,16 @@ def adore_cache_import_state(cache: int, host_buf: np.ndarray) -> None:
     _check(_lib().adore_cache_import_state(cache, _ptr(host_buf), host_buf.nbytes), "adore_cache_import_state")
 
 
-def adore_cache_set_stage_timing(cache: int, enable: bool) -> None:
+def adore_cache_set_stage_timing(cache: int, enable) -> None:
+    """enable: 0/False off, 1/True per-stage timing, 2 group timing."""
     _check(_lib().adore_cache_set_stage_timing(cache, int(enable)), "adore_cache_set_stage_timing")
+
+
+def adore_cache_group_times(cache: int):
+    """Returns (ms, steps): device time of the attention + selection group summed over the steps since the last call."""
+    ms, n = C.c_double(), C.c_int64()
+    _check(_lib().adore_cache_group_times(cache, C.byref(ms), C.byref(n)), "adore_cache_group_times")
+    return ms.value, n.value
 
 
 def adore_cache_stage_times(cache: int):
@@ -278,12 +285,6 @@ def adore_controller_score_static(weights_dev: Dict[str, object], dtype: str, ba
     _check(_lib().adore_controller_score_static(C.byref(w), ADORE_F32 if dtype == "f32" else ADORE_BF16, batch, hidden,
                                                 ctrl_hidden, _ptr(x), _ptr(z), position, pos_scale, _ptr(score),
                                                 _ptr(sigma), cuda_stream or None), "adore_controller_score_static")
-
-
-def adore_probe_read_bandwidth(buffer, n_blocks: int, block_rows: int, row_bytes: int, kept_rows: int, gather: bool,
-                               ctas: int, scratch4, cuda_stream: int = 0) -> None:
-    _check(_lib().adore_probe_read_bandwidth(_ptr(buffer), n_blocks, block_rows, row_bytes, kept_rows, int(gather), ctas,
-                                             _ptr(scratch4), cuda_stream or None), "adore_probe_read_bandwidth")
 
 
 def adore_status_string(status: int) -> str:

@@ -8,8 +8,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB = os.path.join(HERE, "libadore.so")
-SOURCES = [os.path.join(HERE, "csrc", "adore_api.cu"), os.path.join(HERE, "csrc", "controller_static.cu"),
-           os.path.join(HERE, "csrc", "probe.cu")]
+SOURCES = [os.path.join(HERE, "csrc", "adore_api.cu"), os.path.join(HERE, "csrc", "controller_static.cu")]
 
 
 def _newest_source_mtime() -> float:

@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <initializer_list>
 #include <new>
 #include <vector>
 
@@ -136,6 +137,14 @@ struct adore_cache {
   std::vector<int> ev_stage;
   double stage_ms[4] = {0, 0, 0, 0};        // attention, controller+selection, rebuild, admit (layer 0)
   int64_t stage_launches[4] = {0, 0, 0, 0};
+  // optional group timing: the step's schedule is left as it is (side streams and all); three events per step mark where
+  // the attention + selection group starts, where its main-stream part ends (the last layer's attention, or the new
+  // token's row of a one-layer cache) and where the controller chain ends
+  bool group_timing = false;
+  std::vector<cudaEvent_t> grp_pool;
+  size_t grp_used = 0;
+  double grp_ms = 0;
+  int64_t grp_steps = 0;
   double* part = nullptr;
   size_t part_doubles = 0;
   int ksplit = 1;
@@ -217,6 +226,22 @@ struct StageScope {
   ~StageScope() { if (on) cudaEventRecord(c->ev_pool[idx + 1], st); }
 };
 
+// Group timing: the idx-th event (0 start, 1 end on the main stream, 2 end of the controller chain) of the open step.
+adore_status_t group_mark(adore_cache* c, int idx, cudaStream_t stream) {
+  if (!c->group_timing) return ADORE_OK;
+  if (idx == 0) {
+    if (c->grp_used + 3 > c->grp_pool.size())
+      for (int i = 0; i < 3; ++i) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) return ADORE_ERR_CUDA;
+        c->grp_pool.push_back(e);
+      }
+    c->grp_used += 3;
+  }
+  if (c->grp_used < 3) return ADORE_OK;
+  return cudaEventRecord(c->grp_pool[c->grp_used - 3 + idx], stream) == cudaSuccess ? ADORE_OK : ADORE_ERR_CUDA;
+}
+
 adore_status_t cuda_fail(cudaError_t e) {
   if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return ADORE_ERR_OOM; }
   return ADORE_ERR_CUDA;
@@ -253,6 +278,25 @@ adore_status_t dev_alloc(adore_cache* c, P** out, size_t bytes, bool zero) {
   c->owned.push_back(p);
   if (zero) CUDA_OK(cudaMemsetAsync(p, 0, bytes ? bytes : 16, c->stream));
   *out = static_cast<P*>(p);
+  return ADORE_OK;
+}
+
+// A group of device buffers that only make sense together: either all exist afterwards (owned by the cache), or none
+// does and nothing is left behind.
+struct GroupItem { void** out; size_t bytes; };
+adore_status_t alloc_group(adore_cache* c, std::initializer_list<GroupItem> items) {
+  std::vector<void*> got;
+  for (const GroupItem& it : items) {
+    void* p = nullptr;
+    if (cudaMalloc(&p, it.bytes ? it.bytes : 16) != cudaSuccess) {
+      cudaGetLastError();
+      for (void* g : got) cudaFree(g);
+      return ADORE_ERR_OOM;
+    }
+    got.push_back(p);
+  }
+  size_t i = 0;
+  for (const GroupItem& it : items) { *it.out = got[i]; c->owned.push_back(got[i]); ++i; }
   return ADORE_OK;
 }
 
@@ -312,7 +356,7 @@ adore_status_t launch_gates(adore_cache* c, const T* x, long long seq_stride, in
   g.w_ih = c->w_ih; g.part = c->part; g.ksplit = ksplit;
   const int per = (c->cfg.hidden + ksplit - 1) / ksplit;
   g.kslice = ((per + kGateKInner - 1) / kGateKInner) * kGateKInner;
-  static const bool narrow_only = std::getenv("ADORE_GATES_NARROW") != nullptr;   // A/B switch
+  static const bool narrow_only = dev_switch("ADORE_GATES_NARROW");
   if (g.rows >= kGateWideMinRows && !narrow_only) {
     dim3 grid((g.G + kGateWideG - 1) / kGateWideG, (g.rows + kGateWideR - 1) / kGateWideR, ksplit);
     ctrl_gates_wide_kernel<T><<<grid, kGateWideThreads, kGateWideSmem, stream>>>(g);
@@ -350,7 +394,7 @@ bool launch_attention_rows_as(adore_cache* c, int layer, const AttnParams<__nv_b
 template <>
 bool launch_attention_rows<__nv_bfloat16>(adore_cache* c, int layer, const AttnParams<__nv_bfloat16>& p, int rows_q) {
   const adore_config_t& f = c->cfg;
-  static const bool off = std::getenv("ADORE_ROWS_SIMT") != nullptr;     // A/B switch
+  static const bool off = dev_switch("ADORE_ROWS_SIMT");
   const size_t smem = rows_smem_bytes(f.capacity, f.head_dim, std::min(rows_q, kRowsMaxQ));
   const int per_lane = (f.capacity + 1 + 31) / 32;
   if (off || c->map_k.empty() || per_lane > kRowsKeysPerLaneMax || smem > 200 * 1024) return false;
@@ -394,8 +438,6 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
   const int grid = f.batch * f.n_heads * rows_q;
   StageScope scope(c, 0);
   cudaError_t e;
-  // ADORE_ATTN_DIRECT=1 selects the variant without shared-memory staging (for A/B timing)
-  static const bool direct = std::getenv("ADORE_ATTN_DIRECT") != nullptr;
   // Few (b, h) pairs: a cluster of CTAs shares each of them. Not at layer 0: there the controller's
   // one-CTA-per-sequence kernel (200 KB of shared memory each) runs beside the attention and needs
   // SMs that the extra CTAs would occupy; measured at batch 1 the step got slower, not faster.
@@ -409,18 +451,10 @@ adore_status_t launch_attention(adore_cache* c, int layer, const void* q, const 
     CUDA_OK(er);
     return ADORE_OK;
   }
-  const int split = (direct || layer == 0) ? 1 : attn_split_factor(grid, f.capacity, c->sms);
+  if (!attn_tma_usable<T>(f.capacity, f.head_dim)) return ADORE_ERR_UNSUPPORTED;
+  const int split = layer == 0 ? 1 : attn_split_factor(grid, f.capacity, c->sms);
   if (split > 1) e = launch_attention_split<T>(p, f.head_dim, grid, split, c->stream);
-  else if (!direct && attn_tma_usable<T>(f.capacity, f.head_dim)) e = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
-  else if (f.head_dim == 64) {
-    const size_t smem = attn_smem_bytes(f.capacity, 64);
-    attention_kernel<T, 64><<<grid, kAttnThreads, smem, c->stream>>>(p);
-    e = cudaGetLastError();
-  } else {
-    const size_t smem = attn_smem_bytes(f.capacity, 128);
-    attention_kernel<T, 128><<<grid, kAttnThreads, smem, c->stream>>>(p);
-    e = cudaGetLastError();
-  }
+  else e = launch_attention_tma<T>(p, f.head_dim, grid, c->stream);
   ++c->launches;
   CUDA_OK(e);
   return ADORE_OK;
@@ -446,7 +480,7 @@ adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, co
     // Rows gathered from the token store for this step's table serve every layer that rebuilds from the store.
     const bool from_store = step_table && x_table == nullptr && size_t(m_max) <= c->tc.a_rows;
     int launched = 0;
-    static const int lean_mode = std::getenv("ADORE_REBUILD_LEAN") ? std::atoi(std::getenv("ADORE_REBUILD_LEAN")) : 1;   // A/B switch
+    static const int lean_mode = dev_switch_int("ADORE_REBUILD_LEAN", 1);
     cudaError_t e = launch_rebuild_tc(c->tc, p, layer, m_max, stream, &launched, from_store && c->rows_gathered,
                                       lean_mode != 0 && stream != c->stream);
     c->launches += launched;
@@ -796,9 +830,8 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   for (void* p : c->owned) cudaFree(p);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->grp_pool) cudaEventDestroy(e);
   for (cudaEvent_t e : c->ev_stage_free) cudaEventDestroy(e);
-  void* hosts[] = {c->h_q, c->h_k, c->h_v, c->h_x, c->h_out, c->h_list, c->h_count, c->hq_all, c->hq_x, c->hq_list, c->hq_count};
-  for (void* p : hosts) if (p) cudaFree(p);
   cudaGetLastError();
   delete c;
   return ADORE_OK;
@@ -905,6 +938,7 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     // the attention is the longest of the three and is launched first; the side streams start from the same point
     // (with per-stage timing on: from the end of the attention, so that no stage overlaps another)
     if (!c->timing) CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
+    if (group_mark(c, 0, c->stream) != ADORE_OK) return ADORE_ERR_CUDA;
     c->attn = c->cur;
     st = f.dtype == ADORE_F32 ? launch_attention<float>(c, 0, q, k_new, v_new, out, weights, false)
                               : launch_attention<__nv_bfloat16>(c, 0, q, k_new, v_new, out, weights, false);
@@ -914,6 +948,7 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
     st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel, true);
     if (st != ADORE_OK) return st;
+    if (group_mark(c, 2, c->ctl) != ADORE_OK) return ADORE_ERR_CUDA;
     c->joined = sel == c->stream;
     if (!c->joined) CUDA_OK(cudaEventRecord(c->ev_join, sel));
     c->cur = 1 - c->cur;
@@ -926,8 +961,9 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     if (wait_rebuild(c, layer, c->stream) != ADORE_OK) return ADORE_ERR_CUDA;
     adore_status_t st = f.dtype == ADORE_F32 ? launch_attention<float>(c, layer, q, k_new, v_new, out, weights, true)
                                              : launch_attention<__nv_bfloat16>(c, layer, q, k_new, v_new, out, weights, true);
-    if (st != ADORE_OK || !from_attention) return st;
-    return launch_add_attention(c, weights);
+    if (st == ADORE_OK && from_attention) st = launch_add_attention(c, weights);
+    if (st == ADORE_OK && layer == f.n_layers - 1) st = group_mark(c, 1, c->stream);
+    return st;
   }
   if (!c->joined) CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
   c->joined = true;
@@ -942,7 +978,11 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     CUDA_OK(cudaGetLastError());
   }
   // after the join: this step's selection has read the scores it ranks by, the weights count from the next step on
-  if (from_attention) return launch_add_attention(c, weights);
+  if (from_attention) {
+    adore_status_t st = launch_add_attention(c, weights);
+    if (st != ADORE_OK) return st;
+  }
+  if (f.n_layers == 1) return group_mark(c, 1, c->stream);
   return ADORE_OK;
 }
 
@@ -999,10 +1039,10 @@ adore_status_t decode_step_host_impl(adore_cache_t* c, int32_t layer, const void
   const adore_config_t& f = c->cfg;
   const size_t qb = size_t(f.batch) * f.n_heads * f.head_dim * c->esz, xb = size_t(f.batch) * f.hidden * c->esz;
   if (!c->h_q) {
-    CUDA_OK(cudaMalloc(&c->h_q, qb)); CUDA_OK(cudaMalloc(&c->h_k, qb)); CUDA_OK(cudaMalloc(&c->h_v, qb));
-    CUDA_OK(cudaMalloc(&c->h_out, qb)); CUDA_OK(cudaMalloc(&c->h_x, xb));
-    CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->h_list), size_t(f.batch) * f.max_tokens * sizeof(int)));
-    CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->h_count), size_t(f.batch) * sizeof(int)));
+    adore_status_t sa = alloc_group(c, {{&c->h_q, qb}, {&c->h_k, qb}, {&c->h_v, qb}, {&c->h_out, qb}, {&c->h_x, xb},
+                                        {reinterpret_cast<void**>(&c->h_list), size_t(f.batch) * f.max_tokens * sizeof(int)},
+                                        {reinterpret_cast<void**>(&c->h_count), size_t(f.batch) * sizeof(int)}});
+    if (sa != ADORE_OK) return sa;
   }
   if (r_in < 0 || r_in > f.max_tokens) return ADORE_ERR_INVALID_ARG;
   // The staging buffers are free (the previous call waited for every kernel that read them), so the
@@ -1066,17 +1106,27 @@ adore_status_t adore_decode_rebuild_host_queued(adore_cache_t* c, int32_t layer,
   if (r_in < 0 || r_in > f.max_tokens) return ADORE_ERR_INVALID_ARG;
   if (layer == 0 && !x_new) return ADORE_ERR_INVALID_ARG;
   if (!c->hq_all) {
-    CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->hq_all), size_t(f.n_layers) * 4 * qb));
-    CUDA_OK(cudaMalloc(&c->hq_x, xb));
-    CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->hq_list), size_t(f.batch) * f.max_tokens * sizeof(int)));
-    CUDA_OK(cudaMalloc(reinterpret_cast<void**>(&c->hq_count), size_t(f.batch) * sizeof(int)));
-    CUDA_OK(cudaStreamCreateWithFlags(&c->d2h, cudaStreamNonBlocking));
-    for (int l = 0; l < f.n_layers; ++l) {
+    // stream and events first (cheap to undo), the buffers last: the set exists as a whole or not at all
+    cudaStream_t d2h = nullptr;
+    std::vector<cudaEvent_t> evs;
+    bool ok = cudaStreamCreateWithFlags(&d2h, cudaStreamNonBlocking) == cudaSuccess;
+    for (int l = 0; ok && l < f.n_layers; ++l) {
       cudaEvent_t e = nullptr;
-      CUDA_OK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-      c->ev_stage_free.push_back(e);
-      CUDA_OK(cudaEventRecord(e, c->stream));
+      ok = cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+      if (ok) { evs.push_back(e); ok = cudaEventRecord(e, c->stream) == cudaSuccess; }
     }
+    adore_status_t sa = ok ? alloc_group(c, {{reinterpret_cast<void**>(&c->hq_all), size_t(f.n_layers) * 4 * qb}, {&c->hq_x, xb},
+                                             {reinterpret_cast<void**>(&c->hq_list), size_t(f.batch) * f.max_tokens * sizeof(int)},
+                                             {reinterpret_cast<void**>(&c->hq_count), size_t(f.batch) * sizeof(int)}})
+                           : ADORE_ERR_CUDA;
+    if (sa != ADORE_OK) {
+      for (cudaEvent_t e : evs) cudaEventDestroy(e);
+      if (d2h) cudaStreamDestroy(d2h);
+      cudaGetLastError();
+      return sa;
+    }
+    c->d2h = d2h;
+    c->ev_stage_free = evs;
   }
   unsigned char* set = c->hq_all + size_t(layer) * 4 * qb;
   void *dq = set, *dk = set + qb, *dv = set + 2 * qb, *dout = set + 3 * qb;
@@ -1122,7 +1172,7 @@ adore_status_t adore_rebuild(adore_cache_t* c, int32_t layer, const void* x_tabl
   // layer, so the rebuild goes to its own stream, behind everything queued so far (this layer's attention, the
   // selection, the new token's row), and the attention of the following layers runs beside it. (Not with per-stage
   // timing on, where stages must not overlap, and not in the rebuild-first order, whose attention reads these rows.)
-  static const bool inline_only = std::getenv("ADORE_REBUILD_INLINE") != nullptr;   // A/B switch
+  static const bool inline_only = dev_switch("ADORE_REBUILD_INLINE");
   // In the rebuild-first order the attention of layer l reads what rebuild(l) writes, but rebuild(l + 1) needs only the
   // step's selection: on the side stream it starts from the end of adore_step_begin and runs beside the attention of
   // layer l; adore_attend_rows(l + 1) waits for it.
@@ -1204,8 +1254,29 @@ int64_t adore_cache_launch_count(const adore_cache_t* c) { return c ? c->launche
 
 adore_status_t adore_cache_set_stage_timing(adore_cache_t* c, int32_t enable) {
   if (!c) return ADORE_ERR_INVALID_ARG;
+  if (enable < 0 || enable > 2) return ADORE_ERR_INVALID_ARG;
   if (join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
-  c->timing = enable != 0;
+  c->timing = enable == 1;
+  c->group_timing = enable == 2;
+  return ADORE_OK;
+}
+
+adore_status_t adore_cache_group_times(adore_cache_t* c, double* ms, int64_t* steps) {
+  if (!c || !ms || !steps) return ADORE_ERR_INVALID_ARG;
+  if (join_controller(c) != ADORE_OK || join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
+  for (size_t i = 0; i + 3 <= c->grp_used; i += 3) {
+    float a = 0.f, b = 0.f;
+    if (cudaEventElapsedTime(&a, c->grp_pool[i], c->grp_pool[i + 1]) != cudaSuccess) { cudaGetLastError(); continue; }   // a step left open
+    if (cudaEventElapsedTime(&b, c->grp_pool[i], c->grp_pool[i + 2]) != cudaSuccess) { cudaGetLastError(); b = 0.f; }
+    c->grp_ms += double(a > b ? a : b);
+    c->grp_steps += 1;
+  }
+  c->grp_used = 0;
+  *ms = c->grp_ms;
+  *steps = c->grp_steps;
+  c->grp_ms = 0;
+  c->grp_steps = 0;
   return ADORE_OK;
 }
 
@@ -1275,6 +1346,47 @@ void add_relative_state(adore_cache* c, std::vector<StateSection>& sec) {
 }
 inline size_t pad8(size_t v) { return (v + 7) & ~size_t(7); }
 
+// Index checks of a snapshot's integer sections before any of it reaches the device: the selection, the gather and the
+// GEMM's scatter use these values as indices. `sec` is the cache's own section list (sizes only are used).
+bool snapshot_consistent(const adore_config_t& f, const StateHeader& hd, const unsigned char* buf, const std::vector<StateSection>& sec) {
+  std::vector<const unsigned char*> at(sec.size());
+  size_t off = sizeof(StateHeader);
+  for (size_t i = 0; i < sec.size(); ++i) { at[i] = buf + off; off += pad8(sec[i].bytes); }
+  const int B = f.batch, C = f.capacity, MT = f.max_tokens, R = f.rebuild_max, m = C - R, n = hd.n;
+  auto i32 = [&](size_t section, size_t idx) { int v; std::memcpy(&v, at[section] + idx * sizeof(int), sizeof(int)); return v; };
+  for (int map = 0; map < 2; ++map)
+    for (int b = 0; b < B; ++b) {
+      int retained = 0, rebuilt = 0;
+      for (int s = 0; s < C; ++s) {
+        const int tok = i32(size_t(map), size_t(b) * C + s);
+        const unsigned role = at[2 + map][size_t(b) * C + s];
+        if (tok < -1 || tok >= n || role > ROLE_REBUILT || ((tok < 0) != (role == ROLE_EMPTY))) return false;
+        retained += role == ROLE_RETAINED;
+        rebuilt += role == ROLE_REBUILT;
+      }
+      if (retained > m || rebuilt > R) return false;
+    }
+  for (int b = 0; b < B; ++b) {
+    for (int t = 0; t < MT; ++t) {
+      const int s = i32(4, size_t(b) * MT + t);
+      if (s < -1 || s >= C) return false;
+    }
+    const int adm = i32(8, b), ev = i32(9, b), cnt = i32(12, b);
+    if (adm < -1 || adm >= C || ev < -1 || ev >= std::max(n, 1) || cnt < 0 || cnt > R) return false;
+    for (int i = 0; i < cnt; ++i) {
+      const int tok = i32(10, size_t(b) * R + i), slot = i32(11, size_t(b) * R + i);
+      if (tok < 0 || tok >= n || slot < 0 || slot >= C) return false;
+    }
+  }
+  const int total = i32(16, 0);
+  if (total < 0 || total > B * R) return false;
+  for (int i = 0; i < total; ++i) {
+    const int b = i32(13, i), tok = i32(14, i), slot = i32(15, i);
+    if (b < 0 || b >= B || tok < 0 || tok >= n || slot < 0 || slot >= C) return false;
+  }
+  return true;
+}
+
 }  // namespace
 
 adore_status_t adore_cache_export_state(adore_cache_t* c, void* host_buf, size_t* bytes) {
@@ -1315,13 +1427,15 @@ adore_status_t adore_cache_import_state(adore_cache_t* c, const void* host_buf, 
   const adore_config_t& f = c->cfg;
   if (hd.magic != kStateMagic || hd.version != 1 || hd.batch != f.batch || hd.capacity != f.capacity ||
       hd.rebuild_max != f.rebuild_max || hd.max_tokens != f.max_tokens || hd.ctrl_hidden != f.ctrl_hidden ||
-      hd.reserved[0] != (f.flags & ADORE_FLAG_RELATIVE_POSITION) || hd.n < 0 || hd.n > f.max_tokens || (hd.cur != 0 && hd.cur != 1) || (hd.attn != 0 && hd.attn != 1))
+      hd.reserved[0] != (f.flags & ADORE_FLAG_RELATIVE_POSITION) || hd.n < 0 || hd.n > f.max_tokens || (hd.cur != 0 && hd.cur != 1) ||
+      (hd.attn != 0 && hd.attn != 1) || hd.step_open < 0 || hd.step_open > 2)
     return ADORE_ERR_INVALID_ARG;
   std::vector<StateSection> sec = state_sections(c);
   add_relative_state(c, sec);
   size_t need = sizeof(StateHeader);
   for (const StateSection& s : sec) need += pad8(s.bytes);
   if (bytes < need) return ADORE_ERR_INVALID_ARG;
+  if (!snapshot_consistent(f, hd, static_cast<const unsigned char*>(host_buf), sec)) return ADORE_ERR_INVALID_ARG;
   if (join_controller(c) != ADORE_OK || join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
   if (c->aux && cudaStreamSynchronize(c->aux) != cudaSuccess) return ADORE_ERR_CUDA;
@@ -1349,7 +1463,7 @@ adore_status_t adore_label_tokens(const float* weights, int32_t n_layers, int32_
   const size_t smem = size_t(label_pow2(n_slots)) * sizeof(unsigned long long);
   CUDA_OK(cudaMemsetAsync(count, 0, size_t(batch) * n_slots * sizeof(int), st));
   const int n_rows = n_layers * batch * n_heads;
-  static const bool full_sort = std::getenv("ADORE_LABELS_FULL_SORT") != nullptr;   // A/B switch
+  static const bool full_sort = dev_switch("ADORE_LABELS_FULL_SORT");
   if (!full_sort && half <= kLabelWarpMaxHalf && n_slots <= 32 * kLabelWarpKeysPerLane) {
     int P = 32;
     while (P < half) P <<= 1;

@@ -7,9 +7,11 @@
 // out per slot. Finally the current token's key/value row is written into its slot (append of
 // the most recent state, Section 2.2 third bullet).
 //
-// One CTA per (b, h). The K block of a (b, h) is one contiguous C*dh array, so phase 1 streams it
-// with 16-byte loads, phase 2 finds the K-th largest logit with a 4-pass radix select in shared
-// memory, phase 3 is the softmax, phase 4 reads ONLY the kept value rows.
+// This header holds the phases the attention kernels share: given the logits of a (b, h) pair in shared
+// memory, phase 2 finds the K-th largest logit with a 4-pass radix select, phase 3 is the softmax, phase 4
+// reads ONLY the kept value rows, and the tail writes the output and the current token's row. Phase 1 (the
+// logits) belongs to the kernels: attention_tma.cuh stages the contiguous C*dh key block of a pair through
+// shared memory, attention_split.cuh spreads it over a thread-block cluster.
 #pragma once
 
 #include "common.cuh"
@@ -215,20 +217,14 @@ __device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, 
   constexpr int LPR = DH / EPL;
   constexpr int RPW = 32 / LPR;
   constexpr int U = kAttnUnroll;
-  float* s_logit = sm.logit;
-  int* s_list = sm.list;
-  float* s_red = sm.red;
+  const float* s_logit = sm.logit;
+  const int* s_list = sm.list;
   const int C = p.C;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int sub = lane / LPR, li = lane % LPR;
-  const int b = bh / p.H;
   const size_t row_bytes = size_t(DH) * sizeof(T);
-  const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * row_bytes;
   const unsigned char* Vb = reinterpret_cast<const unsigned char*>(p.Vc) + size_t(bh) * C * row_bytes;
-  const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * row_bytes;
   const unsigned char* vnew = reinterpret_cast<const unsigned char*>(p.v_new) + size_t(bh) * row_bytes;
-  (void)NW; (void)RPW; (void)U; (void)s_logit; (void)s_list; (void)s_red; (void)warp; (void)sub; (void)li; (void)b;
-  (void)Kb; (void)Vb; (void)knew; (void)vnew;
   // ---- phase 4: weighted sum of the kept value rows ----------------------------------------
   for (int j0 = j_begin + warp * RPW; j0 < n_kept; j0 += NW * RPW * U) {   // entries [j_begin, n_kept) of the kept list
     uint4 vv[U];
@@ -263,22 +259,16 @@ __device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const A
   constexpr int NW = NT / 32;
   constexpr int EPL = Elem<T>::kPer16B;
   constexpr int LPR = DH / EPL;
-  constexpr int RPW = 32 / LPR;
-  constexpr int U = kAttnUnroll;
-  float* s_logit = sm.logit;
-  int* s_list = sm.list;
   float* s_red = sm.red;
   const int C = p.C;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane / LPR, li = lane % LPR;
   const int b = bh / p.H;
   const size_t row_bytes = size_t(DH) * sizeof(T);
-  const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * row_bytes;
-  const unsigned char* Vb = reinterpret_cast<const unsigned char*>(p.Vc) + size_t(bh) * C * row_bytes;
+  unsigned char* Kb = reinterpret_cast<unsigned char*>(p.Kc) + size_t(bh) * C * row_bytes;
+  unsigned char* Vb = reinterpret_cast<unsigned char*>(p.Vc) + size_t(bh) * C * row_bytes;
   const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * row_bytes;
   const unsigned char* vnew = reinterpret_cast<const unsigned char*>(p.v_new) + size_t(bh) * row_bytes;
-  (void)NW; (void)RPW; (void)U; (void)s_logit; (void)s_list; (void)s_red; (void)warp; (void)sub; (void)li; (void)b;
-  (void)Kb; (void)Vb; (void)knew; (void)vnew;
 #pragma unroll
   for (int o = LPR; o < 32; o <<= 1)
 #pragma unroll
@@ -299,83 +289,14 @@ __device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const A
     const int s = p.admit_slot[b];
     if (s >= 0 && s < C) {
       constexpr int V16 = int(sizeof(T)) * DH / 16;
-      unsigned char* kd = const_cast<unsigned char*>(Kb) + size_t(s) * row_bytes;
-      unsigned char* vd = const_cast<unsigned char*>(Vb) + size_t(s) * row_bytes;
+      unsigned char* kd = Kb + size_t(s) * row_bytes;
+      unsigned char* vd = Vb + size_t(s) * row_bytes;
       if (tid < V16) reinterpret_cast<uint4*>(kd)[tid] = reinterpret_cast<const uint4*>(knew)[tid];
       else if (tid < 2 * V16) reinterpret_cast<uint4*>(vd)[tid - V16] = reinterpret_cast<const uint4*>(vnew)[tid - V16];
     } else if (tid == 0) {
       set_error(p.err, ERRW_BOUNDS);
     }
   }
-}
-
-// Phases 2-4 and the admit write for kernels that gather the value rows with direct loads.
-template <typename T, int DH, int NT = kAttnThreads>
-__device__ __forceinline__ void attention_tail(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh) {
-  const int n_kept = attention_keep_and_weights<T, DH, NT>(p, sm, bh);
-  float acc[Elem<T>::kPer16B];
-#pragma unroll
-  for (int e = 0; e < Elem<T>::kPer16B; ++e) acc[e] = 0.f;
-  attention_values_direct<T, DH, NT>(p, sm, bh, n_kept, acc);
-  attention_finish<T, DH, NT>(p, sm, bh, acc);
-}
-
-template <typename T, int DH>
-__global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParams<T> p) {
-  constexpr int NT = kAttnThreads;
-  constexpr int NW = NT / 32;
-  constexpr int EPL = Elem<T>::kPer16B;   // elements per lane (one 16-byte load)
-  constexpr int LPR = DH / EPL;           // lanes that share one row
-  constexpr int RPW = 32 / LPR;           // rows per warp-wide load
-  static_assert(LPR >= 1 && LPR <= 32 && (LPR & (LPR - 1)) == 0, "row must split over a warp");
-  constexpr int U = kAttnUnroll;
-
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  const int C = p.C, rows = C + 1;
-  const AttnSmem<DH> sm(smem_raw, rows);
-  float* s_logit = sm.logit;
-
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int sub = lane / LPR, li = lane % LPR;
-  const int bh = blockIdx.x, b = bh / p.H;
-  const size_t row_bytes = size_t(DH) * sizeof(T);
-  const unsigned char* Kb = reinterpret_cast<const unsigned char*>(p.Kc) + size_t(bh) * C * row_bytes;
-  const unsigned char* knew = reinterpret_cast<const unsigned char*>(p.k_new) + size_t(bh) * row_bytes;
-  const int* map = p.slot_tok + size_t(b) * C;
-
-  // ---- phase 1: logits -------------------------------------------------------------------
-  float qf[EPL];
-  {
-    const uint4 qr = *reinterpret_cast<const uint4*>(
-        reinterpret_cast<const unsigned char*>(p.q) + size_t(bh) * row_bytes + li * 16);
-    Elem<T>::unpack(qr, qf);
-  }
-  for (int r0 = warp * RPW; r0 < rows; r0 += NW * RPW * U) {
-    uint4 kv[U];
-    bool ok[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int row = r0 + u * NW * RPW + sub;
-      ok[u] = row < rows && (row == C || map[row] >= 0);
-      kv[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (ok[u]) kv[u] = ldg_stream((row == C ? knew : Kb + size_t(row) * row_bytes) + li * 16);
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int row = r0 + u * NW * RPW + sub;
-      float kf[EPL];
-      Elem<T>::unpack(kv[u], kf);
-      float dot = 0.f;
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) dot = fmaf(qf[e], kf[e], dot);
-#pragma unroll
-      for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-      if (li == 0 && row < rows) s_logit[row] = ok[u] ? dot * p.scale : -INFINITY;
-    }
-  }
-  __syncthreads();
-
-  attention_tail<T, DH>(p, sm, bh);
 }
 
 }  // namespace adore

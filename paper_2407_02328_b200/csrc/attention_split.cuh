@@ -1,7 +1,7 @@
 // Split-slot decode attention for launches with few (sequence, head) pairs.
 //
-// Same computation as attention_kernel (Section 2.1 target attention with the top-K mask of
-// Section 2.2). With a small batch there are fewer (b, h) blocks than SMs and one CTA per block leaves
+// Section 2.1 target attention with the top-K mask of Section 2.2 (the phases after the logits are
+// shared, attention.cuh). With a small batch there are fewer (b, h) blocks than SMs and one CTA per block leaves
 // most of the memory system idle, so a thread-block cluster of S CTAs shares one (b, h):
 //   phase 1   CTA r computes the logits of slots [r*C/S, (r+1)*C/S) (the last CTA also takes the
 //             current token's own key);

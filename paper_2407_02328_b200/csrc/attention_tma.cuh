@@ -1,7 +1,7 @@
 // Decode attention, phase 1 staged through shared memory by the bulk-copy engine (TMA).
 //
-// Same computation as attention_kernel (Section 2.1 target attention with the top-K mask of
-// Section 2.2); only the way the key rows reach the SM differs. The K block of one (sequence,
+// Section 2.1 target attention with the top-K mask of Section 2.2 (the phases after the logits are
+// shared, attention.cuh); only the way the key rows reach the SM differs. The K block of one (sequence,
 // head) is a contiguous C*dh array, so one elected thread streams it in 8 KB chunks with
 // cp.async.bulk into a 4-deep ring; an mbarrier per stage counts the bytes. The warps read the
 // rows from shared memory (conflict-free 16-byte accesses). This keeps 24-32 KB in flight per

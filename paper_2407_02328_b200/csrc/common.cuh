@@ -98,6 +98,17 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
   return r;
 }
 
+// ---- development switches -------------------------------------------------------------------------
+// A build with -DADORE_DEVTOOLS reads a few environment variables that turn a launch choice off, for A/B timing of
+// the variant that then serves the launch. The ordinary build reads no environment variable at all.
+#ifdef ADORE_DEVTOOLS
+inline bool dev_switch(const char* name) { return std::getenv(name) != nullptr; }
+inline int dev_switch_int(const char* name, int dflt) { const char* v = std::getenv(name); return v ? std::atoi(v) : dflt; }
+#else
+inline bool dev_switch(const char*) { return false; }
+inline int dev_switch_int(const char*, int dflt) { return dflt; }
+#endif
+
 // ---- programmatic dependent launch ----------------------------------------------------------------
 // A kernel launched with launch_dependent() may be placed on the SMs while the kernel ahead of it in the stream is
 // still finishing, which hides its launch latency. Such a kernel calls wait_for_prior_grid() before it reads anything
@@ -111,7 +122,7 @@ __device__ __forceinline__ void let_next_grid_start() { asm volatile("griddepcon
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                                     Args&&... args) {
-  static const bool off = std::getenv("ADORE_NO_DEPENDENT_LAUNCH") != nullptr;   // A/B switch
+  static const bool off = dev_switch("ADORE_NO_DEPENDENT_LAUNCH");
   cudaLaunchConfig_t lc{};
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -83,6 +83,12 @@ extern "C" adore_status_t adore_controller_score_static(const adore_controller_w
   if (!w->gru_w_ih || !w->gru_w_hh || !w->gru_b_ih || !w->gru_b_hh || !w->pos_w || !w->pos_b || !w->mlp_w1 ||
       !w->mlp_b1 || !w->mlp_w2 || !w->mlp_b2)
     return ADORE_ERR_INVALID_ARG;
+  // The gate product reads x and W_ih in 16-byte pieces, 32 elements of a row at a time with no bound inside a piece:
+  // rows must be whole pieces and start on a 16-byte boundary (the cache-based path has the same rule for `hidden`).
+  if (hidden % 64 != 0) return ADORE_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(x) % 16 != 0 || reinterpret_cast<uintptr_t>(w->gru_w_ih) % 16 != 0 ||
+      reinterpret_cast<uintptr_t>(z) % 8 != 0)
+    return ADORE_ERR_UNSUPPORTED;
   const int G = 3 * ctrl_hidden;
   // the partial sums of one k-slice must fit the fixed array
   if (size_t(batch) * size_t(G) > kStaticPartDoubles) return ADORE_ERR_UNSUPPORTED;

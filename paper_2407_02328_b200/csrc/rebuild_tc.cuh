@@ -487,7 +487,7 @@ inline adore_status_t tc_init(TcState& s, const adore_config_t& f, std::vector<v
   s.N = 2 * f.n_heads * f.head_dim;
   s.K = f.hidden;
   if (s.N % 128 != 0 || s.K % kTcBK != 0) return ADORE_OK;          // shape not tiled: the ALU path serves it
-  if (std::getenv("ADORE_REBUILD_SIMT") != nullptr) return ADORE_OK; // cross-check switch
+  if (dev_switch("ADORE_REBUILD_SIMT")) return ADORE_OK;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult q;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || fn == nullptr ||
@@ -523,7 +523,7 @@ inline adore_status_t tc_init(TcState& s, const adore_config_t& f, std::vector<v
                            int(TcSmem<128, kTcLeanStages>::kTotal)) != cudaSuccess)
     return ADORE_ERR_CUDA;
   // the two-SM kernel needs pairs of SMs that can host a cluster of two 1-CTA-per-SM blocks
-  if (s.N % kPairBN == 0 && std::getenv("ADORE_REBUILD_ONE_SM") == nullptr &&
+  if (s.N % kPairBN == 0 && !dev_switch("ADORE_REBUILD_ONE_SM") &&
       cudaFuncSetAttribute(rebuild_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kPairSmemBytes)) == cudaSuccess) {
     cudaLaunchConfig_t lc{};
     cudaLaunchAttribute at[1];
@@ -583,7 +583,7 @@ inline cudaError_t launch_rebuild_tc<__nv_bfloat16>(TcState& s, const RebuildPar
     g.Kc = rp.Kc; g.Vc = rp.Vc; g.row_b = rp.row_b + base; g.row_tok = rp.row_tok + base; g.row_slot = rp.row_slot + base;
     g.row_total = rp.row_total; g.row_base = base; g.row_limit = limit;
     g.rope_cos = rp.rope_cos; g.rope_sin = rp.rope_sin; g.H = rp.H; g.DH = rp.DH; g.C = rp.C; g.N = rp.N; g.K = rp.d; g.err = rp.err;
-    static const int max_split = std::getenv("ADORE_TC_KSPLIT_MAX") ? std::atoi(std::getenv("ADORE_TC_KSPLIT_MAX")) : 4;
+    static const int max_split = dev_switch_int("ADORE_TC_KSPLIT_MAX", 4);
     const TcPlan plan = tc_plan(limit, s.N, s.K, s.sms, s.pairs, max_split);
     g.ksplit = plan.ksplit; g.partial = s.partial; g.unit_cnt = s.unit_cnt;
     if (plan.kind == 2) {
@@ -593,7 +593,7 @@ inline cudaError_t launch_rebuild_tc<__nv_bfloat16>(TcState& s, const RebuildPar
       at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
       at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
       at[1].val.programmaticStreamSerializationAllowed = 1;
-      static const bool no_dep = std::getenv("ADORE_NO_DEPENDENT_LAUNCH") != nullptr;
+      static const bool no_dep = dev_switch("ADORE_NO_DEPENDENT_LAUNCH");
       lc.gridDim = dim3(unsigned(plan.grid)); lc.blockDim = dim3(kTcThreads); lc.dynamicSmemBytes = kPairSmemBytes;
       lc.stream = stream; lc.attrs = at; lc.numAttrs = no_dep ? 1 : 2;
       e = cudaLaunchKernelEx(&lc, rebuild_tc_pair_kernel, s.map_a, s.map_w128[layer], g);

@@ -54,3 +54,25 @@ def test_roofline_arithmetic():
     assert nbytes == (8192 * 4096 + 16384 * 4096 + 16384 * 8192) * 2
     peaks, kind = bench.measured_peaks()
     assert kind in ("measured", "fallback") and peaks["hbm_gbs"] > 1000
+
+
+def test_workload_for_a_few_sequences_and_layers_draws_the_same_numbers_as_the_full_one():
+    """The parity tests of the large configurations check some sequences and some layers of a run in which the GPU
+    holds all of them: the reduced workload must hand out exactly the rows, flags and weights of the full one."""
+    import numpy as np
+    import workloads as wl
+    from oracle.harness import Workload
+    cfg = wl.WorkloadConfig(name="sub", dtype="bf16", n_layers=4, batch=6, n_heads=2, head_dim=64, hidden=64, capacity=16,
+                            topk=8, rebuild_max=4, prompt=5, steps=9, rope_theta=1.0e4, rebuild_mode="explicit",
+                            rebuild_p=0.3, seed=5, per_layer_inputs=True)
+    full = Workload(cfg)
+    part = Workload(cfg, batch=2, layers=[0, 3])
+    assert part.cfg.n_layers == 2 and part.r_in == full.r_in
+    assert np.array_equal(part.prompt(1), full.prompt(3)[:2]) and np.array_equal(part.prompt(0), full.prompt(0)[:2])
+    assert np.array_equal(part.x_new(7, 1), full.x_new(7, 3)[:2])
+    assert np.array_equal(part.w_kv[1], full.w_kv[3]) and np.array_equal(part.w_q[1], full.w_q[3])
+    for a, b in zip(part.explicit(4, 9), full.explicit(4, 9)):
+        assert np.array_equal(a, b[:2])
+    x = full.x_new(6, 3)
+    for a, b in zip(part.qkv(6, 1, x[:2]), full.qkv(6, 3, x)):
+        assert np.allclose(a, b[:2], rtol=0, atol=1e-6)

@@ -134,3 +134,34 @@ def test_a_cache_that_cannot_fit_is_refused_with_out_of_memory_and_leaves_the_de
         lib.adore_cache_sync_status(g.handle)
     finally:
         g.close()
+
+
+def test_a_bounded_device_wait_that_runs_out_sets_the_timeout_bit_and_returns():
+    """Every mbarrier wait of the library is bounded (mbar_wait_bounded): on expiry the kernel sets the timeout bit of an
+    error word and leaves through its ordinary exit. Here that path is taken in the safe form: a test-only kernel built
+    from the library's own mbarrier header waits on a barrier nobody arrives on, with nothing in flight. The kernel must
+    return, the word must carry the timeout bit (the one adore_cache_sync_status reports as ADORE_ERR_TIMEOUT), and a
+    cache must work as usual afterwards."""
+    import ctypes
+    from tests.native import build_wait_probe
+    torch, lib, w, g, to_dev = _setup()
+    try:
+        probe = ctypes.CDLL(build_wait_probe())
+        probe.wait_probe_run.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+        probe.wait_probe_timeout_bit.restype = ctypes.c_uint
+        words = torch.zeros(2, dtype=torch.int32, device="cuda")
+        ctas = 4
+        rc = probe.wait_probe_run(words.data_ptr(), words.data_ptr() + 4, ctas, torch.cuda.current_stream().cuda_stream)
+        assert rc == 0
+        torch.cuda.synchronize()                              # the kernel came back: the wait is bounded
+        err_word, reached = (int(v) for v in words.cpu())
+        assert err_word == probe.wait_probe_timeout_bit() == 1
+        assert reached == ctas, "every CTA must leave through the common exit"
+        assert lib.STATUS_NAMES[7] == "TIMEOUT"
+        n = lib.adore_cache_num_tokens(g.handle)
+        q, k, v, x = _inputs(w, to_dev, n)
+        lib.adore_decode_step(g.handle, 0, q, k, v, x, None, None, 0, g.out, None)    # the device and the cache are fine
+        lib.adore_rebuild(g.handle, 0, None)
+        lib.adore_cache_sync_status(g.handle)
+    finally:
+        g.close()

@@ -11,16 +11,25 @@ SMALL = wl.WorkloadConfig(name="small_bf16", dtype="bf16", n_layers=1, batch=3, 
                           rope_theta=1.0e4, rebuild_mode="policy", rebuild_p=0.0, seed=101, ctrl_hidden=128)
 
 
+def _check(name, rep):
+    print("\n" + rep.line(name))
+    # the one exemption of the parity bar: kept sets that differ by a near-tie (float64 logits within 1e-6 of the row's
+    # logit scale); at most 2 per 1000 (sequence, head) rows
+    assert rep.near_ties <= max(2, rep.topk_rows // 500)
+    return rep
+
+
 def _run(cfg, **kw):
     from tests.gpu_driver import run_parity
-    rep = run_parity(cfg, **kw)
-    print(f"\n[{cfg.name}] steps={rep.steps} near_ties={rep.near_ties}+{rep.rounding_ties}r/{rep.topk_rows} rows "
-          f"max_out_err={rep.max_out_err:.3e} max_w_err={rep.max_w_err:.3e} max_kv_ulp={rep.max_kv_ulp:.2f} "
-          f"score_mismatch={rep.score_mismatch}")
-    assert rep.near_ties <= max(2, rep.topk_rows // 1000)
-    # every cache row that came out of the projection can sit one bf16 unit away from the oracle's,
-    # so the share of rows whose K-th logit is decided by such a unit grows with the capacity
-    assert rep.rounding_ties <= max(2, rep.topk_rows // 50)
+    return _check(cfg.name, run_parity(cfg, **kw))
+
+
+def _run_and_repeat_free(cfg, mode="device", sync_every=0, **kw):
+    """Lockstep parity, then the same workload with no host wait between the calls: bit-identical outputs and state."""
+    from tests.gpu_driver import run_parity, run_free, assert_same_run
+    rep = _check(cfg.name, run_parity(cfg, record=True, **kw))
+    record, final = run_free(cfg, batch=kw.get("batch"), steps=kw.get("steps"), mode=mode, sync_every=sync_every)
+    assert_same_run(rep, record, final, f"{cfg.name} ({mode})")
     return rep
 
 
@@ -61,12 +70,14 @@ def test_three_layers_with_their_own_inputs():
 
 def test_rebuilds_beside_the_following_layers_without_a_host_wait_between_steps():
     """In a cache of several layers the rebuild of a layer runs on the library's own stream beside the attention of the
-    layers after it (and of the next step's first layers). The state is only read every fifth step here, so nothing but
-    the library's own stream dependencies orders the rebuilds against the next step's selection, gather and attention."""
-    _run(SMALL.scaled(name="L4_free_running", n_layers=4, batch=2, per_layer_inputs=True, seed=150, steps=20), state_every=5)
-    _run(SMALL.scaled(name="L3_explicit_free_running", n_layers=3, batch=4, n_heads=8, per_layer_inputs=True, rebuild_mode="explicit",
-                      rebuild_p=0.5, rebuild_max=30, capacity=64, topk=20, prompt=100, seed=151, steps=15), state_every=5)
-    _run(SMALL.scaled(name="L2_store_rows_free_running", n_layers=2, batch=2, seed=152, steps=15), state_every=15)
+    layers after it (and of the next step's first layers). The lockstep run reads the rebuilt rows after every call; the
+    free run that must repeat it bit for bit has nothing but the library's own stream dependencies to order the rebuilds
+    against the next step's selection, gather and attention."""
+    _run_and_repeat_free(SMALL.scaled(name="L4_free_running", n_layers=4, batch=2, per_layer_inputs=True, seed=150, steps=20), state_every=5)
+    _run_and_repeat_free(SMALL.scaled(name="L3_explicit_free_running", n_layers=3, batch=4, n_heads=8, per_layer_inputs=True,
+                                      rebuild_mode="explicit", rebuild_p=0.5, rebuild_max=30, capacity=64, topk=20, prompt=100,
+                                      seed=151, steps=15), state_every=5)
+    _run_and_repeat_free(SMALL.scaled(name="L2_store_rows_free_running", n_layers=2, batch=2, seed=152, steps=15), state_every=15)
 
 
 def test_host_buffer_entry_point():
@@ -79,16 +90,14 @@ def test_host_buffer_entry_point():
 
 def test_queued_host_buffer_entry_point():
     """adore_decode_rebuild_host_queued: the calls of all layers (and of several steps) are issued without a host wait in
-    between, every layer through a staging set of its own; outputs are read after one sync."""
-    from tests.gpu_driver import run_parity_queued_host
-    for cfg, kw in ((SMALL.scaled(name="queued_L3", n_layers=3, batch=2, per_layer_inputs=True, seed=153, steps=12), dict(sync_every=1)),
-                    (SMALL.scaled(name="queued_L2_three_steps_in_flight", n_layers=2, batch=2, per_layer_inputs=True, seed=154, steps=12,
-                                  rebuild_mode="explicit", rebuild_p=0.4, rebuild_max=10), dict(sync_every=3)),
-                    (SMALL.scaled(name="queued_one_layer", seed=155, steps=10), dict(sync_every=2))):
-        rep = run_parity_queued_host(cfg, **kw)
-        print(f"\n[{cfg.name}] steps={rep.steps} near_ties={rep.near_ties}+{rep.rounding_ties}r/{rep.topk_rows} rows "
-              f"max_out_err={rep.max_out_err:.3e} max_w_err={rep.max_w_err:.3e} max_kv_ulp={rep.max_kv_ulp:.2f}")
-        assert rep.steps == cfg.steps and rep.near_ties <= 2
+    between, every layer through a staging set of its own; the outputs, read after the waits, must repeat the lockstep
+    run's bit for bit."""
+    for cfg, every in ((SMALL.scaled(name="queued_L3", n_layers=3, batch=2, per_layer_inputs=True, seed=153, steps=12), 1),
+                       (SMALL.scaled(name="queued_L2_three_steps_in_flight", n_layers=2, batch=2, per_layer_inputs=True, seed=154,
+                                     steps=12, rebuild_mode="explicit", rebuild_p=0.4, rebuild_max=10), 3),
+                       (SMALL.scaled(name="queued_one_layer", seed=155, steps=10), 0)):
+        rep = _run_and_repeat_free(cfg, mode="queued_host", sync_every=every)
+        assert rep.steps == cfg.steps
 
 
 def test_capacity_spanning_several_tiles_with_ragged_tail():
@@ -164,6 +173,25 @@ def test_config4_shapes_two_layers_full_batch():
     _run(wl.get_config(4).scaled(name="cfg4_two_layers", n_layers=2), steps=2)
 
 
+def test_config3_steady_state_after_600_free_steps():
+    """Config 3 where `bench.py` times it: all 64 sequences run 600 decode steps with no host wait (every explicit list at
+    its full 256 rows, 16k rebuilt rows per step), while the oracle follows two sequences' scoring and selection on its
+    own. Then the small states must be equal, the oracle takes over the library's exported state and cache rows (each
+    row within one unit of its by-definition value), and two more steps are compared output by output."""
+    from tests.gpu_driver import run_sampled_parity
+    rep = _check("cfg3_steady_state", run_sampled_parity(wl.get_config(3), free_steps=600, check_steps=2, seqs=2))
+    assert rep.steps == 2 and rep.rows_adopted >= 2 * 512 + 2 * 2 * 256
+
+
+def test_config4_full_depth_all_32_layers():
+    """Config 4 as `bench.py` runs it: 32 layers, 32 sequences, C = 1024, prompt 2048, every layer with its own input rows
+    and projection, one slot map for all layers. Eight free steps, then two steps in which the oracle checks layers 0, 15
+    and 31 of two sequences (the layers share nothing but the map, Section 2.2 second bullet)."""
+    from tests.gpu_driver import run_sampled_parity
+    rep = _check("cfg4_full_depth", run_sampled_parity(wl.get_config(4), free_steps=8, check_steps=2, seqs=2, layers=[0, 15, 31]))
+    assert rep.steps == 2
+
+
 def test_controller_widths_off_the_default():
     """d' = 160 takes the controller path that streams its matrices from global memory, d' = 96 the
     shared-memory-resident one with partly filled warps."""
@@ -181,12 +209,7 @@ def test_controller_ablations_width_64_and_no_recurrence():
 
 def _run_rebuild_first(cfg, **kw):
     from tests.gpu_driver import run_parity_rebuild_first
-    rep = run_parity_rebuild_first(cfg, **kw)
-    print(f"\n[{cfg.name}] steps={rep.steps} near_ties={rep.near_ties}+{rep.rounding_ties}r/{rep.topk_rows} rows "
-          f"max_out_err={rep.max_out_err:.3e} max_w_err={rep.max_w_err:.3e} max_kv_ulp={rep.max_kv_ulp:.2f}")
-    assert rep.near_ties <= max(2, rep.topk_rows // 1000)
-    assert rep.rounding_ties <= max(2, rep.topk_rows // 50)
-    return rep
+    return _check(cfg.name, run_parity_rebuild_first(cfg, **kw))
 
 
 def test_rebuild_first_step_with_query_rows_of_the_rebuilt_tokens():

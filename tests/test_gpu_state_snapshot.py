@@ -85,6 +85,56 @@ def test_export_import_rewinds_the_cache(CFG):
         g.close()
 
 
+def test_import_refuses_a_snapshot_whose_indices_do_not_fit_the_cache():
+    """A truncated or damaged snapshot must not turn into out-of-range device accesses: every integer section is checked
+    on the host, and a snapshot that fails is refused with the cache unchanged and still working."""
+    import torch
+    from paper_2407_02328_b200 import adore as lib
+    from oracle.harness import Workload
+    from tests.gpu_driver import GpuCache, to_dev, parse_snapshot
+    w = Workload(CFG, None)
+    g = GpuCache(w)
+    try:
+        lib.adore_cache_append_tokens(g.handle, to_dev(w.prompt(), CFG), CFG.prompt)
+        _steps(g, w, lib, torch, to_dev, 0, 3)
+        snap = np.zeros(lib.adore_cache_export_state(g.handle, None), np.uint8)
+        lib.adore_cache_export_state(g.handle, snap)
+        fields = parse_snapshot(snap, CFG, g.B)
+        B, C, MT, R = g.B, CFG.capacity, CFG.max_tokens, CFG.rebuild_max
+        off_slot_tok0 = 64
+        off_role0 = off_slot_tok0 + 2 * B * C * 4
+        off_tok_slot = off_role0 + 2 * ((B * C + 7) & ~7)
+        off_z = off_tok_slot + 3 * B * MT * 4
+        off_admit = off_z + B * CFG.ctrl_hidden * 8
+        off_count = off_admit + 2 * ((B * 4 + 7) & ~7) + 2 * ((B * R * 4 + 7) & ~7)
+        off_row_b = off_count + ((B * 4 + 7) & ~7)
+        assert np.array_equal(snap[off_tok_slot: off_tok_slot + B * MT * 4].view(np.int32).reshape(B, MT), fields["tok_slot"])
+        assert np.array_equal(snap[off_count: off_count + B * 4].view(np.int32), fields["rebuild_count"])
+
+        def tampered(offset, value, dtype=np.int32):
+            bad = snap.copy()
+            bad[offset: offset + np.dtype(dtype).itemsize] = np.array([value], dtype).view(np.uint8)
+            return bad
+
+        n = int(fields["n"])
+        cases = [tampered(off_slot_tok0, 10 ** 6), tampered(off_slot_tok0, n), tampered(off_role0, 7, np.uint8),
+                 tampered(off_tok_slot + 4, C), tampered(off_admit, -2), tampered(off_count, R + 1),
+                 tampered(40, 3)]                                              # header word 10: step_open
+        if int(fields["row_total"][0]) > 0:
+            cases.append(tampered(off_row_b, B))
+        for bad in cases:
+            with pytest.raises(lib.AdoreError) as e:
+                lib.adore_cache_import_state(g.handle, bad)
+            assert e.value.status == 1
+        again = np.zeros_like(snap)
+        lib.adore_cache_export_state(g.handle, again)
+        assert (again == snap).all(), "a refused import changed the cache"
+        lib.adore_cache_import_state(g.handle, snap)                             # the untouched snapshot is accepted
+        _steps(g, w, lib, torch, to_dev, 3, 2)
+    finally:
+        g.close()
+
+
 def test_import_rejects_a_snapshot_of_another_shape():
     from paper_2407_02328_b200 import adore as lib
     from oracle.harness import Workload

@@ -5,7 +5,7 @@ gone through every other test. Some callers of this library may not allocate dev
 thread working next to CUDA-graph capture, a process whose device memory belongs to another
 allocator); for them adore_controller_score_static keeps its scratch in a fixed array inside the
 library. Here it must reproduce, on two calls in a row that share that array, the scores the
-cache-based path computes for the same tokens.
+cache-based path computes for the same tokens, and the scores the CPU oracle's controller gives.
 """
 import numpy as np
 import pytest
@@ -19,7 +19,9 @@ CFG = wl.WorkloadConfig(name="no_alloc", dtype="bf16", n_layers=1, batch=5, n_he
                         rebuild_mode="policy", rebuild_p=0.0, seed=77, ctrl_hidden=128, pos_scale=64.0)
 
 
-@pytest.mark.parametrize("cfg", [CFG, CFG.scaled(name="no_alloc_f32", dtype="f32", batch=3, ctrl_hidden=96, seed=78)])
+@pytest.mark.parametrize("cfg", [CFG, CFG.scaled(name="no_alloc_f32", dtype="f32", batch=3, ctrl_hidden=96, seed=78),
+                                 CFG.scaled(name="no_alloc_wide", batch=4, ctrl_hidden=256, hidden=256, seed=79)],
+                         ids=lambda c: c.name)
 def test_static_scoring_matches_cache_path_on_two_calls_in_a_row(cfg):
     import torch
     from oracle.harness import Workload
@@ -53,6 +55,18 @@ def test_static_scoring_matches_cache_path_on_two_calls_in_a_row(cfg):
     torch.cuda.synchronize()
     assert np.allclose(score.cpu().numpy().T, ref_score, rtol=1e-6, atol=1e-9)
     assert np.allclose(sigma.cpu().numpy().T, ref_sigma, rtol=1e-6, atol=1e-9)
+    # and against the oracle's controller (Section 2.2 Eq. 2 in float64, rounded once to float32): equal, or one unit in
+    # the last place where the float64 sums were split differently
+    from oracle import adore_oracle as ao
+    zo = np.zeros((cfg.batch, cfg.ctrl_hidden), np.float64)
+    for n in range(2):
+        zo = ao.gru_step(w.x_new(n), zo, w.ctrl)
+        so = ao.controller_score(zo, n, cfg.pos_scale, w.ctrl).astype(np.float32)
+        got = score[n].cpu().numpy()
+        assert (np.abs(got - so) <= np.spacing(np.abs(so))).all(), f"scores of call {n} differ from the oracle's"
+        sig = (1.0 / (1.0 + np.exp(-ao.controller_score(zo, n, cfg.pos_scale, w.ctrl)))).astype(np.float32)
+        assert np.allclose(sigma[n].cpu().numpy(), sig, rtol=1e-6, atol=0)
+    assert np.allclose(z.cpu().numpy(), zo, rtol=1e-12, atol=1e-15)
 
 
 def test_static_scoring_rejects_oversized_requests():
@@ -63,3 +77,17 @@ def test_static_scoring_rejects_oversized_requests():
     with pytest.raises(lib.AdoreError) as e:                 # 700 * 3 * 128 doubles exceed the 2 MiB array
         lib.adore_controller_score_static(wdev, "bf16", 700, 4096, 128, dummy, dummy, 0, 4096.0, dummy, dummy)
     assert e.value.status == 8
+
+
+def test_static_scoring_rejects_rows_it_cannot_read_in_16_byte_pieces():
+    """Refused on the host, nothing launched: a hidden size that is not a multiple of 64, and an input that does not
+    start on a 16-byte boundary."""
+    import torch
+    from paper_2407_02328_b200 import adore as lib
+    dummy = torch.zeros(4096, dtype=torch.float32, device="cuda")
+    wdev = {k: dummy for k, _ in lib.adore_controller_weights_t._fields_}
+    for hidden, x in ((100, dummy), (128, dummy[1:])):
+        with pytest.raises(lib.AdoreError) as e:
+            lib.adore_controller_score_static(wdev, "f32", 2, hidden, 64, x.data_ptr(), dummy, 0, 64.0, dummy, dummy)
+        assert e.value.status == 8
+    torch.cuda.synchronize()
