@@ -103,8 +103,13 @@ struct AttnSmem {
 // kept set, turns the logits into weights in place (0 for rows not kept), writes the weights out and
 // builds the ordered list of kept row indices. Returns the number of kept rows. Every thread of the
 // block calls it after a __syncthreads(); the results are published by a final __syncthreads().
-template <typename T, int DH, int NT = kAttnThreads>
-__device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh /* row of out/weights */) {
+//
+// Every warp owns one contiguous segment of the rows and every lane keeps its rows' order-preserving keys in
+// registers (row seg_begin + 32 k + lane in register k, KPT registers): the passes of the radix select, the maximum
+// and the exponentials are then unrolled loops over registers with no shared-memory load in their dependency chains,
+// and the kept rows are counted and placed with ballots; the block meets only to exchange counts.
+template <typename T, int DH, int NT, int KPT>
+__device__ __forceinline__ int attention_keep_and_weights_impl(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh, int seg) {
   constexpr int NW = NT / 32;
   float* s_logit = sm.logit;
   int* s_list = sm.list;
@@ -113,27 +118,34 @@ __device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p
   int* s_sel = sm.sel;
   const int rows = p.C + 1;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int seg_begin = warp * seg, seg_end = min(rows, seg_begin + seg);
 
   // ---- phase 2: which logits are kept (K largest, lower index wins ties) -------------------
+  uint32_t key[KPT];                      // 0 for positions past the segment: below every real key
   int cnt = 0;
-  for (int i = tid; i < rows; i += NT) cnt += (s_logit[i] > -INFINITY) ? 1 : 0;
-  const int n_cand = __float2int_rn(block_sum_f<NT>(float(cnt), s_tmp));
+#pragma unroll
+  for (int k = 0; k < KPT; ++k) {
+    const int i = seg_begin + 32 * k + lane;
+    const float l = i < seg_end ? s_logit[i] : -INFINITY;
+    key[k] = i < seg_end ? float_key(l) : 0u;
+    cnt += (l > -INFINITY) ? 1 : 0;
+  }
+  for (int i = tid; i < 256; i += NT) s_hist[i] = 0u;
+  const int n_cand = __float2int_rn(block_sum_f<NT>(float(cnt), s_tmp));   // (its barriers also publish the zeroed bins)
   uint32_t thr_key = 0u;                  // keep every candidate unless there are more than K
   if (n_cand > p.topk) {
     uint32_t prefix = 0u, mask = 0u;
     int need = p.topk;
+#pragma unroll
     for (int shift = 24; shift >= 0; shift -= 8) {
-      for (int i = tid; i < 256; i += NT) s_hist[i] = 0u;
-      __syncthreads();
-      for (int i = tid; i < rows; i += NT) {
-        const uint32_t key = float_key(s_logit[i]);
-        if ((key & mask) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1u);
-      }
+#pragma unroll
+      for (int k = 0; k < KPT; ++k)
+        if (key[k] != 0u && (key[k] & mask) == prefix) atomicAdd(&s_hist[(key[k] >> shift) & 255u], 1u);
       __syncthreads();
       if (warp == 0) {
         int c[8], tot = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { c[j] = int(s_hist[lane * 8 + j]); tot += c[j]; }
+        for (int j = 0; j < 8; ++j) { c[j] = int(s_hist[lane * 8 + j]); tot += c[j]; s_hist[lane * 8 + j] = 0u; }   // bins ready for the next digit
         int incl = tot;                   // suffix sum: this lane's bins and all higher ones
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -157,66 +169,88 @@ __device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p
     }
     thr_key = prefix;
     const int n_eq = s_sel[2];
-    __syncthreads();
-    if (n_eq != need && tid == 0) {       // exact ties at the threshold: keep the lowest indices
-      int left = need;
-      for (int i = 0; i < rows; ++i)
-        if (float_key(s_logit[i]) == thr_key) { if (left > 0) --left; else s_logit[i] = -INFINITY; }
+    if (n_eq != need) {                   // exact ties at the threshold (block-uniform): keep the lowest indices
+      __syncthreads();
+      if (tid == 0) {
+        int left = need;
+        for (int i = 0; i < rows; ++i)
+          if (float_key(s_logit[i]) == thr_key) { if (left > 0) --left; else s_logit[i] = -INFINITY; }
+      }
+      __syncthreads();
+#pragma unroll
+      for (int k = 0; k < KPT; ++k) {     // the dropped rows now read -inf
+        const int i = seg_begin + 32 * k + lane;
+        if (i < seg_end) key[k] = float_key(s_logit[i]);
+      }
     }
-    __syncthreads();
   }
 
   // ---- phase 3: softmax over the kept logits ----------------------------------------------
+  // kept: a real key (float_key(-inf) = 0x007fffff and the padding 0 are below every finite logit's key) at or above the threshold
+  constexpr uint32_t kMinusInfKey = 0x007fffffu;
+  const uint32_t keep_from = thr_key > kMinusInfKey ? thr_key : kMinusInfKey + 1u;
+  uint32_t kmax = 0u;
+#pragma unroll
+  for (int k = 0; k < KPT; ++k) kmax = (key[k] >= keep_from && key[k] > kmax) ? key[k] : kmax;
+  // the largest key is the largest logit: undo the order-preserving map
   float mx = -INFINITY;
-  for (int i = tid; i < rows; i += NT) {
-    const float l = s_logit[i];
-    if (l > -INFINITY && float_key(l) >= thr_key) mx = fmaxf(mx, l);
-  }
+  if (kmax != 0u) mx = __uint_as_float((kmax & 0x80000000u) ? (kmax & 0x7fffffffu) : ~kmax);
   mx = block_max_f<NT>(mx, s_tmp);
   float part = 0.f;
-  for (int i = tid; i < rows; i += NT) {
-    const float l = s_logit[i];
-    const bool keep = l > -INFINITY && float_key(l) >= thr_key;
-    const float e = keep ? expf(l - mx) : -1.f;   // -1 marks "not kept"
-    s_logit[i] = e;
-    part += keep ? e : 0.f;
-  }
-  const float inv = 1.f / block_sum_f<NT>(part, s_tmp);
-  // ordered compaction of the kept indices; weights replace the logits in place
-  int n_kept = 0;
-  for (int i0 = 0; i0 < rows; i0 += NT) {
-    const int i = i0 + tid;
-    const float e = i < rows ? s_logit[i] : -1.f;
-    const bool keep = e >= 0.f;
-    const unsigned bal = __ballot_sync(0xffffffffu, keep);
-    __syncthreads();
-    if (lane == 0) s_sel[8 + warp] = __popc(bal);
-    __syncthreads();
-    int base = n_kept, total = 0;
+  int kept_here = 0;
+  float ev[KPT];
 #pragma unroll
-    for (int w = 0; w < NW; ++w) { const int c = s_sel[8 + w]; if (w < warp) base += c; total += c; }
-    const float wgt = keep ? e * inv : 0.f;
-    if (i < rows) {
+  for (int k = 0; k < KPT; ++k) {
+    const bool keep = key[k] >= keep_from;
+    const float l = __uint_as_float((key[k] & 0x80000000u) ? (key[k] & 0x7fffffffu) : ~key[k]);
+    ev[k] = keep ? expf(l - mx) : -1.f;   // -1 marks "not kept"
+    part += keep ? ev[k] : 0.f;
+    kept_here += __popc(__ballot_sync(0xffffffffu, keep));
+  }
+  if (lane == 0) s_sel[8 + warp] = kept_here;
+  const float inv = 1.f / block_sum_f<NT>(part, s_tmp);     // (its barriers also publish the warps' counts)
+  int base = 0, n_kept = 0;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) { const int c = s_sel[8 + w]; if (w < warp) base += c; n_kept += c; }
+  // ordered compaction of the kept indices; weights replace the logits in place
+#pragma unroll
+  for (int k = 0; k < KPT; ++k) {
+    const int i = seg_begin + 32 * k + lane;
+    const bool keep = ev[k] >= 0.f;
+    const unsigned bal = __ballot_sync(0xffffffffu, keep);
+    const float wgt = keep ? ev[k] * inv : 0.f;
+    if (i < seg_end) {
       s_logit[i] = wgt;
       if (p.weights) p.weights[size_t(bh) * rows + i] = wgt;
     }
     if (keep) s_list[base + __popc(bal & ((1u << lane) - 1u))] = i;
-    n_kept += total;
+    base += __popc(bal);
   }
   __syncthreads();
   return n_kept;
 }
 
-// Phase 4 with direct loads: adds w_s * V[s] of the kept rows [j_begin, n_kept) of the list into acc (this lane's 16-byte column
-// slice; lanes of different row groups and warps hold partial sums).
 template <typename T, int DH, int NT = kAttnThreads>
+__device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh /* row of out/weights */) {
+  constexpr int NW = NT / 32;
+  const int rows = p.C + 1;
+  const int seg = (((rows + NW - 1) / NW) + 31) & ~31;      // rows per warp, a multiple of 32
+  // 9 registers per lane cover C <= 1151 with 4 warps and C <= 2303 with 8; kernels of 4 warps are launched for
+  // C <= 1024 only, those of 8 warps for any capacity up to 4096 (17 registers)
+  if (NT <= 128 || seg <= 9 * 32) return attention_keep_and_weights_impl<T, DH, NT, 9>(p, sm, bh, seg);
+  return attention_keep_and_weights_impl<T, DH, NT, 17>(p, sm, bh, seg);
+}
+
+// Phase 4 with direct loads: adds w_s * V[s] of the kept rows [j_begin, n_kept) of the list into acc (this lane's 16-byte column
+// slice; lanes of different row groups and warps hold partial sums). U loads of 16 bytes are in flight per lane: a gather of
+// 256-byte rows needs on the order of 100 KB in flight per SM to run at the memory system's rate.
+template <typename T, int DH, int NT = kAttnThreads, int U = kAttnUnroll>
 __device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh, int n_kept,
                                                         float (&acc)[Elem<T>::kPer16B], int j_begin = 0) {
   constexpr int NW = NT / 32;
   constexpr int EPL = Elem<T>::kPer16B;
   constexpr int LPR = DH / EPL;
   constexpr int RPW = 32 / LPR;
-  constexpr int U = kAttnUnroll;
   const float* s_logit = sm.logit;
   const int* s_list = sm.list;
   const int C = p.C;

@@ -13,14 +13,15 @@
 // reported as failed by adore_cache_sync_status).
 #pragma once
 
+#include <algorithm>
+
 #include "attention.cuh"
 #include "mbarrier.cuh"
 
 namespace adore {
 
-constexpr int kRingChunkBytes = 8192;
-__host__ __device__ inline size_t attn_tma_smem_bytes(int C, int DH, int threads, int kRingStages) {
-  // ring first (needs 128-byte alignment at most), then barriers, then the common carve-up
+__host__ __device__ inline size_t attn_tma_smem_bytes(int C, int DH, int threads, int kRingStages, int kRingChunkBytes) {
+  // ring first (needs 128-byte alignment at most), then barriers (up to 8), then the common carve-up
   return size_t(kRingStages) * kRingChunkBytes + 64 + attn_smem_bytes(C, DH, threads);
 }
 
@@ -29,8 +30,8 @@ __host__ __device__ inline size_t attn_tma_smem_bytes(int C, int DH, int threads
 // give each pair more threads (better when there are few pairs or very long key blocks).
 // MULTI: several query rows per pair (Section 2.3's rebuilt tokens' rows); the plain decode step compiles without any
 // of that logic.
-template <typename T, int DH, int NT, int kRingStages, bool MULTI>
-__global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p) {
+template <typename T, int DH, int NT, int kRingStages, int kRingChunkBytes, bool MULTI>
+__global__ void __launch_bounds__(NT, NT <= 128 ? 7 : 4) attention_tma_kernel(const AttnParams<T> p) {
   constexpr int NW = NT / 32;
   constexpr int EPL = Elem<T>::kPer16B;
   constexpr int LPR = DH / EPL;
@@ -38,6 +39,7 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
   constexpr int ROW_BYTES = DH * int(sizeof(T));
   constexpr int CHUNK_ROWS = kRingChunkBytes / ROW_BYTES;
   static_assert(CHUNK_ROWS % (NW * RPW) == 0, "a chunk must be a whole number of block-wide passes");
+  static_assert(kRingStages <= 8, "eight barriers are laid out");
   constexpr int PASSES = CHUNK_ROWS / (NW * RPW);
 
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -170,41 +172,71 @@ __global__ void __launch_bounds__(NT) attention_tma_kernel(const AttnParams<T> p
   float acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-  attention_values_direct<T, DH, NT>(p, sm, bh, n_kept, acc);
+  constexpr int UV = NT <= 128 ? 8 : 4;     // value-row loads in flight per lane: small CTAs have few warps to hide the latency
+  attention_values_direct<T, DH, NT, UV>(p, sm, bh, n_kept, acc);
   attention_finish<T, DH, NT>(p, sm, bh, acc, item, last_row);
 }
 
 template <typename T>
 inline bool attn_tma_usable(int /*C*/, int DH) { return DH == 64 || DH == 128; }
 
-template <typename T, int DH, int NT, int STAGES, bool MULTI>
+// CTAs per SM that spread `grid` CTAs evenly over the waves the launch needs anyway. With at most `fit` CTAs on an SM
+// it takes w = ceil(grid / (sms * fit)) waves; ceil(grid / (sms * w)) CTAs per SM fill every one of them equally,
+// where the greedy placement would run a full wave and then a part-empty one with fewer loads in flight per SM
+// (2048 CTAs, fit 8: two waves of 7 per SM instead of 8 and 5.8).
+inline int attn_balanced_ctas_per_sm(int grid, int sms, int fit) {
+  if (fit < 1 || sms < 1) return fit;
+  const int waves = (grid + sms * fit - 1) / (sms * fit);
+  return std::min(fit, (grid + sms * waves - 1) / (sms * waves));
+}
+
+template <typename T, int DH, int NT, int STAGES, int CHUNK, bool MULTI>
 inline cudaError_t launch_attention_tma_as(const AttnParams<T>& p, int grid, cudaStream_t stream) {
-  const size_t smem = attn_tma_smem_bytes(p.C, DH, NT, STAGES);
+  size_t smem = attn_tma_smem_bytes(p.C, DH, NT, STAGES, CHUNK);
+  constexpr size_t kSmBytes = 228 * 1024, kCtaReserve = 1024;   // shared memory of an SM, and what the system adds to every CTA
   static bool opted_in = false;            // per instantiation; the attribute is per function
+  static int sms = 0, fit_smem = -1, fit = 0;
+  auto kernel = attention_tma_kernel<T, DH, NT, STAGES, CHUNK, MULTI>;
   if (!opted_in) {
-    cudaError_t e = cudaFuncSetAttribute(attention_tma_kernel<T, DH, NT, STAGES, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 120 * 1024);
     if (e != cudaSuccess) return e;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 0;
     opted_in = true;
   }
-  return launch_dependent(attention_tma_kernel<T, DH, NT, STAGES, MULTI>, dim3(grid), dim3(NT), smem, stream, p);
+  if (fit_smem != int(smem)) {             // resident CTAs per SM at this shared-memory size (registers and threads included)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kernel, NT, smem) != cudaSuccess) { cudaGetLastError(); fit = 0; }
+    fit_smem = int(smem);
+  }
+  const int want = attn_balanced_ctas_per_sm(grid, sms, fit);
+  if (want >= 1 && want < fit) {
+    // the smallest size that keeps a (want + 1)-th CTA off the SM; whatever is left stays free for kernels that run beside
+    const size_t pad = (kSmBytes / size_t(want + 1) - kCtaReserve + 128) & ~size_t(127);
+    if (pad > smem && pad <= 120 * 1024) smem = pad;
+  }
+  return launch_dependent(kernel, dim3(grid), dim3(NT), smem, stream, p);
 }
-template <typename T, int DH, int NT, int STAGES>
+template <typename T, int DH, int NT, int STAGES, int CHUNK>
 inline cudaError_t launch_attention_tma_cfg(const AttnParams<T>& p, int grid, cudaStream_t stream) {
-  return p.rows_q > 1 ? launch_attention_tma_as<T, DH, NT, STAGES, true>(p, grid, stream)
-                      : launch_attention_tma_as<T, DH, NT, STAGES, false>(p, grid, stream);
+  return p.rows_q > 1 ? launch_attention_tma_as<T, DH, NT, STAGES, CHUNK, true>(p, grid, stream)
+                      : launch_attention_tma_as<T, DH, NT, STAGES, CHUNK, false>(p, grid, stream);
 }
 
 // Many (b, h) pairs with key blocks of moderate length: small CTAs; otherwise large ones (measured on the
 // capacity x batch sweep: 128 threads win from ~1000 pairs on up to C = 1024, 256 threads elsewhere).
+// Ring: 2 x 8 KB for the small CTAs, 4 x 8 KB for the large ones (the same bytes cut into 4 x 4 KB or 8 x 2 KB stages
+// were measured no faster, resp. slower: the key pass is bound by the work per row, not by the bytes in flight).
+constexpr int kSmallRingStages = 2, kSmallRingChunk = 8192;
+constexpr int kLargeRingStages = 4, kLargeRingChunk = 8192;
 template <typename T>
 inline cudaError_t launch_attention_tma(const AttnParams<T>& p, int DH, int grid, cudaStream_t stream) {
   const bool small_ctas = grid >= 1024 && p.C <= 1024;
   if (DH == 64) {
-    if (small_ctas) return launch_attention_tma_cfg<T, 64, 128, 2>(p, grid, stream);
-    return launch_attention_tma_cfg<T, 64, 256, 4>(p, grid, stream);
+    if (small_ctas) return launch_attention_tma_cfg<T, 64, 128, kSmallRingStages, kSmallRingChunk>(p, grid, stream);
+    return launch_attention_tma_cfg<T, 64, 256, kLargeRingStages, kLargeRingChunk>(p, grid, stream);
   }
-  if (small_ctas) return launch_attention_tma_cfg<T, 128, 128, 2>(p, grid, stream);
-  return launch_attention_tma_cfg<T, 128, 256, 4>(p, grid, stream);
+  if (small_ctas) return launch_attention_tma_cfg<T, 128, 128, kSmallRingStages, kSmallRingChunk>(p, grid, stream);
+  return launch_attention_tma_cfg<T, 128, 256, kLargeRingStages, kLargeRingChunk>(p, grid, stream);
 }
 
 }  // namespace adore
