@@ -256,10 +256,12 @@ adore_status_t adore_cache_stage_times(adore_cache_t *cache, double *ms, int64_t
  * the following layers. Per attend-first step three events are recorded: where the group starts (before the attention
  * of layer 0), where its main-stream part ends (after the last layer's attention; in a one-layer cache after the new
  * token's row has been written) and where the controller chain ends. adore_cache_group_times waits for the streams and
- * returns, summed over the steps since the last call, the time from the first event to the later of the other two,
- * and the number of steps; both are reset. ms, steps: HOST pointers. In a cache of several layers the rebuilds of
- * layers 0..L-2 run inside that window, on their own stream. */
-adore_status_t adore_cache_group_times(adore_cache_t *cache, double *ms, int64_t *steps);
+ * returns, summed over the steps since the last call, in *ms the time from the first event to the later of the other
+ * two, in *ms_main the time from the first event to the second alone (what the rest of the step waits for: the
+ * controller of token n starts when the attention of layer 0 is done and its score is first read by the next step's
+ * selection), and the number of steps; all are reset. ms, ms_main, steps: HOST pointers. In a cache of several layers
+ * the rebuilds of layers 0..L-2 run inside that window, on their own stream. */
+adore_status_t adore_cache_group_times(adore_cache_t *cache, double *ms, double *ms_main, int64_t *steps);
 
 /* Total number of rows rebuilt by decode steps so far (Section 2.3: sum over steps and sequences
  * of the rebuild-list lengths); waits for the stream. rows: HOST pointer. */

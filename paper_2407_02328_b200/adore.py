@@ -95,7 +95,7 @@ def _lib():
         lib.adore_cache_wait_outputs.argtypes = [vp]
         lib.adore_cache_set_stage_timing.argtypes = [vp, i32]
         lib.adore_cache_stage_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
-        lib.adore_cache_group_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+        lib.adore_cache_group_times.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         lib.adore_cache_rebuild_rows.argtypes = [vp, C.POINTER(C.c_int64)]
         lib.adore_cache_export_state.argtypes = [vp, vp, C.POINTER(C.c_size_t)]
         lib.adore_cache_import_state.argtypes = [vp, vp, C.c_size_t]
@@ -257,10 +257,11 @@ def adore_cache_set_stage_timing(cache: int, enable) -> None:
 
 
 def adore_cache_group_times(cache: int):
-    """Returns (ms, steps): device time of the attention + selection group summed over the steps since the last call."""
-    ms, n = C.c_double(), C.c_int64()
-    _check(_lib().adore_cache_group_times(cache, C.byref(ms), C.byref(n)), "adore_cache_group_times")
-    return ms.value, n.value
+    """Returns (ms, ms_main, steps): device time of the attention + selection group summed over the steps since the last
+    call, to the later of {main-stream part, controller chain} and to the end of the main-stream part alone."""
+    ms, ms_main, n = C.c_double(), C.c_double(), C.c_int64()
+    _check(_lib().adore_cache_group_times(cache, C.byref(ms), C.byref(ms_main), C.byref(n)), "adore_cache_group_times")
+    return ms.value, ms_main.value, n.value
 
 
 def adore_cache_stage_times(cache: int):

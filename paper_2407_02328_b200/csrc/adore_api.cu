@@ -128,6 +128,7 @@ struct adore_cache {
   int* frow_slot = nullptr;
   int* frow_total = nullptr;
   unsigned long long* rows_accum = nullptr;
+  unsigned* sel_done = nullptr;     // arrivals of a selection launch's CTAs (the last one builds the row table)
   int sms = 148;
   unsigned* err = nullptr;
   // optional per-stage timing
@@ -143,7 +144,7 @@ struct adore_cache {
   bool group_timing = false;
   std::vector<cudaEvent_t> grp_pool;
   size_t grp_used = 0;
-  double grp_ms = 0;
+  double grp_ms = 0, grp_main_ms = 0;
   int64_t grp_steps = 0;
   double* part = nullptr;
   size_t part_doubles = 0;
@@ -159,7 +160,7 @@ struct adore_cache {
   // second side stream: the controller (gates, then GRU + MLP) of the new token. Its score is first needed by
   // the NEXT step's selection, so it may run on past the end of the step that launched it.
   cudaStream_t ctl = nullptr;
-  cudaEvent_t ev_gates = nullptr, ev_ctrl = nullptr;
+  cudaEvent_t ev_xrow = nullptr, ev_attn = nullptr, ev_ctrl = nullptr;   // the token's row is in the store / the attention of layer 0 is done
   bool ctrl_pending = false;    // ev_ctrl was recorded and the main stream has not waited for it yet
   // uploads of the host-buffer entry point run on their own stream, beside the previous rebuild
   cudaStream_t copy = nullptr;
@@ -350,21 +351,23 @@ SelectParams select_params(adore_cache* c, int n, int P, int old_map, int new_ma
 }
 
 template <typename T>
-adore_status_t launch_gates(adore_cache* c, const T* x, long long seq_stride, int tc, int ksplit, cudaStream_t stream) {
+adore_status_t launch_gates(adore_cache* c, const T* x, long long seq_stride, int tc, int ksplit, cudaStream_t stream,
+                            int hh_slices = 0) {
   GateParams<T> g{};
+  g.hh_slices = hh_slices; g.h = c->cfg.ctrl_hidden; g.w_hh = c->w_hh; g.z = c->z;
   g.x = x; g.seq_stride = seq_stride; g.tc = tc; g.rows = c->cfg.batch * tc; g.d = c->cfg.hidden; g.G = 3 * c->cfg.ctrl_hidden;
   g.w_ih = c->w_ih; g.part = c->part; g.ksplit = ksplit;
   const int per = (c->cfg.hidden + ksplit - 1) / ksplit;
   g.kslice = ((per + kGateKInner - 1) / kGateKInner) * kGateKInner;
   static const bool narrow_only = dev_switch("ADORE_GATES_NARROW");
   if (g.rows >= kGateWideMinRows && !narrow_only) {
-    dim3 grid((g.G + kGateWideG - 1) / kGateWideG, (g.rows + kGateWideR - 1) / kGateWideR, ksplit);
+    dim3 grid((g.G + kGateWideG - 1) / kGateWideG, (g.rows + kGateWideR - 1) / kGateWideR, ksplit + hh_slices);
     ctrl_gates_wide_kernel<T><<<grid, kGateWideThreads, kGateWideSmem, stream>>>(g);
     ++c->launches;
     CUDA_OK(cudaGetLastError());
     return ADORE_OK;
   }
-  dim3 grid((g.G + kGateTileG - 1) / kGateTileG, (g.rows + kGateTileR - 1) / kGateTileR, ksplit);
+  dim3 grid((g.G + kGateTileG - 1) / kGateTileG, (g.rows + kGateTileR - 1) / kGateTileR, ksplit + hh_slices);
   ctrl_gates_kernel<T><<<grid, kGateThreads, 0, stream>>>(g);
   ++c->launches;
   CUDA_OK(cudaGetLastError());
@@ -578,6 +581,10 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
   sp.explicit_list = ex && r_in > 0 ? explicit_list : nullptr;
   sp.explicit_count = ex && r_in > 0 ? explicit_count : nullptr;
   sp.r_in = r_in;
+  if (f.rebuild_max > 0) {                      // the last CTA of the launch writes the rebuild's row table
+    sp.row_b = c->row_b; sp.row_tok = c->row_tok; sp.row_slot = c->row_slot; sp.row_total = c->row_total;
+    sp.rows_accum = c->rows_accum; sp.done_count = c->sel_done;
+  }
   const size_t smem = select_smem_bytes(f.capacity, P);
   if (f.dtype == ADORE_F32)
     select_kernel<float><<<f.batch, select_threads(c), smem, sel>>>(
@@ -587,8 +594,10 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
         sp, static_cast<const __nv_bfloat16*>(x_new), static_cast<__nv_bfloat16*>(c->x_store), f.hidden);
   ++c->launches;
   CUDA_OK(cudaGetLastError());
-  st = launch_row_table(c, true, sel);
-  if (st != ADORE_OK) return st;
+  // the selection kernel has put the token's row into the token store: the controller reads it from there, so that
+  // x_new is borrowed only until the selection has run (which the main stream waits for anyway)
+  CUDA_OK(cudaEventRecord(c->ev_xrow, sel));
+  CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_xrow, 0));
   // A short list's rows are copied out of the token store into the GEMM's compact input right away, beside the
   // attention, so that the rebuild that follows starts with its GEMM. Long lists are copied after the attention:
   // side by side the two slow each other down by more than the copy takes (measured at 15k rows: attention
@@ -607,17 +616,30 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
       c->rows_gathered = true;
     }
   }
-  if (controller) {
-    if (f.dtype == ADORE_F32) st = launch_gates<float>(c, static_cast<const float*>(x_new), 1, 1, c->ksplit, c->ctl);
-    else st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(x_new), 1, 1, c->ksplit, c->ctl);
+  // the recurrent product rides in the gate product when the state has whole 32-element chunks and is not ignored
+  const int hh_slices = (f.ctrl_hidden % kGateKInner == 0 && !(f.flags & ADORE_FLAG_NO_RECURRENCE))
+                            ? (f.ctrl_hidden + kGateHhSlice - 1) / kGateHhSlice : 0;
+  if (!controller) return ADORE_OK;
+  {
+    const size_t row0 = size_t(c->n) * f.hidden;        // token n of sequence 0 in the store [B][max_tokens][d]
+    if (f.dtype == ADORE_F32)
+      st = launch_gates<float>(c, static_cast<const float*>(c->x_store) + row0, f.max_tokens, 1, c->ksplit, c->ctl, hh_slices);
+    else
+      st = launch_gates<__nv_bfloat16>(c, static_cast<const __nv_bfloat16*>(c->x_store) + row0, f.max_tokens, 1, c->ksplit, c->ctl, hh_slices);
     if (st != ADORE_OK) return st;
   }
-  CUDA_OK(cudaEventRecord(c->ev_gates, c->ctl));
-  if (!controller) return ADORE_OK;
   RecurParams rp = recur_params(c, f.batch, 1, c->ksplit, c->n);
-  ctrl_recur_kernel<<<f.batch, select_threads(c), ctrl_smem(c), c->ctl>>>(rp, ctrl_resident_ok(f.ctrl_hidden) ? 1 : 0, c->err);
+  rp.hh_slices = hh_slices;
+  if (f.ctrl_hidden % 4 == 0) {
+    // (an ordinary launch: while a programmatic dependent of the gate product was pending, kernels of the other streams
+    // -- the new token's row, the gather -- were not started either)
+    ctrl_decode_tail_kernel<<<f.batch, kTailThreads, ctrl_tail_smem_bytes(f.ctrl_hidden), c->ctl>>>(rp);
+    CUDA_OK(cudaGetLastError());
+  } else {                                            // rows that are not whole 16-byte pieces: the scalar-load kernel of the prompt scan
+    ctrl_recur_kernel<<<f.batch, select_threads(c), ctrl_smem(c), c->ctl>>>(rp, 0, c->err);
+    CUDA_OK(cudaGetLastError());
+  }
   ++c->launches;
-  CUDA_OK(cudaGetLastError());
   CUDA_OK(cudaEventRecord(c->ev_ctrl, c->ctl));
   c->ctrl_pending = true;
   if (c->timing) { CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_ctrl, 0)); c->ctrl_pending = false; }
@@ -690,6 +712,7 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   TRY(dev_alloc(c, &c->frow_slot, B * C * sizeof(int), true));
   TRY(dev_alloc(c, &c->frow_total, sizeof(int), true));
   TRY(dev_alloc(c, &c->rows_accum, sizeof(unsigned long long), true));
+  TRY(dev_alloc(c, &c->sel_done, sizeof(unsigned), true));
   {
     int dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, dev);
@@ -697,19 +720,19 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
   TRY(dev_alloc(c, &c->err, sizeof(unsigned), true));
   if (f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION)
     TRY(dev_alloc(c, &c->w_internal, B * f.n_heads * (C + 1) * sizeof(float), true));
-  // decode splits the d-long dot products so that roughly one wave of CTAs is busy
+  // decode splits the d-long dot products into k-slices (whole 32-element chunks) so that the launch has about one CTA per SM
   {
-    int ks = 1;
-    if (int(B) >= kGateWideMinRows) {     // decode uses the 128 x 64 tile kernel: one CTA per SM at most
-      const int tiles = int((G + kGateWideG - 1) / kGateWideG) * int((B + kGateWideR - 1) / kGateWideR);
-      while (ks < 32 && tiles * ks * 2 <= 192 && int(d) / (ks * 2) >= 2 * kGateKInner) ks *= 2;
-    } else {
-      const int tiles = int((G + kGateTileG - 1) / kGateTileG) * int((B + kGateTileR - 1) / kGateTileR);
-      while (ks < 16 && tiles * ks * 2 <= 296 && int(d) / (ks * 2) >= kGateKChunk) ks *= 2;
-    }
+    const bool wide = int(B) >= kGateWideMinRows;
+    const int tiles = wide ? int((G + kGateWideG - 1) / kGateWideG) * int((B + kGateWideR - 1) / kGateWideR)
+                           : int((G + kGateTileG - 1) / kGateTileG) * int((B + kGateTileR - 1) / kGateTileR);
+    const int chunks = int(d) / kGateKInner;
+    const int ks_cap = h % 4 == 0 ? 64 : 32;       // odd widths go through the prompt kernel, which adds at most 32 slices
+    const int ks_max = std::max(1, std::min(ks_cap, c->sms / std::max(1, tiles)));
+    const int slice_chunks = (chunks + ks_max - 1) / ks_max;
+    const int ks = (chunks + slice_chunks - 1) / slice_chunks;
     c->ksplit = ks;
     const size_t rows_prefill = std::min<size_t>(B * MT, std::max<size_t>(kMaxPrefillRows, B));
-    c->part_doubles = std::max<size_t>(size_t(ks) * B, rows_prefill) * G;
+    c->part_doubles = std::max<size_t>(size_t(ks + 4) * B, rows_prefill) * G;   // + 4: the recurrent product's slices (d' <= 256)
     TRY(dev_alloc(c, &c->part, c->part_doubles * sizeof(double), false));
   }
   TRY(upload(c, &c->w_hh, w->gru_w_hh, G * h));
@@ -761,7 +784,8 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
       cudaStreamCreateWithPriority(&c->ctl, cudaStreamNonBlocking, prio_high) != cudaSuccess ||
-      cudaEventCreateWithFlags(&c->ev_gates, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_xrow, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_attn, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_ctrl, cudaEventDisableTiming) != cudaSuccess ||
       cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_copy, cudaEventDisableTiming) != cudaSuccess ||
@@ -821,7 +845,8 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (c->ev_rb_fork) cudaEventDestroy(c->ev_rb_fork);
   if (c->ev_step_open) cudaEventDestroy(c->ev_step_open);
   for (cudaEvent_t e : c->ev_rebuilt) cudaEventDestroy(e);
-  if (c->ev_gates) cudaEventDestroy(c->ev_gates);
+  if (c->ev_xrow) cudaEventDestroy(c->ev_xrow);
+  if (c->ev_attn) cudaEventDestroy(c->ev_attn);
   if (c->ev_ctrl) cudaEventDestroy(c->ev_ctrl);
   if (c->copy) { cudaStreamSynchronize(c->copy); cudaStreamDestroy(c->copy); }
   if (c->ev_copy) cudaEventDestroy(c->ev_copy);
@@ -945,7 +970,11 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     if (st != ADORE_OK) return st;
     if (c->timing) CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
     if (sel != c->stream) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_fork, 0));
-    CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
+    // The controller's float64 products would take SM time from the attention, which fills the GPU and is on the step's
+    // critical path, while their result is first needed by the NEXT step's selection: they start when the attention
+    // of layer 0 is done and run beside what follows it (the gather of a long rebuild list, the next layers).
+    CUDA_OK(cudaEventRecord(c->ev_attn, c->stream));
+    CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_attn, 0));
     st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel, true);
     if (st != ADORE_OK) return st;
     if (group_mark(c, 2, c->ctl) != ADORE_OK) return ADORE_ERR_CUDA;
@@ -967,7 +996,6 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
   }
   if (!c->joined) CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
   c->joined = true;
-  CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_gates, 0));   // x_new is borrowed only until the main stream passes the call
   {
     StageScope scope(c, 3);
     const size_t row_bytes = size_t(f.head_dim) * c->esz;
@@ -1009,7 +1037,6 @@ adore_status_t adore_step_begin(adore_cache_t* c, const void* x_new, const int32
     CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
   }
   c->joined = true;
-  CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_gates, 0));
   if (c->ev_step_open) CUDA_OK(cudaEventRecord(c->ev_step_open, c->stream));
   c->cur = 1 - c->cur;
   c->attn = c->cur;             // this step's attention reads the NEW map
@@ -1261,8 +1288,8 @@ adore_status_t adore_cache_set_stage_timing(adore_cache_t* c, int32_t enable) {
   return ADORE_OK;
 }
 
-adore_status_t adore_cache_group_times(adore_cache_t* c, double* ms, int64_t* steps) {
-  if (!c || !ms || !steps) return ADORE_ERR_INVALID_ARG;
+adore_status_t adore_cache_group_times(adore_cache_t* c, double* ms, double* ms_main, int64_t* steps) {
+  if (!c || !ms || !ms_main || !steps) return ADORE_ERR_INVALID_ARG;
   if (join_controller(c) != ADORE_OK || join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return ADORE_ERR_CUDA;
   for (size_t i = 0; i + 3 <= c->grp_used; i += 3) {
@@ -1270,12 +1297,14 @@ adore_status_t adore_cache_group_times(adore_cache_t* c, double* ms, int64_t* st
     if (cudaEventElapsedTime(&a, c->grp_pool[i], c->grp_pool[i + 1]) != cudaSuccess) { cudaGetLastError(); continue; }   // a step left open
     if (cudaEventElapsedTime(&b, c->grp_pool[i], c->grp_pool[i + 2]) != cudaSuccess) { cudaGetLastError(); b = 0.f; }
     c->grp_ms += double(a > b ? a : b);
+    c->grp_main_ms += double(a);
     c->grp_steps += 1;
   }
   c->grp_used = 0;
   *ms = c->grp_ms;
+  *ms_main = c->grp_main_ms;
   *steps = c->grp_steps;
-  c->grp_ms = 0;
+  c->grp_ms = c->grp_main_ms = 0;
   c->grp_steps = 0;
   return ADORE_OK;
 }

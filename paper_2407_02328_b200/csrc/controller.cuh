@@ -28,13 +28,21 @@ struct GateParams {
   int rows;              // B * tc
   int d, G;              // input width (multiple of 64), 3*d'
   const float* w_ih;     // [G, d]
-  double* part;          // [ksplit, rows, G]
+  double* part;          // [ksplit + hh_slices, rows, G]
   int ksplit, kslice;    // kslice is a multiple of kGateKInner
+  // Decode step only (tc == 1): the recurrent product W_hh z of the same token as hh_slices further k-slices of 64,
+  // so that it runs as part of this tiled product (every weight converted once per CTA, shared by all sequences of the
+  // tile) instead of once per sequence. CTAs with blockIdx.z >= ksplit take it: k runs over 0 .. h - 1, the weights are
+  // w_hh [G, h] and the input row of sequence r is the float64 state z[r, :]. Needs h % 32 == 0.
+  int hh_slices, h;
+  const float* w_hh;
+  const double* z;
 };
 
 // 64 gates x 32 rows per CTA, 4 x 2 outputs per thread, float64 FMA, k in chunks of 32. The next
 // chunk is fetched into registers while the current one is consumed from shared memory.
 constexpr int kGateKInner = 32;
+constexpr int kGateHhSlice = 64;   // k-slice of the recurrent product when it rides in the gate product (decode step)
 
 template <typename T>
 __global__ void __launch_bounds__(kGateThreads) ctrl_gates_kernel(const GateParams<T> p) {
@@ -43,7 +51,11 @@ __global__ void __launch_bounds__(kGateThreads) ctrl_gates_kernel(const GatePara
   __shared__ __align__(16) double Xs[kGateKInner][XS];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int g0 = blockIdx.x * kGateTileG, r0 = blockIdx.y * kGateTileR, ks = blockIdx.z;
-  const int k_begin = ks * p.kslice, k_end = min(p.d, k_begin + p.kslice);
+  let_next_grid_start();                       // a dependent launch may start the part of its work that does not need these sums
+  const bool is_hh = ks >= p.ksplit;           // this CTA multiplies the recurrent matrix with the state (decode step)
+  const int ld = is_hh ? p.h : p.d;
+  const int k_begin = is_hh ? (ks - p.ksplit) * kGateHhSlice : ks * p.kslice;
+  const int k_end = is_hh ? min(p.h, k_begin + kGateHhSlice) : min(p.d, k_begin + p.kslice);
   // per chunk this thread fetches two float4 of W (gates wg, wg+32; k offset 4*wk) and 4 elements of one x row
   const int wk = tid & 7, wg = tid >> 3;
   const int xr = tid >> 3, xk = tid & 7;
@@ -53,7 +65,7 @@ __global__ void __launch_bounds__(kGateThreads) ctrl_gates_kernel(const GatePara
   for (int j = 0; j < 2; ++j) {
     const int g = g0 + wg + 32 * j;
     wok[j] = g < p.G;
-    wsrc[j] = p.w_ih + size_t(wok[j] ? g : 0) * p.d + 4 * wk;
+    wsrc[j] = (is_hh ? p.w_hh : p.w_ih) + size_t(wok[j] ? g : 0) * ld + 4 * wk;
   }
   const bool xok = r0 + xr < p.rows;
   const T* xsrc = p.x;
@@ -67,7 +79,7 @@ __global__ void __launch_bounds__(kGateThreads) ctrl_gates_kernel(const GatePara
 #pragma unroll
     for (int j = 0; j < 2; ++j)
       wreg[j] = wok[j] ? __ldg(reinterpret_cast<const float4*>(wsrc[j] + k0)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    if (!xok) {
+    if (!xok || is_hh) {                          // (the state is float64: it goes to shared memory directly, below)
       xreg[0] = xreg[1] = xreg[2] = xreg[3] = 0.f;
     } else if (sizeof(T) == 2) {
       const uint2 v = __ldg(reinterpret_cast<const uint2*>(xsrc + k0));
@@ -91,8 +103,13 @@ __global__ void __launch_bounds__(kGateThreads) ctrl_gates_kernel(const GatePara
       Ws[4 * wk + 2][g] = double(wreg[j].z);
       Ws[4 * wk + 3][g] = double(wreg[j].w);
     }
+    if (is_hh) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) Xs[4 * xk + e][xr] = double(xreg[e]);
+      for (int e = 0; e < 4; ++e) Xs[4 * xk + e][xr] = xok ? p.z[size_t(r0 + xr) * p.h + k0 + 4 * xk + e] : 0.0;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) Xs[4 * xk + e][xr] = double(xreg[e]);
+    }
     __syncthreads();
     if (k0 + kGateKInner < k_end) fetch(k0 + kGateKInner);
 #pragma unroll 8
@@ -133,7 +150,11 @@ __global__ void __launch_bounds__(kGateWideThreads) ctrl_gates_wide_kernel(const
   double (*Xs)[kGateWideXS] = reinterpret_cast<double (*)[kGateWideXS]>(gw_smem + kGateKInner * kGateWideWS);
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int g0 = blockIdx.x * kGateWideG, r0 = blockIdx.y * kGateWideR, ks = blockIdx.z;
-  const int k_begin = ks * p.kslice, k_end = min(p.d, k_begin + p.kslice);
+  let_next_grid_start();
+  const bool is_hh = ks >= p.ksplit;           // this CTA multiplies the recurrent matrix with the state (decode step)
+  const int ld = is_hh ? p.h : p.d;
+  const int k_begin = is_hh ? (ks - p.ksplit) * kGateHhSlice : ks * p.kslice;
+  const int k_end = is_hh ? min(p.h, k_begin + kGateHhSlice) : min(p.d, k_begin + p.kslice);
   // fetch roles: 8 float4 of W (gate (tid + 128 q) / 8, k offset 4 * ((tid + 128 q) % 8)) and 2 x 8 elements of x
   // (row (tid + 128 q) / 4, k offset 8 * ((tid + 128 q) % 4)) per chunk of 32 k
   const float* wsrc[8];
@@ -142,7 +163,7 @@ __global__ void __launch_bounds__(kGateWideThreads) ctrl_gates_wide_kernel(const
   for (int q = 0; q < 8; ++q) {
     const int idx = tid + kGateWideThreads * q, g = g0 + (idx >> 3);
     wok[q] = g < p.G;
-    wsrc[q] = p.w_ih + size_t(wok[q] ? g : 0) * p.d + 4 * (idx & 7);
+    wsrc[q] = (is_hh ? p.w_hh : p.w_ih) + size_t(wok[q] ? g : 0) * ld + 4 * (idx & 7);
   }
   const T* xsrc[2];
   bool xok[2];
@@ -162,7 +183,7 @@ __global__ void __launch_bounds__(kGateWideThreads) ctrl_gates_wide_kernel(const
       wreg[q] = wok[q] ? __ldg(reinterpret_cast<const float4*>(wsrc[q] + k0)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
-      if (!xok[q]) {
+      if (!xok[q] || is_hh) {                     // (the state is float64: it goes to shared memory directly, below)
 #pragma unroll
         for (int e = 0; e < 8; ++e) xreg[q][e] = 0.f;
       } else if (sizeof(T) == 2) {
@@ -199,8 +220,13 @@ __global__ void __launch_bounds__(kGateWideThreads) ctrl_gates_wide_kernel(const
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
       const int idx = tid + kGateWideThreads * q, r = idx >> 2, kk = 8 * (idx & 3);
+      if (is_hh) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) Xs[kk + e][r] = double(xreg[q][e]);
+        for (int e = 0; e < 8; ++e) Xs[kk + e][r] = xok[q] ? p.z[size_t(r0 + r) * p.h + k0 + kk + e] : 0.0;
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) Xs[kk + e][r] = double(xreg[q][e]);
+      }
     }
     __syncthreads();
     if (k0 + kGateKInner < k_end) fetch(k0 + kGateKInner);
@@ -237,7 +263,7 @@ __global__ void __launch_bounds__(kGateWideThreads) ctrl_gates_wide_kernel(const
 }
 
 struct RecurParams {
-  const double* part;    // [ksplit, rows, G], row = b*tc + t; ksplit <= 32
+  const double* part;    // [ksplit, rows, G], row = b*tc + t; ksplit <= 32 for the prompt kernels, <= 64 for the decode kernel
   int ksplit, rows, tc;
   int h;                 // d'
   const float* b_ih;     // [3h]
@@ -256,6 +282,7 @@ struct RecurParams {
   int n0;                // position of the first token of this call
   double pos_scale;
   int no_recurrence;     // 1: every token sees a zero state (the ablation without the GRU's memory, Section 3.5.3)
+  int hh_slices;         // decode kernel: k-slices of `part` after the first ksplit that hold W_hh z (0: it computes that product itself)
   double* a_tab;         // [B, max_tokens, h] or null. Set: positions are relative to the current token; the token is
                          // scored at distance 0 and the input of its Tanh layer is kept for later re-scoring
 };
@@ -549,6 +576,170 @@ __device__ __forceinline__ void controller_tokens_resident(const RecurParams& p,
     __syncthreads();
   }
   if (tid < h) p.z[size_t(b) * h + tid] = s_z[tid];
+}
+
+// ---- decode step: one new token per sequence, small footprint ---------------------------------------
+// The controller of token n runs beside the attention of layer 0, whose CTAs fill the SMs. The prompt kernel above keeps
+// the whole recurrent matrix in shared memory (right for a scan of thousands of tokens), so one CTA needs an SM to itself
+// and has to wait until an SM has drained. For the single token of a decode step the recurrent product W_hh z rides in the
+// tiled gate product (GateParams::hh_slices) and this kernel does the rest per sequence: it adds the k-slices, applies
+// the gates, updates z and runs the two small layers of the MLP. It needs 14 d' doubles of shared memory and shares SMs
+// with whatever else is running. Its rows of the interaction matrix are fetched into registers first, so that their
+// latency overlaps the k-slice sums. Every sum runs over the same indices in a fixed order (reproducible; float64 as
+// everywhere in the controller).
+constexpr int kTailThreads = 512;
+constexpr int kTailWarps = kTailThreads / 32;
+constexpr int kTailRows = 8;                    // matrix rows a warp has in flight
+
+__host__ __device__ inline size_t ctrl_tail_smem_bytes(int h) { return sizeof(double) * (14 * size_t(h) + 32); }
+
+// Rows r0 .. r0 + kTailRows - 1 of a row-major [n_rows, h] float matrix (h % 4 == 0) into registers: lane l takes
+// columns 4 l .. 4 l + 3 (and 128 + 4 l .. for h > 128) with 16-byte loads, all of them in flight at once.
+__device__ __forceinline__ void tail_rows_load(const float* __restrict__ W, int n_rows, int h, int r0, int lane,
+                                               float4 (&w)[kTailRows][2]) {
+#pragma unroll
+  for (int a = 0; a < kTailRows; ++a) {
+    const int r = min(r0 + a, n_rows - 1);
+#pragma unroll
+    for (int jj = 0; jj < 2; ++jj) {
+      const int j = 4 * lane + 128 * jj;
+      w[a][jj] = j < h ? __ldg(reinterpret_cast<const float4*>(W + size_t(r) * h + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+}
+// y[a] = sum_j w[a][j] v[j]: the lane's columns, then a shuffle tree over the lanes. Results in every lane.
+__device__ __forceinline__ void tail_rows_dot(const float4 (&w)[kTailRows][2], const double (&v)[2][4], double (&y)[kTailRows]) {
+#pragma unroll
+  for (int a = 0; a < kTailRows; ++a) {
+    double acc = 0.0;
+#pragma unroll
+    for (int jj = 0; jj < 2; ++jj) {
+      acc = fma(double(w[a][jj].x), v[jj][0], acc);
+      acc = fma(double(w[a][jj].y), v[jj][1], acc);
+      acc = fma(double(w[a][jj].z), v[jj][2], acc);
+      acc = fma(double(w[a][jj].w), v[jj][3], acc);
+    }
+    y[a] = acc;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+    for (int a = 0; a < kTailRows; ++a) y[a] += __shfl_xor_sync(0xffffffffu, y[a], o);
+}
+// this lane's columns of a shared-memory vector of length h, in the layout of tail_rows_load
+__device__ __forceinline__ void tail_lane_columns(const double* s_v, int h, int lane, double (&v)[2][4]) {
+#pragma unroll
+  for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { const int j = 4 * lane + 128 * jj + e; v[jj][e] = j < h ? s_v[j] : 0.0; }
+}
+// sum of part[i * stride] for i = i_begin .. i_end - 1, ascending, 24 loads in flight at a time
+__device__ __forceinline__ double tail_sum_slices(const double* __restrict__ part, size_t stride, int i_begin, int i_end) {
+  double acc = 0.0;
+  for (int i0 = i_begin; i0 < i_end; i0 += 24) {
+    double t[24];
+#pragma unroll
+    for (int i = 0; i < 24; ++i) t[i] = i0 + i < i_end ? part[size_t(i0 + i) * stride] : 0.0;
+#pragma unroll
+    for (int i = 0; i < 24; ++i) acc += t[i];
+  }
+  return acc;
+}
+
+// grid = B CTAs; p.tc must be 1, p.rows = B and p.h a multiple of 4. p.part holds ksplit partial sums of W_ih x per
+// (sequence, gate), followed by hh_slices partial sums of W_hh z (hh_slices == 0: the recurrent product is done here).
+static __global__ void __launch_bounds__(kTailThreads) ctrl_decode_tail_kernel(const RecurParams p) {
+  extern __shared__ __align__(16) unsigned char tail_smem[];
+  double* sm = reinterpret_cast<double*>(tail_smem);
+  const int h = p.h, G = 3 * h, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, b = blockIdx.x;
+  double* s_z = sm;            // [h]
+  double* s_gi = sm + h;       // [3h]  input side of every gate (+ bias)
+  double* s_gh = sm + 4 * h;   // [3h]  hidden side of every gate (+ bias)
+  double* s_pz = sm + 7 * h;   // [h]
+  double* s_half = sm + 8 * h; // [2][3h] the two halves of the k-slice sums
+  double* s_t = s_gi;          // [h]   w2[i] * tanh(.), reuses the gate sums once they are consumed
+  let_next_grid_start();
+  // ---- independent of the gate product: the state, this warp's rows of the interaction matrix, and the recurrent half if
+  // the gate product does not carry it ----
+  for (int i = tid; i < h; i += kTailThreads) s_z[i] = p.no_recurrence ? 0.0 : p.z[size_t(b) * h + i];
+  float4 w1r[kTailRows][2];
+  const bool mlp_once = h <= kTailWarps * kTailRows;            // every warp has its rows of W1 in registers (d' <= 128)
+  if (mlp_once) tail_rows_load(p.w1, h, h, warp * kTailRows, lane, w1r);
+  __syncthreads();
+  if (p.hh_slices == 0 && !p.no_recurrence) {
+    double v[2][4];
+    tail_lane_columns(s_z, h, lane, v);
+    for (int g0 = warp * kTailRows; g0 < G; g0 += kTailWarps * kTailRows) {
+      float4 w[kTailRows][2];
+      double y[kTailRows];
+      tail_rows_load(p.w_hh, G, h, g0, lane, w);
+      tail_rows_dot(w, v, y);
+      if (lane < kTailRows && g0 + lane < G) {
+        double mine = y[0];
+#pragma unroll
+        for (int a = 1; a < kTailRows; ++a) if (lane == a) mine = y[a];
+        s_gh[g0 + lane] = mine + double(__ldg(p.b_hh + g0 + lane));
+      }
+    }
+  }
+  // ---- the k-slices of the input-side product: two threads per gate, each adds one half of the slices in ascending
+  // order; then first half + second half ----
+  wait_for_prior_grid();
+  {
+    const size_t stride = size_t(p.rows) * G;
+    const int mid = (p.ksplit + 1) / 2;
+    for (int item = tid; item < 2 * G; item += kTailThreads) {
+      const int g = item % G, half = item / G;
+      s_half[half * G + g] = tail_sum_slices(p.part + size_t(b) * G + g, stride, half ? mid : 0, half ? p.ksplit : mid);
+    }
+    if (p.hh_slices > 0 || p.no_recurrence)
+      for (int g = tid; g < G; g += kTailThreads)
+        s_gh[g] = double(__ldg(p.b_hh + g)) +
+                  (p.no_recurrence ? 0.0 : tail_sum_slices(p.part + size_t(b) * G + g, stride, p.ksplit, p.ksplit + p.hh_slices));
+  }
+  __syncthreads();
+  for (int g = tid; g < G; g += kTailThreads) s_gi[g] = double(__ldg(p.b_ih + g)) + (s_half[g] + s_half[G + g]);
+  __syncthreads();
+  const int pos = p.n0;
+  for (int i = tid; i < h; i += kTailThreads) {
+    const double r = 1.0 / (1.0 + exp(-(s_gi[i] + s_gh[i])));
+    const double u = 1.0 / (1.0 + exp(-(s_gi[h + i] + s_gh[h + i])));
+    const double c = tanh(s_gi[2 * h + i] + r * s_gh[2 * h + i]);
+    const double zn = (1.0 - u) * c + u * s_z[i];
+    p.z[size_t(b) * h + i] = zn;
+    const double upos = p.a_tab ? 0.0 : double(pos) / p.pos_scale;
+    s_pz[i] = double(p.pos_w[i]) * upos + double(p.pos_b[i]) + zn;
+  }
+  __syncthreads();
+  {
+    double v[2][4];
+    tail_lane_columns(s_pz, h, lane, v);
+    for (int i0 = warp * kTailRows; i0 < h; i0 += kTailWarps * kTailRows) {
+      double y[kTailRows];
+      if (!mlp_once) tail_rows_load(p.w1, h, h, i0, lane, w1r);
+      tail_rows_dot(w1r, v, y);
+      if (lane < kTailRows && i0 + lane < h) {
+        double mine = y[0];
+#pragma unroll
+        for (int a = 1; a < kTailRows; ++a) if (lane == a) mine = y[a];
+        const int i = i0 + lane;
+        const double pre = mine + double(__ldg(p.b1 + i));
+        s_t[i] = double(__ldg(p.w2 + i)) * tanh(pre);
+        if (p.a_tab) p.a_tab[(size_t(b) * p.max_tokens + pos) * h + i] = pre;
+      }
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    double acc = 0.0;
+    for (int i = lane; i < h; i += 32) acc += s_t[i];
+    acc = warp_sum(acc);
+    if (lane == 0) {
+      const double sc = acc + double(p.b2[0]);
+      p.score[size_t(b) * p.max_tokens + pos] = float(sc);
+      p.sigma[size_t(b) * p.max_tokens + pos] = float(1.0 / (1.0 + exp(-sc)));
+    }
+  }
 }
 
 // ---- relative positions: every earlier token scored anew at every step ---------------------------

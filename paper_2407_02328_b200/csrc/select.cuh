@@ -41,6 +41,19 @@ __device__ __forceinline__ unsigned long long block_min_u64(unsigned long long v
   for (int w = 0; w < int(blockDim.x >> 5); ++w) r = tmp[w] < r ? tmp[w] : r;
   return r;
 }
+__device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v, unsigned long long* tmp) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long t = __shfl_xor_sync(0xffffffffu, v, o);
+    v = t > v ? t : v;
+  }
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) tmp[threadIdx.x >> 5] = v;
+  __syncthreads();
+  unsigned long long r = 0ull;
+  for (int w = 0; w < int(blockDim.x >> 5); ++w) r = tmp[w] > r ? tmp[w] : r;
+  return r;
+}
 // Exclusive position of this thread's flag among the block's flags (thread order); total out.
 __device__ __forceinline__ int block_rank(bool flag, int* tmp, int* total) {
   const unsigned bal = __ballot_sync(0xffffffffu, flag);
@@ -52,6 +65,24 @@ __device__ __forceinline__ int block_rank(bool flag, int* tmp, int* total) {
   for (int w = 0; w < int(blockDim.x >> 5); ++w) { const int c = tmp[w]; if (w < warp) base += c; tot += c; }
   *total = tot;
   return base + __popc(bal & ((1u << lane) - 1u));
+}
+
+// Exclusive prefix sum of v over the block's threads (thread order); total out. tmp: 64 words.
+__device__ __forceinline__ int block_scan_excl(int v, int* tmp, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  __syncthreads();
+  if (lane == 31) tmp[warp] = incl;
+  __syncthreads();
+  int base = 0, tot = 0;
+  for (int w = 0; w < int(blockDim.x >> 5); ++w) { const int c = tmp[w]; if (w < warp) base += c; tot += c; }
+  *total = tot;
+  return base + incl - v;
 }
 
 // ---- bitonic sort, DESCENDING, P a power of two -------------------------------------------------
@@ -174,12 +205,19 @@ struct SelectParams {
   int* rebuild_slot;          // [B,r_max]
   int* rebuild_count;         // [B]
   unsigned* err;
+  // decode step: the CTA that finishes last also compacts all sequences' lists into the row table of the rebuild
+  int* row_b;                 // [B * r_max] or null (no table: the bulk load builds it with row_table_kernel)
+  int* row_tok;
+  int* row_slot;
+  int* row_total;
+  unsigned long long* rows_accum;   // running total of rebuilt rows, or null
+  unsigned* done_count;       // arrivals of this launch's CTAs; left at zero by the last one
 };
 
 __host__ __device__ inline size_t select_smem_bytes(int C, int P) {
-  // keys[P] u64 | tok[C] | lst[C] | slots[C] int | role[C] u8 (padded) | 64 words scratch | 32 u64
+  // keys[P] u64 | tok[C] | lst[C] | slots[C] int | 64 words scratch + 512 offsets (row table) | role[C] u8 (padded) | 32 u64
   return sizeof(unsigned long long) * size_t(P) + sizeof(int) * 3 * size_t(C) + ((size_t(C) + 15) & ~size_t(15)) +
-         sizeof(int) * 64 + sizeof(unsigned long long) * 32;
+         sizeof(int) * (64 + 512) + sizeof(unsigned long long) * 32;
 }
 
 struct SelectSmem {
@@ -197,9 +235,14 @@ struct SelectSmem {
     lst = tok + C;
     slots = lst + C;
     tmp = slots + C;
-    role = reinterpret_cast<uint8_t*>(tmp + 64);
+    role = reinterpret_cast<uint8_t*>(tmp + 64 + 512);     // (selection kernels run with at most 512 threads)
   }
 };
+
+constexpr int kSelectIterMax = 16;     // lists up to this length are picked by repeated block-wide maxima
+constexpr int kSelectIterKeys = 16;    // keys a thread holds for that (512 threads x 16 = the largest token table)
+
+__device__ inline int place_rebuild_list(const struct SelectParams& p, const struct SelectSmem& sm, int b, int* tok_slot, int found);
 
 // Candidate keys -> sorted -> first r_max distinct tokens -> ascending empty slots.
 // Expects sm.tok / sm.role to hold the map with the new token already placed. Returns the count.
@@ -218,6 +261,29 @@ __device__ inline int assign_rebuild_list(const SelectParams& p, const SelectSme
       }
       sm.keys[i] = key;
     }
+  } else if (p.r_max <= kSelectIterMax && p.P <= kSelectIterKeys * NT) {
+    // A short list out of many released tokens (the paper's R = 8 of thousands): no sort. Every thread keeps its
+    // candidates' keys in registers and the block takes the largest key below the previous one, r_max times (keys are
+    // distinct: the token position is part of the key).
+    unsigned long long k[kSelectIterKeys];
+#pragma unroll
+    for (int j = 0; j < kSelectIterKeys; ++j) {
+      const int i = tid + j * NT;
+      k[j] = (i < n_seen && tok_slot[i] < 0) ? value_key(score[i], i) : 0ull;
+    }
+    unsigned long long prev = ~0ull;
+    int found = 0;
+    for (int r = 0; r < p.r_max; ++r) {
+      unsigned long long m = 0ull;
+#pragma unroll
+      for (int j = 0; j < kSelectIterKeys; ++j) m = (k[j] < prev && k[j] > m) ? k[j] : m;
+      m = block_max_u64(m, sm.tmp64);
+      if (m == 0ull) break;                                 // block-uniform: no released token is left
+      if (tid == 0) sm.lst[r] = int(m & 0xffffffffull);
+      prev = m;
+      ++found;
+    }
+    return place_rebuild_list(p, sm, b, tok_slot, found);
   } else {
     for (int i = tid; i < p.P; i += NT)
       sm.keys[i] = (i < n_seen && tok_slot[i] < 0) ? value_key(score[i], i) : 0ull;
@@ -233,8 +299,15 @@ __device__ inline int assign_rebuild_list(const SelectParams& p, const SelectSme
     if (f && pos < p.r_max) sm.lst[pos] = int(sm.keys[i] & 0xffffffffull);
     found += tot;
   }
+  return place_rebuild_list(p, sm, b, tok_slot, found);
+}
+
+// The first min(found, r_max) tokens of sm.lst (most valuable first) take the empty slots in ascending order.
+__device__ inline int place_rebuild_list(const SelectParams& p, const SelectSmem& sm, int b, int* tok_slot, int found) {
+  const int tid = threadIdx.x, NT = blockDim.x;
   const int cnt = min(found, p.r_max);
   int seen = 0;
+  __syncthreads();
   for (int s0 = 0; s0 < p.C && seen < cnt; s0 += NT) {
     const int s = s0 + tid;
     const bool f = s < p.C && sm.role[s] == ROLE_EMPTY;
@@ -290,6 +363,51 @@ __global__ void __launch_bounds__(128) row_table_kernel(const int* rebuild_tok, 
   }
 }
 
+// Called by every thread of every CTA of a decode step's selection launch once its sequence's list is written: the CTA
+// that arrives last turns the per-sequence lists into the compact row table (b-major, list order) that the gather and
+// the GEMM of the rebuild walk, so that no further launch stands between the selection and them.
+__device__ inline void select_finish_row_table(const SelectParams& p, int* s_tmp) {
+  if (p.row_b == nullptr) return;
+  const int tid = threadIdx.x, NT = blockDim.x;
+  __threadfence();                                   // this CTA's list is visible before its arrival is
+  __syncthreads();
+  if (tid == 0) s_tmp[63] = (atomicAdd(p.done_count, 1u) == unsigned(p.B - 1)) ? 1 : 0;
+  __syncthreads();
+  if (s_tmp[63] == 0) return;
+  __threadfence();
+  // offsets: sequences in chunks of blockDim.x, an exclusive scan of the counts per chunk (every thread ends up with the
+  // same running total); then all threads copy the chunk's entries, one (sequence, list position) pair each per round
+  int* s_off = s_tmp + 64;                           // [blockDim.x], provided by the caller behind its scratch words
+  int base = 0;
+  for (int b0 = 0; b0 < p.B; b0 += NT) {
+    const int b = b0 + tid;
+    const int mine = b < p.B ? min(__ldcg(p.rebuild_count + b), p.r_max) : 0;
+    int tot;
+    const int excl = block_scan_excl(mine, s_tmp, &tot);
+    s_off[tid] = base + excl;
+    __syncthreads();
+    const int nb = min(NT, p.B - b0);
+#pragma unroll 4
+    for (int idx = tid; idx < nb * p.r_max; idx += NT) {
+      const int bb = idx / p.r_max, j = idx - bb * p.r_max;
+      const int next = bb + 1 < nb ? s_off[bb + 1] : base + tot;
+      if (j < next - s_off[bb]) {
+        const size_t src = size_t(b0 + bb) * p.r_max + j;
+        p.row_b[s_off[bb] + j] = b0 + bb;
+        p.row_tok[s_off[bb] + j] = __ldcg(p.rebuild_tok + src);
+        p.row_slot[s_off[bb] + j] = __ldcg(p.rebuild_slot + src);
+      }
+    }
+    base += tot;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    *p.row_total = base;
+    if (p.rows_accum) *p.rows_accum += static_cast<unsigned long long>(base);
+    *p.done_count = 0u;                              // ready for the next launch
+  }
+}
+
 // One decode step's selection for sequence blockIdx.x.
 __device__ inline void select_step(const SelectParams& p, unsigned char* smem) {
   const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x, C = p.C;
@@ -338,6 +456,7 @@ __device__ inline void select_step(const SelectParams& p, unsigned char* smem) {
     p.slot_tok_new[size_t(b) * C + s] = sm.tok[s];
     p.slot_role_new[size_t(b) * C + s] = sm.role[s];
   }
+  select_finish_row_table(p, sm.tmp);
 }
 
 // Bulk load of T tokens into an empty cache: the newest token plus the min(m-1, T-1) most
