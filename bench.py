@@ -42,9 +42,13 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES = {
     ("rebuild projection", "cfg3_llama7b_b64_c512_rebuild20pct"):
         {"bytes": 284.9e6 + 144.9e6, "rows": 9950.0, "profile": "profiles/rebuild_tc_pair_kernel_cfg3.md"},
-    ("attention kernel", "cfg3_llama7b_b64_c512_rebuild20pct"): None,
-    ("attention kernel", "cfg4_llama7b_L32_b32_c1024"): None,
-    ("attention kernel", "cfg5_sweep_c1024_b32"): None,
+    ("attention kernel", "cfg3_llama7b_b64_c512_rebuild20pct"):
+        {"bytes": 359.1e6 + 6.7e6, "rows": None, "profile": "profiles/attention_tma_kernel_cfg3.md"},
+    # config 4's per-layer launch, captured on a one-layer cache of the same shape (the sweep point C=1024, B=32)
+    ("attention kernel", "cfg4_llama7b_L32_b32_c1024"):
+        {"bytes": 403.4e6 + 4.5e6, "rows": None, "profile": "profiles/attention_tma_kernel_cfg4_shape.md"},
+    ("attention kernel", "cfg5_sweep_c1024_b32"):
+        {"bytes": 403.4e6 + 4.5e6, "rows": None, "profile": "profiles/attention_tma_kernel_cfg4_shape.md"},
 }
 
 

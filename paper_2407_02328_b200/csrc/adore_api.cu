@@ -581,7 +581,10 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
   sp.explicit_list = ex && r_in > 0 ? explicit_list : nullptr;
   sp.explicit_count = ex && r_in > 0 ? explicit_count : nullptr;
   sp.r_in = r_in;
-  if (f.rebuild_max > 0) {                      // the last CTA of the launch writes the rebuild's row table
+  // Short lists (the paper's R = 8): the last CTA of the launch also writes the rebuild's row table. Long lists keep the
+  // table's own launch, one CTA per sequence: one CTA copying 16k entries took longer (16 us) than that launch (5 us).
+  const bool table_in_select = f.rebuild_max > 0 && size_t(f.batch) * f.rebuild_max <= 4096;
+  if (table_in_select) {
     sp.row_b = c->row_b; sp.row_tok = c->row_tok; sp.row_slot = c->row_slot; sp.row_total = c->row_total;
     sp.rows_accum = c->rows_accum; sp.done_count = c->sel_done;
   }
@@ -598,6 +601,10 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
   // x_new is borrowed only until the selection has run (which the main stream waits for anyway)
   CUDA_OK(cudaEventRecord(c->ev_xrow, sel));
   CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_xrow, 0));
+  if (!table_in_select) {
+    st = launch_row_table(c, true, sel);
+    if (st != ADORE_OK) return st;
+  }
   // A short list's rows are copied out of the token store into the GEMM's compact input right away, beside the
   // attention, so that the rebuild that follows starts with its GEMM. Long lists are copied after the attention:
   // side by side the two slow each other down by more than the copy takes (measured at 15k rows: attention
