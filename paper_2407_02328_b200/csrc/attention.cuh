@@ -54,25 +54,36 @@ __host__ __device__ inline size_t attn_smem_bytes(int C, int DH, int threads = k
          sizeof(float) * (threads / 32) * DH + sizeof(float) * 64;
 }
 
-template <int NT>
+// Who "the block" of the shared phases is: the whole CTA, or one 128-thread group of a CTA that works on two pairs at
+// once (threads 0..127 and 128..255, each group with a named barrier of its own; further warps of the CTA stay out).
+struct CtaScope {
+  static __device__ __forceinline__ int tid() { return threadIdx.x; }
+  static __device__ __forceinline__ void sync() { __syncthreads(); }
+};
+struct GroupScope {
+  static __device__ __forceinline__ int tid() { return threadIdx.x & 127; }
+  static __device__ __forceinline__ void sync() { asm volatile("bar.sync %0, 128;" ::"r"(1 + (threadIdx.x >> 7)) : "memory"); }
+};
+
+template <int NT, typename SY = CtaScope>
 __device__ __forceinline__ float block_sum_f(float v, float* tmp) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = SY::tid() & 31, warp = SY::tid() >> 5;
   v = warp_sum(v);
-  __syncthreads();                       // tmp may still be read from a previous reduction
+  SY::sync();                       // tmp may still be read from a previous reduction
   if (lane == 0) tmp[warp] = v;
-  __syncthreads();
+  SY::sync();
   float r = 0.f;
 #pragma unroll
   for (int w = 0; w < NT / 32; ++w) r += tmp[w];
   return r;
 }
-template <int NT>
+template <int NT, typename SY = CtaScope>
 __device__ __forceinline__ float block_max_f(float v, float* tmp) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = SY::tid() & 31, warp = SY::tid() >> 5;
   v = warp_max(v);
-  __syncthreads();
+  SY::sync();
   if (lane == 0) tmp[warp] = v;
-  __syncthreads();
+  SY::sync();
   float r = tmp[0];
 #pragma unroll
   for (int w = 1; w < NT / 32; ++w) r = fmaxf(r, tmp[w]);
@@ -102,13 +113,13 @@ struct AttnSmem {
 // Phases 2-3, given the logits of all C+1 rows in shared memory (-inf for empty slots): decides the
 // kept set, turns the logits into weights in place (0 for rows not kept), writes the weights out and
 // builds the ordered list of kept row indices. Returns the number of kept rows. Every thread of the
-// block calls it after a __syncthreads(); the results are published by a final __syncthreads().
+// block (scope SY) calls it after a barrier of that scope; the results are published by a final barrier.
 //
 // Every warp owns one contiguous segment of the rows and every lane keeps its rows' order-preserving keys in
 // registers (row seg_begin + 32 k + lane in register k, KPT registers): the passes of the radix select, the maximum
 // and the exponentials are then unrolled loops over registers with no shared-memory load in their dependency chains,
 // and the kept rows are counted and placed with ballots; the block meets only to exchange counts.
-template <typename T, int DH, int NT, int KPT>
+template <typename T, int DH, int NT, int KPT, typename SY>
 __device__ __forceinline__ int attention_keep_and_weights_impl(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh, int seg) {
   constexpr int NW = NT / 32;
   float* s_logit = sm.logit;
@@ -117,7 +128,7 @@ __device__ __forceinline__ int attention_keep_and_weights_impl(const AttnParams<
   float* s_tmp = sm.tmp;
   int* s_sel = sm.sel;
   const int rows = p.C + 1;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = SY::tid(), lane = tid & 31, warp = tid >> 5;
   const int seg_begin = warp * seg, seg_end = min(rows, seg_begin + seg);
 
   // ---- phase 2: which logits are kept (K largest, lower index wins ties) -------------------
@@ -131,7 +142,7 @@ __device__ __forceinline__ int attention_keep_and_weights_impl(const AttnParams<
     cnt += (l > -INFINITY) ? 1 : 0;
   }
   for (int i = tid; i < 256; i += NT) s_hist[i] = 0u;
-  const int n_cand = __float2int_rn(block_sum_f<NT>(float(cnt), s_tmp));   // (its barriers also publish the zeroed bins)
+  const int n_cand = __float2int_rn(block_sum_f<NT, SY>(float(cnt), s_tmp));   // (its barriers also publish the zeroed bins)
   uint32_t thr_key = 0u;                  // keep every candidate unless there are more than K
   if (n_cand > p.topk) {
     uint32_t prefix = 0u, mask = 0u;
@@ -141,7 +152,7 @@ __device__ __forceinline__ int attention_keep_and_weights_impl(const AttnParams<
 #pragma unroll
       for (int k = 0; k < KPT; ++k)
         if (key[k] != 0u && (key[k] & mask) == prefix) atomicAdd(&s_hist[(key[k] >> shift) & 255u], 1u);
-      __syncthreads();
+      SY::sync();
       if (warp == 0) {
         int c[8], tot = 0;
 #pragma unroll
@@ -162,7 +173,7 @@ __device__ __forceinline__ int attention_keep_and_weights_impl(const AttnParams<
           }
         }
       }
-      __syncthreads();
+      SY::sync();
       prefix |= uint32_t(s_sel[0]) << shift;
       mask |= 255u << shift;
       need = s_sel[1];
@@ -170,13 +181,13 @@ __device__ __forceinline__ int attention_keep_and_weights_impl(const AttnParams<
     thr_key = prefix;
     const int n_eq = s_sel[2];
     if (n_eq != need) {                   // exact ties at the threshold (block-uniform): keep the lowest indices
-      __syncthreads();
+      SY::sync();
       if (tid == 0) {
         int left = need;
         for (int i = 0; i < rows; ++i)
           if (float_key(s_logit[i]) == thr_key) { if (left > 0) --left; else s_logit[i] = -INFINITY; }
       }
-      __syncthreads();
+      SY::sync();
 #pragma unroll
       for (int k = 0; k < KPT; ++k) {     // the dropped rows now read -inf
         const int i = seg_begin + 32 * k + lane;
@@ -195,7 +206,7 @@ __device__ __forceinline__ int attention_keep_and_weights_impl(const AttnParams<
   // the largest key is the largest logit: undo the order-preserving map
   float mx = -INFINITY;
   if (kmax != 0u) mx = __uint_as_float((kmax & 0x80000000u) ? (kmax & 0x7fffffffu) : ~kmax);
-  mx = block_max_f<NT>(mx, s_tmp);
+  mx = block_max_f<NT, SY>(mx, s_tmp);
   float part = 0.f;
   int kept_here = 0;
   float ev[KPT];
@@ -208,7 +219,7 @@ __device__ __forceinline__ int attention_keep_and_weights_impl(const AttnParams<
     kept_here += __popc(__ballot_sync(0xffffffffu, keep));
   }
   if (lane == 0) s_sel[8 + warp] = kept_here;
-  const float inv = 1.f / block_sum_f<NT>(part, s_tmp);     // (its barriers also publish the warps' counts)
+  const float inv = 1.f / block_sum_f<NT, SY>(part, s_tmp);     // (its barriers also publish the warps' counts)
   int base = 0, n_kept = 0;
 #pragma unroll
   for (int w = 0; w < NW; ++w) { const int c = s_sel[8 + w]; if (w < warp) base += c; n_kept += c; }
@@ -226,25 +237,25 @@ __device__ __forceinline__ int attention_keep_and_weights_impl(const AttnParams<
     if (keep) s_list[base + __popc(bal & ((1u << lane) - 1u))] = i;
     base += __popc(bal);
   }
-  __syncthreads();
+  SY::sync();
   return n_kept;
 }
 
-template <typename T, int DH, int NT = kAttnThreads>
+template <typename T, int DH, int NT = kAttnThreads, typename SY = CtaScope>
 __device__ __forceinline__ int attention_keep_and_weights(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh /* row of out/weights */) {
   constexpr int NW = NT / 32;
   const int rows = p.C + 1;
   const int seg = (((rows + NW - 1) / NW) + 31) & ~31;      // rows per warp, a multiple of 32
   // 9 registers per lane cover C <= 1151 with 4 warps and C <= 2303 with 8; kernels of 4 warps are launched for
   // C <= 1024 only, those of 8 warps for any capacity up to 4096 (17 registers)
-  if (NT <= 128 || seg <= 9 * 32) return attention_keep_and_weights_impl<T, DH, NT, 9>(p, sm, bh, seg);
-  return attention_keep_and_weights_impl<T, DH, NT, 17>(p, sm, bh, seg);
+  if (NT <= 128 || seg <= 9 * 32) return attention_keep_and_weights_impl<T, DH, NT, 9, SY>(p, sm, bh, seg);
+  return attention_keep_and_weights_impl<T, DH, NT, 17, SY>(p, sm, bh, seg);
 }
 
 // Phase 4 with direct loads: adds w_s * V[s] of the kept rows [j_begin, n_kept) of the list into acc (this lane's 16-byte column
 // slice; lanes of different row groups and warps hold partial sums). U loads of 16 bytes are in flight per lane: a gather of
 // 256-byte rows needs on the order of 100 KB in flight per SM to run at the memory system's rate.
-template <typename T, int DH, int NT = kAttnThreads, int U = kAttnUnroll>
+template <typename T, int DH, int NT = kAttnThreads, int U = kAttnUnroll, typename SY = CtaScope>
 __device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh, int n_kept,
                                                         float (&acc)[Elem<T>::kPer16B], int j_begin = 0) {
   constexpr int NW = NT / 32;
@@ -254,7 +265,7 @@ __device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, 
   const float* s_logit = sm.logit;
   const int* s_list = sm.list;
   const int C = p.C;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = SY::tid() & 31, warp = SY::tid() >> 5;
   const int sub = lane / LPR, li = lane % LPR;
   const size_t row_bytes = size_t(DH) * sizeof(T);
   const unsigned char* Vb = reinterpret_cast<const unsigned char*>(p.Vc) + size_t(bh) * C * row_bytes;
@@ -286,7 +297,7 @@ __device__ __forceinline__ void attention_values_direct(const AttnParams<T>& p, 
 
 // Adds the partial sums of all row groups and warps, writes `out`, then writes the current token's
 // row into its slot (append of the most recent state, Section 2.2 third bullet).
-template <typename T, int DH, int NT = kAttnThreads>
+template <typename T, int DH, int NT = kAttnThreads, typename SY = CtaScope>
 __device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const AttnSmem<DH, NT>& sm, int bh,
                                                  float (&acc)[Elem<T>::kPer16B], int out_row = -1, bool admit = true) {
   if (out_row < 0) out_row = bh;
@@ -295,7 +306,7 @@ __device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const A
   constexpr int LPR = DH / EPL;
   float* s_red = sm.red;
   const int C = p.C;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = SY::tid(), lane = tid & 31, warp = tid >> 5;
   const int sub = lane / LPR, li = lane % LPR;
   const int b = bh / p.H;
   const size_t row_bytes = size_t(DH) * sizeof(T);
@@ -310,7 +321,7 @@ __device__ __forceinline__ void attention_finish(const AttnParams<T>& p, const A
   if (sub == 0)
 #pragma unroll
     for (int e = 0; e < EPL; ++e) s_red[warp * DH + li * EPL + e] = acc[e];
-  __syncthreads();
+  SY::sync();
   for (int e = tid; e < DH; e += NT) {
     float s = 0.f;
 #pragma unroll
