@@ -29,18 +29,19 @@ constexpr int kMaxPrefillRows = 8192;       // controller rows per chunk during 
 // One step's selection for sequence blockIdx.x. It ranks tokens 0..n-1 by the scores they already have, so it
 // does not wait for the controller's score of the new token n (that score is first read at step n+1) and runs
 // beside the controller kernels.
-template <typename T>
-__global__ void __launch_bounds__(512) select_kernel(const SelectParams sp, const T* x_new, T* x_store, int d) {
+__global__ void __launch_bounds__(512, 2) select_kernel(const SelectParams sp) {
   extern __shared__ __align__(128) unsigned char smem[];
-  const int b = blockIdx.x;
   let_next_grid_start();
-  // keep the new token's layer-input row: it is what a later rebuild recomputes from
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(x_new + size_t(b) * d);
-    uint4* dst = reinterpret_cast<uint4*>(x_store + (size_t(b) * sp.max_tokens + sp.n) * d);
-    for (int i = threadIdx.x; i < int(d * sizeof(T) / 16); i += blockDim.x) dst[i] = src[i];
-  }
   select_step(sp, smem);
+}
+
+// Keeps the new token's layer-input row (it is what a later rebuild recomputes from, and what the controller reads):
+// row b of x_new goes to position n of sequence b in the token store. One CTA per sequence, 16-byte pieces.
+__global__ void __launch_bounds__(256) store_row_kernel(const uint4* x_new, uint4* x_store, int row_pieces, long long seq_pieces,
+                                                        long long at_pieces) {
+  const uint4* src = x_new + size_t(blockIdx.x) * row_pieces;
+  uint4* dst = x_store + size_t(blockIdx.x) * seq_pieces + at_pieces;
+  for (int i = threadIdx.x; i < row_pieces; i += blockDim.x) dst[i] = src[i];
 }
 
 __global__ void __launch_bounds__(512) ctrl_recur_kernel(const RecurParams rp, int resident, unsigned* err) {
@@ -161,6 +162,8 @@ struct adore_cache {
   // the NEXT step's selection, so it may run on past the end of the step that launched it.
   cudaStream_t ctl = nullptr;
   cudaEvent_t ev_xrow = nullptr, ev_attn = nullptr, ev_ctrl = nullptr;   // the token's row is in the store / the attention of layer 0 is done
+  cudaEvent_t ev_gather = nullptr;  // the early gather of a short list (selection stream) is done: the rebuild waits for it
+  bool xrow_pending = false, gather_pending = false;   // events the main stream / the rebuild's stream has not waited for yet
   bool ctrl_pending = false;    // ev_ctrl was recorded and the main stream has not waited for it yet
   // uploads of the host-buffer entry point run on their own stream, beside the previous rebuild
   cudaStream_t copy = nullptr;
@@ -266,6 +269,10 @@ adore_status_t wait_rebuild(adore_cache* c, int layer, cudaStream_t stream) {
 // Makes the main stream wait for every rebuild that runs beside it. The side stream runs them in order, so the
 // event of the most recent one covers all.
 adore_status_t join_rebuilds(adore_cache* c) {
+  if (c->gather_pending) {        // an early gather that no rebuild on the main stream has waited for
+    CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_gather, 0));
+    c->gather_pending = false;
+  }
   if (c->rb_last >= 0) CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_rebuilt[c->rb_last], 0));
   c->rb_last = -1;
   std::fill(c->rb_pending.begin(), c->rb_pending.end(), char(0));
@@ -320,6 +327,13 @@ adore_status_t fill_i32(adore_cache* c, int* p, int v, size_t n) {
 // One CTA per sequence owns an SM for a latency-bound chain (GRU, MLP, sort): the more warps, the better
 // the loads and barriers are hidden.
 int select_threads(const adore_cache*) { return 512; }
+// The step's selection runs beside the attention of layer 0. With few (batch, head) pairs that launch has 256-thread
+// CTAs of 16k registers, three or four to an SM: a selection CTA of 256 threads x 64 registers still fits beside three
+// of them and starts at once, one of 512 threads waits until an SM has drained (measured: 14 us later).
+int step_select_threads(const adore_cache* c) {
+  const adore_config_t& f = c->cfg;
+  return f.batch * f.n_heads < 1024 && f.max_tokens <= 4096 ? 256 : 512;
+}
 size_t ctrl_smem(const adore_cache* c) {
   const int h = c->cfg.ctrl_hidden;
   return ctrl_resident_ok(h) ? ctrl_resident_smem_bytes(h) : recur_smem_bytes(h);
@@ -483,6 +497,10 @@ adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, co
     // Rows gathered from the token store for this step's table serve every layer that rebuilds from the store.
     const bool from_store = step_table && x_table == nullptr && size_t(m_max) <= c->tc.a_rows;
     int launched = 0;
+    if (from_store && c->rows_gathered && c->gather_pending) {
+      CUDA_OK(cudaStreamWaitEvent(stream, c->ev_gather, 0));
+      if (stream == c->stream) c->gather_pending = false;       // (a side stream: every rebuild of the step waits)
+    }
     static const int lean_mode = dev_switch_int("ADORE_REBUILD_LEAN", 1);
     cudaError_t e = launch_rebuild_tc(c->tc, p, layer, m_max, stream, &launched, from_store && c->rows_gathered,
                                       lean_mode != 0 && stream != c->stream);
@@ -562,16 +580,30 @@ adore_status_t check_config(const adore_config_t* f) {
 
 namespace {
 
-// Launches the controller of token n (gates, then GRU + MLP + score) on the controller stream and the step's
-// selection and row table on `sel`. Both streams must already wait for everything they depend on in the main stream.
+// Launches, on the controller stream, the copy of the new token's row into the token store and the controller of
+// token n (gates, then GRU + MLP + score), and on `sel` the step's selection and row table. Both streams must already
+// wait for the point of the main stream the step starts from; with `ctrl_after_attention` the controller also waits
+// for ev_attn, which the caller has recorded. Records ev_xrow (x_new has been read) and, if `sel` is a side stream,
+// ev_join (map, lists and row table are written); the main stream has to wait for both.
 adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new, const int32_t* explicit_list,
                                              const int32_t* explicit_count, int32_t r_in, cudaStream_t sel,
-                                             bool early_gather) {
+                                             bool early_gather, bool ctrl_after_attention) {
   const adore_config_t& f = c->cfg;
   const bool ex = f.rebuild_mode == ADORE_REBUILD_EXPLICIT;
   adore_status_t st;
   StageScope scope(c, 1);
   const bool controller = !(f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION);   // else the scores come from the attention
+  {
+    const int row_pieces = int(size_t(f.hidden) * c->esz / 16);
+    store_row_kernel<<<f.batch, 256, 0, c->ctl>>>(static_cast<const uint4*>(x_new), static_cast<uint4*>(c->x_store), row_pieces,
+                                                 static_cast<long long>(f.max_tokens) * row_pieces,
+                                                 static_cast<long long>(c->n) * row_pieces);
+    ++c->launches;
+    CUDA_OK(cudaGetLastError());
+    CUDA_OK(cudaEventRecord(c->ev_xrow, c->ctl));
+    c->xrow_pending = true;
+    if (ctrl_after_attention) CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_attn, 0));
+  }
   if (c->ctrl_pending) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_ctrl, 0));   // scores of token n-1
   // The selection chain is what the step waits for, so it is queued first; the controller's launches follow.
   st = launch_rescore(c, c->n, sel);            // relative positions: the ranking below is the one seen from token n
@@ -589,21 +621,19 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
     sp.rows_accum = c->rows_accum; sp.done_count = c->sel_done;
   }
   const size_t smem = select_smem_bytes(f.capacity, P);
-  if (f.dtype == ADORE_F32)
-    select_kernel<float><<<f.batch, select_threads(c), smem, sel>>>(
-        sp, static_cast<const float*>(x_new), static_cast<float*>(c->x_store), f.hidden);
-  else
-    select_kernel<__nv_bfloat16><<<f.batch, select_threads(c), smem, sel>>>(
-        sp, static_cast<const __nv_bfloat16*>(x_new), static_cast<__nv_bfloat16*>(c->x_store), f.hidden);
+  select_kernel<<<f.batch, step_select_threads(c), smem, sel>>>(sp);
   ++c->launches;
   CUDA_OK(cudaGetLastError());
-  // the selection kernel has put the token's row into the token store: the controller reads it from there, so that
-  // x_new is borrowed only until the selection has run (which the main stream waits for anyway)
-  CUDA_OK(cudaEventRecord(c->ev_xrow, sel));
-  CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_xrow, 0));
   if (!table_in_select) {
     st = launch_row_table(c, true, sel);
     if (st != ADORE_OK) return st;
+  }
+  c->joined = sel == c->stream;
+  if (!c->joined) {
+    CUDA_OK(cudaEventRecord(c->ev_join, sel));   // the gather below is not part of what the main stream waits for
+    // The gate product starts when the selection is done: side by side the two were measured several times slower
+    // (gate product 14 -> 70 us, selection 18 -> 28 us at batch 16), whereas beside the rebuild GEMM it loses little.
+    CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_join, 0));
   }
   // A short list's rows are copied out of the token store into the GEMM's compact input right away, beside the
   // attention, so that the rebuild that follows starts with its GEMM. Long lists are copied after the attention:
@@ -621,6 +651,7 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
       CUDA_OK(launch_gather_tc<__nv_bfloat16>(c->tc, gp, m_max, sel));
       ++c->launches;
       c->rows_gathered = true;
+      if (sel != c->stream) { CUDA_OK(cudaEventRecord(c->ev_gather, sel)); c->gather_pending = true; }   // the rebuild waits for it
     }
   }
   // the recurrent product rides in the gate product when the state has whole 32-element chunks and is not ignored
@@ -778,8 +809,7 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
     cudaFuncSetAttribute(ctrl_recur_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     cudaFuncSetAttribute(ctrl_gates_wide_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGateWideSmem));
     cudaFuncSetAttribute(ctrl_gates_wide_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGateWideSmem));
-    cudaFuncSetAttribute(select_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-    cudaFuncSetAttribute(select_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     cudaFuncSetAttribute(bulk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
     if (cudaGetLastError() != cudaSuccess) { adore_cache_destroy(c); return ADORE_ERR_CUDA; }
   }
@@ -792,6 +822,7 @@ adore_status_t adore_cache_create(const adore_config_t* cfg, const adore_control
       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
       cudaStreamCreateWithPriority(&c->ctl, cudaStreamNonBlocking, prio_high) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_xrow, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_gather, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_attn, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_ctrl, cudaEventDisableTiming) != cudaSuccess ||
       cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess ||
@@ -853,6 +884,7 @@ adore_status_t adore_cache_destroy(adore_cache_t* c) {
   if (c->ev_step_open) cudaEventDestroy(c->ev_step_open);
   for (cudaEvent_t e : c->ev_rebuilt) cudaEventDestroy(e);
   if (c->ev_xrow) cudaEventDestroy(c->ev_xrow);
+  if (c->ev_gather) cudaEventDestroy(c->ev_gather);
   if (c->ev_attn) cudaEventDestroy(c->ev_attn);
   if (c->ev_ctrl) cudaEventDestroy(c->ev_ctrl);
   if (c->copy) { cudaStreamSynchronize(c->copy); cudaStreamDestroy(c->copy); }
@@ -980,13 +1012,12 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
     // The controller's float64 products would take SM time from the attention, which fills the GPU and is on the step's
     // critical path, while their result is first needed by the NEXT step's selection: they start when the attention
     // of layer 0 is done and run beside what follows it (the gather of a long rebuild list, the next layers).
+    // The copy of the new token's row into the store, which is all that reads x_new, does start at the fork.
     CUDA_OK(cudaEventRecord(c->ev_attn, c->stream));
-    CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_attn, 0));
-    st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel, true);
+    CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
+    st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel, true, true);
     if (st != ADORE_OK) return st;
     if (group_mark(c, 2, c->ctl) != ADORE_OK) return ADORE_ERR_CUDA;
-    c->joined = sel == c->stream;
-    if (!c->joined) CUDA_OK(cudaEventRecord(c->ev_join, sel));
     c->cur = 1 - c->cur;
     c->n += 1;
     c->step_layer0_done = 1;
@@ -1003,6 +1034,10 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
   }
   if (!c->joined) CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
   c->joined = true;
+  if (c->xrow_pending) {          // x_new is the caller's again once the main stream has passed this point
+    CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_xrow, 0));
+    c->xrow_pending = false;
+  }
   {
     StageScope scope(c, 3);
     const size_t row_bytes = size_t(f.head_dim) * c->esz;
@@ -1037,13 +1072,12 @@ adore_status_t adore_step_begin(adore_cache_t* c, const void* x_new, const int32
   CUDA_OK(cudaEventRecord(c->ev_fork, c->stream));
   if (sel != c->stream) CUDA_OK(cudaStreamWaitEvent(sel, c->ev_fork, 0));
   CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_fork, 0));
-  adore_status_t st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel, false);
+  adore_status_t st = launch_controller_and_selection(c, x_new, explicit_list, explicit_count, r_in, sel, false, false);
   if (st != ADORE_OK) return st;
-  if (sel != c->stream) {
-    CUDA_OK(cudaEventRecord(c->ev_join, sel));
-    CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
-  }
+  if (!c->joined) CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_join, 0));
   c->joined = true;
+  CUDA_OK(cudaStreamWaitEvent(c->stream, c->ev_xrow, 0));      // x_new has been read
+  c->xrow_pending = false;
   if (c->ev_step_open) CUDA_OK(cudaEventRecord(c->ev_step_open, c->stream));
   c->cur = 1 - c->cur;
   c->attn = c->cur;             // this step's attention reads the NEW map

@@ -44,6 +44,21 @@ struct GateParams {
 constexpr int kGateKInner = 32;
 constexpr int kGateHhSlice = 64;   // k-slice of the recurrent product when it rides in the gate product (decode step)
 
+// A decode step's CTA reads a small block of the weight matrix (tile_g rows x a k-slice) through a chain of dependent
+// chunk loads, each one round trip to memory; beside a kernel that saturates HBM (the rebuild GEMM) a round trip takes
+// several microseconds and the chain was measured at 46 us instead of 14. Asking for the whole block at once (L2
+// prefetches, one per 128-byte line, spread over the threads) leaves one such round trip. Blocks above 64 KB (prompt
+// chunks, where k is not split) are streamed as before.
+__device__ __forceinline__ void gate_prefetch_block(const float* w, int ld, int g0, int tile_g, int G, int k_begin, int k_end) {
+  const int cols = k_end - k_begin;
+  if (cols <= 0 || size_t(cols) * tile_g * sizeof(float) > 65536) return;
+  const int lines = (cols * int(sizeof(float)) + 127) / 128;       // per row; rows start 128-byte aligned when k_begin % 32 == 0
+  for (int i = threadIdx.x; i < tile_g * lines; i += blockDim.x) {
+    const int g = g0 + i / lines, l = i % lines;
+    if (g < G) asm volatile("prefetch.global.L2 [%0];" ::"l"(w + size_t(g) * ld + k_begin + l * 32));
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kGateThreads) ctrl_gates_kernel(const GateParams<T> p) {
   constexpr int WS = kGateTileG + 2, XS = kGateTileR + 2;       // padded, rows stay 16-byte aligned
@@ -56,6 +71,7 @@ __global__ void __launch_bounds__(kGateThreads) ctrl_gates_kernel(const GatePara
   const int ld = is_hh ? p.h : p.d;
   const int k_begin = is_hh ? (ks - p.ksplit) * kGateHhSlice : ks * p.kslice;
   const int k_end = is_hh ? min(p.h, k_begin + kGateHhSlice) : min(p.d, k_begin + p.kslice);
+  gate_prefetch_block(is_hh ? p.w_hh : p.w_ih, ld, g0, kGateTileG, p.G, k_begin, k_end);
   // per chunk this thread fetches two float4 of W (gates wg, wg+32; k offset 4*wk) and 4 elements of one x row
   const int wk = tid & 7, wg = tid >> 3;
   const int xr = tid >> 3, xk = tid & 7;
@@ -155,6 +171,7 @@ __global__ void __launch_bounds__(kGateWideThreads) ctrl_gates_wide_kernel(const
   const int ld = is_hh ? p.h : p.d;
   const int k_begin = is_hh ? (ks - p.ksplit) * kGateHhSlice : ks * p.kslice;
   const int k_end = is_hh ? min(p.h, k_begin + kGateHhSlice) : min(p.d, k_begin + p.kslice);
+  gate_prefetch_block(is_hh ? p.w_hh : p.w_ih, ld, g0, kGateWideG, p.G, k_begin, k_end);
   // fetch roles: 8 float4 of W (gate (tid + 128 q) / 8, k offset 4 * ((tid + 128 q) % 8)) and 2 x 8 elements of x
   // (row (tid + 128 q) / 4, k offset 8 * ((tid + 128 q) % 4)) per chunk of 32 k
   const float* wsrc[8];

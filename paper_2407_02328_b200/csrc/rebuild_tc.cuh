@@ -208,23 +208,85 @@ __device__ __forceinline__ void tc_store_partial(uint32_t taddr, float* dst, int
   }
 }
 
+// 32 consecutive output columns of one row, starting at column col0 of [K | V]: rotary embedding on the key half
+// (adjacent pairs, the token's original position), rounding to bfloat16, four 16-byte stores into the token's slot.
+__device__ __forceinline__ void tc_rope_store_32(const TcGemmParams& p, float (&y)[32], int col0, int b, int tok, int slot) {
+  const int HD = p.H * p.DH;
+  const int part = col0 / HD, h = (col0 % HD) / p.DH, e0 = col0 % p.DH;
+  if (part == 0 && p.rope_cos != nullptr) {
+    const float4* cs = reinterpret_cast<const float4*>(p.rope_cos + size_t(tok) * (p.DH / 2) + e0 / 2);
+    const float4* sn = reinterpret_cast<const float4*>(p.rope_sin + size_t(tok) * (p.DH / 2) + e0 / 2);
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      const float4 c4 = __ldg(cs + g), s4 = __ldg(sn + g);
+      const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float a0 = y[8 * g + 2 * j], a1 = y[8 * g + 2 * j + 1];
+        y[8 * g + 2 * j] = a0 * cc[j] - a1 * ss[j];
+        y[8 * g + 2 * j + 1] = a0 * ss[j] + a1 * cc[j];
+      }
+    }
+  }
+  __nv_bfloat16* dst = (part == 0 ? p.Kc : p.Vc) + ((size_t(b) * p.H + h) * p.C + slot) * p.DH + e0;
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    uint4 o;
+    __nv_bfloat162 t0 = __floats2bfloat162_rn(y[8 * g + 0], y[8 * g + 1]);
+    __nv_bfloat162 t1 = __floats2bfloat162_rn(y[8 * g + 2], y[8 * g + 3]);
+    __nv_bfloat162 t2 = __floats2bfloat162_rn(y[8 * g + 4], y[8 * g + 5]);
+    __nv_bfloat162 t3 = __floats2bfloat162_rn(y[8 * g + 6], y[8 * g + 7]);
+    o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
+    o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
+    reinterpret_cast<uint4*>(dst)[g] = o;
+  }
+}
+
+// Asks for the lines of a token's rotary table that the key columns [n0, n0 + BN) of its row will read, so that the
+// epilogue's loads, issued only when the accumulator is complete, find them in the cache.
+template <int BN>
+__device__ __forceinline__ void tc_prefetch_rope(const TcGemmParams& p, int n0, int tok) {
+  const int HD = p.H * p.DH;
+  if (p.rope_cos == nullptr || n0 >= HD) return;            // no rotation, or a value tile
+  for (int col = n0; col < min(n0 + BN, HD); col += 64) {   // 64 columns = 32 angles = one 128-byte line of each table
+    const size_t at = size_t(tok) * (p.DH / 2) + (col % p.DH) / 2;
+    asm volatile("prefetch.global.L1 [%0];" ::"l"(p.rope_cos + at));
+    asm volatile("prefetch.global.L1 [%0];" ::"l"(p.rope_sin + at));
+  }
+}
+
 // `parts` > 1: the row's values are the sum over the stored accumulators parts_base + q * part_stride, q ascending,
-// with this unit's own part (`my_part`) taken from TMEM.
+// with this unit's own part (`my_part`) taken from TMEM. Two parts: the other unit's 32 values of the NEXT column
+// chunk are requested before the current chunk is worked on, so that only the first request's latency shows.
 template <int BN>
 __device__ __forceinline__ void tc_epilogue_row(const TcGemmParams& p, uint32_t taddr, int n0, bool in_range, int b, int tok,
                                                 int slot, int quarter = 0, int lane = 0, int parts = 1, int my_part = 0,
                                                 const float* parts_base = nullptr, size_t part_stride = 0) {
-  const int HD = p.H * p.DH;
+  const bool two = parts == 2;
+  const float* other = two ? parts_base + size_t(1 - my_part) * part_stride + size_t(quarter) * 1024 + lane : nullptr;
+  float nxt[32];
+  if (two && in_range) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) nxt[i] = __ldcg(other + i * 32);
+  }
 #pragma unroll 1
   for (int c = 0; c < BN / 32; ++c) {
     uint32_t v[32];
     __syncwarp();                               // the TMEM load is warp-collective
     tc_ld_32x32(taddr + uint32_t(c * 32), v);
     const int col0 = n0 + c * 32;
-    const int part = col0 / HD, h = (col0 % HD) / p.DH, e0 = col0 % p.DH;
     if (in_range) {
       float y[32];
-      if (parts > 1) {
+      if (two) {
+        // part 0 + part 1 whichever unit runs this: the sum does not depend on who arrived last
+#pragma unroll
+        for (int i = 0; i < 32; ++i) y[i] = my_part == 0 ? __uint_as_float(v[i]) + nxt[i] : nxt[i] + __uint_as_float(v[i]);
+        if (c + 1 < BN / 32) {
+          const float* src = other + size_t(c + 1) * 4096;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) nxt[i] = __ldcg(src + i * 32);
+        }
+      } else if (parts > 1) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) y[i] = 0.f;
         for (int q = 0; q < parts; ++q) {
@@ -241,33 +303,7 @@ __device__ __forceinline__ void tc_epilogue_row(const TcGemmParams& p, uint32_t 
 #pragma unroll
         for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(v[i]);
       }
-      if (part == 0 && p.rope_cos != nullptr) {
-        const float4* cs = reinterpret_cast<const float4*>(p.rope_cos + size_t(tok) * (p.DH / 2) + e0 / 2);
-        const float4* sn = reinterpret_cast<const float4*>(p.rope_sin + size_t(tok) * (p.DH / 2) + e0 / 2);
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          const float4 c4 = __ldg(cs + g), s4 = __ldg(sn + g);
-          const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float a0 = y[8 * g + 2 * j], a1 = y[8 * g + 2 * j + 1];
-            y[8 * g + 2 * j] = a0 * cc[j] - a1 * ss[j];
-            y[8 * g + 2 * j + 1] = a0 * ss[j] + a1 * cc[j];
-          }
-        }
-      }
-      __nv_bfloat16* dst = (part == 0 ? p.Kc : p.Vc) + ((size_t(b) * p.H + h) * p.C + slot) * p.DH + e0;
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        uint4 o;
-        __nv_bfloat162 t0 = __floats2bfloat162_rn(y[8 * g + 0], y[8 * g + 1]);
-        __nv_bfloat162 t1 = __floats2bfloat162_rn(y[8 * g + 2], y[8 * g + 3]);
-        __nv_bfloat162 t2 = __floats2bfloat162_rn(y[8 * g + 4], y[8 * g + 5]);
-        __nv_bfloat162 t3 = __floats2bfloat162_rn(y[8 * g + 6], y[8 * g + 7]);
-        o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
-        o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
-        reinterpret_cast<uint4*>(dst)[g] = o;
-      }
+      tc_rope_store_32(p, y, col0, b, tok, slot);
     }
   }
 }
@@ -399,6 +435,7 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (valid) { b = p.row_b[r]; tok = p.row_tok[r]; slot = p.row_slot[r]; }
       const bool in_range = valid && slot >= 0 && slot < p.C;
       if (valid && !in_range) set_error(p.err, ERRW_BOUNDS);
+      if (in_range) tc_prefetch_rope<BN>(p, n0, tok);
       if (!tc_mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * BN);
@@ -427,6 +464,7 @@ rebuild_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 }  // namespace adore
 
 #include "rebuild_tc_pair.cuh"   // the two-SM variant of the kernel above (uses its wrappers and epilogue)
+#include "rebuild_tc_split.cuh"  // few rows: K split over a pair of CTAs, halves added through distributed shared memory
 
 namespace adore {
 
@@ -441,6 +479,7 @@ struct TcState {
   int sms = 148;
   int N = 0, K = 0;
   int pairs = 0;                      // CTA pairs the two-SM kernel runs with (0: not available)
+  int split_pairs = 0;                // CTA pairs the K-split kernel can hold at once (0: not available)
   size_t a_rows = 0;                  // rows of the gather buffer (multiple of 256)
   __nv_bfloat16* a_buf = nullptr;
   float* partial = nullptr;           // split-K accumulators: one 128 x 256 fp32 block per SM
@@ -458,14 +497,15 @@ constexpr size_t kTcPartialFloatsPerSm = size_t(256) * 128;
 // the two-SM kernel (tensor-bound). Enough 128 x 256 tiles for every SM: those. Otherwise the launch is bound by the
 // latency of streaming each weight tile once (measured: ~1.5 us per 32 KB stage with six stages in flight, i.e.
 // ~0.3 us per k-block whatever the tile), so 128 x 128 tiles, and K split in two when that still leaves SMs idle.
-struct TcPlan { int kind; int ksplit; int grid; };   // kind 0: 128-wide tiles, 1: 256-wide tiles, 2: SM pairs
-inline TcPlan tc_plan(int rows, int N, int K, int sms, int pairs, int max_split) {
+struct TcPlan { int kind; int ksplit; int grid; };   // kind 0: 128-wide tiles, 1: 256-wide tiles, 2: SM pairs, 3: K split over a CTA pair
+inline TcPlan tc_plan(int rows, int N, int K, int sms, int pairs, int max_split, int split_pairs = 0) {
   const int kb = K / kTcBK;
   const int mt128 = (rows + kTcBM - 1) / kTcBM, mt256 = (rows + 2 * kTcBM - 1) / (2 * kTcBM);
   if (pairs > 0 && N % 256 == 0 && mt256 * (N / 256) >= pairs) return TcPlan{2, 1, 2 * pairs};
   if (N % 256 == 0 && mt128 * (N / 256) >= sms) return TcPlan{1, 1, sms};
   const int tiles = mt128 * (N / 128);
   const bool split = max_split >= 2 && kb % 2 == 0 && kb / 2 >= 4 && 2 * tiles <= sms && 4 * tiles <= kTcCounters;
+  if (split && tiles <= split_pairs) return TcPlan{3, 2, 2 * tiles};
   const int units = split ? 2 * tiles : tiles;
   return TcPlan{0, split ? 2 : 1, std::max(1, std::min(sms, units))};
 }
@@ -535,6 +575,20 @@ inline adore_status_t tc_init(TcState& s, const adore_config_t& f, std::vector<v
     if (cudaOccupancyMaxActiveClusters(&clusters, rebuild_tc_pair_kernel, &lc) == cudaSuccess) s.pairs = std::min(clusters, s.sms / 2);
   }
   cudaGetLastError();
+  // the K-split kernel: pairs of SMs again, with its own (larger) shared-memory footprint
+  if (cudaFuncSetAttribute(rebuild_tc_split_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(split_smem_bytes<6>())) == cudaSuccess &&
+      cudaFuncSetAttribute(rebuild_tc_split_kernel<kTcLeanStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(split_smem_bytes<kTcLeanStages>())) == cudaSuccess) {
+    cudaLaunchConfig_t lc{};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    lc.gridDim = dim3(unsigned(s.sms / 2 * 2)); lc.blockDim = dim3(kTcThreads); lc.dynamicSmemBytes = split_smem_bytes<6>();
+    lc.attrs = at; lc.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, rebuild_tc_split_kernel<6>, &lc) == cudaSuccess) s.split_pairs = std::min(clusters, s.sms / 2);
+  }
+  cudaGetLastError();
   s.ready = true;
   return ADORE_OK;
 }
@@ -584,7 +638,7 @@ inline cudaError_t launch_rebuild_tc<__nv_bfloat16>(TcState& s, const RebuildPar
     g.row_total = rp.row_total; g.row_base = base; g.row_limit = limit;
     g.rope_cos = rp.rope_cos; g.rope_sin = rp.rope_sin; g.H = rp.H; g.DH = rp.DH; g.C = rp.C; g.N = rp.N; g.K = rp.d; g.err = rp.err;
     static const int max_split = dev_switch_int("ADORE_TC_KSPLIT_MAX", 4);
-    const TcPlan plan = tc_plan(limit, s.N, s.K, s.sms, s.pairs, max_split);
+    const TcPlan plan = tc_plan(limit, s.N, s.K, s.sms, s.pairs, max_split, s.split_pairs);
     g.ksplit = plan.ksplit; g.partial = s.partial; g.unit_cnt = s.unit_cnt;
     if (plan.kind == 2) {
       cudaLaunchConfig_t lc{};
@@ -597,6 +651,25 @@ inline cudaError_t launch_rebuild_tc<__nv_bfloat16>(TcState& s, const RebuildPar
       lc.gridDim = dim3(unsigned(plan.grid)); lc.blockDim = dim3(kTcThreads); lc.dynamicSmemBytes = kPairSmemBytes;
       lc.stream = stream; lc.attrs = at; lc.numAttrs = no_dep ? 1 : 2;
       e = cudaLaunchKernelEx(&lc, rebuild_tc_pair_kernel, s.map_a, s.map_w128[layer], g);
+      ++*launched;
+      if (e != cudaSuccess) return e;
+      continue;
+    }
+    if (plan.kind == 3) {
+      cudaLaunchConfig_t lc{};
+      // (an ordinary launch: as a programmatic dependent this cluster launch kept the controller's gate product, which
+      // runs beside it on another stream, from finishing before the GEMM did: 14 -> 46 us)
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      lc.gridDim = dim3(unsigned(plan.grid)); lc.blockDim = dim3(kTcThreads); lc.stream = stream; lc.attrs = at; lc.numAttrs = 1;
+      if (lean) {
+        lc.dynamicSmemBytes = split_smem_bytes<kTcLeanStages>();
+        e = cudaLaunchKernelEx(&lc, rebuild_tc_split_kernel<kTcLeanStages>, s.map_a, s.map_w128[layer], g);
+      } else {
+        lc.dynamicSmemBytes = split_smem_bytes<6>();
+        e = cudaLaunchKernelEx(&lc, rebuild_tc_split_kernel<6>, s.map_a, s.map_w128[layer], g);
+      }
       ++*launched;
       if (e != cudaSuccess) return e;
       continue;
