@@ -42,6 +42,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES = {
     ("rebuild projection", "cfg3_llama7b_b64_c512_rebuild20pct"):
         {"bytes": 284.9e6 + 144.9e6, "rows": 9950.0, "profile": "profiles/rebuild_tc_pair_kernel_cfg3.md"},
+    ("rebuild projection", "cfg2_llama7b_b16_c256"):
+        {"bytes": 68.2e6 + 1.1e6, "rows": 128.0, "profile": "profiles/rebuild_tc_split_kernel_cfg2.md"},
     ("attention kernel", "cfg3_llama7b_b64_c512_rebuild20pct"):
         {"bytes": 359.1e6 + 6.7e6, "rows": None, "profile": "profiles/attention_tma_kernel_cfg3.md"},
     # config 4's per-layer launch, captured on a one-layer cache of the same shape (the sweep point C=1024, B=32)
@@ -558,6 +560,8 @@ def main():
     ap.add_argument("--order", default="attend-first", choices=["attend-first", "rebuild-first"],
                     help="rebuild-first: select, rebuild, then one attention with R_max+1 query rows per sequence "
                          "(adore_step_begin / adore_attend_rows); no end-to-end pass in that order")
+    ap.add_argument("--rebuild-max", type=int, default=None,
+                    help="override the configuration's R_max (tokens rebuilt per sequence and step), e.g. the paper's 32")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
@@ -566,6 +570,8 @@ def main():
         run_labels(args)
         return
     cfg = sweep_point(args.capacity, args.batch) if args.config == 5 else wl.get_config(args.config)
+    if args.rebuild_max is not None:
+        cfg = cfg.scaled(name=f"{cfg.name}_r{args.rebuild_max}", rebuild_max=args.rebuild_max)
     if args.steps is None:
         args.steps = default_steps(cfg) if args.impl == "ours" else 3
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

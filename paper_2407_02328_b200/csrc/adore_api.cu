@@ -391,47 +391,61 @@ adore_status_t launch_gates(adore_cache* c, const T* x, long long seq_stride, in
 template <typename T>
 bool launch_attention_rows(adore_cache*, int, const AttnParams<T>&, int) { return false; }
 
-template <int DH, int KPL>
+constexpr size_t kRowsSmemLimit = 226 * 1024;             // dynamic shared memory a CTA of the rows kernel may ask for
+
+template <int DH, int KPL, int RB>
 bool launch_attention_rows_as(adore_cache* c, int layer, const AttnParams<__nv_bfloat16>& p, size_t smem) {
   static bool opted = false;                                // per instantiation
   if (!opted) {
-    if (cudaFuncSetAttribute(attention_rows_kernel<DH, KPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
+    if (cudaFuncSetAttribute(attention_rows_kernel<DH, KPL, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kRowsSmemLimit)) != cudaSuccess) {
       cudaGetLastError();
       return false;
     }
     opted = true;
   }
   const dim3 grid(unsigned(c->cfg.batch * c->cfg.n_heads)), block(kRowsThreads);
-  cudaError_t e = launch_dependent(attention_rows_kernel<DH, KPL>, grid, block, smem, c->stream, c->map_k[layer], c->map_v[layer], p);
+  cudaError_t e = launch_dependent(attention_rows_kernel<DH, KPL, RB>, grid, block, smem, c->stream, c->map_k[layer], c->map_v[layer], p);
   ++c->launches;
   if (e != cudaSuccess) { cudaGetLastError(); return false; }
   return true;
+}
+
+template <int DH, int RB>
+bool launch_attention_rows_kpl(adore_cache* c, int layer, const AttnParams<__nv_bfloat16>& p, size_t smem, int per_lane) {
+  if (per_lane <= 9) return launch_attention_rows_as<DH, 9, RB>(c, layer, p, smem);
+  if (per_lane <= 17) return launch_attention_rows_as<DH, 17, RB>(c, layer, p, smem);
+  return launch_attention_rows_as<DH, 33, RB>(c, layer, p, smem);
 }
 
 template <>
 bool launch_attention_rows<__nv_bfloat16>(adore_cache* c, int layer, const AttnParams<__nv_bfloat16>& p, int rows_q) {
   const adore_config_t& f = c->cfg;
   static const bool off = dev_switch("ADORE_ROWS_SIMT");
-  const size_t smem = rows_smem_bytes(f.capacity, f.head_dim, std::min(rows_q, kRowsMaxQ));
   const int per_lane = (f.capacity + 1 + 31) / 32;
-  if (off || c->map_k.empty() || per_lane > kRowsKeysPerLaneMax || smem > 200 * 1024) return false;
-  // more than 16 rows: one launch per group of 16; the last group holds the current token's row and stores its rows
-  for (int rb = 0; rb < rows_q; rb += kRowsMaxQ) {
+  if (off || c->map_k.empty() || per_lane > kRowsKeysPerLaneMax) return false;
+  // Rows per launch: up to 16 with two CTAs per SM; more rows go through the three-block kernel, as many per launch as
+  // the logits of a pair fit in shared memory (one pass over the pair's keys and values for all of them). What is
+  // left goes in further launches of the same size; the last group holds the current token's row and stores its rows.
+  int group = std::min(rows_q, kRowsMaxQ);
+  if (rows_q > kRowsMaxQ) {
+    group = std::min(rows_q, kRowsMaxQ * kRowsMaxBlocks);
+    while (group > kRowsMaxQ && rows_smem_bytes(f.capacity, f.head_dim, group) > kRowsSmemLimit) --group;
+  }
+  const size_t smem = rows_smem_bytes(f.capacity, f.head_dim, group);
+  if (smem > (group > kRowsMaxQ ? kRowsSmemLimit : size_t(200 * 1024))) return false;
+  for (int rb = 0; rb < rows_q; rb += group) {
     AttnParams<__nv_bfloat16> g = p;
-    g.rows_q = std::min(kRowsMaxQ, rows_q - rb);
+    g.rows_q = std::min(group, rows_q - rb);
     g.row_base = rb;
     g.rows_total = rows_q;
     if (rb + g.rows_q < rows_q) g.admit_slot = nullptr;
     bool ok;
-    if (f.head_dim == 128) {
-      if (per_lane <= 9) ok = launch_attention_rows_as<128, 9>(c, layer, g, smem);
-      else if (per_lane <= 17) ok = launch_attention_rows_as<128, 17>(c, layer, g, smem);
-      else ok = launch_attention_rows_as<128, 33>(c, layer, g, smem);
-    } else {
-      if (per_lane <= 9) ok = launch_attention_rows_as<64, 9>(c, layer, g, smem);
-      else if (per_lane <= 17) ok = launch_attention_rows_as<64, 17>(c, layer, g, smem);
-      else ok = launch_attention_rows_as<64, 33>(c, layer, g, smem);
-    }
+    if (group > kRowsMaxQ)
+      ok = f.head_dim == 128 ? launch_attention_rows_kpl<128, kRowsMaxBlocks>(c, layer, g, smem, per_lane)
+                             : launch_attention_rows_kpl<64, kRowsMaxBlocks>(c, layer, g, smem, per_lane);
+    else
+      ok = f.head_dim == 128 ? launch_attention_rows_kpl<128, 1>(c, layer, g, smem, per_lane)
+                             : launch_attention_rows_kpl<64, 1>(c, layer, g, smem, per_lane);
     // a refused first launch leaves the other kernel to do all rows; a later one cannot fail where the first did not
     if (!ok) return false;
   }

@@ -14,9 +14,12 @@
 //            each warp takes one of a tile's four k-steps and half of the output columns, the partial outputs are
 //            added through shared memory. The current token's own value row is added for the last row.
 // Then the current token's rows are stored in their slot. Every mbarrier wait is bounded.
-// More than 16 rows per pair: one launch per group of 16 rows (row_base / rows_total in the parameters); the groups of
-// a pair read its key and value blocks again (from L2 when the launches follow one another closely), and only the
-// last group, which holds the current token's row, adds that token's own key and value and stores its rows.
+// More than 16 rows per pair (the paper's range goes to R = 32): the kernel exists with RB = 3 blocks of 16 rows, which
+// share every key and value fragment read from shared memory, so that up to 48 rows still take one pass over the pair's
+// keys and one over its values (one CTA per SM then: the logits of 48 rows need most of the shared memory). Rows beyond
+// what fits go in groups, one launch per group (row_base / rows_total in the parameters); the groups of a pair read its
+// key and value blocks again (from L2 when the launches follow one another closely), and only the last group, which
+// holds the current token's row, adds that token's own key and value and stores its rows.
 #pragma once
 
 #include <cuda.h>
@@ -30,7 +33,8 @@ constexpr int kRowsThreads = 256;
 constexpr int kRowsWarps = kRowsThreads / 32;
 constexpr int kRowsTile = 64;            // key / value rows per tile
 constexpr int kRowsStages = 4;
-constexpr int kRowsMaxQ = 16;
+constexpr int kRowsMaxQ = 16;            // rows of one block (the M of one MMA)
+constexpr int kRowsMaxBlocks = 3;        // row blocks a CTA can carry through one pass
 constexpr int kRowsKeysPerLaneMax = 33;  // logits of a row per lane: C + 1 <= 1056
 
 __host__ __device__ inline int rows_logit_stride(int C) {
@@ -39,7 +43,8 @@ __host__ __device__ inline int rows_logit_stride(int C) {
   return sp;
 }
 __host__ __device__ inline size_t rows_smem_bytes(int C, int DH, int rows_q) {
-  return 1024 + size_t(kRowsStages) * kRowsTile * DH * 2 + 64 + 64 + sizeof(int) * size_t((C + 3) & ~3) +
+  return 1024 + size_t(kRowsStages) * kRowsTile * DH * 2 + 64 + sizeof(int) * kRowsMaxQ * kRowsMaxBlocks +
+         sizeof(int) * size_t((C + 3) & ~3) +
          sizeof(float) * size_t(rows_q) * rows_logit_stride(C);
 }
 
@@ -72,7 +77,7 @@ __device__ __forceinline__ uint32_t rows_swz(int row, int c16) { return uint32_t
 
 // KPL: logits of a row held per lane during the selection (C + 1 <= 32 KPL); the counting loops run over all KPL
 // registers without guards (slots past the row hold key 0, which never counts).
-template <int DH, int KPL>
+template <int DH, int KPL, int RB>
 __global__ void __launch_bounds__(kRowsThreads)
 attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                       const AttnParams<__nv_bfloat16> p) {
@@ -84,8 +89,8 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(rows_smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* ring = base;
   uint64_t* full = reinterpret_cast<uint64_t*>(base + size_t(kRowsStages) * TILE_BYTES);
-  int* s_qtok = reinterpret_cast<int*>(full + 8);       // [16] position bound per row (< 0: padding)
-  int* s_tok = s_qtok + 16;                             // [C] the pair's slot map row (token position per slot)
+  int* s_qtok = reinterpret_cast<int*>(full + 8);       // [48] position bound per row (< 0: padding)
+  int* s_tok = s_qtok + kRowsMaxQ * kRowsMaxBlocks;     // [C] the pair's slot map row (token position per slot)
   float* S = reinterpret_cast<float*>(s_tok + ((p.C + 3) & ~3));
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -105,7 +110,7 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   wait_for_prior_grid();
-  if (tid < kRowsMaxQ) {
+  if (tid < kRowsMaxQ * RB) {
     const int g = rb + tid;                             // row index within the pair
     s_qtok[tid] = tid >= R1 ? -1 : (g < RT - 1 ? p.row_tok[size_t(b) * p.r_max + g] : p.n_cur);
   }
@@ -131,17 +136,18 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     for (int i = 0; i < min(kRowsStages, n_loads); ++i) issue(i);
 
   // ---- query block as A fragments: rows lane/4 and lane/4 + 8, columns 16 ks + (lane % 4) * 2 (+8) ----
-  uint32_t qa[KSTEPS][4];
-  {
+  uint32_t qa[RB][KSTEPS][4];
+#pragma unroll
+  for (int k = 0; k < RB; ++k) {
     const T* qb = p.q + (size_t(bh) * RT + rb) * DH;
-    const int r0 = lane >> 2, r1 = r0 + 8, c0 = (lane & 3) * 2;
+    const int r0 = k * kRowsMaxQ + (lane >> 2), r1 = r0 + 8, c0 = (lane & 3) * 2;
 #pragma unroll
     for (int ks = 0; ks < KSTEPS; ++ks) {
       const int col = ks * 16 + c0;
-      qa[ks][0] = r0 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r0) * DH + col) : 0u;
-      qa[ks][1] = r1 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r1) * DH + col) : 0u;
-      qa[ks][2] = r0 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r0) * DH + col + 8) : 0u;
-      qa[ks][3] = r1 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r1) * DH + col + 8) : 0u;
+      qa[k][ks][0] = r0 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r0) * DH + col) : 0u;
+      qa[k][ks][1] = r1 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r1) * DH + col) : 0u;
+      qa[k][ks][2] = r0 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r0) * DH + col + 8) : 0u;
+      qa[k][ks][3] = r1 < R1 ? *reinterpret_cast<const uint32_t*>(qb + size_t(r1) * DH + col + 8) : 0u;
     }
   }
   // the current token's own key: last row only (index C); every other row does not see it
@@ -157,7 +163,9 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
 
   bool failed = false;
   // ---- phase 1: logits, two tiles (two independent accumulator chains per warp) per block barrier ----
-  const int qt0 = s_qtok[lane >> 2], qt1 = s_qtok[(lane >> 2) + 8];
+  int qt[RB][2];
+#pragma unroll
+  for (int k = 0; k < RB; ++k) { qt[k][0] = s_qtok[k * kRowsMaxQ + (lane >> 2)]; qt[k][1] = s_qtok[k * kRowsMaxQ + (lane >> 2) + 8]; }
   for (int t = 0; t < n_tiles; t += 2) {
     const int stage = t % kRowsStages;
     const uint32_t parity = uint32_t(t / kRowsStages) & 1u;
@@ -168,7 +176,11 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
         failed = true;
       }
     const uint32_t tile = smem_u32(ring + size_t(stage) * TILE_BYTES);
-    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    float acc[RB][2][4];
+#pragma unroll
+    for (int k = 0; k < RB; ++k)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { acc[k][0][e] = 0.f; acc[k][1][e] = 0.f; }
     // ldmatrix.x4: matrix j holds keys warp*8 .. +7 (rows) x 8 columns starting at 8 * (4 q + j)
     const int krow = warp * 8 + (lane & 7), mj = lane >> 3;
 #pragma unroll
@@ -178,8 +190,11 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
       for (int h2 = 0; h2 < 2; ++h2) {
         uint32_t bf[4];
         rows_ldmatrix_x4(tile + uint32_t(h2) * TILE_BYTES + uint32_t(c16 >> 3) * (kRowsTile * 128) + rows_swz(krow, c16 & 7), bf);
-        rows_mma(acc[h2], qa[2 * q4], bf[0], bf[1]);
-        rows_mma(acc[h2], qa[2 * q4 + 1], bf[2], bf[3]);
+#pragma unroll
+        for (int k = 0; k < RB; ++k) {                  // every row block uses the key fragments just read
+          rows_mma(acc[k][h2], qa[k][2 * q4], bf[0], bf[1]);
+          rows_mma(acc[k][h2], qa[k][2 * q4 + 1], bf[2], bf[3]);
+        }
       }
     }
     // accumulator: rows lane/4 (+8), keys (lane % 4) * 2 (+1) of this warp's 8 in each tile
@@ -187,13 +202,15 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     for (int h2 = 0; h2 < 2; ++h2) {
       const int key0 = (t + h2) * kRowsTile + warp * 8 + (lane & 3) * 2;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int r = (lane >> 2) + (e >> 1) * 8, key = key0 + (e & 1);
-        if (r < R1 && key < C) {
-          const int tok = s_tok[key], qt = (e >> 1) ? qt1 : qt0;
-          S[size_t(r) * SP + key] = (tok >= 0 && tok <= qt) ? acc[h2][e] * p.scale : -INFINITY;
+      for (int k = 0; k < RB; ++k)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int r = k * kRowsMaxQ + (lane >> 2) + (e >> 1) * 8, key = key0 + (e & 1);
+          if (r < R1 && key < C) {
+            const int tok = s_tok[key];
+            S[size_t(r) * SP + key] = (tok >= 0 && tok <= qt[k][e >> 1]) ? acc[k][h2][e] * p.scale : -INFINITY;
+          }
         }
-      }
     }
     __syncthreads();                                    // everyone is done with these two stages
     if (tid == 0 && !failed) {
@@ -204,10 +221,10 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
 
   // ---- phase 2: per row, which logits are kept, softmax, weights (one warp per row) ----
   const int rows_n = C + 1;
-  // The current token's row always needs a selection (it sees every slot) and goes alone to warp 0; the other rows
-  // follow on warps 1..7, the ninth and later ones are stacked from warp 7 downwards.
-  for (int pass = 0; pass < 2; ++pass) {
-    const int e = pass == 0 ? warp : 15 - warp;          // entry 0: last row; entry e > 0: row e - 1
+  // The current token's row always needs a selection (it sees every slot) and goes first, to warp 0; the other rows
+  // follow on warps 1..7, the ninth and later ones are stacked from warp 7 downwards, the next eight upwards again.
+  for (int pass = 0; pass < 2 * RB; ++pass) {
+    const int e = pass * kRowsWarps + ((pass & 1) ? kRowsWarps - 1 - warp : warp);   // entry 0: last row; entry e > 0: row e - 1
     if (e >= R1) continue;
     const int r = e == 0 ? R1 - 1 : e - 1;
     float* row = S + size_t(r) * SP;
@@ -246,10 +263,10 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
       bool exact = false;
       for (int bit = top; bit >= 0; --bit) {
         const uint32_t cand = thr | (1u << bit);
-        int c = 0;
+        int c = 0;                                        // per-lane count, one warp-wide add per pass
 #pragma unroll
-        for (int j = 0; j < KPL; ++j)
-          c += __popc(__ballot_sync(0xffffffffu, kk[j] >= cand));
+        for (int j = 0; j < KPL; ++j) c += kk[j] >= cand ? 1 : 0;
+        c = __reduce_add_sync(0xffffffffu, c);
         if (c >= p.topk) thr = cand;
         if (c == p.topk) { exact = true; break; }       // exactly K keys are >= thr: that is the kept set
       }
@@ -300,9 +317,11 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
   // fragments of a k-step are built by two warps instead of all eight; the partial outputs meet in shared memory ----
   constexpr int NTW = DH / 16;                          // 8-column n-tiles per warp (8 for dh 128, 4 for dh 64)
   const int my_ks = warp & 3, col_half = warp >> 2;
-  float o[NTW][4];
+  float o[RB][NTW][4];
 #pragma unroll
-  for (int j = 0; j < NTW; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+  for (int k = 0; k < RB; ++k)
+#pragma unroll
+    for (int j = 0; j < NTW; ++j) { o[k][j][0] = o[k][j][1] = o[k][j][2] = o[k][j][3] = 0.f; }
   for (int t = 0; t < n_tiles; t += 2) {
     const int li = n_tiles + t;
     const int stage = li % kRowsStages;
@@ -318,16 +337,19 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
       const uint32_t tile = smem_u32(ring + size_t(stage + h2) * TILE_BYTES);
       // A: weights of rows lane/4 (+8) for keys 16 my_ks + (lane % 4) * 2 (+1, +8, +9) of this tile, head + remainder
       const int key = (t + h2) * kRowsTile + my_ks * 16 + (lane & 3) * 2;
-      const int r0 = lane >> 2, r1 = r0 + 8;
-      uint32_t ah[4], al[4];
+      uint32_t ah[RB][4], al[RB][4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int r = (e & 1) ? r1 : r0, k = key + (e >> 1) * 8;
-        const float w0 = (r < R1 && k < C) ? S[size_t(r) * SP + k] : 0.f;
-        const float w1 = (r < R1 && k + 1 < C) ? S[size_t(r) * SP + k + 1] : 0.f;
-        const __nv_bfloat16 h0 = __float2bfloat16_rn(w0), h1 = __float2bfloat16_rn(w1);
-        ah[e] = rows_pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
-        al[e] = rows_pack_bf16(w0 - __bfloat162float(h0), w1 - __bfloat162float(h1));
+      for (int kb = 0; kb < RB; ++kb) {
+        const int r0 = kb * kRowsMaxQ + (lane >> 2), r1 = r0 + 8;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int r = (e & 1) ? r1 : r0, k = key + (e >> 1) * 8;
+          const float w0 = (r < R1 && k < C) ? S[size_t(r) * SP + k] : 0.f;
+          const float w1 = (r < R1 && k + 1 < C) ? S[size_t(r) * SP + k + 1] : 0.f;
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(w0), h1 = __float2bfloat16_rn(w1);
+          ah[kb][e] = rows_pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
+          al[kb][e] = rows_pack_bf16(w0 - __bfloat162float(h0), w1 - __bfloat162float(h1));
+        }
       }
       // B (transposed load): matrix j: keys 16 my_ks + 8 (j % 2) .. +7 (rows of the tile) x the columns of n-tile j / 2
       const int vrow = my_ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
@@ -336,10 +358,13 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
         const int c16 = col_half * NTW + nt + (lane >> 4);
         uint32_t bf[4];
         rows_ldmatrix_x4_trans(tile + uint32_t(c16 >> 3) * (kRowsTile * 128) + rows_swz(vrow, c16 & 7), bf);
-        rows_mma(o[nt], ah, bf[0], bf[1]);
-        rows_mma(o[nt], al, bf[0], bf[1]);
-        rows_mma(o[nt + 1], ah, bf[2], bf[3]);
-        rows_mma(o[nt + 1], al, bf[2], bf[3]);
+#pragma unroll
+        for (int kb = 0; kb < RB; ++kb) {               // every row block uses the value fragments just read
+          rows_mma(o[kb][nt], ah[kb], bf[0], bf[1]);
+          rows_mma(o[kb][nt], al[kb], bf[0], bf[1]);
+          rows_mma(o[kb][nt + 1], ah[kb], bf[2], bf[3]);
+          rows_mma(o[kb][nt + 1], al[kb], bf[2], bf[3]);
+        }
       }
     }
     __syncthreads();
@@ -349,38 +374,44 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     }
   }
 
-  // ---- the four k-step warps of a column half add up through shared memory (the ring is free now), then rows < R1
-  // go out; the last row also gets the current token's own value row ----
+  // ---- the four k-step warps of a column half add up through shared memory (the ring is free now), one row block
+  // after the other, then rows < R1 go out; the last row also gets the current token's own value row ----
   {
     float* part = reinterpret_cast<float*>(ring);       // [4 k-steps][16 rows][DH] floats: at most 32 KB
-#pragma unroll
-    for (int nt = 0; nt < NTW; ++nt) {
-      const int col = col_half * (DH / 2) + nt * 8 + (lane & 3) * 2;
-#pragma unroll
-      for (int hrow = 0; hrow < 2; ++hrow) {
-        const int r = (lane >> 2) + hrow * 8;
-        float* d = part + (size_t(my_ks) * 16 + r) * DH + col;
-        d[0] = o[nt][hrow * 2];
-        d[1] = o[nt][hrow * 2 + 1];
-      }
-    }
-    __syncthreads();
     const T* vn = p.v_new + size_t(bh) * DH;
     const float w_own = has_last ? S[size_t(R1 - 1) * SP + C] : 0.f;
-    for (int i = tid; i < R1 * (DH / 2); i += kRowsThreads) {
-      const int r = i / (DH / 2), col = (i % (DH / 2)) * 2;
-      float a0 = 0.f, a1 = 0.f;
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        const float* d = part + (size_t(q4) * 16 + r) * DH + col;
-        a0 += d[0];
-        a1 += d[1];
+    for (int kb = 0; kb < RB; ++kb) {
+      if (kb * kRowsMaxQ >= R1) break;                  // (the same in every thread)
+      if (kb > 0) __syncthreads();                      // the previous block's sums have been read
+#pragma unroll
+      for (int nt = 0; nt < NTW; ++nt) {
+        const int col = col_half * (DH / 2) + nt * 8 + (lane & 3) * 2;
+#pragma unroll
+        for (int hrow = 0; hrow < 2; ++hrow) {
+          const int r = (lane >> 2) + hrow * 8;
+          float* d = part + (size_t(my_ks) * 16 + r) * DH + col;
+          d[0] = o[kb][nt][hrow * 2];
+          d[1] = o[kb][nt][hrow * 2 + 1];
+        }
       }
-      if (has_last && r == R1 - 1) {
-        a0 = fmaf(w_own, __bfloat162float(vn[col]), a0);
-        a1 = fmaf(w_own, __bfloat162float(vn[col + 1]), a1);
+      __syncthreads();
+      const int rows_here = min(kRowsMaxQ, R1 - kb * kRowsMaxQ);
+      for (int i = tid; i < rows_here * (DH / 2); i += kRowsThreads) {
+        const int rl = i / (DH / 2), col = (i % (DH / 2)) * 2, r = kb * kRowsMaxQ + rl;
+        float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const float* d = part + (size_t(q4) * 16 + rl) * DH + col;
+          a0 += d[0];
+          a1 += d[1];
+        }
+        if (has_last && r == R1 - 1) {
+          a0 = fmaf(w_own, __bfloat162float(vn[col]), a0);
+          a1 = fmaf(w_own, __bfloat162float(vn[col + 1]), a1);
+        }
+        *reinterpret_cast<uint32_t*>(p.out + (size_t(bh) * RT + rb + r) * DH + col) = rows_pack_bf16(a0, a1);
       }
-      *reinterpret_cast<uint32_t*>(p.out + (size_t(bh) * RT + rb + r) * DH + col) = rows_pack_bf16(a0, a1);
     }
   }
   // ---- admit: the current token's rows go into their slot (all tiles of this pair have been consumed) ----

@@ -235,15 +235,25 @@ def test_rebuild_first_step_on_the_tensor_core_kernel_shapes():
     _run_rebuild_first(wl.get_config(2).scaled(name="rows_cfg2_shape", batch=2, steps=4))
 
 
-def test_rebuild_first_step_with_more_than_sixteen_query_rows_in_groups():
-    """More than 16 rows per pair on bfloat16 caches: one launch of the tensor-core kernel per group of 16 rows; only the
-    last group holds the current token's row (own key and value, rows stored in their slot). 39 + 1 rows = 16 + 16 + 8,
-    32 + 1 rows = 16 + 16 + a group with the current token alone, explicit lists leave padding rows in every group."""
+def test_rebuild_first_step_with_more_than_sixteen_query_rows():
+    """More than 16 rows per pair on bfloat16 caches. Up to 48 rows go through the tensor-core kernel's three-block form
+    in ONE pass over the pair's keys and values (39 + 1 rows, the paper's R = 32 + 1, 20 + 1 at head dim 64; explicit
+    lists leave padding rows in every block). More rows than that go in groups, one launch per group; only the last
+    group holds the current token's row (own key and value, rows stored in their slot): 59 + 1 rows = 48 + 12 and
+    96 + 1 rows = 48 + 48 + a group with the current token alone. A long key block whose logits do not fit for 48 rows
+    is cut into smaller groups (C = 1024: 39 + 10 rows)."""
     _run_rebuild_first(SMALL.scaled(name="rows_40", rebuild_max=39, capacity=90, topk=30, prompt=140, steps=10, seed=146))
     _run_rebuild_first(SMALL.scaled(name="rows_33_explicit", rebuild_mode="explicit", rebuild_p=0.4, rebuild_max=32, capacity=80,
                                     topk=24, prompt=0, steps=70, seed=147))
     _run_rebuild_first(SMALL.scaled(name="rows_21_dh64_two_layers", head_dim=64, n_heads=3, hidden=192, n_layers=2, batch=2,
                                     rebuild_max=20, capacity=300, topk=100, prompt=400, steps=6, seed=148))
+    _run_rebuild_first(SMALL.scaled(name="rows_60_in_two_groups", rebuild_max=59, capacity=130, topk=40, prompt=200, steps=6, seed=156))
+    _run_rebuild_first(SMALL.scaled(name="rows_97_explicit_in_three_groups", rebuild_mode="explicit", rebuild_p=0.5, rebuild_max=96,
+                                    capacity=200, topk=64, prompt=260, steps=5, batch=2, seed=157))
+    _run_rebuild_first(wl.get_config(4).scaled(name="rows_49_cfg4_shape", n_layers=1, batch=2, per_layer_inputs=False, rebuild_max=48,
+                                               steps=2, seed=158))
+    _run_rebuild_first(wl.get_config(4).scaled(name="rows_33_cfg4_shape", n_layers=1, batch=2, per_layer_inputs=False, rebuild_max=32,
+                                               steps=2, seed=159))
 
 
 def test_cumulative_attention_as_the_score_source():
