@@ -101,8 +101,9 @@ def run_sweep(args):
         print(json.dumps({"workload": cfg.name, "capacity": cap, "batch": b, "steps_per_s": d["steps_per_s"],
                           "tokens_per_s": d["value"], "ms_per_step": d["ms_per_step"],
                           "attention_hbm_frac": st["attention"]["frac"],
-                          "attention_plus_selection_hbm_frac": st["attention_plus_selection"]["frac"],
-                          "attention_plus_selection_frac_is": st["attention_plus_selection"]["frac_is"],
+                          "attention_plus_selection_hbm_frac": {
+                              k: (st["attention_plus_selection"].get(k) or {}).get("frac")
+                              for k in ("stages_added", "overlapped", "overlapped_without_controller_tail")},
                           "rebuild": {k: st.get("rebuild", {}).get(k) for k in ("bound", "frac", "rows_per_launch", "ms_per_launch")},
                           "clocks": d["clocks"]}), flush=True)
 
