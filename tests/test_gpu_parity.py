@@ -123,13 +123,22 @@ def test_rebuild_on_sm_pairs_with_ragged_row_count():
                       rebuild_mode="explicit", rebuild_p=0.6, seed=117))
 
 
-def test_rebuild_with_the_reduction_dimension_split_over_work_units():
-    # few output tiles: the launch plan splits K in two so that more SMs stream the weights; whichever unit of a tile
-    # finishes last adds the two parts in a fixed order
+def test_rebuild_with_the_reduction_dimension_split_over_a_cta_pair():
+    # few output tiles: the launch plan splits K over the two CTAs of a cluster so that more SMs stream the weights; the
+    # halves are exchanged through distributed shared memory and each CTA finishes 64 of the tile's 128 columns
     _run(SMALL.scaled(name="ksplit2", hidden=1024, rebuild_max=12, capacity=48, topk=20, rebuild_mode="explicit", rebuild_p=0.5,
                       prompt=60, steps=8, seed=118))
     _run(SMALL.scaled(name="ksplit2_two_row_tiles", hidden=1024, batch=5, rebuild_max=40, capacity=100, topk=40,
                       rebuild_mode="explicit", rebuild_p=0.7, prompt=160, steps=6, seed=120))   # 200 rows: 2 x 8 tiles x 2 parts
+    # several layers: the rebuilds run beside the following layers' attention with the small ring (3 stages)
+    _run(SMALL.scaled(name="ksplit2_small_ring_two_layers", hidden=1024, n_layers=2, batch=2, rebuild_max=9, capacity=40, topk=16,
+                      prompt=70, steps=6, seed=160))
+
+
+def test_config2_full_batch_in_the_benchmark_launch_configuration():
+    """All 16 sequences of config 2: 128 listed rows = one full row tile of the K-split GEMM (64 CTA pairs), 512 attention
+    items with the 256-thread selection beside them. Two decode steps, every output compared."""
+    _run(wl.get_config(2), steps=2)
 
 
 def test_largest_capacity_and_token_table_the_library_accepts():
