@@ -256,14 +256,26 @@ class DeviceRun:
         self.tables = None
         if c.per_layer_inputs:
             self.tables = [torch.zeros((B, c.max_tokens, d), dtype=self.dt, device=dev) for _ in range(L)]
+        self.prompt_ms = 0.0        # device time of the prompt's bulk load (controller scan, selection, fill of every layer)
         if c.prompt:
             xp = prompt_rows()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
             lib.adore_cache_append_tokens(self.handle, xp, c.prompt)
+            lib.adore_cache_join(self.handle)
+            e1.record()
+            torch.cuda.synchronize()
+            self.prompt_ms = e0.elapsed_time(e1)
             if c.per_layer_inputs:
                 self.tables[0][:, : c.prompt] = xp
                 for l in range(1, L):
                     self.tables[l][:, : c.prompt] = prompt_rows()
+                    e0.record()
                     lib.adore_cache_fill_layer(self.handle, l, self.tables[l])
+                    lib.adore_cache_join(self.handle)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    self.prompt_ms += e0.elapsed_time(e1)
             del xp
         # per-step inputs
         S = self.S = total_steps
@@ -818,6 +830,13 @@ def main():
                                   "controller_select": st_ms[1] / max(sum(st_ms), 1e-9),
                                   "rebuild": st_ms[2] / max(sum(st_ms), 1e-9)}}
 
+    prompt_load = None
+    if cfg.prompt:
+        n_prompt = cfg.batch * cfg.prompt
+        prompt_load = {"tokens": n_prompt, "layers": cfg.n_layers, "ms": run.prompt_ms,
+                       "tokens_per_s": n_prompt / (run.prompt_ms * 1e-3) if run.prompt_ms > 0 else None,
+                       "what": "adore_cache_append_tokens (controller scan, bulk selection, projection of the residents) "
+                               "+ adore_cache_fill_layer for every further layer; device time, once, before the decode steps"}
     run.close()
     del run, kv_live, kv_keep
     torch.cuda.empty_cache()
@@ -840,7 +859,8 @@ def main():
                 "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
                 "config": dict(workload_desc(cfg), step_order=args.order, score_source=args.score_source), "clocks": clocks,
                 "clocks_stage_pass": clocks_stage, "e2e": e2e, "gpu_launches": int(launches),
-                "roofline": roofline, "stages": stages, "cpu_baseline": cpu, "largest_config": largest}
+                "roofline": roofline, "stages": stages, "prompt_load": prompt_load, "cpu_baseline": cpu,
+                "largest_config": largest}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -849,7 +869,7 @@ def main():
 def run_largest_leg(args):
     """Config 4 (32 layers, B 32, C 1024: the configuration the HBM target is stated for) in a process of its own, a few
     timed steps; returns the part of its line that the metric names."""
-    cmd = [sys.executable, os.path.abspath(__file__), "--config", "4", "--leg", "--no-cpu-baseline", "--no-e2e",
+    cmd = [sys.executable, os.path.abspath(__file__), "--config", "4", "--leg", "--no-cpu-baseline",
            "--steps", str(args.largest_steps), "--warmup", "3", "--min-timed-ms", "400", "--max-repeats", "12"]
     try:
         res = subprocess.run(cmd, capture_output=True, text=True, timeout=900)
@@ -862,7 +882,8 @@ def run_largest_leg(args):
     return {"workload": d["config"]["workload"], "steps": d["steps"], "repeats": d["repeats"], "ms_per_step": d["ms_per_step"],
             "tokens_per_s": d["value"], "steps_per_s": d["steps_per_s"], "gpu_launches": d["gpu_launches"], "clocks": d["clocks"],
             "attention": st["attention"], "attention_plus_selection": st["attention_plus_selection"],
-            "controller_select": st["controller_select"], "rebuild": st.get("rebuild")}
+            "controller_select": st["controller_select"], "rebuild": st.get("rebuild"), "prompt_load": d.get("prompt_load"),
+            "e2e": d.get("e2e")}
 
 
 if __name__ == "__main__":
