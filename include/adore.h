@@ -154,6 +154,9 @@ adore_status_t adore_cache_fill_layer(adore_cache_t *cache, int32_t layer, const
  *   x_new           : T[B, d], read at layer 0 only (stored in the token table), else ignored.
  *   explicit_list   : int32[B, r_in] candidate token positions, explicit_count int32[B] how many
  *                     are valid per sequence; both NULL in POLICY mode. Read at layer 0 only.
+ *                     x_new and the lists are read by kernels on the library's own streams; the
+ *                     caller's stream is made to wait for those reads before the call returns,
+ *                     so work queued on it afterwards may overwrite them.
  *   out             : T[B, H, dh].
  *   weights         : float[B, H, C+1] or NULL. Entry s < C is slot s, entry C the current
  *                     token; masked or empty entries are 0.
