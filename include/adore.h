@@ -149,7 +149,9 @@ adore_status_t adore_cache_fill_layer(adore_cache_t *cache, int32_t layer, const
 
 /* One decode step for one layer (Sections 2.1-2.3). Call layer 0 first in every step; it also
  * runs the controller for the new token, releases / admits / chooses the rebuild list, and
- * advances n. All pointers are DEVICE pointers.
+ * advances n. All pointers are DEVICE pointers; q, k_new, v_new, x_new and out must start on a
+ * 16-byte boundary (INVALID_ARG otherwise; the same holds for the row pointers of
+ * adore_step_begin / adore_attend_rows and for x_table of adore_rebuild / adore_cache_fill_layer).
  *   q, k_new, v_new : T[B, H, dh]; k_new already carries the rotary embedding of position n.
  *   x_new           : T[B, d], read at layer 0 only (stored in the token table), else ignored.
  *   explicit_list   : int32[B, r_in] candidate token positions, explicit_count int32[B] how many

@@ -260,6 +260,10 @@ adore_status_t join_controller(adore_cache* c) {
   return ADORE_OK;
 }
 
+// The kernels fetch rows of q, k, v, x and the row tables' sources in 16-byte pieces: a device pointer that does not
+// start on such a boundary is refused on the host (a misaligned access would fault the device).
+inline bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
 // Makes `stream` wait for the rebuild of `layer` if it is still running beside the main stream.
 adore_status_t wait_rebuild(adore_cache* c, int layer, cudaStream_t stream) {
   if (layer >= 0 && layer < int(c->rb_pending.size()) && c->rb_pending[layer])
@@ -974,7 +978,7 @@ adore_status_t adore_cache_append_tokens(adore_cache_t* c, const void* x, int32_
 }
 
 adore_status_t adore_cache_fill_layer(adore_cache_t* c, int32_t layer, const void* x_table) {
-  if (!c || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || misaligned16(x_table)) return ADORE_ERR_INVALID_ARG;
   if (!c->w_kv[layer]) return ADORE_ERR_STATE;
   if (join_rebuilds(c) != ADORE_OK) return ADORE_ERR_CUDA;
   return fill_layer_impl(c, layer, x_table);
@@ -984,6 +988,8 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
                                  const void* x_new, const int32_t* explicit_list, const int32_t* explicit_count,
                                  int32_t r_in, void* out, float* weights) {
   if (!c || !q || !k_new || !v_new || !out || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (misaligned16(q) || misaligned16(k_new) || misaligned16(v_new) || misaligned16(out) || (layer == 0 && misaligned16(x_new)))
+    return ADORE_ERR_INVALID_ARG;
   const adore_config_t& f = c->cfg;
   const bool from_attention = (f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION) != 0;
   if (from_attention && !weights) weights = c->w_internal;
@@ -1072,7 +1078,7 @@ adore_status_t adore_decode_step(adore_cache_t* c, int32_t layer, const void* q,
 
 adore_status_t adore_step_begin(adore_cache_t* c, const void* x_new, const int32_t* explicit_list,
                                 const int32_t* explicit_count, int32_t r_in) {
-  if (!c || !x_new) return ADORE_ERR_INVALID_ARG;
+  if (!c || !x_new || misaligned16(x_new)) return ADORE_ERR_INVALID_ARG;
   const adore_config_t& f = c->cfg;
   if (f.flags & ADORE_FLAG_SCORE_FROM_ATTENTION) return ADORE_ERR_UNSUPPORTED;   // defined for the attend-first step
   if (c->n >= f.max_tokens) return ADORE_ERR_TOKEN_TABLE_FULL;
@@ -1103,6 +1109,7 @@ adore_status_t adore_step_begin(adore_cache_t* c, const void* x_new, const int32
 adore_status_t adore_attend_rows(adore_cache_t* c, int32_t layer, const void* q_rows, const void* k_new, const void* v_new,
                                  void* out, float* weights) {
   if (!c || !q_rows || !k_new || !v_new || !out || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (misaligned16(q_rows) || misaligned16(k_new) || misaligned16(v_new) || misaligned16(out)) return ADORE_ERR_INVALID_ARG;
   if (c->step_layer0_done != 2) return ADORE_ERR_STATE;
   if (wait_rebuild(c, layer, c->stream) != ADORE_OK) return ADORE_ERR_CUDA;   // this layer's rows may come from the side stream
   const adore_config_t& f = c->cfg;
@@ -1247,7 +1254,7 @@ adore_status_t adore_cache_wait_outputs(adore_cache_t* c) {
 }
 
 adore_status_t adore_rebuild(adore_cache_t* c, int32_t layer, const void* x_table) {
-  if (!c || layer < 0 || layer >= c->cfg.n_layers) return ADORE_ERR_INVALID_ARG;
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || misaligned16(x_table)) return ADORE_ERR_INVALID_ARG;
   if (!c->w_kv[layer] || !c->step_layer0_done) return ADORE_ERR_STATE;
   const adore_config_t& f = c->cfg;
   // Attend-first order with several layers: this layer's rows are next read by the next step's attention of this

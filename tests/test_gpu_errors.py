@@ -75,6 +75,22 @@ def test_full_token_table_and_bad_arguments():
                 call()
             assert e.value.status == 1
         lib.adore_cache_sync_status(g.handle)
+        # device pointers off the 16-byte boundary the kernels' loads need: refused on the host, nothing is launched
+        n_elems = g.B * CFG.n_heads * CFG.head_dim
+        skew = torch.zeros(n_elems + 8, dtype=torch.bfloat16, device="cuda")[1:n_elems + 1]     # 2 bytes off
+        xskew = torch.zeros(g.B * CFG.hidden + 8, dtype=torch.bfloat16, device="cuda")[3:g.B * CFG.hidden + 3]
+        launches = lib.adore_cache_launch_count(g.handle)
+        for call in (lambda: lib.adore_decode_step(g.handle, 1, skew, k, v, None, None, None, 0, g.out, None),
+                     lambda: lib.adore_decode_step(g.handle, 1, q, k, skew, None, None, None, 0, g.out, None),
+                     lambda: lib.adore_decode_step(g.handle, 1, q, k, v, None, None, None, 0, skew, None),
+                     lambda: lib.adore_step_begin(g.handle, xskew, None, None, 0),
+                     lambda: lib.adore_rebuild(g.handle, 0, xskew),
+                     lambda: lib.adore_cache_fill_layer(g.handle, 1, xskew)):
+            with pytest.raises(lib.AdoreError) as e:
+                call()
+            assert e.value.status == 1
+        assert lib.adore_cache_launch_count(g.handle) == launches
+        lib.adore_cache_sync_status(g.handle)
         # flags that exclude each other, and a flag bit that does not exist
         for flags in (lib.ADORE_FLAG_SCORE_FROM_ATTENTION | lib.ADORE_FLAG_RELATIVE_POSITION, 1 << 9):
             with pytest.raises(lib.AdoreError) as e:
