@@ -799,6 +799,13 @@ def main():
         stages["attention_plus_selection"].update(achieved=ov_gbs, frac=ov_gbs / peaks["hbm_gbs"], frac_is="overlapped")
     else:
         stages["attention_plus_selection"].update(achieved=both_gbs, frac=both_gbs / peaks["hbm_gbs"], frac_is="stages_added")
+    # every algorithmic byte of a step (attention of all layers, controller + selection, rebuild of all layers) over the
+    # free-running step time: what the whole step makes of the HBM (the rebuilds share the bandwidth with the attention)
+    step_bytes = group_bytes + (reb_bytes * cfg.n_layers if rows > 0 else 0)
+    step_ms = ms_total / K
+    step_gbs = step_bytes / (step_ms * 1e-3) / 1e9
+    stages["step_hbm"] = {"algorithmic_bytes": step_bytes, "ms_per_step": step_ms, "achieved": step_gbs, "unit": "GB/s",
+                          "peak": peaks["hbm_gbs"], "frac": step_gbs / peaks["hbm_gbs"]}
     tensor_bound = cfg.dtype == "bf16" and rows >= 300
     if reb_ms > 0 and rows > 0:
         if tensor_bound:
@@ -882,8 +889,8 @@ def run_largest_leg(args):
     return {"workload": d["config"]["workload"], "steps": d["steps"], "repeats": d["repeats"], "ms_per_step": d["ms_per_step"],
             "tokens_per_s": d["value"], "steps_per_s": d["steps_per_s"], "gpu_launches": d["gpu_launches"], "clocks": d["clocks"],
             "attention": st["attention"], "attention_plus_selection": st["attention_plus_selection"],
-            "controller_select": st["controller_select"], "rebuild": st.get("rebuild"), "prompt_load": d.get("prompt_load"),
-            "e2e": d.get("e2e")}
+            "controller_select": st["controller_select"], "rebuild": st.get("rebuild"), "step_hbm": st.get("step_hbm"),
+            "prompt_load": d.get("prompt_load"), "e2e": d.get("e2e")}
 
 
 if __name__ == "__main__":
