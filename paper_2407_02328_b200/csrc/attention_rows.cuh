@@ -239,8 +239,8 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     }
     int cnt = 0;
 #pragma unroll
-    for (int j = 0; j < KPL; ++j)
-      cnt += __popc(__ballot_sync(0xffffffffu, kk[j] > kMasked));
+    for (int j = 0; j < KPL; ++j) cnt += kk[j] > kMasked ? 1 : 0;
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
     uint32_t thr_key = 0u;
     if (cnt > p.topk) {
       // K-th largest key by bisection on the key's bits, most significant first: thr is the largest value with at
@@ -251,11 +251,8 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
 #pragma unroll
       for (int j = 0; j < KPL; ++j)
         if (kk[j] > kMasked) { kmin = min(kmin, kk[j]); kmax = max(kmax, kk[j]); }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
-        kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
-      }
+      kmin = __reduce_min_sync(0xffffffffu, kmin);
+      kmax = __reduce_max_sync(0xffffffffu, kmax);
       const uint32_t diff = kmin ^ kmax;
       const int top = diff ? 31 - __clz(diff) : -1;
       uint32_t thr = top >= 31 ? 0u : (kmax & ~((2u << (top < 0 ? 0 : top)) - 1u));
@@ -274,10 +271,9 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
       int gt = 0, eq = 0;
       if (!exact) {
 #pragma unroll
-        for (int j = 0; j < KPL; ++j) {
-          gt += __popc(__ballot_sync(0xffffffffu, kk[j] > thr));
-          eq += __popc(__ballot_sync(0xffffffffu, kk[j] == thr));
-        }
+        for (int j = 0; j < KPL; ++j) { gt += kk[j] > thr ? 1 : 0; eq += kk[j] == thr ? 1 : 0; }
+        gt = __reduce_add_sync(0xffffffffu, gt);
+        eq = __reduce_add_sync(0xffffffffu, eq);
       }
       const int need = p.topk - gt;                     // how many of the keys equal to the threshold stay
       if (!exact && eq != need) {                       // equal logits at the threshold: the lowest indices stay
@@ -287,28 +283,39 @@ attention_rows_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
             if (float_key(row[i]) == thr_key) { if (left > 0) --left; else row[i] = -INFINITY; }
         }
         __syncwarp();
+#pragma unroll
+        for (int j = 0; j < KPL; ++j) {                 // (rare) the keys in registers follow the row
+          const int i = j * 32 + lane;
+          kk[j] = i < rows_n ? float_key(row[i]) : 0u;
+        }
       }
     }
-    float mx = -INFINITY;
-    for (int i = lane; i < rows_n; i += 32) {
-      const float l = row[i];
-      if (l > -INFINITY && float_key(l) >= thr_key) mx = fmaxf(mx, l);
-    }
-    mx = warp_max(mx);
+    // softmax over the kept logits, from the keys in registers (the key of a float is invertible): the largest key is
+    // always kept, so it gives the maximum; weights go back to the row (phase 3 reads them) and out
+    const uint32_t keep_from = thr_key > kMasked ? thr_key : kMasked + 1u;
+    uint32_t kmax_all = 0u;
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) kmax_all = max(kmax_all, kk[j]);
+    kmax_all = __reduce_max_sync(0xffffffffu, kmax_all);
+    const float mx = __uint_as_float((kmax_all & 0x80000000u) ? (kmax_all & 0x7fffffffu) : ~kmax_all);
     float part = 0.f;
-    for (int i = lane; i < rows_n; i += 32) {
-      const float l = row[i];
-      const bool keep = l > -INFINITY && float_key(l) >= thr_key;
-      const float e = keep ? expf(l - mx) : 0.f;
-      row[i] = e;
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) {
+      const float l = __uint_as_float((kk[j] & 0x80000000u) ? (kk[j] & 0x7fffffffu) : ~kk[j]);
+      const float e = kk[j] >= keep_from ? expf(l - mx) : 0.f;
+      kk[j] = __float_as_uint(e);
       part += e;
     }
     part = warp_sum(part);
     const float inv = part > 0.f ? 1.f / part : 0.f;    // a padding row (nothing visible) keeps all-zero weights
-    for (int i = lane; i < rows_n; i += 32) {
-      const float w = row[i] * inv;
-      row[i] = w;
-      if (wout) wout[i] = w;
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) {
+      const int i = j * 32 + lane;
+      if (i < rows_n) {
+        const float w = __uint_as_float(kk[j]) * inv;
+        row[i] = w;
+        if (wout) wout[i] = w;
+      }
     }
   }
   __syncthreads();
