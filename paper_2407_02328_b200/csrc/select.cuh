@@ -41,6 +41,13 @@ __device__ __forceinline__ unsigned long long block_min_u64(unsigned long long v
   for (int w = 0; w < int(blockDim.x >> 5); ++w) r = tmp[w] < r ? tmp[w] : r;
   return r;
 }
+// Largest 64-bit value of a warp: the high words first, then the low words of the lanes that hold the largest high word.
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+  const uint32_t hi = uint32_t(v >> 32);
+  const uint32_t hmax = __reduce_max_sync(0xffffffffu, hi);
+  const uint32_t lmax = __reduce_max_sync(0xffffffffu, hi == hmax ? uint32_t(v) : 0u);
+  return (static_cast<unsigned long long>(hmax) << 32) | lmax;
+}
 __device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v, unsigned long long* tmp) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -271,8 +278,47 @@ __device__ inline int assign_rebuild_list(const SelectParams& p, const SelectSme
       const int i = tid + j * NT;
       k[j] = (i < n_seen && tok_slot[i] < 0) ? value_key(score[i], i) : 0ull;
     }
-    unsigned long long prev = ~0ull;
     int found = 0;
+    const int NW = NT >> 5, lane = tid & 31, warp = tid >> 5;
+    if (p.P >= NW * p.r_max) {
+      // Two levels, two block barriers: every warp picks the r_max largest of its own keys (a warp-wide maximum of a
+      // 64-bit key = two 32-bit ones: the score part, then the position among the lanes that hold that score), the
+      // candidates of all warps meet in shared memory (the key array is free here) and warp 0 picks among them.
+      unsigned long long prev = ~0ull;
+      for (int r = 0; r < p.r_max; ++r) {
+        unsigned long long m = 0ull;
+#pragma unroll
+        for (int j = 0; j < kSelectIterKeys; ++j) m = (k[j] < prev && k[j] > m) ? k[j] : m;
+        m = warp_max_u64(m);
+        if (lane == 0) sm.keys[warp * p.r_max + r] = m;    // (0 once the warp has run out of released tokens)
+        prev = m == 0ull ? 0ull : m;
+      }
+      __syncthreads();
+      if (warp == 0) {
+        unsigned long long c[kSelectIterKeys / 2];           // 16 warps x 16 candidates at most = 8 per lane
+#pragma unroll
+        for (int j = 0; j < kSelectIterKeys / 2; ++j) {
+          const int i = lane + 32 * j;
+          c[j] = i < NW * p.r_max ? sm.keys[i] : 0ull;
+        }
+        unsigned long long top = ~0ull;
+        for (int r = 0; r < p.r_max; ++r) {
+          unsigned long long m = 0ull;
+#pragma unroll
+          for (int j = 0; j < kSelectIterKeys / 2; ++j) m = (c[j] < top && c[j] > m) ? c[j] : m;
+          m = warp_max_u64(m);
+          if (m == 0ull) break;
+          if (lane == 0) sm.lst[r] = int(m & 0xffffffffull);
+          top = m;
+          ++found;
+        }
+        if (lane == 0) sm.tmp[0] = found;
+      }
+      __syncthreads();
+      found = sm.tmp[0];
+      return place_rebuild_list(p, sm, b, tok_slot, found);
+    }
+    unsigned long long prev = ~0ull;
     for (int r = 0; r < p.r_max; ++r) {
       unsigned long long m = 0ull;
 #pragma unroll
