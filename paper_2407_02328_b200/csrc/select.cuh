@@ -469,27 +469,42 @@ __device__ inline void select_step(const SelectParams& p, unsigned char* smem) {
     sm.role[s] = r;
   }
   __syncthreads();
-  // 2. full => release the least valuable retained token
-  int cnt = 0;
+  // 2. + 3. One pass over the map and ONE block-wide reduction give the number of retained tokens, the least valuable of
+  // them and the lowest empty slot. A full cache releases that token; the new token takes the lowest empty slot, which
+  // is the released token's own if that lies lower.
+  int cnt = 0, emin = INT_MAX;
   unsigned long long kmin = ~0ull;
-  for (int s = tid; s < C; s += NT)
-    if (sm.role[s] == ROLE_RETAINED) {
+  for (int s = tid; s < C; s += NT) {
+    const uint8_t r = sm.role[s];
+    if (r == ROLE_RETAINED) {
       ++cnt;
       const unsigned long long k = value_key(score[sm.tok[s]], sm.tok[s]);
       kmin = k < kmin ? k : kmin;
+    } else if (r == ROLE_EMPTY) {
+      emin = min(emin, s);
     }
-  const int n_ret = block_sum_i(cnt, sm.tmp);
-  kmin = block_min_u64(kmin, sm.tmp64);
+  }
+  cnt = warp_sum(cnt);
+  kmin = warp_min(kmin);
+  emin = warp_min(emin);
+  if ((tid & 31) == 0) { sm.tmp[tid >> 5] = cnt; sm.tmp[32 + (tid >> 5)] = emin; sm.tmp64[tid >> 5] = kmin; }
+  if (tid == 0) sm.tmp[31] = INT_MAX;                     // the released token's slot, written below by the thread that holds it
+  __syncthreads();
+  int n_ret = 0;
+  emin = INT_MAX;
+  kmin = ~0ull;
+  for (int w = 0; w < (NT >> 5); ++w) {
+    n_ret += sm.tmp[w];
+    emin = min(emin, sm.tmp[32 + w]);
+    kmin = sm.tmp64[w] < kmin ? sm.tmp64[w] : kmin;
+  }
   const int evicted = (n_ret >= p.m) ? int(kmin & 0xffffffffull) : -1;
   if (evicted >= 0)
     for (int s = tid; s < C; s += NT)
-      if (sm.tok[s] == evicted) { sm.tok[s] = -1; sm.role[s] = ROLE_EMPTY; tok_slot[evicted] = -1; }
+      if (sm.tok[s] == evicted) { sm.tok[s] = -1; sm.role[s] = ROLE_EMPTY; tok_slot[evicted] = -1; sm.tmp[31] = s; }
   __syncthreads();
-  // 3. the new token takes the lowest-index empty slot
-  int amin = INT_MAX;
-  for (int s = tid; s < C; s += NT) if (sm.role[s] == ROLE_EMPTY) amin = min(amin, s);
-  amin = block_min_i(amin, sm.tmp);
   if (tid == 0) {
+    const int amin = min(emin, sm.tmp[31]);
     if (amin < C) { sm.tok[amin] = p.n; sm.role[amin] = ROLE_RETAINED; tok_slot[p.n] = amin; }
     else set_error(p.err, ERRW_BOUNDS);
     p.admit_slot[b] = amin < C ? amin : -1;
