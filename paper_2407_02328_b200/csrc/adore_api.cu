@@ -334,9 +334,10 @@ int select_threads(const adore_cache*) { return 512; }
 // The step's selection runs beside the attention of layer 0. With few (batch, head) pairs that launch has 256-thread
 // CTAs of 16k registers, three or four to an SM: a selection CTA of 256 threads x 64 registers still fits beside three
 // of them and starts at once, one of 512 threads waits until an SM has drained (measured: 14 us later).
-int step_select_threads(const adore_cache* c) {
+// (Eight warps sort or scan at most 4096 keys, 512 each: wider candidate sets keep the 512-thread CTA.)
+int step_select_threads(const adore_cache* c, int P) {
   const adore_config_t& f = c->cfg;
-  return f.batch * f.n_heads < 1024 && f.max_tokens <= 4096 ? 256 : 512;
+  return f.batch * f.n_heads < 1024 && P <= 4096 ? 256 : 512;
 }
 size_t ctrl_smem(const adore_cache* c) {
   const int h = c->cfg.ctrl_hidden;
@@ -639,7 +640,7 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
     sp.rows_accum = c->rows_accum; sp.done_count = c->sel_done;
   }
   const size_t smem = select_smem_bytes(f.capacity, P);
-  select_kernel<<<f.batch, step_select_threads(c), smem, sel>>>(sp);
+  select_kernel<<<f.batch, step_select_threads(c, P), smem, sel>>>(sp);
   ++c->launches;
   CUDA_OK(cudaGetLastError());
   if (!table_in_select) {

@@ -149,6 +149,13 @@ def test_largest_capacity_and_token_table_the_library_accepts():
                       prompt=8184, steps=8, seed=149), state_every=4)
 
 
+def test_explicit_list_wider_than_4096_entries_for_a_few_pairs():
+    """A caller's candidate list of ~4900 entries per sequence (90 % of 5000 tokens flagged) with only two (b, h) pairs:
+    the selection sorts 8192 keys, which needs its 512-thread CTA although the attention launch beside it is small."""
+    _run(SMALL.scaled(name="explicit_4900", batch=1, n_heads=2, head_dim=64, hidden=128, capacity=1024, topk=300, rebuild_max=300,
+                      rebuild_mode="explicit", rebuild_p=0.9, prompt=5000, steps=4, seed=161), state_every=2)
+
+
 def test_capacity_batch_sweep_corner_shapes():
     """Three points of the capacity x batch sweep (context 4096 = prompt 3840 + steps, K = C/2, R_max = C/4, explicit
     flags at 10 %) with the sweep's own shapes per sequence and a sub-batch the oracle finishes in a minute."""
