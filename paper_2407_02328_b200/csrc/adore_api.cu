@@ -648,12 +648,11 @@ adore_status_t launch_controller_and_selection(adore_cache* c, const void* x_new
     if (st != ADORE_OK) return st;
   }
   c->joined = sel == c->stream;
-  if (!c->joined) {
-    CUDA_OK(cudaEventRecord(c->ev_join, sel));   // the gather below is not part of what the main stream waits for
-    // The gate product starts when the selection is done: side by side the two were measured several times slower
-    // (gate product 14 -> 70 us, selection 18 -> 28 us at batch 16), whereas beside the rebuild GEMM it loses little.
-    CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_join, 0));
-  }
+  CUDA_OK(cudaEventRecord(c->ev_join, sel));     // the gather below is not part of what the main stream waits for
+  // The gate product starts when the selection is done: side by side the two were measured several times slower
+  // (gate product 14 -> 70 us, selection 18 -> 28 us at batch 16), whereas beside the rebuild GEMM it loses little.
+  // (Also with per-stage timing on, where the selection runs on the main stream.)
+  CUDA_OK(cudaStreamWaitEvent(c->ctl, c->ev_join, 0));
   // A short list's rows are copied out of the token store into the GEMM's compact input right away, beside the
   // attention, so that the rebuild that follows starts with its GEMM. Long lists are copied after the attention:
   // side by side the two slow each other down by more than the copy takes (measured at 15k rows: attention
