@@ -496,7 +496,9 @@ constexpr size_t kTcPartialFloatsPerSm = size_t(256) * 128;
 // Which kernel and which split of K serve a launch of at most `rows` rows. Enough 256 x 256 tiles for every SM pair:
 // the two-SM kernel (tensor-bound). Enough 128 x 256 tiles for every SM: those. Otherwise the launch is bound by the
 // latency of streaming each weight tile once (measured: ~1.5 us per 32 KB stage with six stages in flight, i.e.
-// ~0.3 us per k-block whatever the tile), so 128 x 128 tiles, and K split in two when that still leaves SMs idle.
+// ~0.3 us per k-block whatever the tile), so 128 x 128 tiles, and K split in two when that still leaves SMs idle: over
+// the two CTAs of a cluster that add their halves through distributed shared memory (kind 3) where the device can hold
+// that many pairs, else over two independent work units that hand over through global memory and a counter (kind 0).
 struct TcPlan { int kind; int ksplit; int grid; };   // kind 0: 128-wide tiles, 1: 256-wide tiles, 2: SM pairs, 3: K split over a CTA pair
 inline TcPlan tc_plan(int rows, int N, int K, int sms, int pairs, int max_split, int split_pairs = 0) {
   const int kb = K / kTcBK;
