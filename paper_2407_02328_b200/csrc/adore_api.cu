@@ -516,7 +516,8 @@ adore_status_t launch_rebuild(adore_cache* c, int layer, const void* x_table, co
     // Rows gathered from the token store for this step's table serve every layer that rebuilds from the store.
     const bool from_store = step_table && x_table == nullptr && size_t(m_max) <= c->tc.a_rows;
     int launched = 0;
-    if (from_store && c->rows_gathered && c->gather_pending) {
+    // the early gather of this step's list (selection stream) writes the buffer that this launch reads or refills
+    if (c->gather_pending) {
       CUDA_OK(cudaStreamWaitEvent(stream, c->ev_gather, 0));
       if (stream == c->stream) c->gather_pending = false;       // (a side stream: every rebuild of the step waits)
     }

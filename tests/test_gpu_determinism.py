@@ -14,7 +14,7 @@ BASE = wl.WorkloadConfig(name="det", dtype="bf16", n_layers=3, batch=4, n_heads=
                          rebuild_p=0.5, seed=161, ctrl_hidden=128, per_layer_inputs=True)
 
 
-def _free_run(cfg, wait_after_every_call=False):
+def _free_run(cfg, wait_after_every_call=False, table_at_layer0=False):
     """All steps queued back to back on the device (or, for comparison, with a host wait after every call); returns
     everything observable at the end."""
     import torch
@@ -57,7 +57,7 @@ def _free_run(cfg, wait_after_every_call=False):
                                       dc if l == 0 else None, w.r_in if l == 0 else 0, outs[s, l], wts[s, l])
                 if wait_after_every_call:
                     lib.adore_cache_sync_status(g.handle)
-                lib.adore_rebuild(g.handle, l, tables[l] if (tables is not None and l > 0) else None)
+                lib.adore_rebuild(g.handle, l, tables[l] if (tables is not None and (l > 0 or table_at_layer0)) else None)
                 if wait_after_every_call:
                     lib.adore_cache_sync_status(g.handle)
         lib.adore_cache_sync_status(g.handle)
@@ -86,3 +86,18 @@ def test_two_free_running_runs_are_bit_identical(cfg):
             for l, (x, y) in enumerate(zip(a[key], other[key])):
                 assert np.array_equal(x, y), f"{key} rows of layer {l} differ between {what}"
     assert np.isfinite(a["out"]).all() and (a["slot_tok"] >= 0).any()
+
+
+def test_rebuild_from_a_caller_table_at_layer_0_equals_rebuild_from_the_store():
+    """Layer 0 rebuilt from the caller's table (the same rows the library keeps in its token store) instead of from the
+    store: the launch then gathers its rows itself, into the buffer that the step's early gather (selection stream) has
+    just filled, so it has to wait for that gather. Everything observable must equal the run that rebuilds from the store."""
+    a = _free_run(BASE)
+    b = _free_run(BASE, table_at_layer0=True)
+    for key in a:
+        if isinstance(a[key], list):
+            for x, y in zip(a[key], b[key]):
+                assert np.array_equal(x, y), key
+        else:
+            assert np.array_equal(a[key], b[key]), key
+
